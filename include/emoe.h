@@ -1,0 +1,257 @@
+/*
+ * emoe.h - C ABI of the ElasticMoE scale-step re-layout library (libemoe.so).
+ *
+ * One scaling step of an elastic MoE serving instance changes the parallel
+ * configuration: expert parallelism EP=a -> EP=b and tensor parallelism
+ * TP=c -> TP=d.  The paper's HMM derives a redistribution plan from the
+ * current and the target configuration (Sec. 5.2 "HMM Reconfigures Memory
+ * Layout") and then (i) provisions attention weights, (ii) carries the KV
+ * cache over and (iii) migrates experts so that every device again holds
+ * its experts as one contiguous tensor (Sec. 4.1 "Virtual Expert
+ * Management", App. D.5).  The paper keeps TP fixed and remaps pages instead
+ * of copying; it names the copy-based reshaping as the naive alternative
+ * (Sec. 4.1) and TP change with KV reshaping as future work (Sec. 9).  This
+ * library implements that copy-based, TP-changing re-layout on ONE GPU,
+ * where every "rank" is a distinct region ("arena") of that GPU's memory.
+ *
+ * All sizes and offsets are in BYTES unless a name says otherwise.  The
+ * library never interprets element values; `elem_bytes` only scales sizes.
+ *
+ * ---------------------------------------------------------------------------
+ * Layouts (row-major, densely packed, no padding)
+ *
+ *   L = n_layers, D = d_model, F = d_ff, b = elem_bytes, hd = head_dim,
+ *   Hq = n_q_heads, Hkv = n_kv_heads, B = kv_block_tokens, m = D*F*b.
+ *
+ *   Experts.  Logical ids 0..n_routed-1 are routed experts, n_routed ..
+ *   n_routed+n_shared-1 are shared experts.  The placement of rank r is the
+ *   ordered id list P[r] (CSR: place_ids[place_off[r] .. place_off[r+1])),
+ *   n_r = |P[r]|.  Expert arena of rank r:
+ *        [L][3 (gate, up, down)][n_r][m bytes]
+ *   i.e. offset(l, p, s) = ((l*3 + p)*n_r + s) * m.
+ *
+ *   Attention.  Logical Wq[Hq*hd][D], Wk/Wv[Hkv*hd][D], Wo[D][Hq*hd].
+ *   TP=T shard t holds rows [t*Hq*hd/T, (t+1)*Hq*hd/T) of Wq, the same row
+ *   slice (over Hkv) of Wk and Wv, and COLUMNS [t*Hq*hd/T, (t+1)*Hq*hd/T) of
+ *   Wo.  Attention arena of rank t:  [L][ q_t | k_t | v_t | o_t ], each piece
+ *   row-major with its own shard row pitch.
+ *
+ *   KV cache.  One pool per (layer, K|V) per TP rank, shared block table:
+ *        [L][2 (K, V)][kv_num_blocks][B][Hkv/T][hd]
+ *   Global KV head g lives on rank g / (Hkv/T) as local head g % (Hkv/T).
+ * ---------------------------------------------------------------------------
+ */
+#ifndef EMOE_H_
+#define EMOE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct emoe_plan emoe_plan_t; /* opaque; owned by the library */
+
+typedef enum {
+  EMOE_OK = 0,
+  EMOE_ERR_INVALID_ARG = 1,  /* NULL pointer, bad enum value, wrong plan kind         */
+  EMOE_ERR_SHAPE = 2,        /* non-positive dimension, TP does not divide the heads  */
+  EMOE_ERR_PLACEMENT = 3,    /* id out of range, duplicate inside one rank, expert    */
+                             /* missing from the old or from the new placement        */
+  EMOE_ERR_BLOCK_TABLE = 4,  /* id out of range, physical block used twice, old/new   */
+                             /* sequence sets differ, table shorter than a sequence   */
+  EMOE_ERR_ALIGNMENT = 5,    /* an arena base pointer is not 16-byte aligned          */
+  EMOE_ERR_OVERLAP = 6,      /* a source arena intersects a destination arena         */
+  EMOE_ERR_OOM = 7,          /* host or device allocation for the plan failed         */
+  EMOE_ERR_CUDA = 8,         /* a CUDA runtime call failed (no device, bad stream...) */
+  EMOE_ERR_UNSUPPORTED = 9,  /* TP > n_kv_heads, more ranks than EMOE_MAX_RANKS, ...  */
+  EMOE_ERR_DEVICE_TIMEOUT = 10 /* a bounded device-side wait expired                  */
+} emoe_status_t;
+
+/* Model shape.  All fields must be > 0 except n_shared (>= 0). */
+typedef struct {
+  int32_t n_layers;
+  int32_t n_routed;        /* routed experts per layer                       */
+  int32_t n_shared;        /* shared experts per layer (ids follow routed)   */
+  int32_t d_model;
+  int32_t d_ff;
+  int32_t n_q_heads;
+  int32_t n_kv_heads;
+  int32_t head_dim;
+  int32_t kv_block_tokens; /* tokens per paged-KV block                      */
+  int32_t elem_bytes;      /* 2 for bf16                                     */
+} emoe_shape_t;
+
+/* One parallel configuration.  Every pointed-to array is caller-owned host
+ * memory; emoe_plan_create deep-copies what it needs. */
+typedef struct {
+  int32_t ep;                 /* expert-parallel ranks (1..EMOE_MAX_RANKS)          */
+  int32_t tp;                 /* tensor-parallel ranks (1..EMOE_MAX_RANKS)          */
+  const int32_t *place_off;   /* [ep+1] CSR offsets into place_ids                  */
+  const int32_t *place_ids;   /* expert ids, rank by rank, in slot order            */
+  int32_t kv_num_blocks;      /* physical blocks per (layer, K|V) pool per rank     */
+  int32_t n_seqs;             /* sequences in the block table                       */
+  int32_t max_blocks;         /* row length of block_table                          */
+  const int32_t *seq_lens;    /* [n_seqs] tokens per sequence                       */
+  const int32_t *block_table; /* [n_seqs][max_blocks] physical ids, -1 padded       */
+} emoe_config_t;
+
+#define EMOE_MAX_RANKS 64
+
+/* emoe_plan_create flags */
+#define EMOE_PLAN_HOST_ONLY 1u /* build and validate the plan on the host only: no CUDA */
+                               /* call is made, the reshard calls return EMOE_ERR_CUDA  */
+
+/* phase / side selectors of the query helpers */
+#define EMOE_PHASE_EXPERTS 0
+#define EMOE_PHASE_ATTN 1
+#define EMOE_PHASE_KV 2
+#define EMOE_SIDE_OLD 0
+#define EMOE_SIDE_NEW 1
+
+/*
+ * emoe_plan_create - host planner (Sec. 5.2: the plan is a function of the
+ * current and the target configuration only).
+ *
+ * Validates shape and both configurations, enumerates the logical moves of
+ * the three phases, picks the source replica of every destination expert
+ * slot (the copy already on the same rank index if there is one, "maximize
+ * zero-copy reuse", otherwise the lexicographically smallest (rank, slot)),
+ * coalesces moves into segments, and uploads the descriptor arrays to the
+ * current CUDA device (unless EMOE_PLAN_HOST_ONLY).
+ *
+ * shape, old_cfg, new_cfg: host pointers, read during the call only.
+ * n_seqs and seq_lens must agree between old_cfg and new_cfg.
+ * out: receives the plan on success, untouched on failure.
+ * Errors: any validation failure is reported before any device work.
+ */
+emoe_status_t emoe_plan_create(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
+                               const emoe_config_t *new_cfg, uint32_t flags,
+                               emoe_plan_t **out);
+
+/*
+ * emoe_reshard_experts - expert re-pack EP=a -> EP=b (Sec. 4.1 "Virtual
+ * Expert Management", Sec. 5.2 "Expert Weights", App. E for b < a).
+ *
+ * For every new rank r', layer l, projection p and slot s' the matrix of
+ * expert P_new[r'][s'] is copied from its source (rank, slot) of the old
+ * layout to offset(l, p, s') of the new arena of r'.
+ *
+ * src: HOST array of ep_old DEVICE pointers (old expert arenas).
+ * dst: HOST array of ep_new DEVICE pointers (new expert arenas).
+ * cuda_stream: a cudaStream_t (NULL = legacy default stream).
+ * Arenas are caller-owned, sized by emoe_plan_arena_bytes, 16-byte aligned,
+ * and no source arena may intersect a destination arena (out of place).
+ * The call only enqueues work on the stream: it neither synchronises nor
+ * allocates.  The pointer arrays are read before the call returns.
+ */
+emoe_status_t emoe_reshard_experts(const emoe_plan_t *plan, const void *const *src,
+                                   void *const *dst, void *cuda_stream);
+
+/*
+ * emoe_reshard_attn - attention q/k/v/o re-slice TP=c -> TP=d (Sec. 2.1:
+ * TP shards the attention operations; Sec. 5.2 "Attention Weights" is the
+ * c == d case, a whole-tensor copy onto added devices; Sec. 9 names c != d
+ * as future work).  q/k/v are split by stored rows (heads), o by stored
+ * columns (heads).  src: [tp_old] device pointers, dst: [tp_new]; otherwise
+ * as emoe_reshard_experts.
+ */
+emoe_status_t emoe_reshard_attn(const emoe_plan_t *plan, const void *const *src,
+                                void *const *dst, void *cuda_stream);
+
+/*
+ * emoe_reshard_kv - paged KV cache head re-split and re-paging (Sec. 5.2
+ * "KV Cache" is the c == d, same-table case; Sec. 9 "reshaping KV caches").
+ *
+ * For every sequence s, block index j < ceil(seq_len/B), layer, K|V, token
+ * slot and global KV head g, head_dim elements move from old rank
+ * g/(Hkv/c), old physical block bt_old[s][j], local head g%(Hkv/c) to new
+ * rank g/(Hkv/d), block bt_new[s][j], local head g%(Hkv/d).  Whole blocks
+ * move; destination blocks that no sequence maps are not written.
+ * src: [tp_old] device pointers, dst: [tp_new]; otherwise as above.
+ */
+emoe_status_t emoe_reshard_kv(const emoe_plan_t *plan, const void *const *src,
+                              void *const *dst, void *cuda_stream);
+
+/*
+ * emoe_reshard_step_host - one whole scale step on HOST buffers: copies
+ * every old arena host->device into caller-provided device staging arenas,
+ * runs the three phases, and copies every new arena device->host, all
+ * enqueued on cuda_stream (no synchronisation, no allocation).
+ *
+ * h_src / h_dst: per phase (index EMOE_PHASE_*), HOST arrays of HOST
+ * pointers ([ranks of the old side] / [ranks of the new side]); pinned
+ * memory is needed for the copies to be asynchronous.
+ * d_src / d_dst: per phase, HOST arrays of DEVICE staging pointers with the
+ * same rank counts and sizes.  Destination staging arenas are fully
+ * overwritten only where the plan writes; bytes the plan does not write are
+ * copied back as the staging arena held them.
+ */
+emoe_status_t emoe_reshard_step_host(const emoe_plan_t *plan, const void *const *const h_src[3],
+                                     void *const *const h_dst[3],
+                                     void *const *const d_src[3], void *const *const d_dst[3],
+                                     void *cuda_stream);
+
+/* emoe_plan_destroy - frees host state and device descriptor buffers.
+ * NULL-safe.  No kernel using the plan may still be in flight. */
+void emoe_plan_destroy(emoe_plan_t *plan);
+
+/* ---- query helpers ------------------------------------------------------ */
+
+/* Number of ranks on one side of a phase (EP for experts, TP otherwise). */
+emoe_status_t emoe_plan_num_ranks(const emoe_plan_t *plan, int phase, int side, int32_t *n);
+
+/* Arena size in bytes of `rank` for (phase, side). */
+emoe_status_t emoe_plan_arena_bytes(const emoe_plan_t *plan, int phase, int side, int rank,
+                                    uint64_t *bytes);
+
+/* bytes_moved: bytes the phase writes to the new layout.  bytes_read: bytes
+ * it reads from the old layout (smaller when one source run feeds several
+ * destinations).  n_segments: descriptors after coalescing. */
+emoe_status_t emoe_plan_stats(const emoe_plan_t *plan, int phase, uint64_t *bytes_moved,
+                              uint64_t *bytes_read, uint64_t *n_segments);
+
+/* One coalesced copy descriptor, as exported for inspection and host-side
+ * replay: n_runs runs of run_bytes each; run i reads
+ * src[src_rank] + src_off + i*src_pitch and writes
+ * dst[dst_rank] + dst_off + i*dst_pitch.  A source run that feeds several
+ * destinations appears once per destination with the same `group` value. */
+typedef struct {
+  uint64_t src_off, dst_off, run_bytes, src_pitch, dst_pitch;
+  uint32_t n_runs, src_rank, dst_rank, group;
+} emoe_segment_t;
+
+/* Copies up to `cap` segments of the phase into `out` (host memory) and
+ * stores the total count in *n.  For the KV phase the block-pair list is
+ * expanded into per-(pair, old rank, new rank) segments. */
+emoe_status_t emoe_plan_segments(const emoe_plan_t *plan, int phase, emoe_segment_t *out,
+                                 uint64_t cap, uint64_t *n);
+
+/* Reads the plan's device status word (EMOE_OK or EMOE_ERR_DEVICE_TIMEOUT).
+ * Synchronises the device copy on the legacy default stream; call it after
+ * the caller has synchronised the stream(s) the plan ran on. */
+emoe_status_t emoe_plan_device_status(const emoe_plan_t *plan, int32_t *status);
+
+/* Launch tuning.  Fields set to 0 keep the library default. */
+typedef struct {
+  int32_t max_ctas;        /* upper bound on CTAs per launch (SM budget when the    */
+                           /* reshard shares the GPU with a live kernel)            */
+  int32_t bulk_tile_bytes; /* bytes per shared-memory stage of the bulk kernel      */
+  int32_t bulk_stages;     /* stages of the bulk kernel's ring                      */
+  int32_t path;            /* 0 default routing, 1 force the vector kernel for all  */
+                           /* segments, 2 force the bulk kernel where aligned       */
+  int32_t kv_mode;         /* 0 default, 1 direct, 2 staged through shared memory   */
+  int32_t reserved[3];
+} emoe_tuning_t;
+
+/* Replaces the plan's launch tuning.  Not thread-safe against reshard calls
+ * running concurrently on other host threads. */
+emoe_status_t emoe_plan_set_tuning(emoe_plan_t *plan, const emoe_tuning_t *tuning);
+
+/* Static string for a status code. */
+const char *emoe_strerror(emoe_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EMOE_H_ */

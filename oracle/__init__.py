@@ -1,0 +1,126 @@
+"""CPU oracle of the scale-step re-layout (ctypes front of emoe_oracle.cpp).
+
+TEST INFRASTRUCTURE: imported only by tests/, by the smoke check and by the
+benchmark's CPU-baseline leg.  It never imports the CUDA package, and the CUDA
+package never imports it.  Arenas are 1-D numpy uint8 arrays, one per rank.
+"""
+from __future__ import annotations
+
+import ctypes
+from typing import List, Sequence
+
+import numpy as np
+
+from .build import build as _build
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(_build())
+        i32, i64, p = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p
+        L.emoe_oracle_expert_arena_bytes.restype = i64
+        L.emoe_oracle_expert_arena_bytes.argtypes = [i32, i32, i64]
+        L.emoe_oracle_attn_arena_bytes.restype = i64
+        L.emoe_oracle_attn_arena_bytes.argtypes = [i32] * 7
+        L.emoe_oracle_kv_arena_bytes.restype = i64
+        L.emoe_oracle_kv_arena_bytes.argtypes = [i32] * 7
+        L.emoe_oracle_reshard_experts.restype = i32
+        L.emoe_oracle_reshard_experts.argtypes = [i32, i64, i32, p, p, i32, p, p, p, p]
+        L.emoe_oracle_reshard_attn.restype = i32
+        L.emoe_oracle_reshard_attn.argtypes = [i32] * 8 + [p, p]
+        L.emoe_oracle_reshard_kv.restype = i32
+        L.emoe_oracle_reshard_kv.argtypes = [i32] * 11 + [p, p, p, p, p]
+        _lib = L
+    return _lib
+
+
+def _csr(placement: Sequence[Sequence[int]]):
+    off = np.zeros(len(placement) + 1, dtype=np.int32)
+    off[1:] = np.cumsum([len(p) for p in placement])
+    ids = np.array([e for p in placement for e in p], dtype=np.int32)
+    return off, ids
+
+
+def _ptrs(arrs: Sequence[np.ndarray]):
+    for a in arrs:
+        if a.dtype != np.uint8 or a.ndim != 1 or not a.flags.c_contiguous:
+            raise TypeError("arenas must be contiguous 1-D uint8 arrays")
+    return (ctypes.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+
+
+def _vp(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+# ---- arena sizes (bytes) ---------------------------------------------------------------
+
+def expert_arena_bytes(shape, placement) -> List[int]:
+    m = shape.d_model * shape.d_ff * shape.elem_bytes
+    return [lib().emoe_oracle_expert_arena_bytes(shape.n_layers, len(p), m) for p in placement]
+
+
+def attn_arena_bytes(shape, tp: int) -> List[int]:
+    n = lib().emoe_oracle_attn_arena_bytes(shape.n_layers, shape.d_model, shape.n_q_heads,
+                                          shape.n_kv_heads, shape.head_dim, shape.elem_bytes, tp)
+    return [n] * tp
+
+
+def kv_arena_bytes(shape, tp: int, num_blocks: int) -> List[int]:
+    n = lib().emoe_oracle_kv_arena_bytes(shape.n_layers, num_blocks, shape.kv_block_tokens,
+                                        shape.n_kv_heads, shape.head_dim, shape.elem_bytes, tp)
+    return [n] * tp
+
+
+# ---- the three phases ------------------------------------------------------------------
+
+def reshard_experts(shape, old_placement, new_placement, src: Sequence[np.ndarray],
+                    dst: Sequence[np.ndarray]) -> None:
+    """Writes the new expert arenas `dst` from the old arenas `src` (in place on dst)."""
+    m = shape.d_model * shape.d_ff * shape.elem_bytes
+    oo, oi = _csr(old_placement)
+    no, ni = _csr(new_placement)
+    need_s = expert_arena_bytes(shape, old_placement)
+    need_d = expert_arena_bytes(shape, new_placement)
+    if [a.size for a in src] != need_s or [a.size for a in dst] != need_d:
+        raise ValueError("expert arena sizes do not match the placements")
+    rc = lib().emoe_oracle_reshard_experts(shape.n_layers, m, len(old_placement), _vp(oo), _vp(oi),
+                                          len(new_placement), _vp(no), _vp(ni), _ptrs(src),
+                                          _ptrs(dst))
+    if rc != 0:
+        raise ValueError("oracle: an expert of the new placement is absent from the old one")
+
+
+def reshard_attn(shape, tp_old: int, tp_new: int, src, dst) -> None:
+    if ([a.size for a in src] != attn_arena_bytes(shape, tp_old)
+            or [a.size for a in dst] != attn_arena_bytes(shape, tp_new)):
+        raise ValueError("attention arena sizes do not match")
+    rc = lib().emoe_oracle_reshard_attn(shape.n_layers, shape.d_model, shape.n_q_heads,
+                                       shape.n_kv_heads, shape.head_dim, shape.elem_bytes,
+                                       tp_old, tp_new, _ptrs(src), _ptrs(dst))
+    if rc != 0:
+        raise ValueError("oracle: TP degree does not divide the head counts")
+
+
+def reshard_kv(shape, old_cfg, new_cfg, src, dst) -> None:
+    """old_cfg / new_cfg carry tp, kv_num_blocks, seq_lens and block_table."""
+    if ([a.size for a in src] != kv_arena_bytes(shape, old_cfg.tp, old_cfg.kv_num_blocks)
+            or [a.size for a in dst] != kv_arena_bytes(shape, new_cfg.tp, new_cfg.kv_num_blocks)):
+        raise ValueError("KV arena sizes do not match")
+    sl = np.ascontiguousarray(old_cfg.seq_lens, dtype=np.int32)
+    if list(sl) != list(new_cfg.seq_lens):
+        raise ValueError("old and new configuration list different sequences")
+    bo = np.ascontiguousarray(old_cfg.block_table, dtype=np.int32)
+    bn = np.ascontiguousarray(new_cfg.block_table, dtype=np.int32)
+    if bo.shape != bn.shape:
+        w = max(bo.shape[1], bn.shape[1])
+        bo = np.pad(bo, ((0, 0), (0, w - bo.shape[1])), constant_values=-1)
+        bn = np.pad(bn, ((0, 0), (0, w - bn.shape[1])), constant_values=-1)
+    rc = lib().emoe_oracle_reshard_kv(shape.n_layers, shape.kv_block_tokens, shape.n_kv_heads,
+                                     shape.head_dim, shape.elem_bytes, old_cfg.tp, new_cfg.tp,
+                                     old_cfg.kv_num_blocks, new_cfg.kv_num_blocks, len(sl),
+                                     bo.shape[1], _vp(sl), _vp(bo), _vp(bn), _ptrs(src), _ptrs(dst))
+    if rc != 0:
+        raise ValueError("oracle: bad block table or TP degree")

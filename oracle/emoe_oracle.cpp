@@ -1,0 +1,174 @@
+// emoe_oracle.cpp - CPU reference of the scale-step re-layout.
+//
+// TEST INFRASTRUCTURE.  Only the tests, the smoke check and the benchmark's
+// CPU-baseline leg may call this file; the product never does.  It shares no
+// code, header, table or helper with the CUDA library.
+//
+// The re-layout reaches a result with a plain definition (a permutation /
+// replication of bytes), so this file IS that definition: nested loops over
+// logical coordinates in the order the definition states them, one memcpy of
+// the innermost contiguous unit, one thread, no segment lists, no coalescing.
+//
+// Where the definitions come from:
+//  * experts: after a scaling step every device holds its experts as one
+//    contiguous tensor in slot order (paper Sec. 4.1 "Virtual Expert
+//    Management", App. D.5); which experts a device holds is given by the old
+//    and new placement (Sec. 5.2 "Expert Weights", App. E for scale-down);
+//    uneven and replicated placements are allowed (Sec. 2.1).
+//  * attention: TP shards the attention operations (Sec. 2.1); with TP fixed
+//    the shards carry over unchanged (Sec. 5.2 "Attention Weights"); changing
+//    TP is the paper's future work (Sec. 9), read here in the usual way:
+//    q/k/v split by head along stored rows, o split by head along stored
+//    columns.
+//  * KV cache: follows TP (Sec. 4.1, Sec. 5.2 "KV Cache"); "reshaping KV
+//    caches" under a TP change (Sec. 9) is read as a contiguous split of the
+//    KV heads, block tables translating physical block ids.
+//
+// Pins: every function below is pinned by tests that do not use it to make
+// their expectation (numpy/torch indexing of logical tensors, hand-written
+// fixtures, identities and round trips); none is "parity unpinned".
+#include <cstdint>
+#include <cstring>
+
+namespace {
+
+struct Csr {
+  int n_ranks;
+  const int32_t *off;
+  const int32_t *ids;
+  int count(int r) const { return off[r + 1] - off[r]; }
+  int id(int r, int s) const { return ids[off[r] + s]; }
+};
+
+// Source replica of expert e for destination rank r_new: the copy held by the
+// old rank with the same index if there is one (that device keeps its copy,
+// Sec. 5.2 "maximize zero-copy reuse"), else the smallest (rank, slot).
+bool find_source(const Csr &old_p, int e, int r_new, int *r_out, int *s_out) {
+  if (r_new < old_p.n_ranks) {
+    for (int s = 0; s < old_p.count(r_new); ++s)
+      if (old_p.id(r_new, s) == e) { *r_out = r_new; *s_out = s; return true; }
+  }
+  for (int r = 0; r < old_p.n_ranks; ++r)
+    for (int s = 0; s < old_p.count(r); ++s)
+      if (old_p.id(r, s) == e) { *r_out = r; *s_out = s; return true; }
+  return false;
+}
+
+}  // namespace
+
+extern "C" {
+
+// Bytes of the expert arena of a rank holding n_slots experts: [L][3][n_slots][m].
+int64_t emoe_oracle_expert_arena_bytes(int n_layers, int n_slots, int64_t m) {
+  return (int64_t)n_layers * 3 * n_slots * m;
+}
+
+// Bytes of the attention arena of one TP rank: [L][q_t | k_t | v_t | o_t].
+int64_t emoe_oracle_attn_arena_bytes(int n_layers, int d_model, int hq, int hkv, int hd, int b,
+                                     int tp) {
+  int64_t q = (int64_t)(hq / tp) * hd * d_model * b;
+  int64_t kv = (int64_t)(hkv / tp) * hd * d_model * b;
+  return (int64_t)n_layers * (q + 2 * kv + q);
+}
+
+// Bytes of the KV arena of one TP rank: [L][2][NB][B][Hkv/T][hd].
+int64_t emoe_oracle_kv_arena_bytes(int n_layers, int nb, int block_tokens, int hkv, int hd, int b,
+                                   int tp) {
+  return (int64_t)n_layers * 2 * nb * block_tokens * (hkv / tp) * hd * b;
+}
+
+// Expert re-pack.  m = bytes of one expert matrix.  Returns 0, or -1 if an
+// expert of the new placement has no copy in the old one.
+int emoe_oracle_reshard_experts(int n_layers, int64_t m, int ep_old, const int32_t *old_off,
+                                const int32_t *old_ids, int ep_new, const int32_t *new_off,
+                                const int32_t *new_ids, const uint8_t *const *src,
+                                uint8_t *const *dst) {
+  Csr po{ep_old, old_off, old_ids}, pn{ep_new, new_off, new_ids};
+  for (int rn = 0; rn < ep_new; ++rn) {
+    const int64_t n_new = pn.count(rn);
+    for (int l = 0; l < n_layers; ++l)
+      for (int p = 0; p < 3; ++p)
+        for (int sn = 0; sn < n_new; ++sn) {
+          int ro, so;
+          if (!find_source(po, pn.id(rn, sn), rn, &ro, &so)) return -1;
+          const int64_t n_old = po.count(ro);
+          const int64_t off_new = (((int64_t)l * 3 + p) * n_new + sn) * m;
+          const int64_t off_old = (((int64_t)l * 3 + p) * n_old + so) * m;
+          std::memcpy(dst[rn] + off_new, src[ro] + off_old, (size_t)m);
+        }
+  }
+  return 0;
+}
+
+// Attention re-slice TP=c -> TP=d.  b = bytes per element.
+int emoe_oracle_reshard_attn(int n_layers, int d_model, int hq, int hkv, int hd, int b, int c,
+                             int d, const uint8_t *const *src, uint8_t *const *dst) {
+  if (hq % c || hq % d || hkv % c || hkv % d) return -1;
+  const int64_t D = d_model;
+  const int64_t row = D * b;  // one stored row of Wq / Wk / Wv
+  // sizes of the four pieces of one layer on a rank of a TP=T group
+  auto q_bytes = [&](int T) { return (int64_t)(hq / T) * hd * row; };
+  auto kv_bytes = [&](int T) { return (int64_t)(hkv / T) * hd * row; };
+  auto layer_bytes = [&](int T) { return 2 * q_bytes(T) + 2 * kv_bytes(T); };
+
+  for (int l = 0; l < n_layers; ++l) {
+    // q, k, v: global stored row g of the logical matrix
+    for (int t = 0; t < 3; ++t) {
+      const int heads = (t == 0) ? hq : hkv;
+      const int64_t rows = (int64_t)heads * hd;
+      const int64_t rows_c = rows / c, rows_d = rows / d;
+      auto piece_off = [&](int T) {
+        return (t == 0) ? 0 : (t == 1) ? q_bytes(T) : q_bytes(T) + kv_bytes(T);
+      };
+      for (int64_t g = 0; g < rows; ++g) {
+        const int64_t ro = g / rows_c, lo = g % rows_c;
+        const int64_t rn = g / rows_d, ln = g % rows_d;
+        std::memcpy(dst[rn] + l * layer_bytes(d) + piece_off(d) + ln * row,
+                    src[ro] + l * layer_bytes(c) + piece_off(c) + lo * row, (size_t)row);
+      }
+    }
+    // o: stored row i, head h owns columns [h*hd, (h+1)*hd) of the logical Wo
+    const int64_t o_off_c = q_bytes(c) + 2 * kv_bytes(c), o_off_d = q_bytes(d) + 2 * kv_bytes(d);
+    const int64_t cols_c = (int64_t)(hq / c) * hd, cols_d = (int64_t)(hq / d) * hd;
+    for (int64_t i = 0; i < D; ++i)
+      for (int h = 0; h < hq; ++h) {
+        const int64_t col = (int64_t)h * hd;
+        const int64_t ro = col / cols_c, lo = col % cols_c;
+        const int64_t rn = col / cols_d, ln = col % cols_d;
+        std::memcpy(dst[rn] + l * layer_bytes(d) + o_off_d + (i * cols_d + ln) * b,
+                    src[ro] + l * layer_bytes(c) + o_off_c + (i * cols_c + lo) * b,
+                    (size_t)hd * b);
+      }
+  }
+  return 0;
+}
+
+// KV head re-split + re-paging.  bt_old / bt_new: [n_seqs][max_blocks].
+// Returns 0, or -1 on an unmapped (negative) entry inside a sequence.
+int emoe_oracle_reshard_kv(int n_layers, int block_tokens, int hkv, int hd, int b, int c, int d,
+                           int nb_old, int nb_new, int n_seqs, int max_blocks,
+                           const int32_t *seq_lens, const int32_t *bt_old, const int32_t *bt_new,
+                           const uint8_t *const *src, uint8_t *const *dst) {
+  if (hkv % c || hkv % d) return -1;
+  const int64_t B = block_tokens, hc = hkv / c, hdn = hkv / d, vec = (int64_t)hd * b;
+  for (int s = 0; s < n_seqs; ++s) {
+    const int n_blk = (int)((seq_lens[s] + B - 1) / B);
+    for (int j = 0; j < n_blk; ++j) {
+      const int64_t po = bt_old[(int64_t)s * max_blocks + j];
+      const int64_t pn = bt_new[(int64_t)s * max_blocks + j];
+      if (po < 0 || pn < 0 || po >= nb_old || pn >= nb_new) return -1;
+      for (int l = 0; l < n_layers; ++l)
+        for (int kv = 0; kv < 2; ++kv)
+          for (int64_t tok = 0; tok < B; ++tok)
+            for (int64_t g = 0; g < hkv; ++g) {
+              const int64_t ro = g / hc, ho = g % hc, rn = g / hdn, hn = g % hdn;
+              const int64_t off_o = (((((int64_t)l * 2 + kv) * nb_old + po) * B + tok) * hc + ho) * vec;
+              const int64_t off_n = (((((int64_t)l * 2 + kv) * nb_new + pn) * B + tok) * hdn + hn) * vec;
+              std::memcpy(dst[rn] + off_n, src[ro] + off_o, (size_t)vec);
+            }
+    }
+  }
+  return 0;
+}
+
+}  // extern "C"

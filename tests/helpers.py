@@ -1,0 +1,88 @@
+"""Test-side helpers: logical tensors and their sharded arenas written with numpy
+indexing (never with byte-offset formulas), used to pin the oracle."""
+from __future__ import annotations
+
+import numpy as np
+
+import workloads as W
+
+FILL = 0xCD
+
+
+def rand_bytes(key, n):
+    tags = key if isinstance(key, tuple) else (key,)
+    return W.rng.fill_bytes(W.rng.stream_key(0xABCD, *tags), n)
+
+
+# ---- experts ---------------------------------------------------------------------------
+
+def logical_experts(shape, key=1):
+    """uint8 [L, 3, E, m] with independent contents per (l, p, e)."""
+    m = shape.d_model * shape.d_ff * shape.elem_bytes
+    n = shape.n_layers * 3 * shape.n_experts * m
+    return rand_bytes(key, n).reshape(shape.n_layers, 3, shape.n_experts, m)
+
+
+def expert_arenas(logical, placement):
+    """Per-rank arena = the rank's experts gathered along the expert axis."""
+    return [np.ascontiguousarray(logical[:, :, list(p), :]).reshape(-1) for p in placement]
+
+
+# ---- attention -------------------------------------------------------------------------
+
+def logical_attn(shape, key=2):
+    L, D, b = shape.n_layers, shape.d_model, shape.elem_bytes
+    q = shape.n_q_heads * shape.head_dim
+    kv = shape.n_kv_heads * shape.head_dim
+    return dict(
+        q=rand_bytes((key, 0), L * q * D * b).reshape(L, q, D * b),
+        k=rand_bytes((key, 1), L * kv * D * b).reshape(L, kv, D * b),
+        v=rand_bytes((key, 2), L * kv * D * b).reshape(L, kv, D * b),
+        o=rand_bytes((key, 3), L * D * q * b).reshape(L, D, q, b),   # [row, column, byte]
+    )
+
+
+def attn_arenas(logical, tp):
+    """Rank t: per layer q_t | k_t | v_t | o_t, pieces cut with numpy.split."""
+    L = logical["q"].shape[0]
+    qs = np.split(logical["q"], tp, axis=1)
+    ks = np.split(logical["k"], tp, axis=1)
+    vs = np.split(logical["v"], tp, axis=1)
+    os_ = np.split(logical["o"], tp, axis=2)
+    out = []
+    for t in range(tp):
+        per_layer = [np.concatenate([np.ascontiguousarray(x[l]).reshape(-1)
+                                     for x in (qs[t], ks[t], vs[t], os_[t])]) for l in range(L)]
+        out.append(np.concatenate(per_layer))
+    return out
+
+
+# ---- KV --------------------------------------------------------------------------------
+
+def logical_kv(shape, cfg, key=3):
+    """uint8 [L, 2, n_logical_blocks, B, Hkv, hd*b]; logical block index runs over
+    (sequence, block-in-sequence) in order."""
+    B = shape.kv_block_tokens
+    nblk = sum(-(-n // B) for n in cfg.seq_lens)
+    vec = shape.head_dim * shape.elem_bytes
+    n = shape.n_layers * 2 * nblk * B * shape.n_kv_heads * vec
+    return rand_bytes(key, n).reshape(shape.n_layers, 2, nblk, B, shape.n_kv_heads, vec)
+
+
+def kv_arenas(logical, shape, cfg, background=None):
+    """Scatters logical blocks into each rank's pool through the block table."""
+    B = shape.kv_block_tokens
+    L, vec = shape.n_layers, shape.head_dim * shape.elem_bytes
+    hl = shape.n_kv_heads // cfg.tp
+    phys = []
+    for s, n in enumerate(cfg.seq_lens):
+        phys += [int(x) for x in cfg.block_table[s, :-(-n // B)]]
+    out = []
+    for t in range(cfg.tp):
+        if background is None:
+            pool = np.full((L, 2, cfg.kv_num_blocks, B, hl, vec), FILL, dtype=np.uint8)
+        else:
+            pool = background[t].reshape(L, 2, cfg.kv_num_blocks, B, hl, vec).copy()
+        pool[:, :, phys] = logical[:, :, :, :, t * hl:(t + 1) * hl]
+        out.append(pool.reshape(-1))
+    return out

@@ -1,0 +1,338 @@
+"""Pins of the CPU oracle against things that are not the oracle: numpy / torch
+indexing of logical tensors, hand-written fixtures, identities and round trips.
+A wrong offset formula, a swapped operand, a dropped loop or a wrong tie-break in
+oracle/emoe_oracle.cpp fails at least one test here.  No GPU needed."""
+from __future__ import annotations
+
+import dataclasses
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as W
+from helpers import (FILL, attn_arenas, expert_arenas, kv_arenas, logical_attn, logical_experts,
+                     logical_kv, rand_bytes)
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def filled(sizes):
+    return [np.full(n, FILL, dtype=np.uint8) for n in sizes]
+
+
+def tiny_shape(**kw):
+    base = dict(n_layers=3, n_routed=12, n_shared=0, d_model=8, d_ff=6, n_q_heads=8,
+                n_kv_heads=4, head_dim=4, kv_block_tokens=4, elem_bytes=2)
+    base.update(kw)
+    return W.Shape(**base)
+
+
+# ======================================================================== experts ======
+
+PLACEMENTS = {
+    "round_robin_2_4": (lambda: W.place_round_robin(12, 2), lambda: W.place_round_robin(12, 4)),
+    "contig_4_6": (lambda: W.place_contiguous(12, 4), lambda: W.place_contiguous(12, 6)),
+    "contig_4_2": (lambda: W.place_contiguous(12, 4), lambda: W.place_contiguous(12, 2)),
+    "uneven_5_7": (lambda: W.place_contiguous(12, 5), lambda: W.place_contiguous(12, 7)),
+    "scrambled": (lambda: [[5, 0, 11], [3, 9, 1, 7], [2, 10, 4, 8, 6]],
+                  lambda: [[6, 5], [0, 1, 2, 3, 4], [11], [10, 9, 8, 7]]),
+    "replicated_new": (lambda: W.place_contiguous(12, 3),
+                       lambda: [[0, 1, 2, 11], [3, 4, 0, 5], [6, 7, 8], [9, 10, 11, 4]]),
+}
+
+
+@pytest.mark.parametrize("name", sorted(PLACEMENTS))
+@pytest.mark.parametrize("elem_bytes", [1, 2, 4])
+def test_experts_equal_numpy_gather_of_logical_tensor(name, elem_bytes):
+    """Brute force: the new arena of rank r' is logical[:, :, P_new[r'], :]."""
+    sh = tiny_shape(elem_bytes=elem_bytes)
+    po, pn = (f() for f in PLACEMENTS[name])
+    logical = logical_experts(sh)
+    src = expert_arenas(logical, po)
+    want = expert_arenas(logical, pn)
+    dst = filled([a.size for a in want])
+    oracle.reshard_experts(sh, po, pn, src, dst)
+    for r, (g, w) in enumerate(zip(dst, want)):
+        assert np.array_equal(g, w), "rank %d" % r
+
+
+def test_experts_shared_experts_on_every_rank():
+    sh = tiny_shape(n_routed=10, n_shared=2)
+    po = W.with_shared(W.place_contiguous(10, 2), [10, 11])
+    pn = W.with_shared(W.place_contiguous(10, 3), [10, 11])
+    logical = logical_experts(sh)
+    dst = filled([a.size for a in expert_arenas(logical, pn)])
+    oracle.reshard_experts(sh, po, pn, expert_arenas(logical, po), dst)
+    for g, w in zip(dst, expert_arenas(logical, pn)):
+        assert np.array_equal(g, w)
+
+
+def test_experts_contiguous_equals_torch_cat_tensor_split():
+    """Library special case: contiguous ranges -> cat along the slot axis, re-split."""
+    sh = tiny_shape()
+    po, pn = W.place_contiguous(12, 4), W.place_contiguous(12, 6)
+    m = sh.d_model * sh.d_ff * sh.elem_bytes
+    src = [rand_bytes((7, r), sh.n_layers * 3 * len(p) * m) for r, p in enumerate(po)]
+    dst = filled([sh.n_layers * 3 * len(p) * m for p in pn])
+    oracle.reshard_experts(sh, po, pn, src, dst)
+    cat = torch.cat([torch.from_numpy(a).view(sh.n_layers, 3, len(p), m)
+                     for a, p in zip(src, po)], dim=2)
+    parts = cat.tensor_split(list(np.cumsum([len(p) for p in pn])[:-1]), dim=2)
+    for g, w in zip(dst, parts):
+        assert np.array_equal(g, w.contiguous().view(-1).numpy())
+
+
+def test_experts_round_robin_equals_strided_slice():
+    sh = tiny_shape()
+    logical = logical_experts(sh)
+    po, pn = W.place_round_robin(12, 2), W.place_round_robin(12, 4)
+    dst = filled([sh.n_layers * 3 * len(p) * logical.shape[3] for p in pn])
+    oracle.reshard_experts(sh, po, pn, expert_arenas(logical, po), dst)
+    for r in range(4):
+        assert np.array_equal(dst[r], np.ascontiguousarray(logical[:, :, r::4, :]).reshape(-1))
+
+
+def test_experts_identity_is_memcpy_and_round_trip_is_identity():
+    sh = tiny_shape()
+    pa, pb = W.place_contiguous(12, 5), W.place_round_robin(12, 3)
+    m = sh.d_model * sh.d_ff * sh.elem_bytes
+    a0 = [rand_bytes((8, r), sh.n_layers * 3 * len(p) * m) for r, p in enumerate(pa)]
+    same = filled([x.size for x in a0])
+    oracle.reshard_experts(sh, pa, pa, a0, same)
+    assert all(np.array_equal(x, y) for x, y in zip(a0, same))
+    mid = filled([sh.n_layers * 3 * len(p) * m for p in pb])
+    oracle.reshard_experts(sh, pa, pb, a0, mid)
+    back = filled([x.size for x in a0])
+    oracle.reshard_experts(sh, pb, pa, mid, back)
+    assert all(np.array_equal(x, y) for x, y in zip(a0, back))
+
+
+def test_experts_multiplicity_and_conservation():
+    """Every expert lands exactly as often as the new placement lists it."""
+    sh = tiny_shape(n_layers=1, d_model=4, d_ff=4, elem_bytes=1)
+    m = 16
+    po = W.place_contiguous(12, 3)
+    pn = [[0, 1, 2, 11], [3, 4, 0, 5], [6, 7, 8], [9, 10, 11, 4]]
+    logical = np.zeros((1, 3, 12, m), dtype=np.uint8)
+    logical[:] = np.arange(12, dtype=np.uint8)[None, None, :, None]
+    dst = filled([3 * len(p) * m for p in pn])
+    oracle.reshard_experts(sh, po, pn, expert_arenas(logical, po), dst)
+    hist = np.bincount(np.concatenate(dst), minlength=256)
+    want = np.bincount([e for p in pn for e in p], minlength=12) * 3 * m
+    assert np.array_equal(hist[:12], want) and hist[12:].sum() == 0
+    assert sum(a.size for a in dst) == sum(len(p) for p in pn) * 3 * m
+
+
+def test_experts_replica_choice_own_rank_first_then_smallest():
+    """Hand-written: replicas with DIFFERENT contents pin which copy is read.
+    old rank0 = [0, 1], old rank1 = [1, 2]; slabs are tagged 10*rank + slot + 1."""
+    sh = tiny_shape(n_layers=1, n_routed=3, d_model=2, d_ff=2, elem_bytes=1)
+    m = 4
+    po = [[0, 1], [1, 2]]
+    pn = [[1], [1], [1, 0, 2]]
+    src = [np.repeat(np.array([[1, 2]] * 3, dtype=np.uint8).reshape(-1), m),
+           np.repeat(np.array([[11, 12]] * 3, dtype=np.uint8).reshape(-1), m)]
+    dst = filled([3 * len(p) * m for p in pn])
+    oracle.reshard_experts(sh, po, pn, src, dst)
+    assert set(dst[0]) == {2}          # new rank 0 keeps old rank 0's copy (slot 1)
+    assert set(dst[1]) == {11}         # new rank 1 keeps old rank 1's copy (slot 0)
+    assert list(dst[2][:3 * m:m]) == [2, 1, 12]   # no old rank 2: smallest (rank, slot)
+
+
+@pytest.mark.parametrize("case,ep_new", [("up", 6), ("down", 2)])
+def test_experts_paper_scenario_fixture(case, ep_new):
+    """The paper's EP4 -> EP6 scale-up and EP4 -> EP2 scale-down, against a
+    hand-written table of (new rank, new slot) <- (old rank, old slot)."""
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "paper_scale_ep4_ep6.txt"))
+            if l.strip() and not l.startswith("#")]
+    rows = [tuple(int(x) for x in r[1:]) for r in rows if r[0] == case]
+    sh = tiny_shape(n_layers=2, d_model=2, d_ff=2, elem_bytes=2)
+    m = 8
+    po, pn = W.place_contiguous(12, 4), W.place_contiguous(12, ep_new)
+    # every old slab (l, p, slot) of every rank carries its own tag
+    src = []
+    for r in range(4):
+        a = np.zeros((2, 3, 3, m), dtype=np.uint8)
+        for l in range(2):
+            for p in range(3):
+                for s in range(3):
+                    a[l, p, s] = 1 + ((r * 3 + s) * 3 + p) * 2 + l
+        src.append(a.reshape(-1))
+    dst = filled([2 * 3 * len(p) * m for p in pn])
+    oracle.reshard_experts(sh, po, pn, src, dst)
+    assert len(rows) == 12
+    for rn, sn, e, ro, so in rows:
+        assert pn[rn][sn] == e and po[ro][so] == e
+        got = dst[rn].reshape(2, 3, len(pn[rn]), m)
+        for l in range(2):
+            for p in range(3):
+                assert set(got[l, p, sn]) == {1 + ((ro * 3 + so) * 3 + p) * 2 + l}
+
+
+def test_experts_missing_source_is_an_error():
+    sh = tiny_shape(n_layers=1, n_routed=3, d_model=2, d_ff=2)
+    with pytest.raises(ValueError):
+        oracle.reshard_experts(sh, [[0, 1]], [[0, 2]], [np.zeros(48, np.uint8)],
+                               [np.zeros(48, np.uint8)])
+
+
+# ====================================================================== attention ======
+
+@pytest.mark.parametrize("c,d", [(1, 2), (2, 4), (4, 1), (2, 2), (4, 2), (1, 4)])
+@pytest.mark.parametrize("elem_bytes", [2, 4])
+def test_attn_equals_numpy_split_of_logical_matrices(c, d, elem_bytes):
+    sh = tiny_shape(elem_bytes=elem_bytes)
+    logical = logical_attn(sh)
+    src, want = attn_arenas(logical, c), attn_arenas(logical, d)
+    dst = filled([a.size for a in want])
+    oracle.reshard_attn(sh, c, d, src, dst)
+    for t, (g, w) in enumerate(zip(dst, want)):
+        assert np.array_equal(g, w), "rank %d" % t
+
+
+def test_attn_gqa_shapes_and_torch_cat_chunk():
+    """Library special case on one layer: cat(shards, dim).chunk(d, dim) with dim 0
+    for q/k/v and dim 1 for o, for a GQA shape (Hq != Hkv)."""
+    sh = tiny_shape(n_layers=1, n_q_heads=8, n_kv_heads=2, head_dim=4, d_model=6)
+    c, d = 1, 2
+    D, b = sh.d_model, sh.elem_bytes
+    q, kv = sh.n_q_heads * sh.head_dim, sh.n_kv_heads * sh.head_dim
+    src = [rand_bytes(11, (2 * q * D + 2 * kv * D) * b)]
+    t = torch.from_numpy(src[0])
+    sizes = [q * D * b, kv * D * b, kv * D * b, D * q * b]
+    Q, K, V, O = t.split(sizes)
+    Q, K, V = Q.view(q, D * b), K.view(kv, D * b), V.view(kv, D * b)
+    O = O.view(D, q, b)
+    dst = filled(oracle.attn_arena_bytes(sh, d))
+    oracle.reshard_attn(sh, c, d, src, dst)
+    for r in range(d):
+        want = torch.cat([Q.chunk(d, 0)[r].reshape(-1), K.chunk(d, 0)[r].reshape(-1),
+                          V.chunk(d, 0)[r].reshape(-1), O.chunk(d, 1)[r].reshape(-1)])
+        assert np.array_equal(dst[r], want.numpy())
+
+
+def test_attn_fixed_tp_is_memcpy_and_round_trip():
+    sh = tiny_shape()
+    a0 = [rand_bytes((12, t), n) for t, n in enumerate(oracle.attn_arena_bytes(sh, 2))]
+    same = filled([a.size for a in a0])
+    oracle.reshard_attn(sh, 2, 2, a0, same)      # the paper's fixed-TP case (Sec. 5.2)
+    assert all(np.array_equal(x, y) for x, y in zip(a0, same))
+    mid = filled(oracle.attn_arena_bytes(sh, 4))
+    oracle.reshard_attn(sh, 2, 4, a0, mid)
+    back = filled([a.size for a in a0])
+    oracle.reshard_attn(sh, 4, 2, mid, back)
+    assert all(np.array_equal(x, y) for x, y in zip(a0, back))
+
+
+def test_attn_rejects_tp_not_dividing_heads():
+    sh = tiny_shape(n_kv_heads=2)
+    with pytest.raises(ValueError):
+        oracle.reshard_attn(sh, 1, 4, [np.zeros(oracle.attn_arena_bytes(sh, 1)[0], np.uint8)],
+                            [np.zeros(1, np.uint8)] * 4)
+
+
+# ============================================================================= KV ======
+
+def kv_cfgs(sh, c, d, seq_lens, nb_old, nb_new, seed=5, new_order="random"):
+    B = sh.kv_block_tokens
+    bo = W.make_block_table(W.rng.stream_key(seed, 1), seq_lens, B, nb_old)
+    bn = W.make_block_table(W.rng.stream_key(seed, 2), seq_lens, B, nb_new, order=new_order)
+    return (W.ParallelConfig(1, c, [[]], nb_old, seq_lens, bo),
+            W.ParallelConfig(1, d, [[]], nb_new, seq_lens, bn))
+
+
+@pytest.mark.parametrize("c,d", [(1, 2), (2, 4), (4, 2), (1, 1), (2, 2), (4, 1)])
+def test_kv_equals_numpy_scatter_of_logical_cache(c, d):
+    """Tokens keep sequence, position and head identity: both layouts are
+    scatters of the same logical [L,2,block,B,Hkv,hd] cache through the tables."""
+    sh = tiny_shape()
+    old, new = kv_cfgs(sh, c, d, [9, 4, 13, 1], 11, 14)
+    logical = logical_kv(sh, old)
+    src = kv_arenas(logical, sh, old)
+    want = kv_arenas(logical, sh, new)          # unmapped blocks keep the 0xCD fill
+    dst = filled([a.size for a in want])
+    oracle.reshard_kv(sh, old, new, src, dst)
+    for t, (g, w) in enumerate(zip(dst, want)):
+        assert np.array_equal(g, w), "rank %d" % t
+
+
+def test_kv_same_table_same_tp_leaves_mapped_blocks_unchanged():
+    """The paper's case (fixed TP, cache reused as is): output == input on every
+    mapped block, and nothing else is written."""
+    sh = tiny_shape()
+    old, _ = kv_cfgs(sh, 2, 2, [9, 4, 13], 9, 9)
+    src = [rand_bytes((13, t), n) for t, n in enumerate(oracle.kv_arena_bytes(sh, 2, 9))]
+    dst = filled([a.size for a in src])
+    oracle.reshard_kv(sh, old, old, src, dst)
+    used = sorted(int(x) for x in old.block_table.reshape(-1) if x >= 0)
+    free = [p for p in range(9) if p not in used]
+    for s, g in zip(src, dst):
+        s6 = s.reshape(sh.n_layers, 2, 9, -1)
+        g6 = g.reshape(sh.n_layers, 2, 9, -1)
+        assert np.array_equal(g6[:, :, used], s6[:, :, used])
+        assert (g6[:, :, free] == FILL).all()
+
+
+def test_kv_round_trip_and_byte_conservation():
+    sh = tiny_shape()
+    old, new = kv_cfgs(sh, 2, 4, [16, 7, 5], 8, 10)
+    logical = logical_kv(sh, old)
+    src = kv_arenas(logical, sh, old)
+    mid = filled(oracle.kv_arena_bytes(sh, 4, 10))
+    oracle.reshard_kv(sh, old, new, src, mid)
+    back = filled([a.size for a in src])
+    oracle.reshard_kv(sh, new, old, mid, back)
+    assert all(np.array_equal(x, y) for x, y in zip(src, back))
+    n_blocks = sum(-(-n // sh.kv_block_tokens) for n in old.seq_lens)
+    moved = sum(int((a != FILL).sum()) for a in mid)
+    total = (sh.n_layers * 2 * n_blocks * sh.kv_block_tokens * sh.n_kv_heads * sh.head_dim
+             * sh.elem_bytes)
+    # random payload bytes equal the fill value now and then: bound, not equality
+    assert total * 0.98 <= moved <= total
+
+
+def test_kv_hand_written_two_heads_split():
+    """One layer, one block of 2 tokens, 2 heads of 1 two-byte element, TP1 -> TP2,
+    old physical block 1 of 2, new physical block 0 of 1: written out by hand."""
+    sh = tiny_shape(n_layers=1, n_kv_heads=2, head_dim=1, kv_block_tokens=2, elem_bytes=2)
+    old = W.ParallelConfig(1, 1, [[]], 2, [2], np.array([[1]], np.int32))
+    new = W.ParallelConfig(1, 2, [[]], 1, [2], np.array([[0]], np.int32))
+    # old arena: [K|V][block 0, block 1][tok][head][2 bytes]
+    K = [0, 0, 0, 0, 0, 0, 0, 0, 1, 2, 3, 4, 5, 6, 7, 8]        # block 1: t0h0 t0h1 t1h0 t1h1
+    V = [0, 0, 0, 0, 0, 0, 0, 0, 21, 22, 23, 24, 25, 26, 27, 28]
+    src = [np.array(K + V, dtype=np.uint8)]
+    dst = filled([8, 8])
+    oracle.reshard_kv(sh, old, new, src, dst)
+    assert list(dst[0]) == [1, 2, 5, 6, 21, 22, 25, 26]      # head 0: K t0,t1 then V t0,t1
+    assert list(dst[1]) == [3, 4, 7, 8, 23, 24, 27, 28]      # head 1
+
+
+# ===================================================================== arena sizes =====
+
+def test_arena_sizes_match_numpy_shapes():
+    sh = tiny_shape()
+    logical = logical_experts(sh)
+    pl = W.place_contiguous(12, 5)
+    assert oracle.expert_arena_bytes(sh, pl) == [a.size for a in expert_arenas(logical, pl)]
+    assert oracle.attn_arena_bytes(sh, 2) == [a.size for a in attn_arenas(logical_attn(sh), 2)]
+    old, _ = kv_cfgs(sh, 2, 2, [9, 4], 6, 6)
+    assert oracle.kv_arena_bytes(sh, 2, 6) == [a.size for a in
+                                               kv_arenas(logical_kv(sh, old), sh, old)]
+
+
+def test_published_step_bytes_of_the_five_configs():
+    """Whole-step byte counts of C1..C4, computed independently from the shapes."""
+    want = {"c1_tiny": 31457280, "c2_mid": 32161923072, "c3_fine": 56509857792,
+            "c4_large": 25434259456}
+    for name, total in want.items():
+        wl = W.make_workload(name)
+        sh = wl.shape
+        used = sum(-(-n // sh.kv_block_tokens) for n in wl.old.seq_lens)
+        kv_moved = (sh.n_layers * 2 * used * sh.kv_block_tokens * sh.n_kv_heads * sh.head_dim
+                    * sh.elem_bytes)
+        got = (sum(oracle.expert_arena_bytes(sh, wl.new.placement))
+               + sum(oracle.attn_arena_bytes(sh, wl.new.tp)) + kv_moved)
+        assert got == total, name
