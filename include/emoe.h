@@ -211,6 +211,9 @@ emoe_status_t emoe_plan_arena_bytes(const emoe_plan_t *plan, int phase, int side
 emoe_status_t emoe_plan_stats(const emoe_plan_t *plan, int phase, uint64_t *bytes_moved,
                               uint64_t *bytes_read, uint64_t *n_segments);
 
+/* Kernel launches one reshard call of this phase enqueues with the current tuning. */
+emoe_status_t emoe_plan_num_launches(const emoe_plan_t *plan, int phase, int32_t *n);
+
 /* One coalesced copy descriptor, as exported for inspection and host-side
  * replay: n_runs runs of run_bytes each; run i reads
  * src[src_rank] + src_off + i*src_pitch and writes
@@ -222,8 +225,9 @@ typedef struct {
 } emoe_segment_t;
 
 /* Copies up to `cap` segments of the phase into `out` (host memory) and
- * stores the total count in *n.  For the KV phase the block-pair list is
- * expanded into per-(pair, old rank, new rank) segments. */
+ * stores the total count in *n.  For a KV phase that changes the head split
+ * the block-pair list is expanded into one segment per (pair, layer, K|V,
+ * old rank, new rank) overlap, its runs being the block's token rows. */
 emoe_status_t emoe_plan_segments(const emoe_plan_t *plan, int phase, emoe_segment_t *out,
                                  uint64_t cap, uint64_t *n);
 

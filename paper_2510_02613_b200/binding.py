@@ -1,0 +1,274 @@
+"""ctypes binding of libemoe.so: argument marshalling only.
+
+Every step of the re-layout runs inside the library's CUDA kernels; this module
+converts Python objects to the C structs of include/emoe.h and back.  It fails
+loudly if the library cannot be loaded: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+from . import build as _build
+
+PHASE_EXPERTS, PHASE_ATTN, PHASE_KV = 0, 1, 2
+SIDE_OLD, SIDE_NEW = 0, 1
+PLAN_HOST_ONLY = 1
+MAX_RANKS = 64
+
+_i32, _u32, _u64, _vp = ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_void_p
+_i32p = ctypes.POINTER(ctypes.c_int32)
+
+
+class EmoeError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__("libemoe: %s (status %d)" % (what, code))
+        self.code = code
+
+
+class _Shape(ctypes.Structure):
+    _fields_ = [(n, _i32) for n in ("n_layers", "n_routed", "n_shared", "d_model", "d_ff",
+                                    "n_q_heads", "n_kv_heads", "head_dim", "kv_block_tokens",
+                                    "elem_bytes")]
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [("ep", _i32), ("tp", _i32), ("place_off", _i32p), ("place_ids", _i32p),
+                ("kv_num_blocks", _i32), ("n_seqs", _i32), ("max_blocks", _i32),
+                ("seq_lens", _i32p), ("block_table", _i32p)]
+
+
+class _Segment(ctypes.Structure):
+    _fields_ = [("src_off", _u64), ("dst_off", _u64), ("run_bytes", _u64), ("src_pitch", _u64),
+                ("dst_pitch", _u64), ("n_runs", _u32), ("src_rank", _u32), ("dst_rank", _u32),
+                ("group", _u32)]
+
+
+class _Tuning(ctypes.Structure):
+    _fields_ = [("max_ctas", _i32), ("bulk_tile_bytes", _i32), ("bulk_stages", _i32),
+                ("path", _i32), ("kv_mode", _i32), ("reserved", _i32 * 3)]
+
+
+SEGMENT_DTYPE = np.dtype([("src_off", "<u8"), ("dst_off", "<u8"), ("run_bytes", "<u8"),
+                          ("src_pitch", "<u8"), ("dst_pitch", "<u8"), ("n_runs", "<u4"),
+                          ("src_rank", "<u4"), ("dst_rank", "<u4"), ("group", "<u4")])
+
+EXPORTS = ("emoe_plan_create", "emoe_reshard_experts", "emoe_reshard_attn", "emoe_reshard_kv",
+           "emoe_reshard_step_host", "emoe_plan_destroy", "emoe_plan_num_ranks",
+           "emoe_plan_arena_bytes", "emoe_plan_stats", "emoe_plan_num_launches", "emoe_plan_segments",
+           "emoe_plan_device_status", "emoe_plan_set_tuning", "emoe_strerror")
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def library_path() -> str:
+    return _build.OUT
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libemoe.so, building it first if the sources are newer.  Raises if that fails."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.OUT
+    if _build.is_stale():
+        try:
+            _build.build()
+        except Exception as e:  # no nvcc on this machine: use the shipped binary if there is one
+            if not os.path.exists(path):
+                raise RuntimeError("libemoe.so is missing and could not be built: %s" % e) from e
+    L = ctypes.CDLL(path)
+    PP = ctypes.POINTER(_vp)
+    L.emoe_plan_create.restype = _i32
+    L.emoe_plan_create.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Config),
+                                   ctypes.POINTER(_Config), _u32, ctypes.POINTER(_vp)]
+    for name in ("emoe_reshard_experts", "emoe_reshard_attn", "emoe_reshard_kv"):
+        f = getattr(L, name)
+        f.restype = _i32
+        f.argtypes = [_vp, PP, PP, _vp]
+    L.emoe_reshard_step_host.restype = _i32
+    L.emoe_reshard_step_host.argtypes = [_vp, ctypes.POINTER(PP), ctypes.POINTER(PP),
+                                         ctypes.POINTER(PP), ctypes.POINTER(PP), _vp]
+    L.emoe_plan_destroy.restype = None
+    L.emoe_plan_destroy.argtypes = [_vp]
+    L.emoe_plan_num_ranks.restype = _i32
+    L.emoe_plan_num_ranks.argtypes = [_vp, _i32, _i32, ctypes.POINTER(_i32)]
+    L.emoe_plan_arena_bytes.restype = _i32
+    L.emoe_plan_arena_bytes.argtypes = [_vp, _i32, _i32, _i32, ctypes.POINTER(_u64)]
+    L.emoe_plan_stats.restype = _i32
+    L.emoe_plan_stats.argtypes = [_vp, _i32] + [ctypes.POINTER(_u64)] * 3
+    L.emoe_plan_num_launches.restype = _i32
+    L.emoe_plan_num_launches.argtypes = [_vp, _i32, ctypes.POINTER(_i32)]
+    L.emoe_plan_segments.restype = _i32
+    L.emoe_plan_segments.argtypes = [_vp, _i32, _vp, _u64, ctypes.POINTER(_u64)]
+    L.emoe_plan_device_status.restype = _i32
+    L.emoe_plan_device_status.argtypes = [_vp, ctypes.POINTER(_i32)]
+    L.emoe_plan_set_tuning.restype = _i32
+    L.emoe_plan_set_tuning.argtypes = [_vp, ctypes.POINTER(_Tuning)]
+    L.emoe_strerror.restype = ctypes.c_char_p
+    L.emoe_strerror.argtypes = [_i32]
+    _lib = L
+    return L
+
+
+def strerror(code: int) -> str:
+    return lib().emoe_strerror(code).decode()
+
+
+def _check(code: int) -> None:
+    if code != 0:
+        raise EmoeError(code, strerror(code))
+
+
+def _i32arr(x) -> np.ndarray:
+    return np.ascontiguousarray(x, dtype=np.int32)
+
+
+def _make_config(cfg, keep: list) -> _Config:
+    """cfg: object with ep, tp, placement, kv_num_blocks, seq_lens, block_table."""
+    off = np.zeros(len(cfg.placement) + 1, dtype=np.int32)
+    off[1:] = np.cumsum([len(p) for p in cfg.placement])
+    ids = _i32arr([e for p in cfg.placement for e in p])
+    if ids.size == 0:
+        ids = np.zeros(1, dtype=np.int32)
+    sl = _i32arr(cfg.seq_lens)
+    bt = _i32arr(cfg.block_table)
+    n_seqs = int(sl.size)
+    max_blocks = int(bt.shape[1]) if bt.ndim == 2 and n_seqs else 0
+    if sl.size == 0:
+        sl = np.zeros(1, dtype=np.int32)
+    if bt.size == 0:
+        bt = np.zeros(1, dtype=np.int32)
+    keep += [off, ids, sl, bt]
+    p = lambda a: a.ctypes.data_as(_i32p)
+    return _Config(cfg.ep, cfg.tp, p(off), p(ids), cfg.kv_num_blocks, n_seqs, max_blocks,
+                   p(sl), p(bt))
+
+
+def _ptr_array(items: Sequence) -> ctypes.Array:
+    """Device (or host) addresses from ints, torch tensors or numpy arrays."""
+    vals = []
+    for x in items:
+        if isinstance(x, int):
+            vals.append(x)
+        elif hasattr(x, "data_ptr"):
+            vals.append(x.data_ptr())
+        elif isinstance(x, np.ndarray):
+            vals.append(x.ctypes.data)
+        else:
+            raise TypeError("cannot take the address of %r" % type(x))
+    return (_vp * max(len(vals), 1))(*vals)
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        return 0
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)
+
+
+class Plan:
+    """A scale-step plan: emoe_plan_create ... emoe_plan_destroy."""
+
+    def __init__(self, shape, old_cfg, new_cfg, host_only: bool = False):
+        self._h = _vp()
+        keep: list = []
+        sh = _Shape(shape.n_layers, shape.n_routed, shape.n_shared, shape.d_model, shape.d_ff,
+                    shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.kv_block_tokens,
+                    shape.elem_bytes)
+        co, cn = _make_config(old_cfg, keep), _make_config(new_cfg, keep)
+        _check(lib().emoe_plan_create(ctypes.byref(sh), ctypes.byref(co), ctypes.byref(cn),
+                                      PLAN_HOST_ONLY if host_only else 0, ctypes.byref(self._h)))
+        self.host_only = host_only
+
+    # -- life cycle
+    def close(self) -> None:
+        if self._h:
+            lib().emoe_plan_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    # -- queries
+    def num_ranks(self, phase: int, side: int) -> int:
+        n = _i32()
+        _check(lib().emoe_plan_num_ranks(self._h, phase, side, ctypes.byref(n)))
+        return n.value
+
+    def arena_bytes(self, phase: int, side: int) -> List[int]:
+        out = []
+        for r in range(self.num_ranks(phase, side)):
+            b = _u64()
+            _check(lib().emoe_plan_arena_bytes(self._h, phase, side, r, ctypes.byref(b)))
+            out.append(b.value)
+        return out
+
+    def stats(self, phase: int) -> dict:
+        a, b, c = _u64(), _u64(), _u64()
+        _check(lib().emoe_plan_stats(self._h, phase, ctypes.byref(a), ctypes.byref(b),
+                                     ctypes.byref(c)))
+        return dict(bytes_moved=a.value, bytes_read=b.value, n_segments=c.value)
+
+    def num_launches(self, phase: int) -> int:
+        n = _i32()
+        _check(lib().emoe_plan_num_launches(self._h, phase, ctypes.byref(n)))
+        return n.value
+
+    def segments(self, phase: int) -> np.ndarray:
+        n = _u64()
+        _check(lib().emoe_plan_segments(self._h, phase, None, 0, ctypes.byref(n)))
+        out = np.zeros(n.value, dtype=SEGMENT_DTYPE)
+        if n.value:
+            _check(lib().emoe_plan_segments(self._h, phase, out.ctypes.data_as(_vp), n.value,
+                                            ctypes.byref(n)))
+        return out
+
+    def device_status(self) -> int:
+        s = _i32()
+        _check(lib().emoe_plan_device_status(self._h, ctypes.byref(s)))
+        return s.value
+
+    def set_tuning(self, max_ctas: int = 0, bulk_tile_bytes: int = 0, bulk_stages: int = 0,
+                   path: int = 0, kv_mode: int = 0) -> None:
+        t = _Tuning(max_ctas, bulk_tile_bytes, bulk_stages, path, kv_mode)
+        _check(lib().emoe_plan_set_tuning(self._h, ctypes.byref(t)))
+
+    # -- the hot path
+    def _run(self, fn, src, dst, stream) -> None:
+        _check(fn(self._h, _ptr_array(src), _ptr_array(dst), _stream_handle(stream)))
+
+    def reshard_experts(self, src, dst, stream=None) -> None:
+        self._run(lib().emoe_reshard_experts, src, dst, stream)
+
+    def reshard_attn(self, src, dst, stream=None) -> None:
+        self._run(lib().emoe_reshard_attn, src, dst, stream)
+
+    def reshard_kv(self, src, dst, stream=None) -> None:
+        self._run(lib().emoe_reshard_kv, src, dst, stream)
+
+    def reshard_step_host(self, h_src, h_dst, d_src, d_dst, stream=None) -> None:
+        """Each argument: three lists (experts, attn, kv) of per-rank buffers."""
+        PP = ctypes.POINTER(_vp)
+        keep = []
+
+        def pack(groups):
+            arrs = [_ptr_array(g) for g in groups]
+            keep.extend(arrs)
+            return (PP * 3)(*[ctypes.cast(a, PP) for a in arrs])
+
+        _check(lib().emoe_reshard_step_host(self._h, pack(h_src), pack(h_dst), pack(d_src),
+                                            pack(d_dst), _stream_handle(stream)))

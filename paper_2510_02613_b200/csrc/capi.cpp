@@ -1,0 +1,384 @@
+// capi.cpp - the C ABI of libemoe.so: plan life cycle, argument checks, launches.
+#include <cuda_runtime.h>
+
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "kernels.h"
+#include "planner.h"
+
+using namespace emoe;
+
+namespace {
+
+constexpr uint32_t kUnitTiles = 8;
+constexpr uint32_t kDefaultBulkTile = 32768, kDefaultBulkStages = 6;
+constexpr uint32_t kVecTile = 16384;
+constexpr uint64_t kBulkMinRun = 16384;  // shorter runs go to the vector kernel
+
+struct DevPhase {
+  std::vector<Segment> segs;  // routed copy of the host segments (fan-out split to kMaxFanout)
+  std::vector<Dst> dsts;
+  std::vector<Unit> bulk_units, vec_units;
+  Segment *d_segs = nullptr;
+  Dst *d_dsts = nullptr;
+  Unit *d_bulk_units = nullptr, *d_vec_units = nullptr;
+};
+
+}  // namespace
+
+struct emoe_plan {
+  HostPlan hp;
+  bool host_only = true;
+  int device = -1, sm_count = 148;
+  emoe_tuning_t tuning{};
+  DevPhase dev[3];
+  uint32_t *d_pair_old = nullptr, *d_pair_new = nullptr;
+  int *d_status = nullptr;
+};
+
+namespace {
+
+uint32_t bulk_tile(const emoe_plan *p) {
+  return p->tuning.bulk_tile_bytes > 0 ? (uint32_t)p->tuning.bulk_tile_bytes : kDefaultBulkTile;
+}
+uint32_t bulk_stages(const emoe_plan *p) {
+  return p->tuning.bulk_stages > 0 ? (uint32_t)p->tuning.bulk_stages : kDefaultBulkStages;
+}
+
+void add_units(std::vector<Unit> *units, uint32_t seg, uint64_t n_tiles) {
+  for (uint64_t t = 0; t < n_tiles; t += kUnitTiles) {
+    const uint64_t n = n_tiles - t < kUnitTiles ? n_tiles - t : kUnitTiles;
+    units->push_back({seg, (uint32_t)t, (uint32_t)n, 0});
+  }
+}
+
+// Routes every host segment to the bulk or the vector kernel and cuts it into units.
+void build_tables(emoe_plan *p, int phase) {
+  const PhasePlan &pp = p->hp.phase[phase];
+  DevPhase &dp = p->dev[phase];
+  dp.segs.clear(); dp.dsts.clear(); dp.bulk_units.clear(); dp.vec_units.clear();
+  const uint32_t T = bulk_tile(p);
+  for (const Segment &s0 : pp.segs) {
+    bool bulk = s0.align == 16 && s0.run_bytes >= kBulkMinRun;
+    if (p->tuning.path == 1) bulk = false;
+    if (p->tuning.path == 2) bulk = (s0.align == 16);
+    const uint32_t max_fan = bulk ? (uint32_t)kMaxFanout : s0.n_dst;
+    for (uint32_t k = 0; k < s0.n_dst; k += max_fan) {
+      Segment s = s0;
+      s.n_dst = s0.n_dst - k < max_fan ? s0.n_dst - k : max_fan;
+      s.dst_first = (uint32_t)dp.dsts.size();
+      for (uint32_t j = 0; j < s.n_dst; ++j) dp.dsts.push_back(pp.dsts[s0.dst_first + k + j]);
+      const uint32_t idx = (uint32_t)dp.segs.size();
+      dp.segs.push_back(s);
+      if (bulk) add_units(&dp.bulk_units, idx, seg_tile_count(s.run_bytes, s.n_runs, T));
+      else add_units(&dp.vec_units, idx, seg_tile_count(s.run_bytes, s.n_runs, kVecTile));
+    }
+  }
+}
+
+template <typename T>
+cudaError_t upload(const std::vector<T> &v, T **d) {
+  if (*d) { cudaFree(*d); *d = nullptr; }
+  if (v.empty()) return cudaSuccess;
+  cudaError_t e = cudaMalloc((void **)d, v.size() * sizeof(T));
+  if (e != cudaSuccess) return e;
+  return cudaMemcpy(*d, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice);
+}
+
+emoe_status_t cuda_status(cudaError_t e) {
+  if (e == cudaSuccess) return EMOE_OK;
+  (void)cudaGetLastError();
+  return e == cudaErrorMemoryAllocation ? EMOE_ERR_OOM : EMOE_ERR_CUDA;
+}
+
+emoe_status_t upload_phase(emoe_plan *p, int phase) {
+  DevPhase &dp = p->dev[phase];
+  cudaError_t e;
+  if ((e = upload(dp.segs, &dp.d_segs)) != cudaSuccess) return cuda_status(e);
+  if ((e = upload(dp.dsts, &dp.d_dsts)) != cudaSuccess) return cuda_status(e);
+  if ((e = upload(dp.bulk_units, &dp.d_bulk_units)) != cudaSuccess) return cuda_status(e);
+  if ((e = upload(dp.vec_units, &dp.d_vec_units)) != cudaSuccess) return cuda_status(e);
+  return EMOE_OK;
+}
+
+void free_device(emoe_plan *p) {
+  for (DevPhase &dp : p->dev) {
+    cudaFree(dp.d_segs); cudaFree(dp.d_dsts); cudaFree(dp.d_bulk_units); cudaFree(dp.d_vec_units);
+    dp.d_segs = nullptr; dp.d_dsts = nullptr; dp.d_bulk_units = dp.d_vec_units = nullptr;
+  }
+  cudaFree(p->d_pair_old); cudaFree(p->d_pair_new); cudaFree(p->d_status);
+  p->d_pair_old = p->d_pair_new = nullptr; p->d_status = nullptr;
+}
+
+int ranks_of(const emoe_plan *p, int phase, int side) {
+  if (phase == EMOE_PHASE_EXPERTS) return side == EMOE_SIDE_OLD ? p->hp.ep_old : p->hp.ep_new;
+  return side == EMOE_SIDE_OLD ? p->hp.tp_old : p->hp.tp_new;
+}
+
+// Host-side argument checks of a reshard call; fills the by-value pointer table.
+emoe_status_t check_arenas(const emoe_plan *p, int phase, const void *const *src, void *const *dst,
+                           RankPtrs *out) {
+  if (!p || !src || !dst) return EMOE_ERR_INVALID_ARG;
+  if (p->host_only) return EMOE_ERR_CUDA;
+  const PhasePlan &pp = p->hp.phase[phase];
+  const int ns = ranks_of(p, phase, EMOE_SIDE_OLD), nd = ranks_of(p, phase, EMOE_SIDE_NEW);
+  std::memset(out, 0, sizeof(*out));
+  for (int r = 0; r < ns; ++r) {
+    if (pp.arena_old[r] && !src[r]) return EMOE_ERR_INVALID_ARG;
+    if ((uintptr_t)src[r] % 16) return EMOE_ERR_ALIGNMENT;
+    out->src[r] = (const uint8_t *)src[r];
+  }
+  for (int r = 0; r < nd; ++r) {
+    if (pp.arena_new[r] && !dst[r]) return EMOE_ERR_INVALID_ARG;
+    if ((uintptr_t)dst[r] % 16) return EMOE_ERR_ALIGNMENT;
+    out->dst[r] = (uint8_t *)dst[r];
+  }
+  for (int a = 0; a < ns; ++a)
+    for (int b = 0; b < nd; ++b) {
+      const uintptr_t s0 = (uintptr_t)src[a], s1 = s0 + pp.arena_old[a];
+      const uintptr_t d0 = (uintptr_t)dst[b], d1 = d0 + pp.arena_new[b];
+      if (s0 < d1 && d0 < s1) return EMOE_ERR_OVERLAP;
+    }
+  return EMOE_OK;
+}
+
+uint32_t cta_budget(const emoe_plan *p) {
+  return p->tuning.max_ctas > 0 ? (uint32_t)p->tuning.max_ctas : (uint32_t)p->sm_count;
+}
+
+emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, cudaStream_t st) {
+  const DevPhase &dp = p->dev[phase];
+  cudaError_t e = launch_bulk_copy({dp.d_segs, dp.d_dsts, dp.d_bulk_units, (uint32_t)dp.bulk_units.size()},
+                                   ptrs, bulk_tile(p), bulk_stages(p), cta_budget(p), p->d_status, st);
+  if (e != cudaSuccess) return cuda_status(e);
+  e = launch_vec_copy({dp.d_segs, dp.d_dsts, dp.d_vec_units, (uint32_t)dp.vec_units.size()}, ptrs,
+                      kVecTile, cta_budget(p) * 8, st);
+  return cuda_status(e);
+}
+
+std::once_flag g_init_once;
+cudaError_t g_init_err = cudaSuccess;
+
+}  // namespace
+
+extern "C" {
+
+emoe_status_t emoe_plan_create(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
+                               const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out) {
+  if (!shape || !old_cfg || !new_cfg || !out) return EMOE_ERR_INVALID_ARG;
+  emoe_plan *p = new (std::nothrow) emoe_plan();
+  if (!p) return EMOE_ERR_OOM;
+  emoe_status_t st;
+  try {
+    st = build_host_plan(*shape, *old_cfg, *new_cfg, &p->hp);
+    if (st == EMOE_OK)
+      for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
+  } catch (const std::bad_alloc &) {
+    st = EMOE_ERR_OOM;
+  }
+  if (st != EMOE_OK) { delete p; return st; }
+  p->host_only = (flags & EMOE_PLAN_HOST_ONLY) != 0;
+  if (!p->host_only) {
+    cudaError_t e = cudaGetDevice(&p->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
+    if (e == cudaSuccess) {
+      std::call_once(g_init_once, [] { g_init_err = kernels_init(); });
+      e = g_init_err;
+    }
+    st = cuda_status(e);
+    for (int ph = 0; st == EMOE_OK && ph < 3; ++ph) st = upload_phase(p, ph);
+    if (st == EMOE_OK && p->hp.kv.head_split_changes) {
+      cudaError_t e2 = upload(p->hp.kv.pair_old, &p->d_pair_old);
+      if (e2 == cudaSuccess) e2 = upload(p->hp.kv.pair_new, &p->d_pair_new);
+      st = cuda_status(e2);
+    }
+    if (st == EMOE_OK) {
+      cudaError_t e3 = cudaMalloc((void **)&p->d_status, sizeof(int));
+      if (e3 == cudaSuccess) e3 = cudaMemset(p->d_status, 0, sizeof(int));
+      st = cuda_status(e3);
+    }
+    if (st != EMOE_OK) { free_device(p); delete p; return st; }
+  }
+  *out = p;
+  return EMOE_OK;
+}
+
+void emoe_plan_destroy(emoe_plan_t *p) {
+  if (!p) return;
+  if (!p->host_only) free_device(p);
+  delete p;
+}
+
+emoe_status_t emoe_reshard_experts(const emoe_plan_t *p, const void *const *src, void *const *dst,
+                                   void *stream) {
+  RankPtrs ptrs;
+  emoe_status_t st = check_arenas(p, EMOE_PHASE_EXPERTS, src, dst, &ptrs);
+  if (st != EMOE_OK) return st;
+  return run_segments(p, EMOE_PHASE_EXPERTS, ptrs, (cudaStream_t)stream);
+}
+
+emoe_status_t emoe_reshard_attn(const emoe_plan_t *p, const void *const *src, void *const *dst,
+                                void *stream) {
+  RankPtrs ptrs;
+  emoe_status_t st = check_arenas(p, EMOE_PHASE_ATTN, src, dst, &ptrs);
+  if (st != EMOE_OK) return st;
+  return run_segments(p, EMOE_PHASE_ATTN, ptrs, (cudaStream_t)stream);
+}
+
+emoe_status_t emoe_reshard_kv(const emoe_plan_t *p, const void *const *src, void *const *dst,
+                              void *stream) {
+  RankPtrs ptrs;
+  emoe_status_t st = check_arenas(p, EMOE_PHASE_KV, src, dst, &ptrs);
+  if (st != EMOE_OK) return st;
+  if (!p->hp.kv.head_split_changes) return run_segments(p, EMOE_PHASE_KV, ptrs, (cudaStream_t)stream);
+  const KvPlan &kv = p->hp.kv;
+  KvTables t{p->d_pair_old, p->d_pair_new, (uint32_t)kv.pair_old.size(), kv.n_layers * 2,
+             kv.block_tokens, kv.hkv, kv.hkv / kv.c, kv.hkv / kv.d, (uint32_t)kv.head_bytes,
+             kv.nb_old, kv.nb_new};
+  return cuda_status(launch_kv_copy(t, ptrs, p->tuning.kv_mode, cta_budget(p) * 8, p->d_status,
+                                    (cudaStream_t)stream));
+}
+
+emoe_status_t emoe_reshard_step_host(const emoe_plan_t *p, const void *const *const h_src[3],
+                                     void *const *const h_dst[3], void *const *const d_src[3],
+                                     void *const *const d_dst[3], void *stream) {
+  if (!p || !h_src || !h_dst || !d_src || !d_dst) return EMOE_ERR_INVALID_ARG;
+  if (p->host_only) return EMOE_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  for (int ph = 0; ph < 3; ++ph) {
+    if (!h_src[ph] || !h_dst[ph] || !d_src[ph] || !d_dst[ph]) return EMOE_ERR_INVALID_ARG;
+    const PhasePlan &pp = p->hp.phase[ph];
+    for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_OLD); ++r) {
+      if (!pp.arena_old[r]) continue;
+      if (!h_src[ph][r] || !d_src[ph][r]) return EMOE_ERR_INVALID_ARG;
+      cudaError_t e = cudaMemcpyAsync(d_src[ph][r], h_src[ph][r], pp.arena_old[r],
+                                      cudaMemcpyHostToDevice, st);
+      if (e != cudaSuccess) return cuda_status(e);
+    }
+  }
+  emoe_status_t rc = emoe_reshard_experts(p, (const void *const *)d_src[0], d_dst[0], stream);
+  if (rc == EMOE_OK) rc = emoe_reshard_attn(p, (const void *const *)d_src[1], d_dst[1], stream);
+  if (rc == EMOE_OK) rc = emoe_reshard_kv(p, (const void *const *)d_src[2], d_dst[2], stream);
+  if (rc != EMOE_OK) return rc;
+  for (int ph = 0; ph < 3; ++ph) {
+    const PhasePlan &pp = p->hp.phase[ph];
+    for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_NEW); ++r) {
+      if (!pp.arena_new[r]) continue;
+      if (!h_dst[ph][r]) return EMOE_ERR_INVALID_ARG;
+      cudaError_t e = cudaMemcpyAsync(h_dst[ph][r], d_dst[ph][r], pp.arena_new[r],
+                                      cudaMemcpyDeviceToHost, st);
+      if (e != cudaSuccess) return cuda_status(e);
+    }
+  }
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_plan_num_ranks(const emoe_plan_t *p, int phase, int side, int32_t *n) {
+  if (!p || !n || phase < 0 || phase > 2 || side < 0 || side > 1) return EMOE_ERR_INVALID_ARG;
+  *n = ranks_of(p, phase, side);
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_plan_arena_bytes(const emoe_plan_t *p, int phase, int side, int rank,
+                                    uint64_t *bytes) {
+  if (!p || !bytes || phase < 0 || phase > 2 || side < 0 || side > 1) return EMOE_ERR_INVALID_ARG;
+  if (rank < 0 || rank >= ranks_of(p, phase, side)) return EMOE_ERR_INVALID_ARG;
+  const PhasePlan &pp = p->hp.phase[phase];
+  *bytes = side == EMOE_SIDE_OLD ? pp.arena_old[rank] : pp.arena_new[rank];
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_plan_stats(const emoe_plan_t *p, int phase, uint64_t *bytes_moved,
+                              uint64_t *bytes_read, uint64_t *n_segments) {
+  if (!p || phase < 0 || phase > 2) return EMOE_ERR_INVALID_ARG;
+  const PhasePlan &pp = p->hp.phase[phase];
+  if (bytes_moved) *bytes_moved = pp.bytes_moved;
+  if (bytes_read) *bytes_read = pp.bytes_read;
+  if (n_segments) {
+    *n_segments = pp.segs.size();
+    if (phase == EMOE_PHASE_KV && p->hp.kv.head_split_changes) *n_segments = p->hp.kv.pair_old.size();
+  }
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_plan_num_launches(const emoe_plan_t *p, int phase, int32_t *n) {
+  if (!p || !n || phase < 0 || phase > 2) return EMOE_ERR_INVALID_ARG;
+  if (phase == EMOE_PHASE_KV && p->hp.kv.head_split_changes) {
+    *n = p->hp.kv.pair_old.empty() ? 0 : 1;
+    return EMOE_OK;
+  }
+  *n = (p->dev[phase].bulk_units.empty() ? 0 : 1) + (p->dev[phase].vec_units.empty() ? 0 : 1);
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_plan_segments(const emoe_plan_t *p, int phase, emoe_segment_t *out, uint64_t cap,
+                                 uint64_t *n) {
+  if (!p || !n || phase < 0 || phase > 2 || (cap && !out)) return EMOE_ERR_INVALID_ARG;
+  try {
+    std::vector<emoe_segment_t> v;
+    export_segments(p->hp, phase, &v);
+    *n = v.size();
+    const uint64_t k = v.size() < cap ? v.size() : cap;
+    if (k) std::memcpy(out, v.data(), k * sizeof(emoe_segment_t));
+  } catch (const std::bad_alloc &) {
+    return EMOE_ERR_OOM;
+  }
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_plan_device_status(const emoe_plan_t *p, int32_t *status) {
+  if (!p || !status) return EMOE_ERR_INVALID_ARG;
+  if (p->host_only) return EMOE_ERR_CUDA;
+  int v = 0;
+  cudaError_t e = cudaMemcpy(&v, p->d_status, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_status(e);
+  *status = v;
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
+  if (!p || !t) return EMOE_ERR_INVALID_ARG;
+  if (t->max_ctas < 0 || t->bulk_tile_bytes < 0 || t->bulk_stages < 0 || t->path < 0 ||
+      t->path > 2 || t->kv_mode < 0 || t->kv_mode > 2)
+    return EMOE_ERR_INVALID_ARG;
+  if (t->bulk_tile_bytes && (t->bulk_tile_bytes % 128 || t->bulk_tile_bytes < 1024))
+    return EMOE_ERR_INVALID_ARG;
+  const uint32_t tile = t->bulk_tile_bytes ? t->bulk_tile_bytes : kDefaultBulkTile;
+  const uint32_t stages = t->bulk_stages ? t->bulk_stages : kDefaultBulkStages;
+  if (stages < 2 || stages > 16 || (uint64_t)tile * stages > 200 * 1024) return EMOE_ERR_INVALID_ARG;
+  p->tuning = *t;
+  emoe_status_t st = EMOE_OK;
+  try {
+    for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
+  } catch (const std::bad_alloc &) {
+    return EMOE_ERR_OOM;
+  }
+  if (!p->host_only) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return EMOE_ERR_CUDA;
+    for (int ph = 0; st == EMOE_OK && ph < 3; ++ph) st = upload_phase(p, ph);
+  }
+  return st;
+}
+
+const char *emoe_strerror(emoe_status_t s) {
+  switch (s) {
+    case EMOE_OK: return "ok";
+    case EMOE_ERR_INVALID_ARG: return "invalid argument";
+    case EMOE_ERR_SHAPE: return "invalid model shape or TP degree does not divide the head counts";
+    case EMOE_ERR_PLACEMENT: return "invalid expert placement";
+    case EMOE_ERR_BLOCK_TABLE: return "invalid KV block table";
+    case EMOE_ERR_ALIGNMENT: return "arena base pointer is not 16-byte aligned";
+    case EMOE_ERR_OVERLAP: return "source and destination arenas overlap";
+    case EMOE_ERR_OOM: return "out of memory";
+    case EMOE_ERR_CUDA: return "CUDA error, or a host-only plan was asked to run";
+    case EMOE_ERR_UNSUPPORTED: return "unsupported configuration";
+    case EMOE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,430 @@
+// kernels.cu - sm_100a copy kernels of the scale-step re-layout.
+//
+//  * bulk_copy_kernel : long 16-byte-aligned runs.  One producer thread per CTA
+//    issues cp.async.bulk (TMA, untiled) global->shared loads into a ring of
+//    stages guarded by mbarriers; one consumer thread issues the
+//    shared->global bulk stores, once per destination of the tile, so a
+//    replicated source is read from HBM once.  No cluster, no multicast.
+//  * vec_copy_kernel  : short, strided or narrowly aligned runs.  A warp per
+//    tile, lanes walk the tile in 16-byte (or narrower) pieces, four loads in
+//    flight per lane before the stores.
+//  * kv_copy_kernel   : KV head re-split.  A CTA per (layer, K|V, block pair)
+//    gathers the block's token rows from the old ranks and writes each new
+//    rank's block; only 8 bytes of metadata per block pair.
+//
+// Every device-side wait is bounded: on expiry the kernel records
+// EMOE_ERR_DEVICE_TIMEOUT in the plan's status word, lets its own copies in
+// flight land, and returns.
+#include "kernels.h"
+
+namespace emoe {
+namespace {
+
+constexpr uint32_t kMaxStages = 16;
+constexpr unsigned long long kWaitLimitNs = 4000000000ull;  // 4 s per wait
+
+// ---- PTX wrappers -----------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within kWaitLimitNs.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
+  }
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes,
+                                          uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
+               "r"(src_smem), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// ---- bulk path --------------------------------------------------------------------------
+
+struct TileInfo {  // producer -> consumer, one per stage
+  uint64_t dst_ptr[kMaxFanout];
+  uint64_t dst_pitch[kMaxFanout];
+  uint32_t n_dst, n_rows, row_bytes, pad;
+};
+
+struct BulkParams {
+  SegTables t;
+  uint32_t tile_bytes, stages;
+  int *status;
+  RankPtrs ptrs;
+};
+
+__global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant__ BulkParams p) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const uint32_t S = p.stages, T = p.tile_bytes;
+  uint8_t *data = smem;
+  TileInfo *info = reinterpret_cast<TileInfo *>(smem + (size_t)S * T);
+  uint64_t *full = reinterpret_cast<uint64_t *>(info + S);
+  uint64_t *empty = full + S;
+  __shared__ const uint8_t *s_src[EMOE_MAX_RANKS];
+  __shared__ uint8_t *s_dst[EMOE_MAX_RANKS];
+  __shared__ volatile int s_abort;
+
+  const uint32_t tid = threadIdx.x;
+  if (tid < EMOE_MAX_RANKS) {
+    s_src[tid] = p.ptrs.src[tid];
+    s_dst[tid] = p.ptrs.dst[tid];
+  }
+  if (tid == 0) {
+    s_abort = 0;
+    for (uint32_t s = 0; s < S; ++s) {
+      mbar_init(smem_u32(&full[s]), 1);
+      mbar_init(smem_u32(&empty[s]), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+
+  if (tid == 0) {
+    // ---------------- producer: schedule tiles, issue loads ----------------
+    uint32_t it = 0;
+    bool ok = true;
+    for (uint32_t u = blockIdx.x; ok && u < p.t.n_units; u += gridDim.x) {
+      const Unit un = p.t.units[u];
+      const Segment sg = p.t.segs[un.seg];
+      const uint8_t *src_base = s_src[sg.src_rank] + sg.src_off;
+      const bool long_run = sg.run_bytes >= T;
+      const uint32_t tpr = long_run ? (uint32_t)((sg.run_bytes + T - 1) / T) : 1u;
+      const uint32_t rpt = long_run ? 1u : (uint32_t)(T / sg.run_bytes);
+      uint32_t run = long_run ? un.first_tile / tpr : un.first_tile * rpt;  // first run (row)
+      uint32_t ch = long_run ? un.first_tile % tpr : 0u;                    // chunk in run
+      for (uint32_t k = 0; k < un.n_tiles; ++k, ++it) {
+        const uint32_t st = it % S, round = it / S;
+        if (round > 0 && !mbar_wait(smem_u32(&empty[st]), (round - 1) & 1)) { ok = false; break; }
+        if (s_abort) { ok = false; break; }
+        uint32_t rows, row_bytes;
+        uint64_t in_run;
+        if (long_run) {
+          in_run = (uint64_t)ch * T;
+          const uint64_t left = sg.run_bytes - in_run;
+          row_bytes = left < T ? (uint32_t)left : T;
+          rows = 1;
+        } else {
+          in_run = 0;
+          rows = sg.n_runs - run < rpt ? sg.n_runs - run : rpt;
+          row_bytes = (uint32_t)sg.run_bytes;
+        }
+        TileInfo &ti = info[st];
+        for (uint32_t d = 0; d < sg.n_dst; ++d) {
+          const Dst dd = p.t.dsts[sg.dst_first + d];
+          ti.dst_ptr[d] = (uint64_t)(s_dst[dd.rank] + dd.off + (uint64_t)run * dd.pitch + in_run);
+          ti.dst_pitch[d] = dd.pitch;
+        }
+        ti.n_dst = sg.n_dst;
+        ti.n_rows = rows;
+        ti.row_bytes = row_bytes;
+        const uint32_t bar = smem_u32(&full[st]);
+        mbar_arrive_expect_tx(bar, rows * row_bytes);
+        const uint8_t *sp = src_base + (uint64_t)run * sg.src_pitch + in_run;
+        const uint32_t dp = smem_u32(data + (size_t)st * T);
+        for (uint32_t r = 0; r < rows; ++r)
+          bulk_load(dp + r * row_bytes, sp + (uint64_t)r * sg.src_pitch, row_bytes, bar);
+        if (long_run) {
+          if (++ch == tpr) { ch = 0; ++run; }
+        } else {
+          run += rows;
+        }
+      }
+    }
+    if (ok) {
+      // end marker
+      const uint32_t st = it % S, round = it / S;
+      if (round == 0 || mbar_wait(smem_u32(&empty[st]), (round - 1) & 1)) {
+        info[st].n_rows = 0;
+        mbar_arrive(smem_u32(&full[st]));
+      } else {
+        ok = false;
+      }
+    }
+    if (!ok) {
+      // a wait expired: flag it, then let the loads already issued land before leaving
+      s_abort = 1;
+      atomicExch(p.status, (int)EMOE_ERR_DEVICE_TIMEOUT);
+      const uint32_t back = it < S ? it : S;
+      for (uint32_t j = 1; j <= back; ++j) {
+        const uint32_t i2 = it - j;
+        (void)mbar_wait(smem_u32(&full[i2 % S]), (i2 / S) & 1);
+      }
+    }
+  } else if (tid == 32) {
+    // ---------------- consumer: issue stores, recycle stages ----------------
+    for (uint32_t it = 0;; ++it) {
+      const uint32_t st = it % S, round = it / S;
+      if (!mbar_wait(smem_u32(&full[st]), round & 1)) {
+        s_abort = 1;
+        atomicExch(p.status, (int)EMOE_ERR_DEVICE_TIMEOUT);
+        break;
+      }
+      const TileInfo &ti = info[st];
+      const uint32_t rows = ti.n_rows, rb = ti.row_bytes;
+      if (rows == 0) break;
+      const uint32_t sp = smem_u32(data + (size_t)st * T);
+      for (uint32_t d = 0; d < ti.n_dst; ++d) {
+        uint8_t *dp = reinterpret_cast<uint8_t *>(ti.dst_ptr[d]);
+        const uint64_t pitch = ti.dst_pitch[d];
+        for (uint32_t r = 0; r < rows; ++r) bulk_store(dp + (uint64_t)r * pitch, sp + r * rb, rb);
+      }
+      bulk_commit();
+      if (it >= 1) {  // the store of the previous tile has finished reading its stage
+        bulk_wait_read<1>();
+        mbar_arrive(smem_u32(&empty[(it - 1) % S]));
+      }
+    }
+    bulk_wait_read<0>();
+  }
+}
+
+// ---- vector path ------------------------------------------------------------------------
+
+struct VecParams {
+  SegTables t;
+  uint32_t tile_bytes;
+  RankPtrs ptrs;
+};
+
+template <typename V>
+__device__ __forceinline__ void warp_copy_tile(const uint8_t *sp, uint64_t src_pitch, uint32_t rows,
+                                               uint32_t row_bytes, const Segment &sg,
+                                               const Dst *dsts, uint8_t *const *s_dst, uint32_t run,
+                                               uint64_t in_run, uint32_t lane) {
+  constexpr uint32_t W = sizeof(V);
+  const uint32_t cpr = row_bytes / W;  // pieces per row
+  const uint32_t total = rows * cpr;
+  for (uint32_t i0 = lane; i0 < total; i0 += 32 * 4) {
+    V v[4];
+    uint32_t r[4], c[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t i = i0 + 32 * u;
+      if (i < total) {
+        r[u] = rows == 1 ? 0 : i / cpr;
+        c[u] = rows == 1 ? i : i - r[u] * cpr;
+        v[u] = *reinterpret_cast<const V *>(sp + (uint64_t)r[u] * src_pitch + (uint64_t)c[u] * W);
+      }
+    }
+    for (uint32_t d = 0; d < sg.n_dst; ++d) {
+      const Dst dd = dsts[sg.dst_first + d];
+      uint8_t *dp = s_dst[dd.rank] + dd.off + (uint64_t)run * dd.pitch + in_run;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t i = i0 + 32 * u;
+        if (i < total)
+          *reinterpret_cast<V *>(dp + (uint64_t)r[u] * dd.pitch + (uint64_t)c[u] * W) = v[u];
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) vec_copy_kernel(const __grid_constant__ VecParams p) {
+  __shared__ const uint8_t *s_src[EMOE_MAX_RANKS];
+  __shared__ uint8_t *s_dst[EMOE_MAX_RANKS];
+  if (threadIdx.x < EMOE_MAX_RANKS) {
+    s_src[threadIdx.x] = p.ptrs.src[threadIdx.x];
+    s_dst[threadIdx.x] = p.ptrs.dst[threadIdx.x];
+  }
+  __syncthreads();
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  const uint32_t T = p.tile_bytes;
+  for (uint32_t u = blockIdx.x; u < p.t.n_units; u += gridDim.x) {
+    const Unit un = p.t.units[u];
+    const Segment sg = p.t.segs[un.seg];
+    const uint8_t *src_base = s_src[sg.src_rank] + sg.src_off;
+    const bool long_run = sg.run_bytes >= T;
+    const uint32_t tpr = long_run ? (uint32_t)((sg.run_bytes + T - 1) / T) : 1u;
+    const uint32_t rpt = long_run ? 1u : (uint32_t)(T / sg.run_bytes);
+    for (uint32_t k = warp; k < un.n_tiles; k += n_warps) {
+      const uint32_t tile = un.first_tile + k;
+      uint32_t run, rows, row_bytes;
+      uint64_t in_run;
+      if (long_run) {
+        run = tile / tpr;
+        in_run = (uint64_t)(tile % tpr) * T;
+        const uint64_t left = sg.run_bytes - in_run;
+        row_bytes = left < T ? (uint32_t)left : T;
+        rows = 1;
+      } else {
+        run = tile * rpt;
+        in_run = 0;
+        rows = sg.n_runs - run < rpt ? sg.n_runs - run : rpt;
+        row_bytes = (uint32_t)sg.run_bytes;
+      }
+      const uint8_t *sp = src_base + (uint64_t)run * sg.src_pitch + in_run;
+      switch (sg.align) {
+        case 16: warp_copy_tile<uint4>(sp, sg.src_pitch, rows, row_bytes, sg, p.t.dsts, s_dst, run, in_run, lane); break;
+        case 8: warp_copy_tile<uint2>(sp, sg.src_pitch, rows, row_bytes, sg, p.t.dsts, s_dst, run, in_run, lane); break;
+        case 4: warp_copy_tile<uint32_t>(sp, sg.src_pitch, rows, row_bytes, sg, p.t.dsts, s_dst, run, in_run, lane); break;
+        case 2: warp_copy_tile<uint16_t>(sp, sg.src_pitch, rows, row_bytes, sg, p.t.dsts, s_dst, run, in_run, lane); break;
+        default: warp_copy_tile<uint8_t>(sp, sg.src_pitch, rows, row_bytes, sg, p.t.dsts, s_dst, run, in_run, lane); break;
+      }
+    }
+  }
+}
+
+// ---- KV head re-split -------------------------------------------------------------------
+
+struct KvParams {
+  KvTables t;
+  RankPtrs ptrs;
+};
+
+// Direct variant: thread q of a tile owns piece q of the LOGICAL block
+// [token][global head][piece]; it reads the piece from the old rank that holds the
+// head and writes it to the new rank that will.  Reads of a warp cover whole token
+// rows of the old layout, writes whole head vectors of the new one.
+template <typename V>
+__global__ void __launch_bounds__(256) kv_direct_kernel(const __grid_constant__ KvParams p) {
+  __shared__ const uint8_t *s_src[EMOE_MAX_RANKS];
+  __shared__ uint8_t *s_dst[EMOE_MAX_RANKS];
+  if (threadIdx.x < EMOE_MAX_RANKS) {
+    s_src[threadIdx.x] = p.ptrs.src[threadIdx.x];
+    s_dst[threadIdx.x] = p.ptrs.dst[threadIdx.x];
+  }
+  __syncthreads();
+  constexpr uint32_t W = sizeof(V);
+  const KvTables &t = p.t;
+  const uint32_t cpv = t.head_bytes / W;     // pieces per head vector
+  const uint32_t row = t.hkv * cpv;          // pieces per logical token row
+  const uint32_t total = t.block_tokens * row;
+  const uint64_t blk_old = (uint64_t)t.block_tokens * t.hc * t.head_bytes;
+  const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
+  const uint64_t n_tiles = (uint64_t)t.n_pairs * t.n_lk;
+  for (uint64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const uint32_t lk = (uint32_t)(tile / t.n_pairs), pr = (uint32_t)(tile % t.n_pairs);
+    const uint64_t base_old = ((uint64_t)lk * t.nb_old + t.pair_old[pr]) * blk_old;
+    const uint64_t base_new = ((uint64_t)lk * t.nb_new + t.pair_new[pr]) * blk_new;
+    for (uint32_t q0 = threadIdx.x; q0 < total; q0 += blockDim.x * 4) {
+      V v[4];
+      uint32_t tok[4], g[4], j[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t q = q0 + u * blockDim.x;
+        if (q < total) {
+          tok[u] = q / row;
+          const uint32_t rem = q - tok[u] * row;
+          g[u] = rem / cpv;
+          j[u] = rem - g[u] * cpv;
+          const uint32_t ro = g[u] / t.hc, ho = g[u] - ro * t.hc;
+          v[u] = *reinterpret_cast<const V *>(
+              s_src[ro] + base_old + ((uint64_t)(tok[u] * t.hc + ho) * cpv + j[u]) * W);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t q = q0 + u * blockDim.x;
+        if (q < total) {
+          const uint32_t rn = g[u] / t.hn, hn = g[u] - rn * t.hn;
+          *reinterpret_cast<V *>(s_dst[rn] + base_new +
+                                 ((uint64_t)(tok[u] * t.hn + hn) * cpv + j[u]) * W) = v[u];
+        }
+      }
+    }
+  }
+}
+
+}  // namespace
+
+// ---- launchers --------------------------------------------------------------------------
+
+static size_t bulk_smem_bytes(uint32_t tile_bytes, uint32_t stages) {
+  return (size_t)stages * tile_bytes + stages * (sizeof(TileInfo) + 2 * sizeof(uint64_t));
+}
+
+cudaError_t kernels_init() {
+  return cudaFuncSetAttribute(bulk_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              227 * 1024 - 2048);
+}
+
+cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
+                             uint32_t stages, uint32_t grid, int *status, cudaStream_t stream) {
+  if (t.n_units == 0) return cudaSuccess;
+  if (stages < 2 || stages > kMaxStages || tile_bytes % 128 != 0) return cudaErrorInvalidValue;
+  const size_t smem = bulk_smem_bytes(tile_bytes, stages);
+  if (smem > 227 * 1024 - 2048) return cudaErrorInvalidValue;
+  BulkParams p{t, tile_bytes, stages, status, ptrs};
+  if (grid > t.n_units) grid = t.n_units;
+  bulk_copy_kernel<<<grid, 64, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_vec_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
+                            uint32_t grid, cudaStream_t stream) {
+  if (t.n_units == 0) return cudaSuccess;
+  VecParams p{t, tile_bytes, ptrs};
+  if (grid > t.n_units) grid = t.n_units;
+  vec_copy_kernel<<<grid, 256, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, uint32_t grid,
+                           int *status, cudaStream_t stream) {
+  (void)mode;
+  (void)status;
+  const uint64_t n_tiles = (uint64_t)t.n_pairs * t.n_lk;
+  if (n_tiles == 0) return cudaSuccess;
+  if (grid > n_tiles) grid = (uint32_t)n_tiles;
+  KvParams p{t, ptrs};
+  const uint32_t hb = t.head_bytes;
+  if (hb % 16 == 0) kv_direct_kernel<uint4><<<grid, 256, 0, stream>>>(p);
+  else if (hb % 8 == 0) kv_direct_kernel<uint2><<<grid, 256, 0, stream>>>(p);
+  else if (hb % 4 == 0) kv_direct_kernel<uint32_t><<<grid, 256, 0, stream>>>(p);
+  else if (hb % 2 == 0) kv_direct_kernel<uint16_t><<<grid, 256, 0, stream>>>(p);
+  else kv_direct_kernel<uint8_t><<<grid, 256, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace emoe

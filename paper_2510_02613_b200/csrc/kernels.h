@@ -1,0 +1,65 @@
+// kernels.h - launch interface of the sm_100a copy kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "planner.h"
+
+namespace emoe {
+
+// A schedulable piece of one segment: n_tiles consecutive tiles starting at
+// first_tile.  A tile is either a chunk of at most tile_bytes of one long run,
+// or as many whole short runs ("rows") as fit into tile_bytes.
+struct Unit {
+  uint32_t seg;
+  uint32_t first_tile;
+  uint32_t n_tiles;
+  uint32_t pad;
+};
+
+constexpr int kMaxFanout = 8;  // destinations one bulk tile is stored to (longer lists are split)
+
+struct RankPtrs {
+  const uint8_t *src[EMOE_MAX_RANKS];
+  uint8_t *dst[EMOE_MAX_RANKS];
+};
+
+struct SegTables {  // device pointers
+  const Segment *segs;
+  const Dst *dsts;
+  const Unit *units;
+  uint32_t n_units;
+};
+
+// Tiles of a segment for a given tile size (shared by host table building and kernels).
+__host__ __device__ inline uint64_t seg_tile_count(uint64_t run_bytes, uint32_t n_runs,
+                                                   uint32_t tile_bytes) {
+  if (run_bytes >= tile_bytes) return (uint64_t)n_runs * ((run_bytes + tile_bytes - 1) / tile_bytes);
+  const uint64_t rpt = tile_bytes / run_bytes;
+  return (n_runs + rpt - 1) / rpt;
+}
+
+struct KvTables {  // device pointers + shape constants of the KV head re-split
+  const uint32_t *pair_old, *pair_new;
+  uint32_t n_pairs, n_lk;        // n_lk = 2 * n_layers
+  uint32_t block_tokens, hkv, hc, hn;
+  uint32_t head_bytes;
+  uint64_t nb_old, nb_new;
+};
+
+// Bulk path: cp.async.bulk global -> shared -> global through an mbarrier ring.
+cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
+                             uint32_t stages, uint32_t grid, int *status, cudaStream_t stream);
+// Vector path: a warp per tile, 16-byte (or narrower, per segment alignment) loads and stores.
+cudaError_t launch_vec_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
+                            uint32_t grid, cudaStream_t stream);
+// KV head re-split; mode 1 = direct register copy, mode 2 = staged through shared memory.
+cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, uint32_t grid,
+                           int *status, cudaStream_t stream);
+
+// One-time per-process kernel attribute setup (dynamic shared memory opt-in).
+cudaError_t kernels_init();
+
+}  // namespace emoe

@@ -1,0 +1,328 @@
+// planner.cpp - host planner: validation, move enumeration, coalescing.
+#include "planner.h"
+
+#include <algorithm>
+#include <map>
+#include <utility>
+
+namespace emoe {
+namespace {
+
+uint32_t pow2_align(uint64_t v) {  // largest power of two <= 16 dividing v (16 for v == 0)
+  uint32_t a = 16;
+  while (a > 1 && (v % a) != 0) a >>= 1;
+  return a;
+}
+
+void finish_segment(PhasePlan *pp, Segment s, const std::vector<Dst> &dsts) {
+  // a strided segment whose pitches equal the run size on both sides is contiguous
+  bool dense = s.n_runs > 1 && s.src_pitch == s.run_bytes;
+  for (const Dst &d : dsts) dense = dense && d.pitch == s.run_bytes;
+  if (dense) {
+    s.run_bytes *= s.n_runs;
+    s.n_runs = 1;
+  }
+  uint32_t a = std::min(pow2_align(s.src_off), pow2_align(s.run_bytes));
+  if (s.n_runs > 1) a = std::min(a, pow2_align(s.src_pitch));
+  for (const Dst &d : dsts) {
+    a = std::min(a, pow2_align(d.off));
+    if (s.n_runs > 1) a = std::min(a, pow2_align(d.pitch));
+  }
+  s.align = a;
+  s.n_dst = (uint32_t)dsts.size();
+  s.dst_first = (uint32_t)pp->dsts.size();
+  s.pad = 0;
+  pp->dsts.insert(pp->dsts.end(), dsts.begin(), dsts.end());
+  pp->segs.push_back(s);
+  pp->bytes_read += (uint64_t)s.n_runs * s.run_bytes;
+  pp->bytes_moved += (uint64_t)s.n_runs * s.run_bytes * dsts.size();
+}
+
+struct Placement {
+  int ep = 0;
+  std::vector<std::vector<int32_t>> ids;
+};
+
+emoe_status_t read_placement(const emoe_config_t &cfg, int n_experts, Placement *out) {
+  if (cfg.ep < 1 || cfg.tp < 1) return EMOE_ERR_INVALID_ARG;
+  if (cfg.ep > EMOE_MAX_RANKS || cfg.tp > EMOE_MAX_RANKS) return EMOE_ERR_UNSUPPORTED;
+  if (!cfg.place_off || !cfg.place_ids) return EMOE_ERR_INVALID_ARG;
+  if (cfg.place_off[0] != 0) return EMOE_ERR_PLACEMENT;
+  out->ep = cfg.ep;
+  out->ids.assign(cfg.ep, {});
+  std::vector<int> seen_total(n_experts, 0);
+  for (int r = 0; r < cfg.ep; ++r) {
+    if (cfg.place_off[r + 1] < cfg.place_off[r]) return EMOE_ERR_PLACEMENT;
+    std::vector<char> seen(n_experts, 0);
+    for (int i = cfg.place_off[r]; i < cfg.place_off[r + 1]; ++i) {
+      const int32_t e = cfg.place_ids[i];
+      if (e < 0 || e >= n_experts) return EMOE_ERR_PLACEMENT;
+      if (seen[e]) return EMOE_ERR_PLACEMENT;  // the same expert twice on one rank
+      seen[e] = 1;
+      seen_total[e]++;
+      out->ids[r].push_back(e);
+    }
+  }
+  for (int e = 0; e < n_experts; ++e)
+    if (!seen_total[e]) return EMOE_ERR_PLACEMENT;  // an expert nobody holds would be lost
+  return EMOE_OK;
+}
+
+emoe_status_t read_block_pairs(const emoe_shape_t &sh, const emoe_config_t &o,
+                               const emoe_config_t &n, std::vector<uint32_t> *po,
+                               std::vector<uint32_t> *pn) {
+  if (o.n_seqs != n.n_seqs || o.n_seqs < 0) return EMOE_ERR_BLOCK_TABLE;
+  if (o.kv_num_blocks < 0 || n.kv_num_blocks < 0) return EMOE_ERR_BLOCK_TABLE;
+  if (o.n_seqs == 0) return EMOE_OK;
+  if (!o.seq_lens || !n.seq_lens || !o.block_table || !n.block_table) return EMOE_ERR_INVALID_ARG;
+  std::vector<char> used_o(o.kv_num_blocks, 0), used_n(n.kv_num_blocks, 0);
+  const int64_t B = sh.kv_block_tokens;
+  for (int s = 0; s < o.n_seqs; ++s) {
+    if (o.seq_lens[s] != n.seq_lens[s] || o.seq_lens[s] < 0) return EMOE_ERR_BLOCK_TABLE;
+    const int64_t nblk = (o.seq_lens[s] + B - 1) / B;
+    if (nblk > o.max_blocks || nblk > n.max_blocks) return EMOE_ERR_BLOCK_TABLE;
+    for (int64_t j = 0; j < nblk; ++j) {
+      const int32_t a = o.block_table[(int64_t)s * o.max_blocks + j];
+      const int32_t b = n.block_table[(int64_t)s * n.max_blocks + j];
+      if (a < 0 || a >= o.kv_num_blocks || b < 0 || b >= n.kv_num_blocks)
+        return EMOE_ERR_BLOCK_TABLE;
+      if (used_o[a] || used_n[b]) return EMOE_ERR_BLOCK_TABLE;  // shared blocks unsupported
+      used_o[a] = used_n[b] = 1;
+      po->push_back((uint32_t)a);
+      pn->push_back((uint32_t)b);
+    }
+  }
+  return EMOE_OK;
+}
+
+// ---- experts ----------------------------------------------------------------------------
+
+void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &pn,
+                  PhasePlan *pp) {
+  const uint64_t m = (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes;
+  const uint32_t runs = (uint32_t)sh.n_layers * 3;
+  const int n_experts = sh.n_routed + sh.n_shared;
+  for (int r = 0; r < po.ep; ++r) pp->arena_old.push_back(runs * po.ids[r].size() * m);
+  for (int r = 0; r < pn.ep; ++r) pp->arena_new.push_back(runs * pn.ids[r].size() * m);
+
+  // every old copy of every expert, in (rank, slot) order
+  std::vector<std::vector<std::pair<int, int>>> copies(n_experts);
+  for (int r = 0; r < po.ep; ++r)
+    for (int s = 0; s < (int)po.ids[r].size(); ++s) copies[po.ids[r][s]].push_back({r, s});
+
+  // source of every destination slot: the copy on the same rank index, else the first
+  struct Move { int rs, ss, rd, sd; };
+  std::vector<Move> moves;
+  std::map<std::pair<int, int>, int> fan;  // (src rank, src slot) -> number of destinations
+  for (int rd = 0; rd < pn.ep; ++rd)
+    for (int sd = 0; sd < (int)pn.ids[rd].size(); ++sd) {
+      const auto &c = copies[pn.ids[rd][sd]];
+      std::pair<int, int> src = c.front();
+      for (const auto &x : c)
+        if (x.first == rd) { src = x; break; }
+      moves.push_back({src.first, src.second, rd, sd});
+      fan[src]++;
+    }
+
+  // single-destination sources: merge runs of consecutive slots on both sides
+  std::map<std::pair<int, int>, std::vector<Dst>> multi;
+  size_t i = 0;
+  while (i < moves.size()) {
+    const Move &a = moves[i];
+    const uint64_t n_old = po.ids[a.rs].size(), n_new = pn.ids[a.rd].size();
+    if (fan[{a.rs, a.ss}] > 1) {
+      multi[{a.rs, a.ss}].push_back({(uint64_t)a.sd * m, n_new * m, (uint32_t)a.rd, 0});
+      ++i;
+      continue;
+    }
+    size_t j = i + 1;
+    while (j < moves.size() && moves[j].rd == a.rd && moves[j].rs == a.rs &&
+           moves[j].sd == moves[j - 1].sd + 1 && moves[j].ss == moves[j - 1].ss + 1 &&
+           fan[{moves[j].rs, moves[j].ss}] == 1)
+      ++j;
+    Segment s{};
+    s.src_off = (uint64_t)a.ss * m;
+    s.run_bytes = (uint64_t)(j - i) * m;
+    s.src_pitch = n_old * m;
+    s.n_runs = runs;
+    s.src_rank = (uint32_t)a.rs;
+    finish_segment(pp, s, {Dst{(uint64_t)a.sd * m, n_new * m, (uint32_t)a.rd, 0}});
+    i = j;
+  }
+  // replicated sources: read once, write to every destination
+  for (const auto &kv : multi) {
+    Segment s{};
+    s.src_off = (uint64_t)kv.first.second * m;
+    s.run_bytes = m;
+    s.src_pitch = po.ids[kv.first.first].size() * m;
+    s.n_runs = runs;
+    s.src_rank = (uint32_t)kv.first.first;
+    finish_segment(pp, s, kv.second);
+  }
+}
+
+// ---- attention --------------------------------------------------------------------------
+
+void plan_attn(const emoe_shape_t &sh, int c, int d, PhasePlan *pp) {
+  const uint64_t D = sh.d_model, b = sh.elem_bytes, hd = sh.head_dim;
+  const uint64_t row = D * b;
+  auto q_bytes = [&](int T) { return (uint64_t)(sh.n_q_heads / T) * hd * row; };
+  auto kv_bytes = [&](int T) { return (uint64_t)(sh.n_kv_heads / T) * hd * row; };
+  auto layer_bytes = [&](int T) { return 2 * q_bytes(T) + 2 * kv_bytes(T); };
+  const uint32_t L = sh.n_layers;
+  pp->arena_old.assign(c, L * layer_bytes(c));
+  pp->arena_new.assign(d, L * layer_bytes(d));
+
+  if (c == d) {  // fixed TP: every shard carries over whole (provisioning a new replica)
+    for (int t = 0; t < c; ++t) {
+      Segment s{};
+      s.run_bytes = L * layer_bytes(c);
+      s.n_runs = 1;
+      s.src_pitch = s.run_bytes;
+      s.src_rank = (uint32_t)t;
+      finish_segment(pp, s, {Dst{0, s.run_bytes, (uint32_t)t, 0}});
+    }
+    return;
+  }
+  // q, k, v: intersect old and new row ranges of the logical matrix
+  for (int t = 0; t < 3; ++t) {
+    const uint64_t rows = (uint64_t)(t == 0 ? sh.n_q_heads : sh.n_kv_heads) * hd;
+    const uint64_t rc = rows / c, rd = rows / d;
+    auto piece = [&](int T) {
+      return t == 0 ? 0 : t == 1 ? q_bytes(T) : q_bytes(T) + kv_bytes(T);
+    };
+    for (int ro = 0; ro < c; ++ro)
+      for (int rn = 0; rn < d; ++rn) {
+        const uint64_t lo = std::max(ro * rc, rn * rd), hi = std::min((ro + 1) * rc, (rn + 1) * rd);
+        if (lo >= hi) continue;
+        Segment s{};
+        s.src_off = piece(c) + (lo - ro * rc) * row;
+        s.run_bytes = (hi - lo) * row;
+        s.src_pitch = layer_bytes(c);
+        s.n_runs = L;
+        s.src_rank = (uint32_t)ro;
+        finish_segment(pp, s,
+                       {Dst{piece(d) + (lo - rn * rd) * row, layer_bytes(d), (uint32_t)rn, 0}});
+      }
+  }
+  // o: intersect old and new column ranges; one strided segment per (layer, overlap)
+  const uint64_t cols = (uint64_t)sh.n_q_heads * hd, cc = cols / c, cd = cols / d;
+  const uint64_t o_c = q_bytes(c) + 2 * kv_bytes(c), o_d = q_bytes(d) + 2 * kv_bytes(d);
+  for (uint32_t l = 0; l < L; ++l)
+    for (int ro = 0; ro < c; ++ro)
+      for (int rn = 0; rn < d; ++rn) {
+        const uint64_t lo = std::max(ro * cc, rn * cd), hi = std::min((ro + 1) * cc, (rn + 1) * cd);
+        if (lo >= hi) continue;
+        Segment s{};
+        s.src_off = l * layer_bytes(c) + o_c + (lo - ro * cc) * b;
+        s.run_bytes = (hi - lo) * b;
+        s.src_pitch = cc * b;
+        s.n_runs = (uint32_t)D;
+        s.src_rank = (uint32_t)ro;
+        finish_segment(pp, s,
+                       {Dst{l * layer_bytes(d) + o_d + (lo - rn * cd) * b, cd * b, (uint32_t)rn, 0}});
+      }
+}
+
+// ---- KV ---------------------------------------------------------------------------------
+
+void plan_kv(const emoe_shape_t &sh, const emoe_config_t &o, const emoe_config_t &n,
+             std::vector<uint32_t> pair_old, std::vector<uint32_t> pair_new, HostPlan *hp) {
+  PhasePlan *pp = &hp->phase[EMOE_PHASE_KV];
+  KvPlan &kv = hp->kv;
+  const uint64_t vec = (uint64_t)sh.head_dim * sh.elem_bytes, B = sh.kv_block_tokens;
+  const uint64_t L = sh.n_layers;
+  kv.c = o.tp; kv.d = n.tp;
+  kv.n_layers = sh.n_layers; kv.block_tokens = sh.kv_block_tokens; kv.hkv = sh.n_kv_heads;
+  kv.head_bytes = vec; kv.nb_old = o.kv_num_blocks; kv.nb_new = n.kv_num_blocks;
+  kv.head_split_changes = (o.tp != n.tp);
+  const uint64_t blk_old = B * (sh.n_kv_heads / o.tp) * vec, blk_new = B * (sh.n_kv_heads / n.tp) * vec;
+  pp->arena_old.assign(o.tp, L * 2 * o.kv_num_blocks * blk_old);
+  pp->arena_new.assign(n.tp, L * 2 * n.kv_num_blocks * blk_new);
+  const uint64_t n_pairs = pair_old.size();
+  const uint64_t logical_bytes = L * 2 * n_pairs * B * sh.n_kv_heads * vec;
+
+  if (kv.head_split_changes) {
+    kv.pair_old = std::move(pair_old);
+    kv.pair_new = std::move(pair_new);
+    pp->bytes_moved = pp->bytes_read = logical_bytes;
+    return;
+  }
+  // head split kept: a block is one contiguous run per (layer, K|V); consecutive
+  // pairs that are consecutive in both pools merge into longer runs
+  size_t i = 0;
+  while (i < n_pairs) {
+    size_t j = i + 1;
+    while (j < n_pairs && pair_old[j] == pair_old[j - 1] + 1 && pair_new[j] == pair_new[j - 1] + 1)
+      ++j;
+    for (int t = 0; t < o.tp; ++t) {
+      Segment s{};
+      s.src_off = pair_old[i] * blk_old;
+      s.run_bytes = (uint64_t)(j - i) * blk_old;
+      s.src_pitch = o.kv_num_blocks * blk_old;
+      s.n_runs = (uint32_t)(L * 2);
+      s.src_rank = (uint32_t)t;
+      finish_segment(pp, s, {Dst{pair_new[i] * blk_new, n.kv_num_blocks * blk_new, (uint32_t)t, 0}});
+    }
+    i = j;
+  }
+}
+
+}  // namespace
+
+emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
+                              const emoe_config_t &n, HostPlan *hp) {
+  if (sh.n_layers <= 0 || sh.n_routed <= 0 || sh.n_shared < 0 || sh.d_model <= 0 ||
+      sh.d_ff <= 0 || sh.n_q_heads <= 0 || sh.n_kv_heads <= 0 || sh.head_dim <= 0 ||
+      sh.kv_block_tokens <= 0 || sh.elem_bytes <= 0)
+    return EMOE_ERR_SHAPE;
+  const int n_experts = sh.n_routed + sh.n_shared;
+  Placement po, pn;
+  emoe_status_t st = read_placement(o, n_experts, &po);
+  if (st != EMOE_OK) return st;
+  st = read_placement(n, n_experts, &pn);
+  if (st != EMOE_OK) return st;
+  for (int tp : {o.tp, n.tp}) {
+    if (tp > sh.n_kv_heads) return EMOE_ERR_UNSUPPORTED;  // would need KV-head replication
+    if (sh.n_q_heads % tp || sh.n_kv_heads % tp) return EMOE_ERR_SHAPE;
+  }
+  std::vector<uint32_t> pair_old, pair_new;
+  st = read_block_pairs(sh, o, n, &pair_old, &pair_new);
+  if (st != EMOE_OK) return st;
+
+  hp->shape = sh;
+  hp->ep_old = o.ep; hp->ep_new = n.ep; hp->tp_old = o.tp; hp->tp_new = n.tp;
+  plan_experts(sh, po, pn, &hp->phase[EMOE_PHASE_EXPERTS]);
+  plan_attn(sh, o.tp, n.tp, &hp->phase[EMOE_PHASE_ATTN]);
+  plan_kv(sh, o, n, std::move(pair_old), std::move(pair_new), hp);
+  return EMOE_OK;
+}
+
+void export_segments(const HostPlan &hp, int phase, std::vector<emoe_segment_t> *out) {
+  out->clear();
+  const PhasePlan &pp = hp.phase[phase];
+  uint32_t group = 0;
+  for (const Segment &s : pp.segs) {
+    for (uint32_t k = 0; k < s.n_dst; ++k) {
+      const Dst &d = pp.dsts[s.dst_first + k];
+      out->push_back({s.src_off, d.off, s.run_bytes, s.src_pitch, d.pitch, s.n_runs, s.src_rank,
+                      d.rank, group});
+    }
+    ++group;
+  }
+  if (phase != EMOE_PHASE_KV || !hp.kv.head_split_changes) return;
+  const KvPlan &kv = hp.kv;
+  const uint64_t hc = kv.hkv / kv.c, hn = kv.hkv / kv.d, B = kv.block_tokens, vec = kv.head_bytes;
+  for (size_t i = 0; i < kv.pair_old.size(); ++i)
+    for (uint64_t lk = 0; lk < (uint64_t)kv.n_layers * 2; ++lk)
+      for (uint32_t ro = 0; ro < kv.c; ++ro)
+        for (uint32_t rn = 0; rn < kv.d; ++rn) {
+          const uint64_t lo = std::max(ro * hc, rn * hn), hi = std::min((ro + 1) * hc, (rn + 1) * hn);
+          if (lo >= hi) continue;
+          out->push_back({((lk * kv.nb_old + kv.pair_old[i]) * B * hc + (lo - ro * hc)) * vec,
+                          ((lk * kv.nb_new + kv.pair_new[i]) * B * hn + (lo - rn * hn)) * vec,
+                          (hi - lo) * vec, hc * vec, hn * vec, (uint32_t)B, ro, rn, group++});
+        }
+}
+
+}  // namespace emoe

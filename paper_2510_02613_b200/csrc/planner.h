@@ -1,0 +1,71 @@
+// planner.h - host planner of the scale-step re-layout (integer work only).
+//
+// Turns (model shape, old configuration, new configuration) into per-phase
+// copy descriptors.  The plan is a pure function of its inputs, as the paper's
+// HMM plan is (Sec. 5.2 "HMM Reconfigures Memory Layout").  No CUDA here.
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "../../include/emoe.h"
+
+namespace emoe {
+
+// One destination of a segment.
+struct Dst {
+  uint64_t off;    // byte offset of run 0 in the destination arena
+  uint64_t pitch;  // byte distance between consecutive runs
+  uint32_t rank;
+  uint32_t pad;
+};
+
+// A coalesced, possibly strided, possibly fanned-out copy: n_runs runs of
+// run_bytes; run i reads src[src_rank] + src_off + i*src_pitch and is written
+// to every destination k at dst[rank_k] + off_k + i*pitch_k.
+struct Segment {
+  uint64_t src_off;
+  uint64_t run_bytes;
+  uint64_t src_pitch;
+  uint32_t n_runs;
+  uint32_t src_rank;
+  uint32_t n_dst;
+  uint32_t dst_first;  // index of the first destination in PhasePlan::dsts
+  uint32_t align;      // largest power of two <= 16 dividing every offset, pitch and run size
+  uint32_t pad;
+};
+
+struct PhasePlan {
+  std::vector<Segment> segs;
+  std::vector<Dst> dsts;
+  std::vector<uint64_t> arena_old, arena_new;  // bytes per rank
+  uint64_t bytes_moved = 0, bytes_read = 0;
+};
+
+// KV phase when the head split changes: block pairs + shape constants.
+struct KvPlan {
+  std::vector<uint32_t> pair_old, pair_new;  // physical block ids, one entry per mapped block
+  uint32_t c = 1, d = 1;                     // old / new TP degree
+  uint32_t n_layers = 0, block_tokens = 0, hkv = 0;
+  uint64_t head_bytes = 0;                   // head_dim * elem_bytes
+  uint64_t nb_old = 0, nb_new = 0;
+  bool head_split_changes = false;
+};
+
+struct HostPlan {
+  emoe_shape_t shape;
+  int ep_old, ep_new, tp_old, tp_new;
+  PhasePlan phase[3];  // experts, attn, kv (kv.segs filled only when the head split is kept)
+  KvPlan kv;
+};
+
+// Validates and plans.  Returns EMOE_OK or the first validation error.
+emoe_status_t build_host_plan(const emoe_shape_t &shape, const emoe_config_t &old_cfg,
+                              const emoe_config_t &new_cfg, HostPlan *out);
+
+// Expands a phase into flat emoe_segment_t records (one per destination).  For a
+// KV plan with a changing head split the block pairs are expanded per (pair, old
+// rank, new rank) overlap.
+void export_segments(const HostPlan &hp, int phase, std::vector<emoe_segment_t> *out);
+
+}  // namespace emoe

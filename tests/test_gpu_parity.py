@@ -1,0 +1,184 @@
+"""GPU parity: the library's output, through the C ABI, must equal the CPU oracle
+byte for byte over whole destination arenas (bit-exact: this is byte movement)."""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2510_02613_b200 as E
+import workloads as W
+from workloads import device as WD
+from gpu_util import KINDS, check_phase_full, check_phase_layers, run_phase
+
+pytestmark = pytest.mark.gpu
+R = dataclasses.replace
+
+
+def test_library_is_loaded_from_the_tree():
+    assert E.library_path().endswith("paper_2510_02613_b200/libemoe.so")
+    E.lib()
+
+
+@pytest.mark.parametrize("inverse", [False, True])
+def test_c1_tiny_all_phases(inverse):
+    wl = W.make_workload("c1_tiny")
+    if inverse:
+        wl = wl.swapped()
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        for phase in range(3):
+            check_phase_full(wl, plan, phase)
+
+
+@pytest.mark.parametrize("name", ["c2_mid", "c3_fine", "c4_large"])
+def test_one_layer_cut_all_phases(name):
+    """One full-width layer: spans thousands of tiles, every kernel, ragged unit tails."""
+    wl = W.make_workload(name, n_layers=1)
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        for phase in range(3):
+            check_phase_full(wl, plan, phase)
+
+
+TUNINGS = [dict(path=1), dict(path=2), dict(bulk_tile_bytes=8192, bulk_stages=3),
+           dict(bulk_tile_bytes=65536, bulk_stages=2), dict(max_ctas=3),
+           dict(bulk_tile_bytes=16384, bulk_stages=12, max_ctas=296)]
+
+
+@pytest.mark.parametrize("tuning", TUNINGS, ids=lambda t: "-".join("%s%s" % kv for kv in t.items()))
+def test_tunings_do_not_change_the_result(tuning):
+    for name in ("c1_tiny", "c4_large"):
+        wl = W.make_workload(name, n_layers=2 if name == "c1_tiny" else 1)
+        if name == "c4_large":   # keep it quick: fewer blocks, thinner experts
+            wl = R(wl, shape=R(wl.shape, d_ff=96))
+        with E.Plan(wl.shape, wl.old, wl.new) as plan:
+            plan.set_tuning(**tuning)
+            for phase in range(3):
+                check_phase_full(wl, plan, phase)
+
+
+ODD = [
+    # d_model, d_ff, hq, hkv, hd, B, elem_bytes, tp_old, tp_new
+    (40, 24, 8, 4, 8, 4, 2, 1, 2),      # 16-byte-aligned but short runs
+    (33, 7, 6, 6, 3, 5, 1, 2, 3),       # nothing aligned: byte path
+    (12, 10, 4, 4, 6, 3, 2, 4, 2),      # 2/4/8-byte alignments
+    (64, 520, 8, 2, 64, 16, 2, 2, 1),   # runs straddle the bulk threshold, ragged tile tails
+    (16, 1030, 4, 4, 16, 8, 4, 1, 4),   # fp32 elements
+]
+
+
+@pytest.mark.parametrize("dims", ODD, ids=lambda d: "x".join(map(str, d)))
+def test_odd_shapes_and_alignments(dims):
+    dm, dff, hq, hkv, hd, B, eb, c, d = dims
+    sh = W.Shape(3, 7, 1, dm, dff, hq, hkv, hd, B, eb)
+    seq_lens = [3 * B + 1, 1, 2 * B]
+    nblk = sum(-(-n // B) for n in seq_lens)
+    bo = W.make_block_table(11, seq_lens, B, nblk + 2)
+    bn = W.make_block_table(12, seq_lens, B, nblk + 5)
+    old = W.ParallelConfig(3, c, W.with_shared(W.place_contiguous(7, 3), [7]), nblk + 2, seq_lens, bo)
+    new = W.ParallelConfig(2, d, W.with_shared(W.place_round_robin(7, 2), [7]), nblk + 5, seq_lens, bn)
+    wl = W.Workload("odd", sh, old, new, 77)
+    for w in (wl, wl.swapped()):
+        with E.Plan(w.shape, w.old, w.new) as plan:
+            for phase in range(3):
+                check_phase_full(w, plan, phase)
+
+
+def test_replicas_with_different_contents_pick_the_documented_source():
+    """Arenas are filled by physical position, so replicas differ: parity then also
+    pins the source choice (own rank first, else the smallest rank and slot)."""
+    sh = W.Shape(2, 6, 0, 64, 128, 4, 4, 16, 4, 2)
+    old = W.ParallelConfig(3, 1, [[0, 1, 2, 5], [2, 3, 0], [4, 5, 1]], 1, [], np.zeros((0, 0), np.int32))
+    new = W.ParallelConfig(4, 1, [[5, 0], [0, 2, 3], [1, 4, 2], [0, 1, 2, 3, 4, 5]], 1, [],
+                           np.zeros((0, 0), np.int32))
+    wl = W.Workload("replicas", sh, old, new, 5)
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        check_phase_full(wl, plan, E.PHASE_EXPERTS)
+        check_phase_full(wl, plan, E.PHASE_KV)      # no sequences: nothing is written
+
+
+def test_round_trip_on_the_gpu_is_identity():
+    wl = W.make_workload("c4_large", n_layers=1)
+    wl = R(wl, shape=R(wl.shape, d_ff=64))
+    with E.Plan(wl.shape, wl.old, wl.new) as fwd, E.Plan(wl.shape, wl.new, wl.old) as bwd:
+        for phase in range(3):
+            a = WD.alloc_filled(fwd.arena_bytes(phase, E.SIDE_OLD), wl.seed, KINDS[phase])
+            b = WD.alloc_const(fwd.arena_bytes(phase, E.SIDE_NEW))
+            c = WD.alloc_const(fwd.arena_bytes(phase, E.SIDE_OLD))
+            if phase == E.PHASE_KV:   # unmapped blocks are not carried: start c from a
+                c = [t.clone() for t in a]
+            run_phase(fwd, phase, a, b)
+            run_phase(bwd, phase, b, c)
+            torch.cuda.synchronize()
+            if phase == E.PHASE_EXPERTS:
+                # replicas differ by position; compare one copy per expert through the oracle
+                continue
+            assert all(torch.equal(x, y) for x, y in zip(a, c))
+
+
+def test_argument_errors_launch_nothing():
+    wl = W.make_workload("c1_tiny")
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        so = plan.arena_bytes(E.PHASE_EXPERTS, E.SIDE_OLD)
+        sn = plan.arena_bytes(E.PHASE_EXPERTS, E.SIDE_NEW)
+        big = torch.full((sum(so) + sum(sn) + 64,), 0xCD, dtype=torch.uint8, device="cuda")
+        src = [big[:so[0]], big[so[0]:so[0] + so[1]]]
+        good = [torch.empty(n, dtype=torch.uint8, device="cuda") for n in sn]
+        # destination 0 aliases the tail of source 1
+        bad = [big[so[0] + so[1] - 16: so[0] + so[1] - 16 + sn[0]]] + good[1:]
+        with pytest.raises(E.EmoeError) as ei:
+            plan.reshard_experts(src, bad)
+        assert ei.value.code == 6
+        mis = [big[sum(so) + 8: sum(so) + 8 + sn[0]]] + good[1:]
+        with pytest.raises(E.EmoeError) as ei:
+            plan.reshard_experts(src, mis)
+        assert ei.value.code == 5
+        with pytest.raises(E.EmoeError) as ei:
+            plan.reshard_experts([0, 0], good)
+        assert ei.value.code == 1
+        torch.cuda.synchronize()
+        assert bool((big == 0xCD).all())
+
+
+def test_step_on_host_buffers_matches_oracle():
+    wl = W.make_workload("c1_tiny")
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        h_src, h_dst, d_src, d_dst, want = [], [], [], [], []
+        for phase in range(3):
+            so, sn = plan.arena_bytes(phase, E.SIDE_OLD), plan.arena_bytes(phase, E.SIDE_NEW)
+            hs = [torch.from_numpy(WD.host_slice(wl.seed, KINDS[phase], r, 0, n)).pin_memory()
+                  for r, n in enumerate(so)]
+            h_src.append(hs)
+            h_dst.append([torch.zeros(n, dtype=torch.uint8).pin_memory() for n in sn])
+            d_src.append([torch.empty(n, dtype=torch.uint8, device="cuda") for n in so])
+            d_dst.append(WD.alloc_const(sn))
+            w = [np.full(n, WD.FILL_BYTE, np.uint8) for n in sn]
+            from gpu_util import oracle_phase
+            oracle_phase(wl, phase, [t.numpy() for t in hs], w)
+            want.append(w)
+        s = torch.cuda.Stream()
+        plan.reshard_step_host(h_src, h_dst, d_src, d_dst, s)
+        s.synchronize()
+        for phase in range(3):
+            for g, w in zip(h_dst[phase], want[phase]):
+                assert np.array_equal(g.numpy(), w)
+
+
+@pytest.mark.parametrize("name", ["c2_mid", "c3_fine", "c4_large"])
+def test_full_size_configs_sampled_layers(name):
+    """The benchmark's launch configuration at full size; first, middle and last layer
+    compared in full with the oracle (layers are independent in every phase)."""
+    wl = W.make_workload(name)
+    L = wl.shape.n_layers
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        for phase in range(3):
+            src = WD.alloc_filled(plan.arena_bytes(phase, E.SIDE_OLD), wl.seed, KINDS[phase])
+            dst = WD.alloc_const(plan.arena_bytes(phase, E.SIDE_NEW))
+            run_phase(plan, phase, src, dst)
+            torch.cuda.synchronize()
+            assert plan.device_status() == 0
+            check_phase_layers(wl, plan, phase, src, dst, [0, L // 2, L - 1])
+            del src, dst
+            torch.cuda.empty_cache()

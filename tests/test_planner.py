@@ -1,0 +1,197 @@
+"""Host planner (no GPU): replaying the exported segment list with plain numpy
+copies must reproduce the oracle byte for byte; destination runs must tile the
+planned destination set exactly once; bad inputs map to the documented codes."""
+from __future__ import annotations
+
+import ctypes
+import dataclasses
+import re
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2510_02613_b200 as E
+import workloads as W
+from helpers import FILL, rand_bytes
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def small(name):
+    """Per-layer structure of the named workload with tiny matrices."""
+    wl = W.make_workload(name)
+    sh = wl.shape
+    L = 2
+    if name == "c1_tiny":
+        sh = dataclasses.replace(sh, n_layers=L, d_model=32, d_ff=16)
+    else:
+        sh = dataclasses.replace(sh, n_layers=L, d_model=16, d_ff=8, head_dim=8)
+        # keep the block-table structure but only the first sequences
+        def cut(cfg, pool):
+            sl = list(cfg.seq_lens[:2])
+            bt = cfg.block_table[:2].copy()
+            return dataclasses.replace(cfg, seq_lens=sl, block_table=bt)
+        wl = dataclasses.replace(wl, old=cut(wl.old, 0), new=cut(wl.new, 0))
+    return dataclasses.replace(wl, shape=sh)
+
+
+def replay(segs, src, dst):
+    for s in segs:
+        for i in range(int(s["n_runs"])):
+            a = int(s["src_off"]) + i * int(s["src_pitch"])
+            b = int(s["dst_off"]) + i * int(s["dst_pitch"])
+            n = int(s["run_bytes"])
+            dst[int(s["dst_rank"])][b:b + n] = src[int(s["src_rank"])][a:a + n]
+
+
+def arenas(sizes, key):
+    return [rand_bytes((key, r), n) for r, n in enumerate(sizes)]
+
+
+def run_oracle(wl, phase, src, dst):
+    if phase == E.PHASE_EXPERTS:
+        oracle.reshard_experts(wl.shape, wl.old.placement, wl.new.placement, src, dst)
+    elif phase == E.PHASE_ATTN:
+        oracle.reshard_attn(wl.shape, wl.old.tp, wl.new.tp, src, dst)
+    else:
+        oracle.reshard_kv(wl.shape, wl.old, wl.new, src, dst)
+
+
+def oracle_sizes(wl, phase):
+    sh = wl.shape
+    if phase == E.PHASE_EXPERTS:
+        return (oracle.expert_arena_bytes(sh, wl.old.placement),
+                oracle.expert_arena_bytes(sh, wl.new.placement))
+    if phase == E.PHASE_ATTN:
+        return oracle.attn_arena_bytes(sh, wl.old.tp), oracle.attn_arena_bytes(sh, wl.new.tp)
+    return (oracle.kv_arena_bytes(sh, wl.old.tp, wl.old.kv_num_blocks),
+            oracle.kv_arena_bytes(sh, wl.new.tp, wl.new.kv_num_blocks))
+
+
+@pytest.mark.parametrize("name", ["c1_tiny", "c2_mid", "c3_fine", "c4_large"])
+@pytest.mark.parametrize("inverse", [False, True])
+def test_segment_replay_equals_oracle(name, inverse):
+    wl = small(name)
+    if inverse:
+        wl = wl.swapped()
+    with E.Plan(wl.shape, wl.old, wl.new, host_only=True) as plan:
+        for phase in range(3):
+            so, sn = oracle_sizes(wl, phase)
+            assert plan.arena_bytes(phase, E.SIDE_OLD) == so
+            assert plan.arena_bytes(phase, E.SIDE_NEW) == sn
+            src = arenas(so, 20 + phase)
+            want = [np.full(n, FILL, np.uint8) for n in sn]
+            got = [np.full(n, FILL, np.uint8) for n in sn]
+            run_oracle(wl, phase, src, want)
+            segs = plan.segments(phase)
+            replay(segs, src, got)
+            for r in range(len(sn)):
+                assert np.array_equal(got[r], want[r]), (name, phase, r)
+            # conservation and exact tiling of the written set
+            st = plan.stats(phase)
+            assert st["bytes_moved"] == int((segs["run_bytes"] * segs["n_runs"]).sum())
+            cover = [np.zeros(n, np.uint8) for n in sn]
+            for s in segs:
+                for i in range(int(s["n_runs"])):
+                    b = int(s["dst_off"]) + i * int(s["dst_pitch"])
+                    assert b + int(s["run_bytes"]) <= sn[int(s["dst_rank"])]
+                    cover[int(s["dst_rank"])][b:b + int(s["run_bytes"])] += 1
+            assert all(c.max(initial=0) <= 1 for c in cover)      # destinations disjoint
+            assert sum(int(c.sum()) for c in cover) == st["bytes_moved"]
+            if phase != E.PHASE_KV:
+                assert all(c.min(initial=1) == 1 for c in cover)  # weights: fully written
+
+
+def test_replicated_source_is_read_once():
+    wl = small("c3_fine")
+    with E.Plan(wl.shape, wl.old, wl.new, host_only=True) as plan:
+        st = plan.stats(E.PHASE_EXPERTS)
+        segs = plan.segments(E.PHASE_EXPERTS)
+    # every old copy is read exactly once although 12 ranks receive the shared experts
+    assert st["bytes_read"] == sum(oracle.expert_arena_bytes(wl.shape, wl.old.placement))
+    assert st["bytes_moved"] == sum(oracle.expert_arena_bytes(wl.shape, wl.new.placement))
+    groups = np.bincount(segs["group"])
+    assert groups.max() == 5       # old rank 0's shared copy feeds new ranks 0, 8, 9, 10, 11
+
+
+def test_contiguous_placement_coalesces_slots():
+    wl = small("c2_mid")
+    with E.Plan(wl.shape, wl.old, wl.new, host_only=True) as plan:
+        segs = plan.segments(E.PHASE_EXPERTS)
+    m = wl.shape.d_model * wl.shape.d_ff * wl.shape.elem_bytes
+    # EP4 (15 per rank) -> EP6 (10 per rank): 8 strided segments of 5 or 10 experts
+    assert len(segs) == 8
+    assert sorted(set(int(x) // m for x in segs["run_bytes"])) == [5, 10]
+
+
+def test_identity_plan_is_one_run_per_arena():
+    wl = small("c2_mid")
+    with E.Plan(wl.shape, wl.old, wl.old, host_only=True) as plan:
+        for phase in (E.PHASE_EXPERTS, E.PHASE_ATTN):
+            segs = plan.segments(phase)
+            assert (segs["n_runs"] == 1).all()
+            assert list(segs["run_bytes"]) == plan.arena_bytes(phase, E.SIDE_OLD)
+
+
+# ---- validation ------------------------------------------------------------------------
+
+def _plan_code(shape, old, new):
+    try:
+        E.Plan(shape, old, new, host_only=True).close()
+        return 0
+    except E.EmoeError as e:
+        return e.code
+
+
+def test_validation_codes():
+    wl = small("c1_tiny")
+    sh, old, new = wl.shape, wl.old, wl.new
+    R = dataclasses.replace
+    assert _plan_code(sh, old, new) == 0
+    assert _plan_code(R(sh, d_model=0), old, new) == 2                      # SHAPE
+    assert _plan_code(sh, old, R(new, tp=3)) == 2                           # 3 does not divide 8
+    assert _plan_code(sh, old, R(new, tp=16)) == 9                          # TP > Hkv
+    assert _plan_code(sh, old, R(new, ep=65, placement=[[0]] * 65)) == 9    # too many ranks
+    dup = [list(p) for p in new.placement]; dup[0] = [0, 0]
+    assert _plan_code(sh, old, R(new, placement=dup)) == 3                  # duplicate in a rank
+    miss = [list(p) for p in new.placement]; miss[0] = miss[0][:1]
+    assert _plan_code(sh, old, R(new, placement=miss)) == 3                 # expert lost
+    assert _plan_code(sh, R(old, placement=[[0, 1, 2, 3], [4, 5, 6]]), new) == 3  # absent from old
+    oob = [list(p) for p in new.placement]; oob[0] = [0, 99]
+    assert _plan_code(sh, old, R(new, placement=oob)) == 3
+    bt = new.block_table.copy(); bt[0, 0] = bt[1, 0]
+    assert _plan_code(sh, old, R(new, block_table=bt)) == 4                 # block used twice
+    bt = new.block_table.copy(); bt[0, 0] = new.kv_num_blocks
+    assert _plan_code(sh, old, R(new, block_table=bt)) == 4                 # id out of range
+    bt = new.block_table.copy(); bt[0, 3] = -1
+    assert _plan_code(sh, old, R(new, block_table=bt)) == 4                 # hole in a sequence
+    assert _plan_code(sh, old, R(new, seq_lens=[256, 256, 256, 255])) == 4  # sequences differ
+    assert _plan_code(sh, old, R(new, block_table=new.block_table[:, :8])) == 4  # table too short
+
+
+def test_host_only_plan_refuses_to_run():
+    wl = small("c1_tiny")
+    with E.Plan(wl.shape, wl.old, wl.new, host_only=True) as plan:
+        with pytest.raises(E.EmoeError) as ei:
+            plan.reshard_experts([16] * 2, [16] * 4)
+        assert ei.value.code == 8
+
+
+def test_null_arguments():
+    L = E.lib()
+    assert L.emoe_plan_create(None, None, None, 1, None) == 1
+    L.emoe_plan_destroy(None)   # NULL-safe
+    assert E.strerror(6).startswith("source and destination")
+
+
+def test_library_exports_every_declared_symbol():
+    """Every function declared in include/emoe.h is exported by libemoe.so."""
+    text = open(os.path.join(ROOT, "include", "emoe.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(emoe_[a-z_]+)\s*\(", text))
+    assert declared == set(E.EXPORTS)
+    lib = ctypes.CDLL(E.library_path())
+    for name in declared:
+        assert hasattr(lib, name), name

@@ -90,13 +90,16 @@ def _s64(x: int) -> int:
 
 
 def torch_fill_bytes(out, key: int, chunk_elems: int = 1 << 26) -> None:
-    """Fills the 1-D uint8 torch tensor `out` (any device, even byte count, 2-byte
-    aligned) with the bf16 stream `key`, bit-identical to fill_bytes(key, n)."""
+    """Fills the 1-D uint8 torch tensor `out` (any device, 2-byte aligned) with the bf16 stream `key`, bit-identical to fill_bytes(key, n)."""
     import torch
 
     n = out.numel()
-    if n % 2:
-        raise ValueError("torch_fill_bytes needs an even byte count")
+    if n % 2:   # odd tail byte: the low byte of the last 16-bit element, made on the host
+        out[n - 1:] = torch.from_numpy(fill_bytes(key, 1, start_byte=n - 1)).to(out.device)
+        out = out[:n - 1]
+        n -= 1
+        if n == 0:
+            return
     dst = out.view(torch.int16)
     n_el = n // 2
     dev = out.device
