@@ -65,7 +65,8 @@ typedef enum {
   EMOE_ERR_OOM = 7,          /* host or device allocation for the plan failed         */
   EMOE_ERR_CUDA = 8,         /* a CUDA runtime call failed (no device, bad stream...) */
   EMOE_ERR_UNSUPPORTED = 9,  /* TP > n_kv_heads, more ranks than EMOE_MAX_RANKS, ...  */
-  EMOE_ERR_DEVICE_TIMEOUT = 10 /* a bounded device-side wait expired                  */
+  EMOE_ERR_DEVICE_TIMEOUT = 10, /* a bounded device-side wait expired                 */
+  EMOE_ERR_TOO_LARGE = 11    /* the problem exceeds a fixed capacity of the entry point */
 } emoe_status_t;
 
 /* Model shape.  All fields must be > 0 except n_shared (>= 0). */
@@ -191,6 +192,46 @@ emoe_status_t emoe_reshard_step_host(const emoe_plan_t *plan, const void *const 
                                      void *const *const h_dst[3],
                                      void *const *const d_src[3], void *const *const d_dst[3],
                                      void *cuda_stream);
+
+/*
+ * emoe_reshard_kv_static - the KV head re-split and re-paging of
+ * emoe_reshard_kv for callers that must not allocate device memory.  (The
+ * paper has no counterpart: this entry point exists for integration only.)
+ *
+ * Who needs it: a serving process whose memory daemon has already claimed
+ * all of HBM for weights and KV pools, so that a cudaMalloc at scaling time
+ * would fail or evict something; a caller inside a latency-critical section
+ * where the implicit device synchronisation of cudaMalloc / cudaFree is not
+ * acceptable; code running under an allocator hook that forbids raw CUDA
+ * allocations.  Such a caller creates its plan with EMOE_PLAN_HOST_ONLY
+ * (which makes no CUDA call at all) and uses this entry point, which calls
+ * no cudaMalloc, no cudaFree and no allocating library routine.
+ *
+ * The block-pair list the kernel reads (8 bytes per mapped block) is kept in
+ * a fixed array inside the library image instead: EMOE_STATIC_KV_MAX_PAIRS
+ * pairs = 512 KiB, resident on every GPU that loads libemoe.so until the
+ * process exits.  A plan with more mapped blocks is rejected with
+ * EMOE_ERR_TOO_LARGE before anything is enqueued.
+ *
+ * plan: any plan, host-only or not.  src / dst / cuda_stream: exactly as for
+ * emoe_reshard_kv (HOST arrays of tp_old / tp_new DEVICE pointers), with the
+ * same alignment and no-overlap rules; the result is byte-identical to
+ * emoe_reshard_kv, whether or not the TP degree changes.
+ *
+ * Each call first copies the plan's pair list into the fixed array on
+ * cuda_stream, then launches the kernel on the same stream.  All calls on a
+ * device share that one array, and it keeps the previous call's list: two
+ * calls whose GPU work can overlap (different streams without an ordering
+ * between them) race on it and must be serialised by the caller.  Nothing in
+ * the array has to start at zero; each call overwrites the prefix it reads.
+ *
+ * The first call on each device looks up the array's device address
+ * (one-time set-up, with that device current).  Make that first call outside
+ * any stream capture.
+ */
+#define EMOE_STATIC_KV_MAX_PAIRS 65536
+emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *plan, const void *const *src,
+                                     void *const *dst, void *cuda_stream);
 
 /* emoe_plan_destroy - frees host state and device descriptor buffers.
  * NULL-safe.  No kernel using the plan may still be in flight. */

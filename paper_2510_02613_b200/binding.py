@@ -57,6 +57,7 @@ SEGMENT_DTYPE = np.dtype([("src_off", "<u8"), ("dst_off", "<u8"), ("run_bytes", 
                           ("src_rank", "<u4"), ("dst_rank", "<u4"), ("group", "<u4")])
 
 EXPORTS = ("emoe_plan_create", "emoe_reshard_experts", "emoe_reshard_attn", "emoe_reshard_kv",
+           "emoe_reshard_kv_static",
            "emoe_reshard_step_host", "emoe_plan_destroy", "emoe_plan_num_ranks",
            "emoe_plan_arena_bytes", "emoe_plan_stats", "emoe_plan_num_launches", "emoe_plan_segments",
            "emoe_plan_device_status", "emoe_plan_set_tuning", "emoe_strerror")
@@ -85,7 +86,8 @@ def lib() -> ctypes.CDLL:
     L.emoe_plan_create.restype = _i32
     L.emoe_plan_create.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Config),
                                    ctypes.POINTER(_Config), _u32, ctypes.POINTER(_vp)]
-    for name in ("emoe_reshard_experts", "emoe_reshard_attn", "emoe_reshard_kv"):
+    for name in ("emoe_reshard_experts", "emoe_reshard_attn", "emoe_reshard_kv",
+                 "emoe_reshard_kv_static"):
         f = getattr(L, name)
         f.restype = _i32
         f.argtypes = [_vp, PP, PP, _vp]
@@ -259,6 +261,15 @@ class Plan:
 
     def reshard_kv(self, src, dst, stream=None) -> None:
         self._run(lib().emoe_reshard_kv, src, dst, stream)
+
+    def reshard_kv_static(self, src, dst, stream=None) -> None:
+        """emoe_reshard_kv for callers that may not allocate device memory (a process
+        whose HBM is fully owned by a memory daemon, a section that cannot afford the
+        implicit synchronisation of cudaMalloc).  Works on host-only plans; the block
+        pair list goes into a fixed 512 KiB array of the library image, shared by all
+        calls on the device, so calls that may overlap on the GPU must be serialised.
+        Make the first call on a device outside stream capture."""
+        self._run(lib().emoe_reshard_kv_static, src, dst, stream)
 
     def reshard_step_host(self, h_src, h_dst, d_src, d_dst, stream=None) -> None:
         """Each argument: three lists (experts, attn, kv) of per-rank buffers."""

@@ -243,6 +243,37 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *p, const void *const *src, void
                                     (cudaStream_t)stream));
 }
 
+emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *p, const void *const *src, void *const *dst,
+                                     void *stream) {
+  if (!p || !src || !dst) return EMOE_ERR_INVALID_ARG;
+  const KvPlan &kv = p->hp.kv;
+  const std::vector<uint32_t> *pair_old = &kv.pair_old, *pair_new = &kv.pair_new;
+  if (pair_old->size() > EMOE_STATIC_KV_MAX_PAIRS) return EMOE_ERR_TOO_LARGE;
+  // the same argument checks as emoe_reshard_kv, but a host-only plan is welcome here
+  const PhasePlan &pp = p->hp.phase[EMOE_PHASE_KV];
+  RankPtrs ptrs;
+  std::memset(&ptrs, 0, sizeof(ptrs));
+  for (int r = 0; r < p->hp.tp_old; ++r) {
+    if (pp.arena_old[r] && !src[r]) return EMOE_ERR_INVALID_ARG;
+    if ((uintptr_t)src[r] % 16) return EMOE_ERR_ALIGNMENT;
+    ptrs.src[r] = (const uint8_t *)src[r];
+  }
+  for (int r = 0; r < p->hp.tp_new; ++r) {
+    if (pp.arena_new[r] && !dst[r]) return EMOE_ERR_INVALID_ARG;
+    if ((uintptr_t)dst[r] % 16) return EMOE_ERR_ALIGNMENT;
+    ptrs.dst[r] = (uint8_t *)dst[r];
+  }
+  for (int a = 0; a < p->hp.tp_old; ++a)
+    for (int b = 0; b < p->hp.tp_new; ++b) {
+      const uintptr_t s0 = (uintptr_t)src[a], s1 = s0 + pp.arena_old[a];
+      const uintptr_t d0 = (uintptr_t)dst[b], d1 = d0 + pp.arena_new[b];
+      if (s0 < d1 && d0 < s1) return EMOE_ERR_OVERLAP;
+    }
+  KvTables t{nullptr, nullptr, (uint32_t)pair_old->size(), kv.n_layers * 2, kv.block_tokens,
+             kv.hkv, kv.hkv / kv.c, kv.hkv / kv.d, (uint32_t)kv.head_bytes, kv.nb_old, kv.nb_new};
+  return launch_kv_copy_static(t, pair_old->data(), pair_new->data(), ptrs, (cudaStream_t)stream);
+}
+
 emoe_status_t emoe_reshard_step_host(const emoe_plan_t *p, const void *const *const h_src[3],
                                      void *const *const h_dst[3], void *const *const d_src[3],
                                      void *const *const d_dst[3], void *stream) {
@@ -377,6 +408,7 @@ const char *emoe_strerror(emoe_status_t s) {
     case EMOE_ERR_CUDA: return "CUDA error, or a host-only plan was asked to run";
     case EMOE_ERR_UNSUPPORTED: return "unsupported configuration";
     case EMOE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case EMOE_ERR_TOO_LARGE: return "problem exceeds the fixed capacity of this entry point";
   }
   return "unknown status";
 }

@@ -17,6 +17,8 @@
 // flight land, and returns.
 #include "kernels.h"
 
+#include <mutex>
+
 namespace emoe {
 namespace {
 
@@ -425,6 +427,71 @@ cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, ui
   else if (hb % 2 == 0) kv_direct_kernel<uint16_t><<<grid, 256, 0, stream>>>(p);
   else kv_direct_kernel<uint8_t><<<grid, 256, 0, stream>>>(p);
   return cudaGetLastError();
+}
+
+// ---- KV re-split without any allocation ---------------------------------------------------
+//
+// For callers that cannot call cudaMalloc (all of HBM already owned by a memory daemon,
+// or no tolerance for the implicit synchronisation of an allocation): the block-pair
+// list lives in this fixed array of the library image, old ids in the first half, new
+// ids in the second.  Every GPU that loads the library holds these 512 KiB until exit.
+// In host code the symbol below is only a handle; its device address is looked up once
+// per device with cudaGetSymbolAddress and handed to the kernel as an ordinary pointer.
+static __device__ __align__(256) uint32_t g_kv_static_pairs[2 * EMOE_STATIC_KV_MAX_PAIRS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+uint32_t *g_static_ptr[kMaxDevices] = {};
+int g_static_sms[kMaxDevices] = {};
+}  // namespace
+
+emoe_status_t launch_kv_copy_static(const KvTables &shape_only, const uint32_t *pair_old,
+                                    const uint32_t *pair_new, const RankPtrs &ptrs,
+                                    cudaStream_t stream) {
+  const uint32_t n = shape_only.n_pairs;
+  if (n > EMOE_STATIC_KV_MAX_PAIRS) return EMOE_ERR_TOO_LARGE;
+  if (n == 0 || shape_only.n_lk == 0) return EMOE_OK;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    (void)cudaGetLastError();
+    return EMOE_ERR_CUDA;
+  }
+  uint32_t *scratch = nullptr;
+  int sms = 0;
+  {
+    // one-time set-up per device, with that device current
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+      void *p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_kv_static_pairs) != cudaSuccess || !p ||
+          cudaDeviceGetAttribute(&g_static_sms[dev], cudaDevAttrMultiProcessorCount, dev) !=
+              cudaSuccess) {
+        (void)cudaGetLastError();
+        return EMOE_ERR_CUDA;
+      }
+      g_static_ptr[dev] = static_cast<uint32_t *>(p);
+    }
+    scratch = g_static_ptr[dev];
+    sms = g_static_sms[dev];
+  }
+  uint32_t *d_old = scratch, *d_new = scratch + EMOE_STATIC_KV_MAX_PAIRS;
+  if (cudaMemcpyAsync(d_old, pair_old, n * sizeof(uint32_t), cudaMemcpyHostToDevice, stream) !=
+          cudaSuccess ||
+      cudaMemcpyAsync(d_new, pair_new, n * sizeof(uint32_t), cudaMemcpyHostToDevice, stream) !=
+          cudaSuccess) {
+    (void)cudaGetLastError();
+    return EMOE_ERR_CUDA;
+  }
+  KvTables t = shape_only;
+  t.pair_old = d_old;
+  t.pair_new = d_new;
+  const cudaError_t e = launch_kv_copy(t, ptrs, 1, (uint32_t)sms * 8, nullptr, stream);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return EMOE_ERR_CUDA;
+  }
+  return EMOE_OK;
 }
 
 }  // namespace emoe

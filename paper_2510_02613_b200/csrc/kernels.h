@@ -59,6 +59,13 @@ cudaError_t launch_vec_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t t
 cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, uint32_t grid,
                            int *status, cudaStream_t stream);
 
+// KV head re-split with its block-pair list in a fixed __device__ array of the library
+// image (no allocation).  pair_old / pair_new: host arrays of n_pairs ids.  Returns
+// EMOE_OK, EMOE_ERR_TOO_LARGE (n_pairs > EMOE_STATIC_KV_MAX_PAIRS) or EMOE_ERR_CUDA.
+emoe_status_t launch_kv_copy_static(const KvTables &shape_only, const uint32_t *pair_old,
+                                    const uint32_t *pair_new, const RankPtrs &ptrs,
+                                    cudaStream_t stream);
+
 // One-time per-process kernel attribute setup (dynamic shared memory opt-in).
 cudaError_t kernels_init();
 

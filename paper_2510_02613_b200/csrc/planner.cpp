@@ -242,9 +242,9 @@ void plan_kv(const emoe_shape_t &sh, const emoe_config_t &o, const emoe_config_t
   const uint64_t n_pairs = pair_old.size();
   const uint64_t logical_bytes = L * 2 * n_pairs * B * sh.n_kv_heads * vec;
 
+  kv.pair_old = pair_old;  // kept in both cases: the fixed-scratch entry point reads them
+  kv.pair_new = pair_new;
   if (kv.head_split_changes) {
-    kv.pair_old = std::move(pair_old);
-    kv.pair_new = std::move(pair_new);
     pp->bytes_moved = pp->bytes_read = logical_bytes;
     return;
   }
