@@ -321,7 +321,7 @@ def run_overlap(torch, E, plan, wl, src, dst, peak, budgets=(0, 96, 48)):
                   if r0.elapsed_time(evs[i + 1]) < t_end and r0.elapsed_time(evs[i]) > 0]
         during_us = (statistics.mean(inside) / n_graph_steps * 1e3) if inside else None
         out["runs"].append({
-            "max_ctas": budget or "all SMs",
+            "max_ctas": budget or "default",
             "reshard_alone_ms": round(alone_ms, 3),
             "reshard_alone_gbs": round(2 * moved / alone_ms / 1e6, 1),
             "reshard_overlapped_ms": round(both_ms, 3),
@@ -387,6 +387,9 @@ def main():
     ap.add_argument("--only-main", action="store_true",
                     help="skip the other configs, the overlap case, e2e and the CPU baseline")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--layers", type=int, default=None,
+                    help="cut the workload to this many layers (for small profiler captures "
+                         "only: the result is then not the named configuration)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "emoe" else args.warmup
 
@@ -413,7 +416,7 @@ def main():
     peak, peak_kind = measured_peak()
     stream = torch.cuda.Stream()
 
-    wl, plan, src, dst, plan_ms = setup(args.workload, torch, E, W, WD)
+    wl, plan, src, dst, plan_ms = setup(args.workload, torch, E, W, WD, n_layers=args.layers)
     sampler = ClockSampler(local)
     sampler.start()
     total_ms, phase_ms = time_steps(torch, plan, src, dst, args.steps, args.warmup, stream, barrier)
@@ -444,7 +447,9 @@ def main():
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 4),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
             "data": "synthetic",
-            "config": {"workload": wl.name, "reconfig": wl.notes, "parallelism": "replicas",
+            "config": {"workload": wl.name if args.layers is None
+                       else "%s cut to %d layers" % (wl.name, args.layers),
+                       "reconfig": wl.notes, "parallelism": "replicas",
                        "l2": "inputs_larger_than_l2", "value_convention": "2 x bytes moved / time",
                        "scale_step_ms": rep["scale_step_ms"],
                        "pct_of_nominal_8000": rep["pct_of_nominal_8000"],

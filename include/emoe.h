@@ -286,7 +286,9 @@ typedef struct {
   int32_t path;            /* 0 default routing, 1 force the vector kernel for all  */
                            /* segments, 2 force the bulk kernel where aligned       */
   int32_t kv_mode;         /* 0 default, 1 direct, 2 staged through shared memory   */
-  int32_t reserved[3];
+  int32_t bulk_hints;      /* 0 default, 1 none, 2 loads evict-first in L2, 3 stores */
+                           /* evict-first, 4 both                                   */
+  int32_t reserved[2];
 } emoe_tuning_t;
 
 /* Replaces the plan's launch tuning.  Not thread-safe against reshard calls

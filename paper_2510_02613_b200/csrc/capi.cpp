@@ -16,6 +16,8 @@ namespace {
 
 constexpr uint32_t kUnitTiles = 8;
 constexpr uint32_t kDefaultBulkTile = 32768, kDefaultBulkStages = 6;
+constexpr uint32_t kDefaultHints = 0;
+constexpr uint32_t kDefaultBulkCtas = 74;  // measured optimum on B200: half the SMs, deep rings
 constexpr uint32_t kVecTile = 16384;
 constexpr uint64_t kBulkMinRun = 16384;  // shorter runs go to the vector kernel
 
@@ -146,14 +148,21 @@ emoe_status_t check_arenas(const emoe_plan *p, int phase, const void *const *src
   return EMOE_OK;
 }
 
+uint32_t bulk_budget(const emoe_plan *p) {
+  if (p->tuning.max_ctas > 0) return (uint32_t)p->tuning.max_ctas;
+  return kDefaultBulkCtas < (uint32_t)p->sm_count ? kDefaultBulkCtas : (uint32_t)p->sm_count;
+}
+
 uint32_t cta_budget(const emoe_plan *p) {
   return p->tuning.max_ctas > 0 ? (uint32_t)p->tuning.max_ctas : (uint32_t)p->sm_count;
 }
 
 emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, cudaStream_t st) {
   const DevPhase &dp = p->dev[phase];
+  const BulkConfig bc{bulk_tile(p), bulk_stages(p),
+                      p->tuning.bulk_hints > 0 ? (uint32_t)p->tuning.bulk_hints - 1 : kDefaultHints};
   cudaError_t e = launch_bulk_copy({dp.d_segs, dp.d_dsts, dp.d_bulk_units, (uint32_t)dp.bulk_units.size()},
-                                   ptrs, bulk_tile(p), bulk_stages(p), cta_budget(p), p->d_status, st);
+                                   ptrs, bc, bulk_budget(p), p->d_status, st);
   if (e != cudaSuccess) return cuda_status(e);
   e = launch_vec_copy({dp.d_segs, dp.d_dsts, dp.d_vec_units, (uint32_t)dp.vec_units.size()}, ptrs,
                       kVecTile, cta_budget(p) * 8, st);
@@ -374,13 +383,15 @@ emoe_status_t emoe_plan_device_status(const emoe_plan_t *p, int32_t *status) {
 emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
   if (!p || !t) return EMOE_ERR_INVALID_ARG;
   if (t->max_ctas < 0 || t->bulk_tile_bytes < 0 || t->bulk_stages < 0 || t->path < 0 ||
-      t->path > 2 || t->kv_mode < 0 || t->kv_mode > 2)
+      t->path > 2 || t->kv_mode < 0 || t->kv_mode > 2 || t->bulk_hints < 0 ||
+      t->bulk_hints > 4)
     return EMOE_ERR_INVALID_ARG;
   if (t->bulk_tile_bytes && (t->bulk_tile_bytes % 128 || t->bulk_tile_bytes < 1024))
     return EMOE_ERR_INVALID_ARG;
   const uint32_t tile = t->bulk_tile_bytes ? t->bulk_tile_bytes : kDefaultBulkTile;
   const uint32_t stages = t->bulk_stages ? t->bulk_stages : kDefaultBulkStages;
-  if (stages < 2 || stages > 16 || (uint64_t)tile * stages > 200 * 1024) return EMOE_ERR_INVALID_ARG;
+  if (stages < 2 || stages > 16 || bulk_smem_bytes(tile, stages) > bulk_smem_limit())
+    return EMOE_ERR_INVALID_ARG;
   p->tuning = *t;
   emoe_status_t st = EMOE_OK;
   try {

@@ -67,6 +67,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
   }
 }
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes,
                                           uint32_t bar) {
   asm volatile(
@@ -74,9 +79,23 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, ui
       ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar)
       : "memory");
 }
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, const void *src, uint32_t bytes,
+                                               uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1], %2, [%3], %4;"
+      ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+      : "memory");
+}
 __device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_t bytes) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
                "r"(src_smem), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_store_hint(void *dst, uint32_t src_smem, uint32_t bytes,
+                                                uint64_t pol) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+               ::"l"(dst), "r"(src_smem), "r"(bytes), "l"(pol)
                : "memory");
 }
 __device__ __forceinline__ void bulk_commit() {
@@ -101,6 +120,7 @@ struct TileInfo {  // producer -> consumer, one per stage
 struct BulkParams {
   SegTables t;
   uint32_t tile_bytes, stages;
+  uint32_t hints;      // bit 0: loads evict-first in L2, bit 1: stores evict-first
   int *status;
   RankPtrs ptrs;
 };
@@ -134,6 +154,8 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
 
   if (tid == 0) {
     // ---------------- producer: schedule tiles, issue loads ----------------
+    const uint64_t pol = policy_evict_first();
+    const bool hint = (p.hints & 1u) != 0;
     uint32_t it = 0;
     bool ok = true;
     for (uint32_t u = blockIdx.x; ok && u < p.t.n_units; u += gridDim.x) {
@@ -174,8 +196,13 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
         mbar_arrive_expect_tx(bar, rows * row_bytes);
         const uint8_t *sp = src_base + (uint64_t)run * sg.src_pitch + in_run;
         const uint32_t dp = smem_u32(data + (size_t)st * T);
-        for (uint32_t r = 0; r < rows; ++r)
-          bulk_load(dp + r * row_bytes, sp + (uint64_t)r * sg.src_pitch, row_bytes, bar);
+        if (hint) {
+          for (uint32_t r = 0; r < rows; ++r)
+            bulk_load_hint(dp + r * row_bytes, sp + (uint64_t)r * sg.src_pitch, row_bytes, bar, pol);
+        } else {
+          for (uint32_t r = 0; r < rows; ++r)
+            bulk_load(dp + r * row_bytes, sp + (uint64_t)r * sg.src_pitch, row_bytes, bar);
+        }
         if (long_run) {
           if (++ch == tpr) { ch = 0; ++run; }
         } else {
@@ -205,6 +232,12 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
     }
   } else if (tid == 32) {
     // ---------------- consumer: issue stores, recycle stages ----------------
+    // A stage is handed back one tile late: when the store of tile i has been issued,
+    // the store of tile i-1 is waited for (reads of shared memory only) and its stage
+    // released.  Releasing a stage right after its own store (a blocking wait per
+    // tile) and several store-issuing threads were both measured slower.
+    const uint64_t pol = policy_evict_first();
+    const bool hint = (p.hints & 2u) != 0;
     for (uint32_t it = 0;; ++it) {
       const uint32_t st = it % S, round = it / S;
       if (!mbar_wait(smem_u32(&full[st]), round & 1)) {
@@ -219,7 +252,12 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
       for (uint32_t d = 0; d < ti.n_dst; ++d) {
         uint8_t *dp = reinterpret_cast<uint8_t *>(ti.dst_ptr[d]);
         const uint64_t pitch = ti.dst_pitch[d];
-        for (uint32_t r = 0; r < rows; ++r) bulk_store(dp + (uint64_t)r * pitch, sp + r * rb, rb);
+        if (hint) {
+          for (uint32_t r = 0; r < rows; ++r)
+            bulk_store_hint(dp + (uint64_t)r * pitch, sp + r * rb, rb, pol);
+        } else {
+          for (uint32_t r = 0; r < rows; ++r) bulk_store(dp + (uint64_t)r * pitch, sp + r * rb, rb);
+        }
       }
       bulk_commit();
       if (it >= 1) {  // the store of the previous tile has finished reading its stage
@@ -382,22 +420,31 @@ __global__ void __launch_bounds__(256) kv_direct_kernel(const __grid_constant__ 
 
 // ---- launchers --------------------------------------------------------------------------
 
-static size_t bulk_smem_bytes(uint32_t tile_bytes, uint32_t stages) {
+size_t bulk_smem_bytes(uint32_t tile_bytes, uint32_t stages) {
   return (size_t)stages * tile_bytes + stages * (sizeof(TileInfo) + 2 * sizeof(uint64_t));
+}
+
+size_t bulk_smem_limit() {
+  cudaFuncAttributes a{};
+  if (cudaFuncGetAttributes(&a, bulk_copy_kernel) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return 200 * 1024;
+  }
+  return 227 * 1024 - a.sharedSizeBytes;
 }
 
 cudaError_t kernels_init() {
   return cudaFuncSetAttribute(bulk_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              227 * 1024 - 2048);
+                              (int)bulk_smem_limit());
 }
 
-cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
-                             uint32_t stages, uint32_t grid, int *status, cudaStream_t stream) {
+cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, const BulkConfig &c,
+                             uint32_t grid, int *status, cudaStream_t stream) {
   if (t.n_units == 0) return cudaSuccess;
-  if (stages < 2 || stages > kMaxStages || tile_bytes % 128 != 0) return cudaErrorInvalidValue;
-  const size_t smem = bulk_smem_bytes(tile_bytes, stages);
-  if (smem > 227 * 1024 - 2048) return cudaErrorInvalidValue;
-  BulkParams p{t, tile_bytes, stages, status, ptrs};
+  if (c.stages < 2 || c.stages > kMaxStages || c.tile_bytes % 128 != 0) return cudaErrorInvalidValue;
+  const size_t smem = bulk_smem_bytes(c.tile_bytes, c.stages);
+  if (bulk_smem_bytes(c.tile_bytes, c.stages) > bulk_smem_limit()) return cudaErrorInvalidValue;
+  BulkParams p{t, c.tile_bytes, c.stages, c.hints, status, ptrs};
   if (grid > t.n_units) grid = t.n_units;
   bulk_copy_kernel<<<grid, 64, smem, stream>>>(p);
   return cudaGetLastError();

@@ -49,9 +49,15 @@ struct KvTables {  // device pointers + shape constants of the KV head re-split
   uint64_t nb_old, nb_new;
 };
 
+struct BulkConfig {
+  uint32_t tile_bytes, stages, hints;
+};
+// Dynamic shared memory the bulk kernel needs / may use at most.
+size_t bulk_smem_bytes(uint32_t tile_bytes, uint32_t stages);
+size_t bulk_smem_limit();
 // Bulk path: cp.async.bulk global -> shared -> global through an mbarrier ring.
-cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
-                             uint32_t stages, uint32_t grid, int *status, cudaStream_t stream);
+cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, const BulkConfig &c,
+                             uint32_t grid, int *status, cudaStream_t stream);
 // Vector path: a warp per tile, 16-byte (or narrower, per segment alignment) loads and stores.
 cudaError_t launch_vec_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
                             uint32_t grid, cudaStream_t stream);
