@@ -116,8 +116,9 @@ typedef struct {
  *
  * Validates shape and both configurations, enumerates the logical moves of
  * the three phases, picks the source replica of every destination expert
- * slot (the copy already on the same rank index if there is one, "maximize
- * zero-copy reuse", otherwise the lexicographically smallest (rank, slot)),
+ * slot (the copy already on the same rank index if there is one, since the
+ * paper's plan prefers data that is already on the device to a transfer;
+ * otherwise the lexicographically smallest (rank, slot)),
  * coalesces moves into segments, and uploads the descriptor arrays to the
  * current CUDA device (unless EMOE_PLAN_HOST_ONLY).
  *

@@ -41,8 +41,9 @@ struct Csr {
 };
 
 // Source replica of expert e for destination rank r_new: the copy held by the
-// old rank with the same index if there is one (that device keeps its copy,
-// Sec. 5.2 "maximize zero-copy reuse"), else the smallest (rank, slot).
+// old rank with the same index if there is one (that device keeps its copy:
+// Sec. 5.2 plans a step so that data already in place is reused rather than
+// transferred), else the smallest (rank, slot).
 bool find_source(const Csr &old_p, int e, int r_new, int *r_out, int *s_out) {
   if (r_new < old_p.n_ranks) {
     for (int s = 0; s < old_p.count(r_new); ++s)
