@@ -289,7 +289,10 @@ typedef struct {
   int32_t kv_mode;         /* 0 default, 1 direct, 2 staged through shared memory   */
   int32_t bulk_hints;      /* 0 default, 1 none, 2 loads evict-first in L2, 3 stores */
                            /* evict-first, 4 both                                   */
-  int32_t reserved[2];
+  int32_t kv_order;        /* order in which mapped KV blocks are visited: 0 default,   */
+                           /* 1 block-table order, 2 by old physical id, 3 by new id    */
+  int32_t unit_order;      /* bulk work order: 0 default (run-major: one layer slab or  */
+                           /* KV pool at a time), 1 segment-major                       */
 } emoe_tuning_t;
 
 /* Replaces the plan's launch tuning.  Not thread-safe against reshard calls

@@ -49,7 +49,8 @@ class _Segment(ctypes.Structure):
 
 class _Tuning(ctypes.Structure):
     _fields_ = [("max_ctas", _i32), ("bulk_tile_bytes", _i32), ("bulk_stages", _i32),
-                ("path", _i32), ("kv_mode", _i32), ("bulk_hints", _i32), ("reserved", _i32 * 2)]
+                ("path", _i32), ("kv_mode", _i32), ("bulk_hints", _i32), ("kv_order", _i32),
+                ("unit_order", _i32)]
 
 
 SEGMENT_DTYPE = np.dtype([("src_off", "<u8"), ("dst_off", "<u8"), ("run_bytes", "<u8"),
@@ -245,8 +246,10 @@ class Plan:
         return s.value
 
     def set_tuning(self, max_ctas: int = 0, bulk_tile_bytes: int = 0, bulk_stages: int = 0,
-                   path: int = 0, kv_mode: int = 0, bulk_hints: int = 0) -> None:
-        t = _Tuning(max_ctas, bulk_tile_bytes, bulk_stages, path, kv_mode, bulk_hints)
+                   path: int = 0, kv_mode: int = 0, bulk_hints: int = 0, kv_order: int = 0,
+                   unit_order: int = 0) -> None:
+        t = _Tuning(max_ctas, bulk_tile_bytes, bulk_stages, path, kv_mode, bulk_hints, kv_order,
+                    unit_order)
         _check(lib().emoe_plan_set_tuning(self._h, ctypes.byref(t)))
 
     # -- the hot path

@@ -1,6 +1,7 @@
 // capi.cpp - the C ABI of libemoe.so: plan life cycle, argument checks, launches.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -17,15 +18,17 @@ namespace {
 constexpr uint32_t kUnitTiles = 8;
 constexpr uint32_t kDefaultBulkTile = 32768, kDefaultBulkStages = 6;
 constexpr uint32_t kDefaultHints = 0;
+constexpr int kDefaultKvMode = 1;   // 1 direct, 2 staged through shared memory
+constexpr int kDefaultKvOrder = 1;  // 1 table order, 2 by old block id, 3 by new block id
 constexpr uint32_t kDefaultBulkCtas = 74;  // measured optimum on B200: half the SMs, deep rings
 constexpr uint32_t kVecTile = 16384;
 constexpr uint64_t kBulkMinRun = 16384;  // shorter runs go to the vector kernel
 
 struct DevPhase {
-  std::vector<Segment> segs;  // routed copy of the host segments (fan-out split to kMaxFanout)
+  std::vector<DevSeg> segs;  // routed copy of the host segments (fan-out split to kMaxFanout)
   std::vector<Dst> dsts;
   std::vector<Unit> bulk_units, vec_units;
-  Segment *d_segs = nullptr;
+  DevSeg *d_segs = nullptr;
   Dst *d_dsts = nullptr;
   Unit *d_bulk_units = nullptr, *d_vec_units = nullptr;
 };
@@ -38,6 +41,7 @@ struct emoe_plan {
   int device = -1, sm_count = 148;
   emoe_tuning_t tuning{};
   DevPhase dev[3];
+  std::vector<uint32_t> pair_old, pair_new;  // block pairs in launch order (see kv_order)
   uint32_t *d_pair_old = nullptr, *d_pair_new = nullptr;
   int *d_status = nullptr;
 };
@@ -50,34 +54,103 @@ uint32_t bulk_tile(const emoe_plan *p) {
 uint32_t bulk_stages(const emoe_plan *p) {
   return p->tuning.bulk_stages > 0 ? (uint32_t)p->tuning.bulk_stages : kDefaultBulkStages;
 }
+int kv_order(const emoe_plan *p) {
+  return p->tuning.kv_order > 0 ? p->tuning.kv_order : kDefaultKvOrder;
+}
 
-void add_units(std::vector<Unit> *units, uint32_t seg, uint64_t n_tiles) {
-  for (uint64_t t = 0; t < n_tiles; t += kUnitTiles) {
-    const uint64_t n = n_tiles - t < kUnitTiles ? n_tiles - t : kUnitTiles;
-    units->push_back({seg, (uint32_t)t, (uint32_t)n, 0});
+struct KeyedUnit {
+  uint32_t run;  // first run the unit touches
+  Unit u;
+};
+
+// Cuts one segment into units of at most kUnitTiles tiles.  A unit of a long-run
+// segment (run >= tile) stays inside one run, so that units can be ordered by run.
+void add_units(std::vector<KeyedUnit> *units, uint32_t seg, const DevSeg &s, uint32_t T) {
+  if (s.run_bytes >= T) {
+    const uint32_t tpr = (uint32_t)((s.run_bytes + T - 1) / T);
+    for (uint32_t run = 0; run < s.n_runs; ++run)
+      for (uint32_t t = 0; t < tpr; t += kUnitTiles) {
+        const uint32_t n = tpr - t < kUnitTiles ? tpr - t : kUnitTiles;
+        units->push_back({run, {seg, run * tpr + t, n, 0}});
+      }
+  } else {
+    const uint32_t rpt = (uint32_t)(T / s.run_bytes);
+    const uint32_t n_tiles = (s.n_runs + rpt - 1) / rpt;
+    for (uint32_t t = 0; t < n_tiles; t += kUnitTiles) {
+      const uint32_t n = n_tiles - t < kUnitTiles ? n_tiles - t : kUnitTiles;
+      units->push_back({t * rpt, {seg, t, n, 0}});
+    }
   }
 }
 
 // Routes every host segment to the bulk or the vector kernel and cuts it into units.
+//
+// Launch order of the bulk units is run-major: all segments' run 0, then all segments'
+// run 1, ...  Runs of one segment are a pitch apart (a whole layer slab, a whole KV pool),
+// so this keeps the CTAs that run at the same time inside one slab - sequential DRAM
+// pages and a small TLB footprint - instead of spread over the whole arena.
 void build_tables(emoe_plan *p, int phase) {
   const PhasePlan &pp = p->hp.phase[phase];
   DevPhase &dp = p->dev[phase];
   dp.segs.clear(); dp.dsts.clear(); dp.bulk_units.clear(); dp.vec_units.clear();
   const uint32_t T = bulk_tile(p);
-  for (const Segment &s0 : pp.segs) {
-    bool bulk = s0.align == 16 && s0.run_bytes >= kBulkMinRun;
-    if (p->tuning.path == 1) bulk = false;
-    if (p->tuning.path == 2) bulk = (s0.align == 16);
-    const uint32_t max_fan = bulk ? (uint32_t)kMaxFanout : s0.n_dst;
+
+  // KV with the head split kept: one segment per block pair and TP rank.  Visit them in
+  // the order kv_order asks for (old or new physical block order instead of table order).
+  std::vector<uint32_t> order(pp.segs.size());
+  for (uint32_t i = 0; i < order.size(); ++i) order[i] = i;
+  if (phase == EMOE_PHASE_KV && kv_order(p) >= 2) {
+    const bool by_new = kv_order(p) == 3;
+    std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
+      const Segment &x = pp.segs[a], &y = pp.segs[b];
+      const uint64_t kx = by_new ? pp.dsts[x.dst_first].off : x.src_off;
+      const uint64_t ky = by_new ? pp.dsts[y.dst_first].off : y.src_off;
+      return kx != ky ? kx < ky : x.src_rank < y.src_rank;
+    });
+  }
+
+  std::vector<KeyedUnit> bulk, vec;
+  for (uint32_t oi : order) {
+    const Segment &s0 = pp.segs[oi];
+    bool is_bulk = s0.align == 16 && s0.run_bytes >= kBulkMinRun;
+    if (p->tuning.path == 1) is_bulk = false;
+    if (p->tuning.path == 2) is_bulk = (s0.align == 16);
+    const uint32_t max_fan = is_bulk ? (uint32_t)kMaxFanout : s0.n_dst;
     for (uint32_t k = 0; k < s0.n_dst; k += max_fan) {
-      Segment s = s0;
+      DevSeg s{};
+      s.src_off = s0.src_off; s.run_bytes = s0.run_bytes; s.src_pitch = s0.src_pitch;
+      s.n_runs = s0.n_runs; s.src_rank = s0.src_rank; s.align = s0.align;
       s.n_dst = s0.n_dst - k < max_fan ? s0.n_dst - k : max_fan;
       s.dst_first = (uint32_t)dp.dsts.size();
-      for (uint32_t j = 0; j < s.n_dst; ++j) dp.dsts.push_back(pp.dsts[s0.dst_first + k + j]);
+      const Dst &d0 = pp.dsts[s0.dst_first + k];
+      s.dst_off = d0.off; s.dst_pitch = d0.pitch; s.dst_rank = d0.rank;
+      if (s.n_dst > 1)  // the one-destination case reads the inlined copy only
+        for (uint32_t j = 0; j < s.n_dst; ++j) dp.dsts.push_back(pp.dsts[s0.dst_first + k + j]);
       const uint32_t idx = (uint32_t)dp.segs.size();
       dp.segs.push_back(s);
-      if (bulk) add_units(&dp.bulk_units, idx, seg_tile_count(s.run_bytes, s.n_runs, T));
-      else add_units(&dp.vec_units, idx, seg_tile_count(s.run_bytes, s.n_runs, kVecTile));
+      if (is_bulk) add_units(&bulk, idx, s, T);
+      else add_units(&vec, idx, s, kVecTile);
+    }
+  }
+  if (p->tuning.unit_order != 1)
+    std::stable_sort(bulk.begin(), bulk.end(),
+                     [](const KeyedUnit &a, const KeyedUnit &b) { return a.run < b.run; });
+  for (const KeyedUnit &k : bulk) dp.bulk_units.push_back(k.u);
+  for (const KeyedUnit &k : vec) dp.vec_units.push_back(k.u);
+
+  if (phase == EMOE_PHASE_KV) {  // block pairs of the head re-split, in launch order
+    const KvPlan &kv = p->hp.kv;
+    std::vector<uint32_t> idx(kv.pair_old.size());
+    for (uint32_t i = 0; i < idx.size(); ++i) idx[i] = i;
+    if (kv_order(p) >= 2) {
+      const std::vector<uint32_t> &key = kv_order(p) == 3 ? kv.pair_new : kv.pair_old;
+      std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) { return key[a] < key[b]; });
+    }
+    p->pair_old.resize(idx.size());
+    p->pair_new.resize(idx.size());
+    for (size_t i = 0; i < idx.size(); ++i) {
+      p->pair_old[i] = kv.pair_old[idx[i]];
+      p->pair_new[i] = kv.pair_new[idx[i]];
     }
   }
 }
@@ -201,8 +274,8 @@ emoe_status_t emoe_plan_create(const emoe_shape_t *shape, const emoe_config_t *o
     st = cuda_status(e);
     for (int ph = 0; st == EMOE_OK && ph < 3; ++ph) st = upload_phase(p, ph);
     if (st == EMOE_OK && p->hp.kv.head_split_changes) {
-      cudaError_t e2 = upload(p->hp.kv.pair_old, &p->d_pair_old);
-      if (e2 == cudaSuccess) e2 = upload(p->hp.kv.pair_new, &p->d_pair_new);
+      cudaError_t e2 = upload(p->pair_old, &p->d_pair_old);
+      if (e2 == cudaSuccess) e2 = upload(p->pair_new, &p->d_pair_new);
       st = cuda_status(e2);
     }
     if (st == EMOE_OK) {
@@ -248,8 +321,8 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *p, const void *const *src, void
   KvTables t{p->d_pair_old, p->d_pair_new, (uint32_t)kv.pair_old.size(), kv.n_layers * 2,
              kv.block_tokens, kv.hkv, kv.hkv / kv.c, kv.hkv / kv.d, (uint32_t)kv.head_bytes,
              kv.nb_old, kv.nb_new};
-  return cuda_status(launch_kv_copy(t, ptrs, p->tuning.kv_mode, cta_budget(p) * 8, p->d_status,
-                                    (cudaStream_t)stream));
+  const int mode = p->tuning.kv_mode > 0 ? p->tuning.kv_mode : kDefaultKvMode;
+  return cuda_status(launch_kv_copy(t, ptrs, mode, cta_budget(p), p->d_status, (cudaStream_t)stream));
 }
 
 emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *p, const void *const *src, void *const *dst,
@@ -384,7 +457,8 @@ emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
   if (!p || !t) return EMOE_ERR_INVALID_ARG;
   if (t->max_ctas < 0 || t->bulk_tile_bytes < 0 || t->bulk_stages < 0 || t->path < 0 ||
       t->path > 2 || t->kv_mode < 0 || t->kv_mode > 2 || t->bulk_hints < 0 ||
-      t->bulk_hints > 4)
+      t->bulk_hints > 4 || t->kv_order < 0 || t->kv_order > 3 || t->unit_order < 0 ||
+      t->unit_order > 1)
     return EMOE_ERR_INVALID_ARG;
   if (t->bulk_tile_bytes && (t->bulk_tile_bytes % 128 || t->bulk_tile_bytes < 1024))
     return EMOE_ERR_INVALID_ARG;
@@ -402,6 +476,11 @@ emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
   if (!p->host_only) {
     if (cudaDeviceSynchronize() != cudaSuccess) return EMOE_ERR_CUDA;
     for (int ph = 0; st == EMOE_OK && ph < 3; ++ph) st = upload_phase(p, ph);
+    if (st == EMOE_OK && p->hp.kv.head_split_changes) {
+      cudaError_t e2 = upload(p->pair_old, &p->d_pair_old);
+      if (e2 == cudaSuccess) e2 = upload(p->pair_new, &p->d_pair_new);
+      st = cuda_status(e2);
+    }
   }
   return st;
 }

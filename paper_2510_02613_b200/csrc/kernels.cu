@@ -154,14 +154,27 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
 
   if (tid == 0) {
     // ---------------- producer: schedule tiles, issue loads ----------------
+    // Descriptors are fetched ahead of their use - the unit record two units ahead, its
+    // segment one unit ahead - so that their latency hides behind the current unit.
     const uint64_t pol = policy_evict_first();
     const bool hint = (p.hints & 1u) != 0;
+    const uint32_t G = gridDim.x, n = p.t.n_units;
     uint32_t it = 0;
     bool ok = true;
-    for (uint32_t u = blockIdx.x; ok && u < p.t.n_units; u += gridDim.x) {
-      const Unit un = p.t.units[u];
-      const Segment sg = p.t.segs[un.seg];
+    uint32_t u = blockIdx.x;                 // < n: the grid never exceeds the unit count
+    Unit un0 = p.t.units[u];
+    DevSeg sg0 = p.t.segs[un0.seg];
+    Unit un1 = un0;
+    if ((uint64_t)u + G < n) un1 = p.t.units[u + G];
+    for (; ok && u < n; u += G) {
+      DevSeg sg1 = sg0;
+      Unit un2 = un1;
+      if ((uint64_t)u + G < n) sg1 = p.t.segs[un1.seg];
+      if ((uint64_t)u + 2ull * G < n) un2 = p.t.units[u + 2 * G];
+      const Unit &un = un0;
+      const DevSeg &sg = sg0;
       const uint8_t *src_base = s_src[sg.src_rank] + sg.src_off;
+      uint8_t *dst_base0 = s_dst[sg.dst_rank] + sg.dst_off;   // the first (often only) destination
       const bool long_run = sg.run_bytes >= T;
       const uint32_t tpr = long_run ? (uint32_t)((sg.run_bytes + T - 1) / T) : 1u;
       const uint32_t rpt = long_run ? 1u : (uint32_t)(T / sg.run_bytes);
@@ -184,10 +197,15 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
           row_bytes = (uint32_t)sg.run_bytes;
         }
         TileInfo &ti = info[st];
-        for (uint32_t d = 0; d < sg.n_dst; ++d) {
-          const Dst dd = p.t.dsts[sg.dst_first + d];
-          ti.dst_ptr[d] = (uint64_t)(s_dst[dd.rank] + dd.off + (uint64_t)run * dd.pitch + in_run);
-          ti.dst_pitch[d] = dd.pitch;
+        if (sg.n_dst == 1) {
+          ti.dst_ptr[0] = (uint64_t)(dst_base0 + (uint64_t)run * sg.dst_pitch + in_run);
+          ti.dst_pitch[0] = sg.dst_pitch;
+        } else {
+          for (uint32_t d = 0; d < sg.n_dst; ++d) {
+            const Dst dd = p.t.dsts[sg.dst_first + d];
+            ti.dst_ptr[d] = (uint64_t)(s_dst[dd.rank] + dd.off + (uint64_t)run * dd.pitch + in_run);
+            ti.dst_pitch[d] = dd.pitch;
+          }
         }
         ti.n_dst = sg.n_dst;
         ti.n_rows = rows;
@@ -209,6 +227,9 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
           run += rows;
         }
       }
+      un0 = un1;
+      sg0 = sg1;
+      un1 = un2;
     }
     if (ok) {
       // end marker
@@ -279,7 +300,7 @@ struct VecParams {
 
 template <typename V>
 __device__ __forceinline__ void warp_copy_tile(const uint8_t *sp, uint64_t src_pitch, uint32_t rows,
-                                               uint32_t row_bytes, const Segment &sg,
+                                               uint32_t row_bytes, const DevSeg &sg,
                                                const Dst *dsts, uint8_t *const *s_dst, uint32_t run,
                                                uint64_t in_run, uint32_t lane) {
   constexpr uint32_t W = sizeof(V);
@@ -298,7 +319,8 @@ __device__ __forceinline__ void warp_copy_tile(const uint8_t *sp, uint64_t src_p
       }
     }
     for (uint32_t d = 0; d < sg.n_dst; ++d) {
-      const Dst dd = dsts[sg.dst_first + d];
+      Dst dd{sg.dst_off, sg.dst_pitch, sg.dst_rank, 0};
+      if (sg.n_dst > 1) dd = dsts[sg.dst_first + d];
       uint8_t *dp = s_dst[dd.rank] + dd.off + (uint64_t)run * dd.pitch + in_run;
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -322,7 +344,7 @@ __global__ void __launch_bounds__(256) vec_copy_kernel(const __grid_constant__ V
   const uint32_t T = p.tile_bytes;
   for (uint32_t u = blockIdx.x; u < p.t.n_units; u += gridDim.x) {
     const Unit un = p.t.units[u];
-    const Segment sg = p.t.segs[un.seg];
+    const DevSeg sg = p.t.segs[un.seg];
     const uint8_t *src_base = s_src[sg.src_rank] + sg.src_off;
     const bool long_run = sg.run_bytes >= T;
     const uint32_t tpr = long_run ? (uint32_t)((sg.run_bytes + T - 1) / T) : 1u;
@@ -416,6 +438,156 @@ __global__ void __launch_bounds__(256) kv_direct_kernel(const __grid_constant__ 
   }
 }
 
+
+// Staged variant: the fused gather-transpose through shared memory.  One producer
+// thread brings the c contiguous pieces of a logical block (one per old rank, each
+// [token][local head][head_dim]) into a stage of a shared-memory ring with
+// cp.async.bulk; 256 consumer threads then read the stage in NEW-layout order and
+// write each new rank's block with coalesced 16-byte stores.  The stage -> destination
+// mapping is the same for every tile, so it is tabulated once per CTA (no division in
+// the steady state); per tile only the two block base offsets change.
+constexpr uint32_t kKvConsumers = 256;
+
+struct KvStagedParams {
+  KvTables t;
+  uint32_t stages, tile_bytes, n_pieces, chunk_bytes;  // chunk = one old rank's share of a block
+  int *status;
+  RankPtrs ptrs;
+};
+
+__global__ void __launch_bounds__(kKvConsumers + 32, 1)
+kv_staged_kernel(const __grid_constant__ KvStagedParams p) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const KvTables &t = p.t;
+  const uint32_t S = p.stages, T = p.tile_bytes;
+  uint8_t *data = smem;
+  uint2 *table = reinterpret_cast<uint2 *>(smem + (size_t)S * T);
+  uint64_t *base_new_of = reinterpret_cast<uint64_t *>(table + p.n_pieces);  // per stage
+  uint64_t *full = base_new_of + S;
+  uint64_t *empty = full + S;
+  __shared__ const uint8_t *s_src[EMOE_MAX_RANKS];
+  __shared__ uint8_t *s_dst[EMOE_MAX_RANKS];
+  __shared__ volatile int s_abort;
+  constexpr uint64_t kEnd = ~0ull;
+
+  const uint32_t tid = threadIdx.x;
+  if (tid < EMOE_MAX_RANKS) {
+    s_src[tid] = p.ptrs.src[tid];
+    s_dst[tid] = p.ptrs.dst[tid];
+  }
+  // stage offset and destination (rank, offset in block) of every 16-byte piece, new-layout order
+  {
+    const uint32_t cpv = t.head_bytes / 16, row_new = t.hn * cpv, ppr = t.block_tokens * row_new;
+    for (uint32_t q = tid; q < p.n_pieces; q += blockDim.x) {
+      const uint32_t rn = q / ppr, r = q - rn * ppr;
+      const uint32_t tok = r / row_new, rem = r - tok * row_new;
+      const uint32_t hl = rem / cpv, j = rem - hl * cpv;
+      const uint32_t g = rn * t.hn + hl, ro = g / t.hc, ho = g - ro * t.hc;
+      table[q] = make_uint2(ro * p.chunk_bytes + ((tok * t.hc + ho) * cpv + j) * 16, (rn << 24) | (r * 16));
+    }
+  }
+  if (tid == 0) {
+    s_abort = 0;
+    for (uint32_t s = 0; s < S; ++s) {
+      mbar_init(smem_u32(&full[s]), 1);
+      mbar_init(smem_u32(&empty[s]), kKvConsumers / 32);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+
+  const uint64_t blk_old = (uint64_t)p.chunk_bytes;
+  const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
+  const uint64_t n_tiles = (uint64_t)t.n_pairs * t.n_lk;
+  const uint32_t c = t.hkv / t.hc;
+
+  if (tid == kKvConsumers) {
+    // ---------------- producer ----------------
+    uint32_t it = 0;
+    bool ok = true;
+    uint64_t tile = blockIdx.x;   // < n_tiles: the grid never exceeds the tile count
+    uint32_t lk = (uint32_t)(tile / t.n_pairs), pr = (uint32_t)(tile % t.n_pairs);
+    uint32_t po = t.pair_old[pr], pn = t.pair_new[pr];
+    for (; tile < n_tiles; tile += gridDim.x, ++it) {
+      // ids of the next tile are fetched now and used one iteration later
+      const uint64_t tile2 = tile + gridDim.x;
+      uint32_t lk2 = lk, pr2 = pr, po2 = po, pn2 = pn;
+      if (tile2 < n_tiles) {
+        lk2 = (uint32_t)(tile2 / t.n_pairs);
+        pr2 = (uint32_t)(tile2 - (uint64_t)lk2 * t.n_pairs);
+        po2 = t.pair_old[pr2];
+        pn2 = t.pair_new[pr2];
+      }
+      const uint32_t st = it % S, round = it / S;
+      if (round > 0 && !mbar_wait(smem_u32(&empty[st]), (round - 1) & 1)) { ok = false; break; }
+      if (s_abort) { ok = false; break; }
+      base_new_of[st] = ((uint64_t)lk * t.nb_new + pn) * blk_new;
+      const uint64_t base_old = ((uint64_t)lk * t.nb_old + po) * blk_old;
+      const uint32_t bar = smem_u32(&full[st]);
+      mbar_arrive_expect_tx(bar, T);
+      const uint32_t dp = smem_u32(data + (size_t)st * T);
+      for (uint32_t ro = 0; ro < c; ++ro)
+        bulk_load(dp + ro * p.chunk_bytes, s_src[ro] + base_old, p.chunk_bytes, bar);
+      lk = lk2; pr = pr2; po = po2; pn = pn2;
+    }
+    if (ok) {  // end marker
+      const uint32_t st = it % S, round = it / S;
+      if (round == 0 || mbar_wait(smem_u32(&empty[st]), (round - 1) & 1)) {
+        base_new_of[st] = kEnd;
+        mbar_arrive(smem_u32(&full[st]));
+      } else {
+        ok = false;
+      }
+    }
+    if (!ok) {
+      // a wait expired: flag it, then let the loads already issued land before leaving
+      s_abort = 1;
+      atomicExch(p.status, (int)EMOE_ERR_DEVICE_TIMEOUT);
+      const uint32_t back = it < S ? it : S;
+      for (uint32_t j = 1; j <= back; ++j) {
+        const uint32_t i2 = it - j;
+        (void)mbar_wait(smem_u32(&full[i2 % S]), (i2 / S) & 1);
+      }
+    }
+  } else if (tid < kKvConsumers) {
+    // ---------------- consumers ----------------
+    const uint32_t n = p.n_pieces;
+    for (uint32_t it = 0;; ++it) {
+      const uint32_t st = it % S, round = it / S;
+      if (!mbar_wait(smem_u32(&full[st]), round & 1)) {
+        s_abort = 1;
+        atomicExch(p.status, (int)EMOE_ERR_DEVICE_TIMEOUT);
+        break;
+      }
+      const uint64_t base_new = base_new_of[st];
+      if (base_new == kEnd) break;
+      const uint8_t *stage = data + (size_t)st * T;
+      for (uint32_t q0 = tid; q0 < n; q0 += kKvConsumers * 4) {
+        uint4 v[4];
+        uint32_t where[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const uint32_t q = q0 + u * kKvConsumers;
+          if (q < n) {
+            const uint2 e = table[q];
+            v[u] = *reinterpret_cast<const uint4 *>(stage + e.x);
+            where[u] = e.y;
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const uint32_t q = q0 + u * kKvConsumers;
+          if (q < n)
+            *reinterpret_cast<uint4 *>(s_dst[where[u] >> 24] + base_new + (where[u] & 0xFFFFFFu)) = v[u];
+        }
+      }
+      __syncwarp();
+      if ((tid & 31) == 0) mbar_arrive(smem_u32(&empty[st]));
+    }
+  }
+}
+
 }  // namespace
 
 // ---- launchers --------------------------------------------------------------------------
@@ -434,8 +606,11 @@ size_t bulk_smem_limit() {
 }
 
 cudaError_t kernels_init() {
-  return cudaFuncSetAttribute(bulk_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)bulk_smem_limit());
+  cudaError_t e = cudaFuncSetAttribute(bulk_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)bulk_smem_limit());
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(kv_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              200 * 1024);
 }
 
 cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, const BulkConfig &c,
@@ -459,15 +634,40 @@ cudaError_t launch_vec_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t t
   return cudaGetLastError();
 }
 
+namespace {
+size_t kv_staged_smem(uint32_t tile_bytes, uint32_t stages) {
+  return (size_t)stages * tile_bytes + (size_t)(tile_bytes / 16) * sizeof(uint2) +
+         (size_t)stages * 3 * sizeof(uint64_t);
+}
+}  // namespace
+
+bool kv_staged_supported(const KvTables &t, uint32_t *stages_out) {
+  const uint64_t tile = (uint64_t)t.block_tokens * t.hkv * t.head_bytes;
+  const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
+  if (t.head_bytes % 16 || tile > 64 * 1024 || blk_new >= (1u << 24) || t.hkv / t.hn > 255) return false;
+  uint32_t stages = (uint32_t)((160 * 1024) / tile);
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) return false;
+  if (stages_out) *stages_out = stages;
+  return true;
+}
+
 cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, uint32_t grid,
                            int *status, cudaStream_t stream) {
-  (void)mode;
-  (void)status;
   const uint64_t n_tiles = (uint64_t)t.n_pairs * t.n_lk;
   if (n_tiles == 0) return cudaSuccess;
-  if (grid > n_tiles) grid = (uint32_t)n_tiles;
   KvParams p{t, ptrs};
   const uint32_t hb = t.head_bytes;
+  uint32_t stages = 0;
+  if (mode == 2 && status && kv_staged_supported(t, &stages)) {
+    const uint32_t tile = t.block_tokens * t.hkv * hb;
+    KvStagedParams sp{t, stages, tile, tile / 16, t.block_tokens * t.hc * hb, status, ptrs};
+    if (grid > n_tiles) grid = (uint32_t)n_tiles;
+    kv_staged_kernel<<<grid, kKvConsumers + 32, kv_staged_smem(tile, stages), stream>>>(sp);
+    return cudaGetLastError();
+  }
+  grid *= 8;  // the direct kernel keeps several small CTAs per SM
+  if (grid > n_tiles) grid = (uint32_t)n_tiles;
   if (hb % 16 == 0) kv_direct_kernel<uint4><<<grid, 256, 0, stream>>>(p);
   else if (hb % 8 == 0) kv_direct_kernel<uint2><<<grid, 256, 0, stream>>>(p);
   else if (hb % 4 == 0) kv_direct_kernel<uint32_t><<<grid, 256, 0, stream>>>(p);
@@ -533,7 +733,7 @@ emoe_status_t launch_kv_copy_static(const KvTables &shape_only, const uint32_t *
   KvTables t = shape_only;
   t.pair_old = d_old;
   t.pair_new = d_new;
-  const cudaError_t e = launch_kv_copy(t, ptrs, 1, (uint32_t)sms * 8, nullptr, stream);
+  const cudaError_t e = launch_kv_copy(t, ptrs, 1, (uint32_t)sms, nullptr, stream);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
     return EMOE_ERR_CUDA;

@@ -26,20 +26,22 @@ struct RankPtrs {
   uint8_t *dst[EMOE_MAX_RANKS];
 };
 
+// Device-side copy descriptor: a planner Segment with its first destination inlined, so
+// that the common one-destination case needs no second table look-up.  With n_dst > 1
+// all destinations (the first included) are dsts[dst_first .. dst_first + n_dst).
+struct DevSeg {
+  uint64_t src_off, run_bytes, src_pitch;
+  uint64_t dst_off, dst_pitch;
+  uint32_t n_runs, src_rank, dst_rank, n_dst, dst_first, align;
+};
+static_assert(sizeof(DevSeg) == 64, "DevSeg is read as four 16-byte words");
+
 struct SegTables {  // device pointers
-  const Segment *segs;
+  const DevSeg *segs;
   const Dst *dsts;
   const Unit *units;
   uint32_t n_units;
 };
-
-// Tiles of a segment for a given tile size (shared by host table building and kernels).
-__host__ __device__ inline uint64_t seg_tile_count(uint64_t run_bytes, uint32_t n_runs,
-                                                   uint32_t tile_bytes) {
-  if (run_bytes >= tile_bytes) return (uint64_t)n_runs * ((run_bytes + tile_bytes - 1) / tile_bytes);
-  const uint64_t rpt = tile_bytes / run_bytes;
-  return (n_runs + rpt - 1) / rpt;
-}
 
 struct KvTables {  // device pointers + shape constants of the KV head re-split
   const uint32_t *pair_old, *pair_new;
@@ -61,7 +63,9 @@ cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, const Bul
 // Vector path: a warp per tile, 16-byte (or narrower, per segment alignment) loads and stores.
 cudaError_t launch_vec_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
                             uint32_t grid, cudaStream_t stream);
-// KV head re-split; mode 1 = direct register copy, mode 2 = staged through shared memory.
+// KV head re-split; mode 1 = direct register copy, mode 2 = staged through shared memory
+// (falls back to direct where the staged kernel does not apply).  grid = CTA budget in SMs.
+bool kv_staged_supported(const KvTables &t, uint32_t *stages_out);
 cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, uint32_t grid,
                            int *status, cudaStream_t stream);
 
