@@ -286,7 +286,9 @@ typedef struct {
   int32_t bulk_stages;     /* stages of the bulk kernel's ring                      */
   int32_t path;            /* 0 default routing, 1 force the vector kernel for all  */
                            /* segments, 2 force the bulk kernel where aligned       */
-  int32_t kv_mode;         /* 0 default, 1 direct, 2 staged through shared memory   */
+  int32_t kv_mode;         /* 0 default, 1 direct, 2 staged through shared memory,  */
+                           /* 3 tiled TMA loads and stores, 4 direct without the    */
+                           /* row-mapped fast path                                  */
   int32_t bulk_hints;      /* 0 default, 1 none, 2 loads evict-first in L2, 3 stores */
                            /* evict-first, 4 both                                   */
   int32_t kv_order;        /* order in which mapped KV blocks are visited: 0 default,   */

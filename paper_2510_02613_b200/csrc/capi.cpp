@@ -238,7 +238,7 @@ emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, 
                                    ptrs, bc, bulk_budget(p), p->d_status, st);
   if (e != cudaSuccess) return cuda_status(e);
   e = launch_vec_copy({dp.d_segs, dp.d_dsts, dp.d_vec_units, (uint32_t)dp.vec_units.size()}, ptrs,
-                      kVecTile, cta_budget(p) * 8, st);
+                      kVecTile, p->tuning.max_ctas > 0 ? cta_budget(p) * 8 : 0xffffffffu, st);
   return cuda_status(e);
 }
 
@@ -322,7 +322,8 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *p, const void *const *src, void
              kv.block_tokens, kv.hkv, kv.hkv / kv.c, kv.hkv / kv.d, (uint32_t)kv.head_bytes,
              kv.nb_old, kv.nb_new};
   const int mode = p->tuning.kv_mode > 0 ? p->tuning.kv_mode : kDefaultKvMode;
-  return cuda_status(launch_kv_copy(t, ptrs, mode, cta_budget(p), p->d_status, (cudaStream_t)stream));
+  return cuda_status(launch_kv_copy(t, ptrs, mode, cta_budget(p), p->tuning.max_ctas <= 0, p->d_status,
+                                    (cudaStream_t)stream));
 }
 
 emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *p, const void *const *src, void *const *dst,
@@ -456,7 +457,7 @@ emoe_status_t emoe_plan_device_status(const emoe_plan_t *p, int32_t *status) {
 emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
   if (!p || !t) return EMOE_ERR_INVALID_ARG;
   if (t->max_ctas < 0 || t->bulk_tile_bytes < 0 || t->bulk_stages < 0 || t->path < 0 ||
-      t->path > 2 || t->kv_mode < 0 || t->kv_mode > 2 || t->bulk_hints < 0 ||
+      t->path > 2 || t->kv_mode < 0 || t->kv_mode > 4 || t->bulk_hints < 0 ||
       t->bulk_hints > 4 || t->kv_order < 0 || t->kv_order > 3 || t->unit_order < 0 ||
       t->unit_order > 1)
     return EMOE_ERR_INVALID_ARG;

@@ -63,11 +63,15 @@ cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, const Bul
 // Vector path: a warp per tile, 16-byte (or narrower, per segment alignment) loads and stores.
 cudaError_t launch_vec_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
                             uint32_t grid, cudaStream_t stream);
-// KV head re-split; mode 1 = direct register copy, mode 2 = staged through shared memory
-// (falls back to direct where the staged kernel does not apply).  grid = CTA budget in SMs.
+// KV head re-split; mode 1 = direct register copy, mode 2 = staged through shared memory,
+// mode 3 = tiled TMA loads and stores (each falls back to direct where it does not apply).
+// grid = CTA budget in SMs; unbounded = no budget was set (the direct kernels then launch
+// one CTA per tile).
+constexpr uint32_t kKvTmaMaxRanks = 12;  // tensor maps travel in the kernel parameters
 bool kv_staged_supported(const KvTables &t, uint32_t *stages_out);
+bool kv_tma_supported(const KvTables &t, uint32_t *stages_out);
 cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, uint32_t grid,
-                           int *status, cudaStream_t stream);
+                           bool unbounded, int *status, cudaStream_t stream);
 
 // KV head re-split with its block-pair list in a fixed __device__ array of the library
 // image (no allocation).  pair_old / pair_new: host arrays of n_pairs ids.  Returns

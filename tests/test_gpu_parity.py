@@ -47,7 +47,8 @@ TUNINGS = [dict(path=1), dict(path=2), dict(bulk_tile_bytes=8192, bulk_stages=3)
            dict(bulk_tile_bytes=16384, bulk_stages=12, max_ctas=296),
            dict(kv_mode=1), dict(kv_mode=2), dict(kv_mode=2, max_ctas=3), dict(kv_order=2),
            dict(kv_order=3, kv_mode=2), dict(kv_order=1, unit_order=1),
-           dict(kv_order=3, bulk_tile_bytes=16384)]
+           dict(kv_order=3, bulk_tile_bytes=16384), dict(kv_mode=3), dict(kv_mode=3, max_ctas=5),
+           dict(kv_mode=3, kv_order=3), dict(kv_mode=4)]
 
 
 @pytest.mark.parametrize("tuning", TUNINGS, ids=lambda t: "-".join("%s%s" % kv for kv in t.items()))
@@ -87,7 +88,7 @@ def test_odd_shapes_and_alignments(dims):
         with E.Plan(w.shape, w.old, w.new) as plan:
             for phase in range(3):
                 check_phase_full(w, plan, phase)
-            for kv_mode in (1, 2):      # both KV kernels (staged falls back where it cannot run)
+            for kv_mode in (1, 2, 3, 4):   # every KV kernel (each falls back where it cannot run)
                 plan.set_tuning(kv_mode=kv_mode, kv_order=3)
                 check_phase_full(w, plan, E.PHASE_KV)
 
