@@ -144,6 +144,27 @@ def time_steps(torch, plan, src, dst, steps, warmup, stream, barrier=None):
     return total, phase
 
 
+def time_graph_steps(torch, plan, src, dst, steps, warmup, stream):
+    """The same step captured once in a CUDA graph and replayed: what a launch-bound
+    (tiny) configuration costs when the host is taken out of the loop.  Returns ms/step."""
+    with torch.cuda.stream(stream):
+        one_step(plan, src, dst, stream)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            one_step(plan, src, dst, stream)
+        for _ in range(warmup):
+            graph.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            graph.replay()
+        e1.record(stream)
+        stream.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
 def config_report(E, plan, wl, total_ms, phase_ms, steps, peak, plan_ms):
     st = [plan.stats(ph) for ph in range(3)]
     moved = sum(s["bytes_moved"] for s in st)
@@ -168,9 +189,10 @@ def config_report(E, plan, wl, total_ms, phase_ms, steps, peak, plan_ms):
 
 # ---- CPU baseline: the oracle, as it stands, on the host cores ---------------------------
 
-def cpu_baseline_sample(wl, src_layer_getter, budget_s=12.0, max_layers=4):
+def cpu_baseline_sample(wl, src_layer_getter, budget_s=12.0, max_layers=64):
     """Times the single-threaded oracle on whole layers of the workload (layers are
-    independent), until `budget_s` of CPU work or `max_layers` layers."""
+    independent; they are taken in order, cyclically), until `budget_s` of CPU work or
+    `max_layers` layer passes."""
     import oracle
     wl1 = wl.with_layers(1)
     sh = wl1.shape
@@ -181,8 +203,8 @@ def cpu_baseline_sample(wl, src_layer_getter, budget_s=12.0, max_layers=4):
     kv_moved = (2 * used * sh.kv_block_tokens * sh.n_kv_heads * sh.head_dim * sh.elem_bytes)
     moved_per_layer = sum(sizes_new[0]) + sum(sizes_new[1]) + kv_moved
     spent, layers = 0.0, 0
-    for l in range(min(max_layers, wl.shape.n_layers)):
-        src = src_layer_getter(l)
+    for i in range(max_layers):
+        src = src_layer_getter(i % wl.shape.n_layers)
         dst = [[np.empty(n, np.uint8) for n in s] for s in sizes_new]
         for group in dst:
             for a in group:
@@ -197,7 +219,7 @@ def cpu_baseline_sample(wl, src_layer_getter, budget_s=12.0, max_layers=4):
             break
     gbs = 2 * moved_per_layer * layers / spent / 1e9
     return {"value": round(gbs, 3), "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": "%d of %d layers of %s, all three phases, single thread; "
+            "sample": "%d layer passes (of %d layers) of %s, all three phases, single thread; "
                       "%.2f s of CPU work" % (layers, wl.shape.n_layers, wl.name, spent),
             "ms_per_layer": round(spent / layers * 1e3, 2),
             "projected_step_ms": round(spent / layers * 1e3 * wl.shape.n_layers, 1)}
@@ -472,8 +494,6 @@ def main():
         except Exception as e:  # report, never hide
             line["e2e"] = {"value": None, "unit": UNIT, "error": repr(e)[:200]}
         # CPU baseline: the oracle on sampled layers of the same arenas
-        for g, kind in zip(src, (W.KIND_EXPERTS, W.KIND_ATTN, W.KIND_KV)):
-            pass
         line["cpu_baseline"] = cpu_baseline_sample(
             wl, device_layer_getter(torch, src, wl.shape.n_layers))
     elif world > 1:
@@ -489,13 +509,14 @@ def main():
             if name == args.workload:
                 others[name] = rep
                 continue
-            base = "c3_fine" if name == "c5_overlap" else name
-            if name == "c5_overlap" and "c3_fine" in others:
-                pass
             wl2, plan2, src2, dst2, pms = setup(name, torch, E, W, WD)
             k = max(5, args.steps // 2) if name != "c1_tiny" else 200
             tot, ph = time_steps(torch, plan2, src2, dst2, k, 3, stream)
             r = config_report(E, plan2, wl2, tot, ph, k, peak, pms)
+            if name == "c1_tiny":    # launch-bound: also as a CUDA-graph replay
+                g_ms = time_graph_steps(torch, plan2, src2, dst2, k, 3, stream)
+                r["cuda_graph"] = {"scale_step_ms": round(g_ms, 4),
+                                   "reshard_gbs": round(2 * r["bytes_moved"] / g_ms / 1e6, 1)}
             if name == "c5_overlap":
                 r["overlap"] = run_overlap(torch, E, plan2, wl2, src2, dst2, peak)
             others[name] = r
