@@ -421,6 +421,7 @@ def main():
 
     import torch
     import paper_2510_02613_b200 as E
+    from paper_2510_02613_b200 import replicas
     import workloads as W
     from workloads import device as WD
 
@@ -443,15 +444,12 @@ def main():
     sampler.start()
     total_ms, phase_ms = time_steps(torch, plan, src, dst, args.steps, args.warmup, stream, barrier)
     clocks = sampler.stop()
-    if dist:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = replicas.job_time_ms(total_ms, dist, device="cuda")   # max over ranks
     rep = config_report(E, plan, wl, total_ms, phase_ms, args.steps, peak, plan_ms)
     if plan.device_status() != 0:
         raise SystemExit("device status word set: a bounded wait expired")
     ms = total_ms / args.steps
-    value = world * 2 * rep["bytes_moved"] / (ms * 1e-3) / 1e9
+    value = replicas.job_throughput_gbs(rep["bytes_moved"], world, ms)
     launches = sum(plan.num_launches(ph) for ph in range(3)) * args.steps
 
     # roofline of the dominant kernel: the expert re-pack's bulk-copy launch
