@@ -485,7 +485,8 @@ def main():
             if psutil.virtual_memory().available < need * 1.15:
                 raise MemoryError("host has %.0f GB available, the step needs %.0f GB pinned"
                                   % (psutil.virtual_memory().available / 1e9, need / 1e9))
-            e_ms, h2d, d2h = run_e2e(torch, plan, src, dst, args.e2e_steps, stream)
+            with E.Plan(wl.shape, wl.old, wl.new, host_step=True) as e2e_plan:   # pipelined form
+                e_ms, h2d, d2h = run_e2e(torch, e2e_plan, src, dst, args.e2e_steps, stream)
             line["e2e"] = {"value": round(2 * rep["bytes_moved"] / (e_ms * 1e-3) / 1e9, 2),
                            "unit": UNIT, "ms_per_step": round(e_ms, 2), "steps": args.e2e_steps,
                            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}

@@ -103,6 +103,9 @@ typedef struct {
 #define EMOE_PLAN_HOST_ONLY 1u /* build and validate the plan on the host only: no CUDA */
                                /* call is made, the reshard calls return EMOE_ERR_CUDA  */
 
+#define EMOE_PLAN_HOST_STEP 2u /* also prepare the pipelined form of emoe_reshard_step_host: */
+                               /* chunk plans, two copy streams and their events           */
+
 /* phase / side selectors of the query helpers */
 #define EMOE_PHASE_EXPERTS 0
 #define EMOE_PHASE_ATTN 1
@@ -188,6 +191,16 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *plan, const void *const *src,
  * same rank counts and sizes.  Destination staging arenas are fully
  * overwritten only where the plan writes; bytes the plan does not write are
  * copied back as the staging arena held them.
+ *
+ * A plan created with EMOE_PLAN_HOST_STEP runs the step as a pipeline over
+ * chunks of layers (layers are independent in every phase): copy-in of one
+ * chunk, the kernels of the previous one and copy-out of the one before
+ * overlap on the plan's own two copy streams, so both directions of the host
+ * link are busy at once.  Work still starts after what cuda_stream held before
+ * the call and cuda_stream ends after the last copy-out.  Calls of this form on
+ * ONE plan must not overlap each other (they share the plan's events).  Without
+ * the flag, or when a layer slice of an arena is not 16-byte aligned, the step
+ * runs serially on cuda_stream alone.
  */
 emoe_status_t emoe_reshard_step_host(const emoe_plan_t *plan, const void *const *const h_src[3],
                                      void *const *const h_dst[3],

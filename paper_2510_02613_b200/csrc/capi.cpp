@@ -35,8 +35,21 @@ struct DevPhase {
 
 }  // namespace
 
+// State of the pipelined host-buffer step (EMOE_PLAN_HOST_STEP): plans for a chunk of
+// layers (layers are independent in every phase and every arena is layer-major, so a
+// plan for lc layers applied to pointers advanced by whole layers does exactly those
+// layers), two copy streams and the events that order copy-in -> kernels -> copy-out.
+struct HostStep {
+  emoe_plan *chunk = nullptr, *tail = nullptr;  // plans for lc layers / for the last L % lc layers
+  int lc = 0, n_chunks = 0;                     // n_chunks counts the tail chunk too
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  std::vector<cudaEvent_t> ev_in, ev_k;
+  cudaEvent_t ev_start = nullptr, ev_done = nullptr;
+};
+
 struct emoe_plan {
   HostPlan hp;
+  HostStep *hs = nullptr;
   bool host_only = true;
   int device = -1, sm_count = 148;
   emoe_tuning_t tuning{};
@@ -245,12 +258,69 @@ emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, 
 std::once_flag g_init_once;
 cudaError_t g_init_err = cudaSuccess;
 
-}  // namespace
+void destroy_host_step(HostStep *hs);
 
-extern "C" {
+emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
+                          const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out);
 
-emoe_status_t emoe_plan_create(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
-                               const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out) {
+// Chunk plans, streams and events of the pipelined host-buffer step.  Leaves p->hs null
+// (the step then runs serially) when a layer slice of some arena is not 16-byte aligned.
+emoe_status_t make_host_step(emoe_plan *p, const emoe_shape_t &shape, const emoe_config_t *old_cfg,
+                             const emoe_config_t *new_cfg) {
+  const int L = shape.n_layers;
+  for (int ph = 0; ph < 3; ++ph) {
+    for (uint64_t b : p->hp.phase[ph].arena_old) if ((b / L) % 16) return EMOE_OK;
+    for (uint64_t b : p->hp.phase[ph].arena_new) if ((b / L) % 16) return EMOE_OK;
+  }
+  HostStep *hs = new (std::nothrow) HostStep();
+  if (!hs) return EMOE_ERR_OOM;
+  hs->lc = (L + 7) / 8;  // about eight chunks: copy-in, kernels and copy-out overlap chunk by chunk
+  const int n_full = L / hs->lc, tail = L % hs->lc;
+  hs->n_chunks = n_full + (tail ? 1 : 0);
+  emoe_shape_t sh = shape;
+  sh.n_layers = hs->lc;
+  emoe_status_t st = create_plan(&sh, old_cfg, new_cfg, 0, &hs->chunk);
+  if (st == EMOE_OK && tail) {
+    sh.n_layers = tail;
+    st = create_plan(&sh, old_cfg, new_cfg, 0, &hs->tail);
+  }
+  cudaError_t e = cudaSuccess;
+  if (st == EMOE_OK) e = cudaStreamCreateWithFlags(&hs->s_in, cudaStreamNonBlocking);
+  if (st == EMOE_OK && e == cudaSuccess) e = cudaStreamCreateWithFlags(&hs->s_out, cudaStreamNonBlocking);
+  if (st == EMOE_OK && e == cudaSuccess) e = cudaEventCreateWithFlags(&hs->ev_start, cudaEventDisableTiming);
+  if (st == EMOE_OK && e == cudaSuccess) e = cudaEventCreateWithFlags(&hs->ev_done, cudaEventDisableTiming);
+  try {
+    for (int i = 0; st == EMOE_OK && e == cudaSuccess && i < hs->n_chunks; ++i) {
+      cudaEvent_t a = nullptr, b = nullptr;
+      e = cudaEventCreateWithFlags(&a, cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b, cudaEventDisableTiming);
+      hs->ev_in.push_back(a);
+      hs->ev_k.push_back(b);
+    }
+  } catch (const std::bad_alloc &) {
+    st = EMOE_ERR_OOM;
+  }
+  if (st == EMOE_OK) st = cuda_status(e);
+  if (st != EMOE_OK) { destroy_host_step(hs); return st; }
+  p->hs = hs;
+  return EMOE_OK;
+}
+
+void destroy_host_step(HostStep *hs) {
+  if (!hs) return;
+  emoe_plan_destroy(hs->chunk);
+  emoe_plan_destroy(hs->tail);
+  for (cudaEvent_t ev : hs->ev_in) if (ev) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : hs->ev_k) if (ev) cudaEventDestroy(ev);
+  if (hs->ev_start) cudaEventDestroy(hs->ev_start);
+  if (hs->ev_done) cudaEventDestroy(hs->ev_done);
+  if (hs->s_in) cudaStreamDestroy(hs->s_in);
+  if (hs->s_out) cudaStreamDestroy(hs->s_out);
+  delete hs;
+}
+
+emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
+                          const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out) {
   if (!shape || !old_cfg || !new_cfg || !out) return EMOE_ERR_INVALID_ARG;
   emoe_plan *p = new (std::nothrow) emoe_plan();
   if (!p) return EMOE_ERR_OOM;
@@ -283,14 +353,25 @@ emoe_status_t emoe_plan_create(const emoe_shape_t *shape, const emoe_config_t *o
       if (e3 == cudaSuccess) e3 = cudaMemset(p->d_status, 0, sizeof(int));
       st = cuda_status(e3);
     }
+    if (st == EMOE_OK && (flags & EMOE_PLAN_HOST_STEP)) st = make_host_step(p, *shape, old_cfg, new_cfg);
     if (st != EMOE_OK) { free_device(p); delete p; return st; }
   }
   *out = p;
   return EMOE_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+emoe_status_t emoe_plan_create(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
+                               const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out) {
+  return create_plan(shape, old_cfg, new_cfg, flags, out);
+}
+
 void emoe_plan_destroy(emoe_plan_t *p) {
   if (!p) return;
+  destroy_host_step(p->hs);
   if (!p->host_only) free_device(p);
   delete p;
 }
@@ -357,12 +438,86 @@ emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *p, const void *const *sr
   return launch_kv_copy_static(t, pair_old->data(), pair_new->data(), ptrs, (cudaStream_t)stream);
 }
 
+}  // extern "C"
+
+namespace {
+
+// Chunk by chunk: copy the layers' slices of every old arena in (stream s_in), run the
+// three phases on them (caller's stream), copy the slices of every new arena out (s_out).
+// The three streams run concurrently, so copy-in of chunk i+1, kernels of chunk i and
+// copy-out of chunk i-1 overlap and both directions of the host link stay busy.
+emoe_status_t step_host_pipelined(const emoe_plan *p, const void *const *const h_src[3],
+                                  void *const *const h_dst[3], void *const *const d_src[3],
+                                  void *const *const d_dst[3], cudaStream_t st) {
+  HostStep *hs = p->hs;
+  const int L = p->hp.shape.n_layers;
+  for (int ph = 0; ph < 3; ++ph) {
+    if (!h_src[ph] || !h_dst[ph] || !d_src[ph] || !d_dst[ph]) return EMOE_ERR_INVALID_ARG;
+    const PhasePlan &pp = p->hp.phase[ph];
+    for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_OLD); ++r)
+      if (pp.arena_old[r] && (!h_src[ph][r] || !d_src[ph][r])) return EMOE_ERR_INVALID_ARG;
+    for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_NEW); ++r)
+      if (pp.arena_new[r] && (!h_dst[ph][r] || !d_dst[ph][r])) return EMOE_ERR_INVALID_ARG;
+  }
+  cudaError_t e = cudaEventRecord(hs->ev_start, st);  // copies start after the stream's earlier work
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(hs->s_in, hs->ev_start, 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(hs->s_out, hs->ev_start, 0);
+  if (e != cudaSuccess) return cuda_status(e);
+  const void *sp[3][EMOE_MAX_RANKS];
+  void *dp[3][EMOE_MAX_RANKS];
+  for (int ci = 0; ci < hs->n_chunks; ++ci) {
+    const int l0 = ci * hs->lc, n = L - l0 < hs->lc ? L - l0 : hs->lc;
+    const emoe_plan *sub = n == hs->lc ? hs->chunk : hs->tail;
+    for (int ph = 0; ph < 3; ++ph) {
+      const PhasePlan &pp = p->hp.phase[ph];
+      for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_OLD); ++r) {
+        const uint64_t lb = pp.arena_old[r] / L;
+        sp[ph][r] = (const uint8_t *)d_src[ph][r] + l0 * lb;
+        if (!lb) continue;
+        e = cudaMemcpyAsync((uint8_t *)d_src[ph][r] + l0 * lb, (const uint8_t *)h_src[ph][r] + l0 * lb,
+                            n * lb, cudaMemcpyHostToDevice, hs->s_in);
+        if (e != cudaSuccess) return cuda_status(e);
+      }
+      for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_NEW); ++r)
+        dp[ph][r] = (uint8_t *)d_dst[ph][r] + l0 * (pp.arena_new[r] / L);
+    }
+    e = cudaEventRecord(hs->ev_in[ci], hs->s_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, hs->ev_in[ci], 0);
+    if (e != cudaSuccess) return cuda_status(e);
+    emoe_status_t rc = emoe_reshard_experts(sub, sp[0], dp[0], st);
+    if (rc == EMOE_OK) rc = emoe_reshard_attn(sub, sp[1], dp[1], st);
+    if (rc == EMOE_OK) rc = emoe_reshard_kv(sub, sp[2], dp[2], st);
+    if (rc != EMOE_OK) return rc;
+    e = cudaEventRecord(hs->ev_k[ci], st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(hs->s_out, hs->ev_k[ci], 0);
+    if (e != cudaSuccess) return cuda_status(e);
+    for (int ph = 0; ph < 3; ++ph) {
+      const PhasePlan &pp = p->hp.phase[ph];
+      for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_NEW); ++r) {
+        const uint64_t lb = pp.arena_new[r] / L;
+        if (!lb) continue;
+        e = cudaMemcpyAsync((uint8_t *)h_dst[ph][r] + l0 * lb, (const uint8_t *)d_dst[ph][r] + l0 * lb,
+                            n * lb, cudaMemcpyDeviceToHost, hs->s_out);
+        if (e != cudaSuccess) return cuda_status(e);
+      }
+    }
+  }
+  e = cudaEventRecord(hs->ev_done, hs->s_out);  // the caller's stream ends after the last copy-out
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(st, hs->ev_done, 0);
+  return cuda_status(e);
+}
+
+}  // namespace
+
+extern "C" {
+
 emoe_status_t emoe_reshard_step_host(const emoe_plan_t *p, const void *const *const h_src[3],
                                      void *const *const h_dst[3], void *const *const d_src[3],
                                      void *const *const d_dst[3], void *stream) {
   if (!p || !h_src || !h_dst || !d_src || !d_dst) return EMOE_ERR_INVALID_ARG;
   if (p->host_only) return EMOE_ERR_CUDA;
   cudaStream_t st = (cudaStream_t)stream;
+  if (p->hs) return step_host_pipelined(p, h_src, h_dst, d_src, d_dst, st);
   for (int ph = 0; ph < 3; ++ph) {
     if (!h_src[ph] || !h_dst[ph] || !d_src[ph] || !d_dst[ph]) return EMOE_ERR_INVALID_ARG;
     const PhasePlan &pp = p->hp.phase[ph];
@@ -450,6 +605,11 @@ emoe_status_t emoe_plan_device_status(const emoe_plan_t *p, int32_t *status) {
   int v = 0;
   cudaError_t e = cudaMemcpy(&v, p->d_status, sizeof(int), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_status(e);
+  if (p->hs && v == 0) {  // the chunk plans of the pipelined host step have status words of their own
+    int32_t sv = 0;
+    for (const emoe_plan *sub : {p->hs->chunk, p->hs->tail})
+      if (sub && v == 0 && emoe_plan_device_status(sub, &sv) == EMOE_OK) v = sv;
+  }
   *status = v;
   return EMOE_OK;
 }
@@ -467,6 +627,12 @@ emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
   const uint32_t stages = t->bulk_stages ? t->bulk_stages : kDefaultBulkStages;
   if (stages < 2 || stages > 16 || bulk_smem_bytes(tile, stages) > bulk_smem_limit())
     return EMOE_ERR_INVALID_ARG;
+  if (p->hs)
+    for (emoe_plan *sub : {p->hs->chunk, p->hs->tail})
+      if (sub) {
+        const emoe_status_t rc = emoe_plan_set_tuning(sub, t);
+        if (rc != EMOE_OK) return rc;
+      }
   p->tuning = *t;
   emoe_status_t st = EMOE_OK;
   try {

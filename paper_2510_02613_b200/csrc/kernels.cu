@@ -315,80 +315,102 @@ struct VecParams {
   RankPtrs ptrs;
 };
 
+// One warp copies one tile to one destination: `rows` rows of cpr pieces, a pitch apart
+// on either side.  Lanes keep a fixed column (or, for rows shorter than a warp pass, a
+// fixed sub-row and column), so the steady state has no division; four loads are in
+// flight per lane before the stores.
 template <typename V>
-__device__ __forceinline__ void warp_copy_tile(const uint8_t *sp, uint64_t src_pitch, uint32_t rows,
-                                               uint32_t row_bytes, const DevSeg &sg,
-                                               const Dst *dsts, uint8_t *const *s_dst, uint32_t run,
-                                               uint64_t in_run, uint32_t lane) {
-  constexpr uint32_t W = sizeof(V);
-  const uint32_t cpr = row_bytes / W;  // pieces per row
-  const uint32_t total = rows * cpr;
-  for (uint32_t i0 = lane; i0 < total; i0 += 32 * 4) {
-    V v[4];
-    uint32_t r[4], c[4];
+__device__ __forceinline__ void warp_copy_tile(const uint8_t *sp, uint64_t src_pitch, uint8_t *dp,
+                                               uint64_t dst_pitch, uint32_t rows, uint32_t cpr,
+                                               uint32_t lane) {
+  if (cpr >= 32) {
+#pragma unroll 1
+    for (uint32_t r = 0; r < rows; ++r) {
+      const V *srow = reinterpret_cast<const V *>(sp + (uint64_t)r * src_pitch);
+      V *drow = reinterpret_cast<V *>(dp + (uint64_t)r * dst_pitch);
+#pragma unroll 1
+      for (uint32_t c0 = lane; c0 < cpr; c0 += 32 * 4) {
+        V v[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const uint32_t i = i0 + 32 * u;
-      if (i < total) {
-        r[u] = rows == 1 ? 0 : i / cpr;
-        c[u] = rows == 1 ? i : i - r[u] * cpr;
-        v[u] = *reinterpret_cast<const V *>(sp + (uint64_t)r[u] * src_pitch + (uint64_t)c[u] * W);
+        for (int u = 0; u < 4; ++u)
+          if (c0 + 32 * u < cpr) v[u] = srow[c0 + 32 * u];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (c0 + 32 * u < cpr) drow[c0 + 32 * u] = v[u];
       }
     }
-    for (uint32_t d = 0; d < sg.n_dst; ++d) {
-      Dst dd{sg.dst_off, sg.dst_pitch, sg.dst_rank, 0};
-      if (sg.n_dst > 1) dd = dsts[sg.dst_first + d];
-      uint8_t *dp = s_dst[dd.rank] + dd.off + (uint64_t)run * dd.pitch + in_run;
+  } else {
+    const uint32_t rpp = 32 / cpr;  // rows per warp pass
+    const uint32_t sub = lane / cpr, c = lane - sub * cpr;
+    if (sub >= rpp) return;
+#pragma unroll 1
+    for (uint32_t r0 = sub; r0 < rows; r0 += rpp * 4) {
+      V v[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const uint32_t i = i0 + 32 * u;
-        if (i < total)
-          *reinterpret_cast<V *>(dp + (uint64_t)r[u] * dd.pitch + (uint64_t)c[u] * W) = v[u];
-      }
+      for (int u = 0; u < 4; ++u)
+        if (r0 + rpp * u < rows)
+          v[u] = reinterpret_cast<const V *>(sp + (uint64_t)(r0 + rpp * u) * src_pitch)[c];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (r0 + rpp * u < rows)
+          reinterpret_cast<V *>(dp + (uint64_t)(r0 + rpp * u) * dst_pitch)[c] = v[u];
     }
   }
 }
 
-__global__ void __launch_bounds__(256) vec_copy_kernel(const __grid_constant__ VecParams p) {
-  __shared__ const uint8_t *s_src[EMOE_MAX_RANKS];
-  __shared__ uint8_t *s_dst[EMOE_MAX_RANKS];
-  if (threadIdx.x < EMOE_MAX_RANKS) {
-    s_src[threadIdx.x] = p.ptrs.src[threadIdx.x];
-    s_dst[threadIdx.x] = p.ptrs.dst[threadIdx.x];
-  }
-  __syncthreads();
+// A CTA takes one unit at a time (its segment is parked in shared memory), a warp one tile.
+__global__ void __launch_bounds__(256, 4) vec_copy_kernel(const __grid_constant__ VecParams p) {
+  __shared__ DevSeg s_sg;
+  __shared__ Unit s_un;
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   const uint32_t T = p.tile_bytes;
   for (uint32_t u = blockIdx.x; u < p.t.n_units; u += gridDim.x) {
-    const Unit un = p.t.units[u];
-    const DevSeg sg = p.t.segs[un.seg];
-    const uint8_t *src_base = s_src[sg.src_rank] + sg.src_off;
-    const bool long_run = sg.run_bytes >= T;
-    const uint32_t tpr = long_run ? (uint32_t)((sg.run_bytes + T - 1) / T) : 1u;
-    const uint32_t rpt = long_run ? 1u : (uint32_t)(T / sg.run_bytes);
-    for (uint32_t k = warp; k < un.n_tiles; k += n_warps) {
-      const uint32_t tile = un.first_tile + k;
+    __syncthreads();  // everyone is done with the previous unit's segment
+    if (threadIdx.x == 0) s_un = p.t.units[u];
+    if (threadIdx.x < 4) {
+      const uint32_t seg = p.t.units[u].seg;
+      reinterpret_cast<uint4 *>(&s_sg)[threadIdx.x] =
+          reinterpret_cast<const uint4 *>(&p.t.segs[seg])[threadIdx.x];
+    }
+    __syncthreads();
+    const uint64_t run_bytes = s_sg.run_bytes;
+    const bool long_run = run_bytes >= T;
+    const uint32_t tpr = long_run ? (uint32_t)((run_bytes + T - 1) / T) : 1u;
+    const uint32_t rpt = long_run ? 1u : (uint32_t)(T / run_bytes);
+    for (uint32_t k = warp; k < s_un.n_tiles; k += n_warps) {
+      const uint32_t tile = s_un.first_tile + k;
       uint32_t run, rows, row_bytes;
       uint64_t in_run;
       if (long_run) {
         run = tile / tpr;
         in_run = (uint64_t)(tile % tpr) * T;
-        const uint64_t left = sg.run_bytes - in_run;
+        const uint64_t left = run_bytes - in_run;
         row_bytes = left < T ? (uint32_t)left : T;
         rows = 1;
       } else {
         run = tile * rpt;
         in_run = 0;
-        rows = sg.n_runs - run < rpt ? sg.n_runs - run : rpt;
-        row_bytes = (uint32_t)sg.run_bytes;
+        rows = s_sg.n_runs - run < rpt ? s_sg.n_runs - run : rpt;
+        row_bytes = (uint32_t)run_bytes;
       }
-      const uint8_t *sp = src_base + (uint64_t)run * sg.src_pitch + in_run;
-      switch (sg.align) {
-        case 16: warp_copy_tile<uint4>(sp, sg.src_pitch, rows, row_bytes, sg, p.t.dsts, s_dst, run, in_run, lane); break;
-        case 8: warp_copy_tile<uint2>(sp, sg.src_pitch, rows, row_bytes, sg, p.t.dsts, s_dst, run, in_run, lane); break;
-        case 4: warp_copy_tile<uint32_t>(sp, sg.src_pitch, rows, row_bytes, sg, p.t.dsts, s_dst, run, in_run, lane); break;
-        case 2: warp_copy_tile<uint16_t>(sp, sg.src_pitch, rows, row_bytes, sg, p.t.dsts, s_dst, run, in_run, lane); break;
-        default: warp_copy_tile<uint8_t>(sp, sg.src_pitch, rows, row_bytes, sg, p.t.dsts, s_dst, run, in_run, lane); break;
+      const uint64_t src_pitch = s_sg.src_pitch;
+      const uint8_t *sp = p.ptrs.src[s_sg.src_rank] + s_sg.src_off + (uint64_t)run * src_pitch + in_run;
+      const uint32_t n_dst = s_sg.n_dst, align = s_sg.align;
+      for (uint32_t d = 0; d < n_dst; ++d) {
+        uint64_t d_off = s_sg.dst_off, d_pitch = s_sg.dst_pitch;
+        uint32_t d_rank = s_sg.dst_rank;
+        if (n_dst > 1) {
+          const Dst dd = p.t.dsts[s_sg.dst_first + d];
+          d_off = dd.off; d_pitch = dd.pitch; d_rank = dd.rank;
+        }
+        uint8_t *dp = p.ptrs.dst[d_rank] + d_off + (uint64_t)run * d_pitch + in_run;
+        switch (align) {
+          case 16: warp_copy_tile<uint4>(sp, src_pitch, dp, d_pitch, rows, row_bytes / 16, lane); break;
+          case 8: warp_copy_tile<uint2>(sp, src_pitch, dp, d_pitch, rows, row_bytes / 8, lane); break;
+          case 4: warp_copy_tile<uint32_t>(sp, src_pitch, dp, d_pitch, rows, row_bytes / 4, lane); break;
+          case 2: warp_copy_tile<uint16_t>(sp, src_pitch, dp, d_pitch, rows, row_bytes / 2, lane); break;
+          default: warp_copy_tile<uint8_t>(sp, src_pitch, dp, d_pitch, rows, row_bytes, lane); break;
+        }
       }
     }
   }

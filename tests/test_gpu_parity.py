@@ -149,9 +149,9 @@ def test_argument_errors_launch_nothing():
         assert bool((big == 0xCD).all())
 
 
-def test_step_on_host_buffers_matches_oracle():
-    wl = W.make_workload("c1_tiny")
-    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+def _step_on_host_buffers(wl, host_step):
+    from gpu_util import oracle_phase
+    with E.Plan(wl.shape, wl.old, wl.new, host_step=host_step) as plan:
         h_src, h_dst, d_src, d_dst, want = [], [], [], [], []
         for phase in range(3):
             so, sn = plan.arena_bytes(phase, E.SIDE_OLD), plan.arena_bytes(phase, E.SIDE_NEW)
@@ -162,15 +162,32 @@ def test_step_on_host_buffers_matches_oracle():
             d_src.append([torch.empty(n, dtype=torch.uint8, device="cuda") for n in so])
             d_dst.append(WD.alloc_const(sn))
             w = [np.full(n, WD.FILL_BYTE, np.uint8) for n in sn]
-            from gpu_util import oracle_phase
             oracle_phase(wl, phase, [t.numpy() for t in hs], w)
             want.append(w)
         s = torch.cuda.Stream()
-        plan.reshard_step_host(h_src, h_dst, d_src, d_dst, s)
-        s.synchronize()
-        for phase in range(3):
-            for g, w in zip(h_dst[phase], want[phase]):
-                assert np.array_equal(g.numpy(), w)
+        for _ in range(2):      # twice: the pipelined form reuses the plan's events
+            for g in h_dst:
+                for t in g:
+                    t.zero_()
+            plan.reshard_step_host(h_src, h_dst, d_src, d_dst, s)
+            s.synchronize()
+            for phase in range(3):
+                for g, w in zip(h_dst[phase], want[phase]):
+                    assert np.array_equal(g.numpy(), w)
+        assert plan.device_status() == 0
+
+
+@pytest.mark.parametrize("host_step", [False, True], ids=["serial", "pipelined"])
+def test_step_on_host_buffers_matches_oracle(host_step):
+    _step_on_host_buffers(W.make_workload("c1_tiny"), host_step)
+
+
+def test_pipelined_host_step_with_a_ragged_last_chunk():
+    """11 layers: chunks of 2 layers and a tail chunk of 1."""
+    wl = W.make_workload("c1_tiny", n_layers=11)
+    wl = R(wl, shape=R(wl.shape, d_ff=64))
+    _step_on_host_buffers(wl, True)
+    _step_on_host_buffers(wl.swapped(), True)
 
 
 @pytest.mark.parametrize("name", ["c2_mid", "c3_fine", "c4_large"])
