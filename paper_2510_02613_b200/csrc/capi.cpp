@@ -23,6 +23,8 @@ constexpr int kDefaultKvOrder = 1;  // 1 table order, 2 by old block id, 3 by ne
 constexpr uint32_t kDefaultBulkCtas = 74;  // measured optimum on B200: half the SMs, deep rings
 constexpr uint32_t kVecTile = 16384;
 constexpr uint64_t kBulkMinRun = 16384;  // shorter runs go to the vector kernel
+constexpr uint64_t kMergeBulkBelow = 1ull << 30;   // see build_tables
+constexpr uint64_t kSmallPhaseBytes = 256ull << 20;
 
 struct DevPhase {
   std::vector<DevSeg> segs;  // routed copy of the host segments (fan-out split to kMaxFanout)
@@ -122,10 +124,23 @@ void build_tables(emoe_plan *p, int phase) {
     });
   }
 
+  // Default routing: long aligned runs to the bulk kernel, the rest to the vector kernel.
+  // A phase that is small, or that needs the vector kernel anyway and has little bulk
+  // work, goes to the vector kernel whole: one launch instead of two, and a short bulk
+  // launch never gets past its ramp-up (measured on the attention phase: 5.3 -> 5.9 TB/s).
+  uint64_t bulk_bytes = 0, vec_bytes = 0;
+  for (const Segment &s0 : pp.segs) {
+    const uint64_t b = (uint64_t)s0.n_runs * s0.run_bytes * s0.n_dst;
+    if (s0.align == 16 && s0.run_bytes >= kBulkMinRun) bulk_bytes += b; else vec_bytes += b;
+  }
+  const bool all_vec = p->tuning.path == 0 &&
+                       ((vec_bytes > 0 && bulk_bytes < kMergeBulkBelow) ||
+                        bulk_bytes + vec_bytes < kSmallPhaseBytes);
+
   std::vector<KeyedUnit> bulk, vec;
   for (uint32_t oi : order) {
     const Segment &s0 = pp.segs[oi];
-    bool is_bulk = s0.align == 16 && s0.run_bytes >= kBulkMinRun;
+    bool is_bulk = s0.align == 16 && s0.run_bytes >= kBulkMinRun && !all_vec;
     if (p->tuning.path == 1) is_bulk = false;
     if (p->tuning.path == 2) is_bulk = (s0.align == 16);
     const uint32_t max_fan = is_bulk ? (uint32_t)kMaxFanout : s0.n_dst;
