@@ -271,7 +271,7 @@ def run_e2e(torch, plan, src, dst, steps, stream):
 
 # ---- C5: reshard on a low-priority stream beside a grouped expert GEMM -------------------
 
-def run_overlap(torch, E, plan, wl, src, dst, peak, budgets=(0, 96, 48)):
+def run_overlap(torch, E, plan, wl, src, dst, peak, budgets=(0, 96, 48, 24)):
     """Victim: 8 active experts x 256 tokens (top-8 routing: every active expert sees all
     tokens), gate/up/down bf16 batched GEMMs (torch.bmm, a measurement fixture, not part
     of the library) on a high-priority stream, weights taken from the old expert arena of

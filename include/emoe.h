@@ -247,6 +247,78 @@ emoe_status_t emoe_reshard_step_host(const emoe_plan_t *plan, const void *const 
 emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *plan, const void *const *src,
                                      void *const *dst, void *cuda_stream);
 
+/* ---- paged expert store: re-layout by re-mapping pages ---------------------
+ *
+ * The paper's own expert mechanism (Sec. 4.1 "Virtual Expert Management",
+ * App. D.5): every expert matrix lives in physical pages of its own, which
+ * are mapped into one contiguous virtual range per device; changing the
+ * expert-parallel degree re-maps the pages a device keeps and transfers only
+ * the experts that arrive.  Here on the CUDA virtual memory API, all ranks
+ * being ranges of ONE GPU.
+ *
+ * Layout of the range of rank r: [L][3 (gate, up, down)][n_r][slab], where
+ * slab = one matrix (m bytes) rounded up to the device's allocation
+ * granularity (2 MiB on B200); the first m bytes of a slab hold the matrix,
+ * the rest is padding.  Apart from the padding this is the dense expert arena.
+ */
+typedef struct emoe_vmm_pool emoe_vmm_pool_t; /* opaque; owns ranges and pages */
+
+typedef struct {
+  uint64_t slabs_remapped; /* (layer, projection, slot) slabs kept by re-mapping        */
+  uint64_t slabs_copied;   /* slabs newly allocated and filled by the copy kernels      */
+  uint64_t bytes_copied;   /* bytes written by the copy kernels (arrivals only)         */
+  uint64_t bytes_read;     /* bytes they read (a source with several arrivals: once)    */
+  uint64_t slab_bytes, matrix_bytes;
+  uint64_t physical_bytes; /* device memory the pool holds after the step               */
+  double map_ms;           /* host time: reserve ranges, allocate and map slabs         */
+  double copy_ms;          /* host time: plan upload, copy kernels, stream synchronise  */
+  double unmap_ms;         /* host time: unmap and free the old ranges, release pages   */
+  double total_ms;
+} emoe_vmm_stats_t;
+
+/* Allocates the store for the placement of `cfg` (ep, place_off, place_ids;
+ * the other fields are ignored) on the current device.  Contents are
+ * undefined until written.  EMOE_ERR_UNSUPPORTED if the driver's virtual
+ * memory API is not available; EMOE_ERR_OOM if pages or address space run out. */
+emoe_status_t emoe_vmm_create(const emoe_shape_t *shape, const emoe_config_t *cfg,
+                              emoe_vmm_pool_t **out);
+
+/* Scale step EP=a -> EP=b in place of emoe_reshard_experts: afterwards the
+ * pool holds the placement of new_cfg.  A destination slot whose expert the
+ * same rank index already holds is re-mapped (no bytes move); every other
+ * slot gets fresh pages filled from its source replica (same source rule as
+ * emoe_plan_create) by the copy kernels on cuda_stream.  The call is
+ * SYNCHRONOUS: it returns after the copies have finished and the old ranges
+ * have been unmapped, so every pointer obtained from emoe_vmm_arena before
+ * the call is invalid after it.  On failure the pool is unchanged.
+ * stats: optional, filled on success. */
+emoe_status_t emoe_vmm_reshard(emoe_vmm_pool_t *pool, const emoe_config_t *new_cfg,
+                               void *cuda_stream, emoe_vmm_stats_t *stats);
+
+/* What emoe_vmm_reshard would do for old_cfg -> new_cfg with slabs of
+ * slab_bytes (>= one matrix), computed on the host without any CUDA call:
+ * fills slabs_remapped, slabs_copied, bytes_copied, bytes_read, slab_bytes,
+ * matrix_bytes and physical_bytes (of the new placement); times stay 0. */
+emoe_status_t emoe_vmm_dry_run(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
+                               const emoe_config_t *new_cfg, uint64_t slab_bytes,
+                               emoe_vmm_stats_t *stats);
+
+/* Number of ranks / the range of one rank: DEVICE base pointer, its size,
+ * the slab stride, the matrix size and the slot count.  NULL outputs are skipped. */
+emoe_status_t emoe_vmm_num_ranks(const emoe_vmm_pool_t *pool, int32_t *n);
+emoe_status_t emoe_vmm_arena(const emoe_vmm_pool_t *pool, int rank, void **base, uint64_t *bytes,
+                             uint64_t *slab_bytes, uint64_t *matrix_bytes, int32_t *n_slots);
+
+/* Copies a DENSE host image [L][3][n_r][m] of rank `rank` into / out of its
+ * paged range (asynchronous on cuda_stream; pinned memory to overlap). */
+emoe_status_t emoe_vmm_write(emoe_vmm_pool_t *pool, int rank, const void *host_dense,
+                             void *cuda_stream);
+emoe_status_t emoe_vmm_read(const emoe_vmm_pool_t *pool, int rank, void *host_dense,
+                            void *cuda_stream);
+
+/* Unmaps and frees everything (synchronises the device first).  NULL-safe. */
+void emoe_vmm_destroy(emoe_vmm_pool_t *pool);
+
 /* emoe_plan_destroy - frees host state and device descriptor buffers.
  * NULL-safe.  No kernel using the plan may still be in flight. */
 void emoe_plan_destroy(emoe_plan_t *plan);

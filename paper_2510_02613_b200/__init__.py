@@ -3,9 +3,9 @@ step (expert re-pack for EP a->b, attention re-slice and KV head re-split for TP
 c->d).  The work is done by libemoe.so (host planner, C ABI, sm_100a copy
 kernels); this package is its thin ctypes binding."""
 from .binding import (EXPORTS, MAX_RANKS, PHASE_ATTN, PHASE_EXPERTS, PHASE_KV, PLAN_HOST_ONLY, PLAN_HOST_STEP,
-                      SEGMENT_DTYPE, SIDE_NEW, SIDE_OLD, EmoeError, Plan, lib, library_path,
-                      strerror)
+                      SEGMENT_DTYPE, SIDE_NEW, SIDE_OLD, EmoeError, Plan, VmmPool, lib, library_path,
+                      strerror, vmm_dry_run)
 
 __all__ = ["EXPORTS", "MAX_RANKS", "PHASE_ATTN", "PHASE_EXPERTS", "PHASE_KV", "PLAN_HOST_ONLY", "PLAN_HOST_STEP",
-           "SEGMENT_DTYPE", "SIDE_NEW", "SIDE_OLD", "EmoeError", "Plan", "lib", "library_path",
-           "strerror"]
+           "SEGMENT_DTYPE", "SIDE_NEW", "SIDE_OLD", "EmoeError", "Plan", "VmmPool", "lib", "library_path",
+           "strerror", "vmm_dry_run"]

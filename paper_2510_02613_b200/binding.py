@@ -54,6 +54,12 @@ class _Tuning(ctypes.Structure):
                 ("unit_order", _i32)]
 
 
+class _VmmStats(ctypes.Structure):
+    _fields_ = [(n, _u64) for n in ("slabs_remapped", "slabs_copied", "bytes_copied", "bytes_read",
+                                    "slab_bytes", "matrix_bytes", "physical_bytes")] + \
+               [(n, ctypes.c_double) for n in ("map_ms", "copy_ms", "unmap_ms", "total_ms")]
+
+
 SEGMENT_DTYPE = np.dtype([("src_off", "<u8"), ("dst_off", "<u8"), ("run_bytes", "<u8"),
                           ("src_pitch", "<u8"), ("dst_pitch", "<u8"), ("n_runs", "<u4"),
                           ("src_rank", "<u4"), ("dst_rank", "<u4"), ("group", "<u4")])
@@ -62,7 +68,9 @@ EXPORTS = ("emoe_plan_create", "emoe_reshard_experts", "emoe_reshard_attn", "emo
            "emoe_reshard_kv_static",
            "emoe_reshard_step_host", "emoe_plan_destroy", "emoe_plan_num_ranks",
            "emoe_plan_arena_bytes", "emoe_plan_stats", "emoe_plan_num_launches", "emoe_plan_segments",
-           "emoe_plan_device_status", "emoe_plan_set_tuning", "emoe_strerror")
+           "emoe_plan_device_status", "emoe_plan_set_tuning", "emoe_strerror",
+           "emoe_vmm_create", "emoe_vmm_reshard", "emoe_vmm_dry_run", "emoe_vmm_num_ranks", "emoe_vmm_arena",
+           "emoe_vmm_write", "emoe_vmm_read", "emoe_vmm_destroy")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -112,6 +120,24 @@ def lib() -> ctypes.CDLL:
     L.emoe_plan_device_status.argtypes = [_vp, ctypes.POINTER(_i32)]
     L.emoe_plan_set_tuning.restype = _i32
     L.emoe_plan_set_tuning.argtypes = [_vp, ctypes.POINTER(_Tuning)]
+    L.emoe_vmm_create.restype = _i32
+    L.emoe_vmm_create.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Config), ctypes.POINTER(_vp)]
+    L.emoe_vmm_reshard.restype = _i32
+    L.emoe_vmm_reshard.argtypes = [_vp, ctypes.POINTER(_Config), _vp, ctypes.POINTER(_VmmStats)]
+    L.emoe_vmm_dry_run.restype = _i32
+    L.emoe_vmm_dry_run.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Config),
+                                   ctypes.POINTER(_Config), _u64, ctypes.POINTER(_VmmStats)]
+    L.emoe_vmm_num_ranks.restype = _i32
+    L.emoe_vmm_num_ranks.argtypes = [_vp, ctypes.POINTER(_i32)]
+    L.emoe_vmm_arena.restype = _i32
+    L.emoe_vmm_arena.argtypes = [_vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_u64),
+                                 ctypes.POINTER(_u64), ctypes.POINTER(_u64), ctypes.POINTER(_i32)]
+    for name in ("emoe_vmm_write", "emoe_vmm_read"):
+        f = getattr(L, name)
+        f.restype = _i32
+        f.argtypes = [_vp, _i32, _vp, _vp]
+    L.emoe_vmm_destroy.restype = None
+    L.emoe_vmm_destroy.argtypes = [_vp]
     L.emoe_strerror.restype = ctypes.c_char_p
     L.emoe_strerror.argtypes = [_i32]
     _lib = L
@@ -288,3 +314,87 @@ class Plan:
 
         _check(lib().emoe_reshard_step_host(self._h, pack(h_src), pack(h_dst), pack(d_src),
                                             pack(d_dst), _stream_handle(stream)))
+
+
+def _placement_config(placement, keep: list) -> _Config:
+    off = np.zeros(len(placement) + 1, dtype=np.int32)
+    off[1:] = np.cumsum([len(p) for p in placement])
+    ids = _i32arr([e for p in placement for e in p])
+    if ids.size == 0:
+        ids = np.zeros(1, dtype=np.int32)
+    keep += [off, ids]
+    p = lambda a: a.ctypes.data_as(_i32p)
+    return _Config(len(placement), 1, p(off), p(ids), 0, 0, 0, None, None)
+
+
+def vmm_dry_run(shape, old_placement, new_placement, slab_bytes: int) -> dict:
+    """What VmmPool.reshard would re-map and copy, computed on the host (no CUDA call)."""
+    keep: list = []
+    sh = _Shape(shape.n_layers, shape.n_routed, shape.n_shared, shape.d_model, shape.d_ff,
+                shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.kv_block_tokens,
+                shape.elem_bytes)
+    st = _VmmStats()
+    _check(lib().emoe_vmm_dry_run(ctypes.byref(sh), ctypes.byref(_placement_config(old_placement, keep)),
+                                  ctypes.byref(_placement_config(new_placement, keep)), slab_bytes,
+                                  ctypes.byref(st)))
+    return {n: getattr(st, n) for n, _ in _VmmStats._fields_}
+
+
+class VmmPool:
+    """Paged expert store: emoe_vmm_create ... emoe_vmm_destroy.  `cfg` objects need
+    `placement` (expert ids per rank) only."""
+
+    def __init__(self, shape, cfg):
+        self._h = _vp()
+        self._keep: list = []
+        sh = _Shape(shape.n_layers, shape.n_routed, shape.n_shared, shape.d_model, shape.d_ff,
+                    shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.kv_block_tokens,
+                    shape.elem_bytes)
+        _check(lib().emoe_vmm_create(ctypes.byref(sh), ctypes.byref(self._config(cfg)),
+                                     ctypes.byref(self._h)))
+
+    def _config(self, cfg) -> _Config:
+        placement = cfg.placement if hasattr(cfg, "placement") else cfg
+        self._keep = []
+        return _placement_config(placement, self._keep)
+
+    def close(self) -> None:
+        if self._h:
+            lib().emoe_vmm_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    def num_ranks(self) -> int:
+        n = _i32()
+        _check(lib().emoe_vmm_num_ranks(self._h, ctypes.byref(n)))
+        return n.value
+
+    def arena(self, rank: int) -> dict:
+        base, b, s, m, n = _vp(), _u64(), _u64(), _u64(), _i32()
+        _check(lib().emoe_vmm_arena(self._h, rank, ctypes.byref(base), ctypes.byref(b),
+                                    ctypes.byref(s), ctypes.byref(m), ctypes.byref(n)))
+        return dict(base=base.value or 0, bytes=b.value, slab_bytes=s.value, matrix_bytes=m.value,
+                    n_slots=n.value)
+
+    def write(self, rank: int, host_dense, stream=None) -> None:
+        _check(lib().emoe_vmm_write(self._h, rank, _ptr_array([host_dense])[0], _stream_handle(stream)))
+
+    def read(self, rank: int, host_dense, stream=None) -> None:
+        _check(lib().emoe_vmm_read(self._h, rank, _ptr_array([host_dense])[0], _stream_handle(stream)))
+
+    def reshard(self, new_cfg, stream=None) -> dict:
+        st = _VmmStats()
+        _check(lib().emoe_vmm_reshard(self._h, ctypes.byref(self._config(new_cfg)),
+                                      _stream_handle(stream), ctypes.byref(st)))
+        return {n: getattr(st, n) for n, _ in _VmmStats._fields_}

@@ -8,6 +8,7 @@
 #include <new>
 #include <vector>
 
+#include "internal.h"
 #include "kernels.h"
 #include "planner.h"
 
@@ -376,6 +377,43 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
 }
 
 }  // namespace
+
+emoe_status_t emoe::run_phase_once(const PhasePlan &pp, const RankPtrs &ptrs, cudaStream_t st) {
+  emoe_plan tmp;
+  tmp.host_only = false;
+  emoe_status_t rc = EMOE_OK;
+  try {
+    tmp.hp.phase[0] = pp;
+    build_tables(&tmp, 0);
+  } catch (const std::bad_alloc &) {
+    return EMOE_ERR_OOM;
+  }
+  cudaError_t e = cudaGetDevice(&tmp.device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&tmp.sm_count, cudaDevAttrMultiProcessorCount, tmp.device);
+  if (e == cudaSuccess) {
+    std::call_once(g_init_once, [] { g_init_err = kernels_init(); });
+    e = g_init_err;
+  }
+  rc = cuda_status(e);
+  if (rc == EMOE_OK) rc = upload_phase(&tmp, 0);
+  if (rc == EMOE_OK) {
+    e = cudaMalloc((void **)&tmp.d_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemsetAsync(tmp.d_status, 0, sizeof(int), st);
+    rc = cuda_status(e);
+  }
+  if (rc == EMOE_OK) rc = run_segments(&tmp, 0, ptrs, st);
+  int status = 0;
+  if (rc == EMOE_OK) {
+    e = cudaMemcpyAsync(&status, tmp.d_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    rc = cuda_status(e);
+    if (rc == EMOE_OK && status != 0) rc = (emoe_status_t)status;
+  } else {
+    (void)cudaStreamSynchronize(st);
+  }
+  free_device(&tmp);
+  return rc;
+}
 
 extern "C" {
 

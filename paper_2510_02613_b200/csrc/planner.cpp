@@ -97,13 +97,17 @@ emoe_status_t read_block_pairs(const emoe_shape_t &sh, const emoe_config_t &o,
 
 // ---- experts ----------------------------------------------------------------------------
 
-void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &pn,
-                  PhasePlan *pp) {
+// slab: distance between consecutive slots of an arena (= m for the dense layout; the
+// paged store pads every matrix to its allocation granularity).  remaps: if non-null,
+// a destination slot whose source sits on the same rank index is recorded there instead
+// of being copied (that device already holds the bytes).
+void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &pn, uint64_t slab,
+                  std::vector<Remap> *remaps, PhasePlan *pp) {
   const uint64_t m = (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes;
   const uint32_t runs = (uint32_t)sh.n_layers * 3;
   const int n_experts = sh.n_routed + sh.n_shared;
-  for (int r = 0; r < po.ep; ++r) pp->arena_old.push_back(runs * po.ids[r].size() * m);
-  for (int r = 0; r < pn.ep; ++r) pp->arena_new.push_back(runs * pn.ids[r].size() * m);
+  for (int r = 0; r < po.ep; ++r) pp->arena_old.push_back(runs * po.ids[r].size() * slab);
+  for (int r = 0; r < pn.ep; ++r) pp->arena_new.push_back(runs * pn.ids[r].size() * slab);
 
   // every old copy of every expert, in (rank, slot) order
   std::vector<std::vector<std::pair<int, int>>> copies(n_experts);
@@ -120,41 +124,45 @@ void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &
       std::pair<int, int> src = c.front();
       for (const auto &x : c)
         if (x.first == rd) { src = x; break; }
+      if (remaps && src.first == rd) {
+        remaps->push_back({(uint32_t)src.first, (uint32_t)src.second, (uint32_t)rd, (uint32_t)sd});
+        continue;
+      }
       moves.push_back({src.first, src.second, rd, sd});
       fan[src]++;
     }
 
-  // single-destination sources: merge runs of consecutive slots on both sides
+  // single-destination sources: merge runs of consecutive slots on both sides (dense layout only)
   std::map<std::pair<int, int>, std::vector<Dst>> multi;
   size_t i = 0;
   while (i < moves.size()) {
     const Move &a = moves[i];
     const uint64_t n_old = po.ids[a.rs].size(), n_new = pn.ids[a.rd].size();
     if (fan[{a.rs, a.ss}] > 1) {
-      multi[{a.rs, a.ss}].push_back({(uint64_t)a.sd * m, n_new * m, (uint32_t)a.rd, 0});
+      multi[{a.rs, a.ss}].push_back({(uint64_t)a.sd * slab, n_new * slab, (uint32_t)a.rd, 0});
       ++i;
       continue;
     }
     size_t j = i + 1;
-    while (j < moves.size() && moves[j].rd == a.rd && moves[j].rs == a.rs &&
+    while (slab == m && j < moves.size() && moves[j].rd == a.rd && moves[j].rs == a.rs &&
            moves[j].sd == moves[j - 1].sd + 1 && moves[j].ss == moves[j - 1].ss + 1 &&
            fan[{moves[j].rs, moves[j].ss}] == 1)
       ++j;
     Segment s{};
-    s.src_off = (uint64_t)a.ss * m;
+    s.src_off = (uint64_t)a.ss * slab;
     s.run_bytes = (uint64_t)(j - i) * m;
-    s.src_pitch = n_old * m;
+    s.src_pitch = n_old * slab;
     s.n_runs = runs;
     s.src_rank = (uint32_t)a.rs;
-    finish_segment(pp, s, {Dst{(uint64_t)a.sd * m, n_new * m, (uint32_t)a.rd, 0}});
+    finish_segment(pp, s, {Dst{(uint64_t)a.sd * slab, n_new * slab, (uint32_t)a.rd, 0}});
     i = j;
   }
   // replicated sources: read once, write to every destination
   for (const auto &kv : multi) {
     Segment s{};
-    s.src_off = (uint64_t)kv.first.second * m;
+    s.src_off = (uint64_t)kv.first.second * slab;
     s.run_bytes = m;
-    s.src_pitch = po.ids[kv.first.first].size() * m;
+    s.src_pitch = po.ids[kv.first.first].size() * slab;
     s.n_runs = runs;
     s.src_rank = (uint32_t)kv.first.first;
     finish_segment(pp, s, kv.second);
@@ -292,9 +300,26 @@ emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
 
   hp->shape = sh;
   hp->ep_old = o.ep; hp->ep_new = n.ep; hp->tp_old = o.tp; hp->tp_new = n.tp;
-  plan_experts(sh, po, pn, &hp->phase[EMOE_PHASE_EXPERTS]);
+  plan_experts(sh, po, pn, (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes, nullptr,
+               &hp->phase[EMOE_PHASE_EXPERTS]);
   plan_attn(sh, o.tp, n.tp, &hp->phase[EMOE_PHASE_ATTN]);
   plan_kv(sh, o, n, std::move(pair_old), std::move(pair_new), hp);
+  return EMOE_OK;
+}
+
+emoe_status_t build_paged_expert_plan(const emoe_shape_t &sh, const emoe_config_t &o,
+                                      const emoe_config_t &n, uint64_t slab, PhasePlan *pp,
+                                      std::vector<Remap> *remaps) {
+  if (sh.n_layers <= 0 || sh.n_routed <= 0 || sh.n_shared < 0 || sh.d_model <= 0 || sh.d_ff <= 0 ||
+      sh.elem_bytes <= 0)
+    return EMOE_ERR_SHAPE;
+  if (slab < (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes) return EMOE_ERR_INVALID_ARG;
+  Placement po, pn;
+  emoe_status_t st = read_placement(o, sh.n_routed + sh.n_shared, &po);
+  if (st != EMOE_OK) return st;
+  st = read_placement(n, sh.n_routed + sh.n_shared, &pn);
+  if (st != EMOE_OK) return st;
+  plan_experts(sh, po, pn, slab, remaps, pp);
   return EMOE_OK;
 }
 

@@ -63,6 +63,17 @@ struct HostPlan {
 emoe_status_t build_host_plan(const emoe_shape_t &shape, const emoe_config_t &old_cfg,
                               const emoe_config_t &new_cfg, HostPlan *out);
 
+// A destination slot that keeps the bytes its rank already holds (paged expert store).
+struct Remap {
+  uint32_t src_rank, src_slot, dst_rank, dst_slot;
+};
+
+// Expert phase for arenas whose slots are `slab` bytes apart (slab >= one matrix).  Slots
+// whose source is on the same rank index go to `remaps` instead of being copied.
+emoe_status_t build_paged_expert_plan(const emoe_shape_t &shape, const emoe_config_t &old_cfg,
+                                      const emoe_config_t &new_cfg, uint64_t slab, PhasePlan *pp,
+                                      std::vector<Remap> *remaps);
+
 // Expands a phase into flat emoe_segment_t records (one per destination).  For a
 // KV plan with a changing head split the block pairs are expanded per (pair, old
 // rank, new rank) overlap.

@@ -206,3 +206,24 @@ def test_full_size_configs_sampled_layers(name):
             check_phase_layers(wl, plan, phase, src, dst, [0, L // 2, L - 1])
             del src, dst
             torch.cuda.empty_cache()
+
+
+def test_maximum_rank_counts():
+    """EMOE_MAX_RANKS = 64 ranks on both sides of every phase: EP 64 -> 63 with replicas,
+    TP 1 -> 64 and back (64 KV heads, one per rank)."""
+    n = E.MAX_RANKS
+    sh = W.Shape(1, 2 * n, 1, 16, 8, n, n, 8, 4, 2)
+    seq_lens = [9, 4]
+    nblk = sum(-(-x // 4) for x in seq_lens)
+    bo = W.make_block_table(21, seq_lens, 4, nblk)
+    bn = W.make_block_table(22, seq_lens, 4, nblk + 3)
+    old = W.ParallelConfig(n, 1, W.with_shared(W.place_round_robin(2 * n, n), [2 * n]), nblk, seq_lens, bo)
+    new = W.ParallelConfig(n - 1, n, W.with_shared(W.place_contiguous(2 * n, n - 1), [2 * n]),
+                           nblk + 3, seq_lens, bn)
+    wl = W.Workload("max_ranks", sh, old, new, 9)
+    for w in (wl, wl.swapped()):
+        with E.Plan(w.shape, w.old, w.new) as plan:
+            for kv_mode in (1, 2, 3):
+                plan.set_tuning(kv_mode=kv_mode)
+                for phase in range(3):
+                    check_phase_full(w, plan, phase)

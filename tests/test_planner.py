@@ -195,3 +195,16 @@ def test_library_exports_every_declared_symbol():
     lib = ctypes.CDLL(E.library_path())
     for name in declared:
         assert hasattr(lib, name), name
+
+
+def test_more_ranks_than_the_library_supports():
+    n = E.MAX_RANKS + 1
+    sh = W.Shape(1, n, 0, 8, 8, n, n, 8, 4, 2)
+    empty = np.zeros((0, 0), np.int32)
+    ok = W.ParallelConfig(1, 1, [list(range(n))], 1, [], empty)
+    too_many_ep = W.ParallelConfig(n, 1, W.place_round_robin(n, n), 1, [], empty)
+    too_many_tp = W.ParallelConfig(1, n, [list(range(n))], 1, [], empty)
+    for bad in (too_many_ep, too_many_tp):
+        with pytest.raises(E.EmoeError) as ei:
+            E.Plan(sh, ok, bad, host_only=True)
+        assert ei.value.code == 9
