@@ -358,6 +358,27 @@ def run_overlap(torch, E, plan, wl, src, dst, peak, budgets=(0, 96, 48, 24)):
     return out
 
 
+# ---- paged expert store: the expert phase as a page re-map plus copies of arrivals -------
+
+def run_vmm(torch, E, wl, copy_all_ms):
+    """Times emoe_vmm_reshard for the workload's expert placements (old -> new) on a pool of
+    uninitialised pages (byte movement does not depend on values) and sets it beside the
+    dense copy-everything expert phase.  Host wall-clock: the call is synchronous."""
+    torch.cuda.empty_cache()
+    try:
+        with E.VmmPool(wl.shape, wl.old.placement) as pool:
+            torch.cuda.synchronize()
+            st = pool.reshard(wl.new.placement)
+    except E.EmoeError as e:
+        return {"error": str(e)}
+    out = {k: (round(v, 3) if isinstance(v, float) else v) for k, v in st.items()}
+    out["copy_gbs"] = round((st["bytes_copied"] + st["bytes_read"]) / st["copy_ms"] / 1e6, 1) \
+        if st["copy_ms"] > 0 and st["bytes_copied"] else None
+    out["dense_copy_all_ms"] = round(copy_all_ms, 3)
+    out["padding_overhead"] = round(st["slab_bytes"] / st["matrix_bytes"] - 1, 4)
+    return out
+
+
 # ---- reference arm: the oracle on the host cores -----------------------------------------
 
 def run_reference(args):
@@ -504,6 +525,8 @@ def main():
     del src, dst
     plan.close()
     torch.cuda.empty_cache()
+    if rank == 0 and not args.only_main:
+        rep["vmm_expert_step"] = run_vmm(torch, E, wl, rep["phases"]["experts"]["ms"])
 
     if not args.only_main and world == 1:
         others = {}
@@ -525,6 +548,8 @@ def main():
             del src2, dst2
             plan2.close()
             torch.cuda.empty_cache()
+            if name != "c5_overlap":
+                r["vmm_expert_step"] = run_vmm(torch, E, wl2, r["phases"]["experts"]["ms"])
         line["configs"] = others
 
     if dist:

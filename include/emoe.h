@@ -270,7 +270,10 @@ typedef struct {
   uint64_t bytes_read;     /* bytes they read (a source with several arrivals: once)    */
   uint64_t slab_bytes, matrix_bytes;
   uint64_t physical_bytes; /* device memory the pool holds after the step               */
-  double map_ms;           /* host time: reserve ranges, allocate and map slabs         */
+  double map_ms;           /* host time: reserve ranges, allocate and map slabs, enable */
+                           /* access; alloc_ms and access_ms are parts of it            */
+  double alloc_ms;         /* ... of which allocating the arrivals' physical pages      */
+  double access_ms;        /* ... of which enabling access to the new ranges            */
   double copy_ms;          /* host time: plan upload, copy kernels, stream synchronise  */
   double unmap_ms;         /* host time: unmap and free the old ranges, release pages   */
   double total_ms;

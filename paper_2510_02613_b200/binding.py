@@ -57,7 +57,8 @@ class _Tuning(ctypes.Structure):
 class _VmmStats(ctypes.Structure):
     _fields_ = [(n, _u64) for n in ("slabs_remapped", "slabs_copied", "bytes_copied", "bytes_read",
                                     "slab_bytes", "matrix_bytes", "physical_bytes")] + \
-               [(n, ctypes.c_double) for n in ("map_ms", "copy_ms", "unmap_ms", "total_ms")]
+               [(n, ctypes.c_double) for n in ("map_ms", "alloc_ms", "access_ms", "copy_ms", "unmap_ms",
+                                               "total_ms")]
 
 
 SEGMENT_DTYPE = np.dtype([("src_off", "<u8"), ("dst_off", "<u8"), ("run_bytes", "<u8"),

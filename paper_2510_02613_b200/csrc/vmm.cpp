@@ -357,14 +357,18 @@ emoe_status_t emoe_vmm_reshard(emoe_vmm_pool_t *pool, const emoe_config_t *new_c
             s.slabs_remapped++;
           } else {
             CUmemGenericAllocationHandle h = 0;
+            const double ta = now_ms();
             rc = new_slab(pool, &h);
+            s.alloc_ms += now_ms() - ta;
             if (rc != EMOE_OK) break;
             rc = map_next(pool, &rg, h);
             if (rc != EMOE_OK) driver().MemRelease(h);
             s.slabs_copied++;
           }
         }
+      const double ta = now_ms();
       if (rc == EMOE_OK) rc = enable_access(pool, rg);
+      s.access_ms += now_ms() - ta;
     }
     const double t1 = now_ms();
     s.map_ms = t1 - t0;
