@@ -24,6 +24,13 @@
 //    caches" under a TP change (Sec. 9) is read as a contiguous split of the
 //    KV heads, block tables translating physical block ids.
 //
+//  * more TP ranks than KV heads (grouped-query attention; the paper is silent):
+//    read in the usual way - with T > Hkv and Hkv | T every KV head is held by
+//    T / Hkv consecutive ranks, one head per rank: rank t holds head
+//    floor(t * Hkv / T).  Which replica a new rank copies from follows the same
+//    rule as for replicated experts: the old rank with the same index if it
+//    holds the head, else the smallest old rank that does.
+//
 // Pins: every function below is pinned by tests that do not use it to make
 // their expectation (numpy/torch indexing of logical tensors, hand-written
 // fixtures, identities and round trips); none is "parity unpinned".
@@ -55,6 +62,24 @@ bool find_source(const Csr &old_p, int e, int r_new, int *r_out, int *s_out) {
   return false;
 }
 
+// KV heads of a TP=T group: heads per rank, first head of rank t, and the old rank
+// a new rank takes global head g from (own index first, else the smallest holder).
+int64_t kv_heads_per_rank(int64_t hkv, int64_t T) { return hkv >= T ? hkv / T : 1; }
+int64_t kv_first_head(int64_t hkv, int64_t T, int64_t t) { return t * hkv / T; }
+bool kv_tp_ok(int64_t hkv, int64_t T) { return T >= 1 && (hkv >= T ? hkv % T == 0 : T % hkv == 0); }
+int64_t kv_source_rank(int64_t hkv, int64_t c, int64_t g, int64_t r_new) {
+  const int64_t h = kv_heads_per_rank(hkv, c);
+  if (r_new < c) {
+    const int64_t f = kv_first_head(hkv, c, r_new);
+    if (f <= g && g < f + h) return r_new;
+  }
+  for (int64_t r = 0; r < c; ++r) {
+    const int64_t f = kv_first_head(hkv, c, r);
+    if (f <= g && g < f + h) return r;
+  }
+  return -1;
+}
+
 }  // namespace
 
 extern "C" {
@@ -68,14 +93,14 @@ int64_t emoe_oracle_expert_arena_bytes(int n_layers, int n_slots, int64_t m) {
 int64_t emoe_oracle_attn_arena_bytes(int n_layers, int d_model, int hq, int hkv, int hd, int b,
                                      int tp) {
   int64_t q = (int64_t)(hq / tp) * hd * d_model * b;
-  int64_t kv = (int64_t)(hkv / tp) * hd * d_model * b;
+  int64_t kv = kv_heads_per_rank(hkv, tp) * hd * d_model * b;
   return (int64_t)n_layers * (q + 2 * kv + q);
 }
 
 // Bytes of the KV arena of one TP rank: [L][2][NB][B][Hkv/T][hd].
 int64_t emoe_oracle_kv_arena_bytes(int n_layers, int nb, int block_tokens, int hkv, int hd, int b,
                                    int tp) {
-  return (int64_t)n_layers * 2 * nb * block_tokens * (hkv / tp) * hd * b;
+  return (int64_t)n_layers * 2 * nb * block_tokens * kv_heads_per_rank(hkv, tp) * hd * b;
 }
 
 // Expert re-pack.  m = bytes of one expert matrix.  Returns 0, or -1 if an
@@ -104,29 +129,38 @@ int emoe_oracle_reshard_experts(int n_layers, int64_t m, int ep_old, const int32
 // Attention re-slice TP=c -> TP=d.  b = bytes per element.
 int emoe_oracle_reshard_attn(int n_layers, int d_model, int hq, int hkv, int hd, int b, int c,
                              int d, const uint8_t *const *src, uint8_t *const *dst) {
-  if (hq % c || hq % d || hkv % c || hkv % d) return -1;
+  if (hq % c || hq % d || !kv_tp_ok(hkv, c) || !kv_tp_ok(hkv, d)) return -1;
   const int64_t D = d_model;
   const int64_t row = D * b;  // one stored row of Wq / Wk / Wv
   // sizes of the four pieces of one layer on a rank of a TP=T group
   auto q_bytes = [&](int T) { return (int64_t)(hq / T) * hd * row; };
-  auto kv_bytes = [&](int T) { return (int64_t)(hkv / T) * hd * row; };
+  auto kv_bytes = [&](int T) { return kv_heads_per_rank(hkv, T) * hd * row; };
   auto layer_bytes = [&](int T) { return 2 * q_bytes(T) + 2 * kv_bytes(T); };
 
   for (int l = 0; l < n_layers; ++l) {
-    // q, k, v: global stored row g of the logical matrix
-    for (int t = 0; t < 3; ++t) {
-      const int heads = (t == 0) ? hq : hkv;
-      const int64_t rows = (int64_t)heads * hd;
+    // q: global stored row g of the logical matrix
+    {
+      const int64_t rows = (int64_t)hq * hd;
       const int64_t rows_c = rows / c, rows_d = rows / d;
-      auto piece_off = [&](int T) {
-        return (t == 0) ? 0 : (t == 1) ? q_bytes(T) : q_bytes(T) + kv_bytes(T);
-      };
       for (int64_t g = 0; g < rows; ++g) {
         const int64_t ro = g / rows_c, lo = g % rows_c;
         const int64_t rn = g / rows_d, ln = g % rows_d;
-        std::memcpy(dst[rn] + l * layer_bytes(d) + piece_off(d) + ln * row,
-                    src[ro] + l * layer_bytes(c) + piece_off(c) + lo * row, (size_t)row);
+        std::memcpy(dst[rn] + l * layer_bytes(d) + ln * row, src[ro] + l * layer_bytes(c) + lo * row,
+                    (size_t)row);
       }
+    }
+    // k, v: every new rank's local heads, each taken from the old rank chosen for that head
+    for (int t = 1; t < 3; ++t) {
+      auto piece_off = [&](int T) { return (t == 1) ? q_bytes(T) : q_bytes(T) + kv_bytes(T); };
+      for (int rn = 0; rn < d; ++rn)
+        for (int64_t hl = 0; hl < kv_heads_per_rank(hkv, d); ++hl) {
+          const int64_t g = kv_first_head(hkv, d, rn) + hl;
+          const int64_t ro = kv_source_rank(hkv, c, g, rn);
+          const int64_t ho = g - kv_first_head(hkv, c, ro);
+          for (int64_t r = 0; r < hd; ++r)
+            std::memcpy(dst[rn] + l * layer_bytes(d) + piece_off(d) + (hl * hd + r) * row,
+                        src[ro] + l * layer_bytes(c) + piece_off(c) + (ho * hd + r) * row, (size_t)row);
+        }
     }
     // o: stored row i, head h owns columns [h*hd, (h+1)*hd) of the logical Wo
     const int64_t o_off_c = q_bytes(c) + 2 * kv_bytes(c), o_off_d = q_bytes(d) + 2 * kv_bytes(d);
@@ -150,8 +184,9 @@ int emoe_oracle_reshard_kv(int n_layers, int block_tokens, int hkv, int hd, int 
                            int nb_old, int nb_new, int n_seqs, int max_blocks,
                            const int32_t *seq_lens, const int32_t *bt_old, const int32_t *bt_new,
                            const uint8_t *const *src, uint8_t *const *dst) {
-  if (hkv % c || hkv % d) return -1;
-  const int64_t B = block_tokens, hc = hkv / c, hdn = hkv / d, vec = (int64_t)hd * b;
+  if (!kv_tp_ok(hkv, c) || !kv_tp_ok(hkv, d)) return -1;
+  const int64_t B = block_tokens, hc = kv_heads_per_rank(hkv, c), hdn = kv_heads_per_rank(hkv, d);
+  const int64_t vec = (int64_t)hd * b;
   for (int s = 0; s < n_seqs; ++s) {
     const int n_blk = (int)((seq_lens[s] + B - 1) / B);
     for (int j = 0; j < n_blk; ++j) {
@@ -161,12 +196,15 @@ int emoe_oracle_reshard_kv(int n_layers, int block_tokens, int hkv, int hd, int 
       for (int l = 0; l < n_layers; ++l)
         for (int kv = 0; kv < 2; ++kv)
           for (int64_t tok = 0; tok < B; ++tok)
-            for (int64_t g = 0; g < hkv; ++g) {
-              const int64_t ro = g / hc, ho = g % hc, rn = g / hdn, hn = g % hdn;
-              const int64_t off_o = (((((int64_t)l * 2 + kv) * nb_old + po) * B + tok) * hc + ho) * vec;
-              const int64_t off_n = (((((int64_t)l * 2 + kv) * nb_new + pn) * B + tok) * hdn + hn) * vec;
-              std::memcpy(dst[rn] + off_n, src[ro] + off_o, (size_t)vec);
-            }
+            for (int64_t rn = 0; rn < d; ++rn)
+              for (int64_t hn = 0; hn < hdn; ++hn) {
+                const int64_t g = kv_first_head(hkv, d, rn) + hn;   // global KV head
+                const int64_t ro = kv_source_rank(hkv, c, g, rn);
+                const int64_t ho = g - kv_first_head(hkv, c, ro);
+                const int64_t off_o = (((((int64_t)l * 2 + kv) * nb_old + po) * B + tok) * hc + ho) * vec;
+                const int64_t off_n = (((((int64_t)l * 2 + kv) * nb_new + pn) * B + tok) * hdn + hn) * vec;
+                std::memcpy(dst[rn] + off_n, src[ro] + off_o, (size_t)vec);
+              }
     }
   }
   return 0;

@@ -42,12 +42,35 @@ def logical_attn(shape, key=2):
     )
 
 
-def attn_arenas(logical, tp):
-    """Rank t: per layer q_t | k_t | v_t | o_t, pieces cut with numpy.split."""
+def kv_heads_of_rank(n_kv_heads, tp, t):
+    """KV heads a TP rank holds: a contiguous share, or - with more ranks than heads -
+    the single head floor(t * Hkv / tp) (every head on tp / Hkv consecutive ranks)."""
+    n = max(1, n_kv_heads // tp)
+    first = t * n_kv_heads // tp
+    return list(range(first, first + n))
+
+
+def _split_kv_rows(x, tp, head_dim):
+    """k or v weight [L, Hkv*hd, row bytes] -> per-rank row slices (whole heads)."""
+    hkv = x.shape[1] // head_dim
+    out = []
+    for t in range(tp):
+        rows = [h * head_dim + r for h in kv_heads_of_rank(hkv, tp, t) for r in range(head_dim)]
+        out.append(x[:, rows])
+    return out
+
+
+def attn_arenas(logical, tp, head_dim=None):
+    """Rank t: per layer q_t | k_t | v_t | o_t, pieces cut with numpy.split (k and v by
+    whole KV heads when head_dim is given, which also covers tp > Hkv)."""
     L = logical["q"].shape[0]
     qs = np.split(logical["q"], tp, axis=1)
-    ks = np.split(logical["k"], tp, axis=1)
-    vs = np.split(logical["v"], tp, axis=1)
+    if head_dim is None:
+        ks = np.split(logical["k"], tp, axis=1)
+        vs = np.split(logical["v"], tp, axis=1)
+    else:
+        ks = _split_kv_rows(logical["k"], tp, head_dim)
+        vs = _split_kv_rows(logical["v"], tp, head_dim)
     os_ = np.split(logical["o"], tp, axis=2)
     out = []
     for t in range(tp):
@@ -73,7 +96,7 @@ def kv_arenas(logical, shape, cfg, background=None):
     """Scatters logical blocks into each rank's pool through the block table."""
     B = shape.kv_block_tokens
     L, vec = shape.n_layers, shape.head_dim * shape.elem_bytes
-    hl = shape.n_kv_heads // cfg.tp
+    hl = max(1, shape.n_kv_heads // cfg.tp)
     phys = []
     for s, n in enumerate(cfg.seq_lens):
         phys += [int(x) for x in cfg.block_table[s, :-(-n // B)]]
@@ -83,6 +106,6 @@ def kv_arenas(logical, shape, cfg, background=None):
             pool = np.full((L, 2, cfg.kv_num_blocks, B, hl, vec), FILL, dtype=np.uint8)
         else:
             pool = background[t].reshape(L, 2, cfg.kv_num_blocks, B, hl, vec).copy()
-        pool[:, :, phys] = logical[:, :, :, :, t * hl:(t + 1) * hl]
+        pool[:, :, phys] = logical[:, :, :, :, kv_heads_of_rank(shape.n_kv_heads, cfg.tp, t)]
         out.append(pool.reshape(-1))
     return out

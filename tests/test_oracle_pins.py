@@ -228,10 +228,25 @@ def test_attn_fixed_tp_is_memcpy_and_round_trip():
 
 
 def test_attn_rejects_tp_not_dividing_heads():
-    sh = tiny_shape(n_kv_heads=2)
-    with pytest.raises(ValueError):
-        oracle.reshard_attn(sh, 1, 4, [np.zeros(oracle.attn_arena_bytes(sh, 1)[0], np.uint8)],
-                            [np.zeros(1, np.uint8)] * 4)
+    sh = tiny_shape(n_kv_heads=2, n_q_heads=12)
+    with pytest.raises(ValueError):      # 3 ranks: neither 2 % 3 nor 3 % 2 is zero
+        oracle.reshard_attn(sh, 1, 3, [np.zeros(oracle.attn_arena_bytes(sh, 1)[0], np.uint8)],
+                            [np.zeros(1, np.uint8)] * 3)
+
+
+@pytest.mark.parametrize("c,d", [(1, 4), (2, 8), (8, 2), (4, 8), (8, 4), (8, 8), (2, 4)])
+def test_attn_more_ranks_than_kv_heads_equals_numpy_head_slices(c, d):
+    """Hkv = 2: with TP > 2 every rank holds ONE k/v head (head floor(t*Hkv/T)), q and o
+    are still split T ways.  Expected arenas are numpy slices of the logical matrices."""
+    sh = tiny_shape(n_q_heads=8, n_kv_heads=2)
+    logical = logical_attn(sh)
+    src = attn_arenas(logical, c, sh.head_dim)
+    want = attn_arenas(logical, d, sh.head_dim)
+    assert [a.size for a in want] == oracle.attn_arena_bytes(sh, d)
+    dst = filled([a.size for a in want])
+    oracle.reshard_attn(sh, c, d, src, dst)
+    for t, (g, w) in enumerate(zip(dst, want)):
+        assert np.array_equal(g, w), "rank %d" % t
 
 
 # ============================================================================= KV ======
@@ -257,6 +272,47 @@ def test_kv_equals_numpy_scatter_of_logical_cache(c, d):
     oracle.reshard_kv(sh, old, new, src, dst)
     for t, (g, w) in enumerate(zip(dst, want)):
         assert np.array_equal(g, w), "rank %d" % t
+
+
+@pytest.mark.parametrize("c,d", [(1, 8), (2, 8), (8, 2), (4, 8), (8, 4), (8, 16), (16, 1)])
+def test_kv_more_ranks_than_heads_equals_numpy_scatter(c, d):
+    """Hkv = 4 and up to 16 ranks: a rank beyond the head count holds one (replicated)
+    head; both layouts are scatters of the same logical cache."""
+    sh = tiny_shape(n_q_heads=16, n_kv_heads=4)
+    old, new = kv_cfgs(sh, c, d, [9, 4, 13, 1], 11, 14)
+    logical = logical_kv(sh, old)
+    src = kv_arenas(logical, sh, old)
+    want = kv_arenas(logical, sh, new)
+    assert [a.size for a in want] == oracle.kv_arena_bytes(sh, d, 14)
+    dst = filled([a.size for a in want])
+    oracle.reshard_kv(sh, old, new, src, dst)
+    for t, (g, w) in enumerate(zip(dst, want)):
+        assert np.array_equal(g, w), "rank %d" % t
+
+
+def test_kv_replicated_head_source_is_own_rank_then_smallest():
+    """Hand-written: one KV head, TP2 -> TP3, the two old replicas hold DIFFERENT bytes
+    (1s and 2s).  New rank 0 keeps old rank 0's, new rank 1 old rank 1's, new rank 2 (no
+    old rank 2) takes the smallest holder's, old rank 0."""
+    sh = tiny_shape(n_layers=1, n_q_heads=6, n_kv_heads=1, head_dim=1, kv_block_tokens=2,
+                    elem_bytes=1)
+    bt = np.array([[0]], np.int32)
+    old = W.ParallelConfig(1, 2, [[]], 1, [2], bt)
+    new = W.ParallelConfig(1, 3, [[]], 1, [2], bt)
+    src = [np.full(4, 1, np.uint8), np.full(4, 2, np.uint8)]       # [K|V][1 block][2 tok][1 head][1 B]
+    dst = filled([4, 4, 4])
+    oracle.reshard_kv(sh, old, new, src, dst)
+    assert [set(a) for a in dst] == [{1}, {2}, {1}]
+    # and the k / v weights follow the same rule (q and o rows are filled with 9s)
+    D = sh.d_model
+    def attn_arena(tag, tp):
+        q = sh.n_q_heads // tp * D
+        return np.concatenate([np.full(q, 9, np.uint8), np.full(2 * D, tag, np.uint8),
+                               np.full(q, 9, np.uint8)])
+    a_dst = filled(oracle.attn_arena_bytes(sh, 3))
+    oracle.reshard_attn(sh, 2, 3, [attn_arena(1, 2), attn_arena(2, 2)], a_dst)
+    q3 = sh.n_q_heads // 3 * D
+    assert [set(a[q3:q3 + 2 * D]) for a in a_dst] == [{1}, {2}, {1}]
 
 
 def test_kv_same_table_same_tp_leaves_mapped_blocks_unchanged():
