@@ -39,6 +39,11 @@
  *   KV cache.  One pool per (layer, K|V) per TP rank, shared block table:
  *        [L][2 (K, V)][kv_num_blocks][B][Hkv/T][hd]
  *   Global KV head g lives on rank g / (Hkv/T) as local head g % (Hkv/T).
+ *   With more TP ranks than KV heads (T > Hkv, Hkv | T) every rank holds ONE
+ *   head, rank t head floor(t*Hkv/T), so each head is on T/Hkv consecutive
+ *   ranks; Wk / Wv rows follow the same rule, Wq / Wo are split T ways.  A new
+ *   rank copies a replicated head from the old rank with its own index if that
+ *   rank holds the head, else from the smallest old rank that does.
  * ---------------------------------------------------------------------------
  */
 #ifndef EMOE_H_
@@ -55,7 +60,8 @@ typedef struct emoe_plan emoe_plan_t; /* opaque; owned by the library */
 typedef enum {
   EMOE_OK = 0,
   EMOE_ERR_INVALID_ARG = 1,  /* NULL pointer, bad enum value, wrong plan kind         */
-  EMOE_ERR_SHAPE = 2,        /* non-positive dimension, TP does not divide the heads  */
+  EMOE_ERR_SHAPE = 2,        /* non-positive dimension, TP does not divide the q heads, */
+                             /* TP neither divides nor is a multiple of the KV heads    */
   EMOE_ERR_PLACEMENT = 3,    /* id out of range, duplicate inside one rank, expert    */
                              /* missing from the old or from the new placement        */
   EMOE_ERR_BLOCK_TABLE = 4,  /* id out of range, physical block used twice, old/new   */
@@ -64,7 +70,7 @@ typedef enum {
   EMOE_ERR_OVERLAP = 6,      /* a source arena intersects a destination arena         */
   EMOE_ERR_OOM = 7,          /* host or device allocation for the plan failed         */
   EMOE_ERR_CUDA = 8,         /* a CUDA runtime call failed (no device, bad stream...) */
-  EMOE_ERR_UNSUPPORTED = 9,  /* TP > n_kv_heads, more ranks than EMOE_MAX_RANKS, ...  */
+  EMOE_ERR_UNSUPPORTED = 9,  /* more ranks than EMOE_MAX_RANKS, no virtual memory API   */
   EMOE_ERR_DEVICE_TIMEOUT = 10, /* a bounded device-side wait expired                 */
   EMOE_ERR_TOO_LARGE = 11    /* the problem exceeds a fixed capacity of the entry point */
 } emoe_status_t;

@@ -271,6 +271,29 @@ emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, 
   return cuda_status(e);
 }
 
+// Shape constants of the KV head re-split as the kernels take them.
+KvTables kv_tables(const KvPlan &kv, const uint32_t *d_pair_old, const uint32_t *d_pair_new) {
+  KvTables t{};
+  t.pair_old = d_pair_old;
+  t.pair_new = d_pair_new;
+  t.n_pairs = (uint32_t)kv.pair_old.size();
+  t.n_lk = kv.n_layers * 2;
+  t.block_tokens = kv.block_tokens;
+  t.hkv = kv.d * kv.hn;
+  t.hc = kv.hc;
+  t.hn = kv.hn;
+  t.head_bytes = (uint32_t)kv.head_bytes;
+  t.nb_old = kv.nb_old;
+  t.nb_new = kv.nb_new;
+  t.use_map = kv.replicated ? 1u : 0u;
+  if (kv.replicated)  // at most max(old ranks, new ranks) <= EMOE_MAX_RANKS slots
+    for (size_t j = 0; j < kv.src_rank.size() && j < kKvMapMax; ++j) {
+      t.map_rank[j] = kv.src_rank[j];
+      t.map_head[j] = (uint8_t)kv.src_head[j];
+    }
+  return t;
+}
+
 std::once_flag g_init_once;
 cudaError_t g_init_err = cudaSuccess;
 
@@ -452,9 +475,7 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *p, const void *const *src, void
   if (st != EMOE_OK) return st;
   if (!p->hp.kv.head_split_changes) return run_segments(p, EMOE_PHASE_KV, ptrs, (cudaStream_t)stream);
   const KvPlan &kv = p->hp.kv;
-  KvTables t{p->d_pair_old, p->d_pair_new, (uint32_t)kv.pair_old.size(), kv.n_layers * 2,
-             kv.block_tokens, kv.hkv, kv.hkv / kv.c, kv.hkv / kv.d, (uint32_t)kv.head_bytes,
-             kv.nb_old, kv.nb_new};
+  KvTables t = kv_tables(kv, p->d_pair_old, p->d_pair_new);
   const int mode = p->tuning.kv_mode > 0 ? p->tuning.kv_mode : kDefaultKvMode;
   return cuda_status(launch_kv_copy(t, ptrs, mode, cta_budget(p), p->tuning.max_ctas <= 0, p->d_status,
                                     (cudaStream_t)stream));
@@ -486,8 +507,7 @@ emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *p, const void *const *sr
       const uintptr_t d0 = (uintptr_t)dst[b], d1 = d0 + pp.arena_new[b];
       if (s0 < d1 && d0 < s1) return EMOE_ERR_OVERLAP;
     }
-  KvTables t{nullptr, nullptr, (uint32_t)pair_old->size(), kv.n_layers * 2, kv.block_tokens,
-             kv.hkv, kv.hkv / kv.c, kv.hkv / kv.d, (uint32_t)kv.head_bytes, kv.nb_old, kv.nb_new};
+  KvTables t = kv_tables(kv, nullptr, nullptr);
   return launch_kv_copy_static(t, pair_old->data(), pair_new->data(), ptrs, (cudaStream_t)stream);
 }
 

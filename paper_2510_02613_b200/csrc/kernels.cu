@@ -459,7 +459,8 @@ __global__ void __launch_bounds__(256) kv_direct_kernel(const __grid_constant__ 
           const uint32_t rem = q - tok[u] * row;
           g[u] = rem / cpv;
           j[u] = rem - g[u] * cpv;
-          const uint32_t ro = g[u] / t.hc, ho = g[u] - ro * t.hc;
+          uint32_t ro = g[u] / t.hc, ho = g[u] - ro * t.hc;
+          if (t.use_map) { ro = t.map_rank[g[u]]; ho = t.map_head[g[u]]; }
           v[u] = *reinterpret_cast<const V *>(
               s_src[ro] + base_old + ((uint64_t)(tok[u] * t.hc + ho) * cpv + j[u]) * W);
         }
@@ -489,7 +490,9 @@ __global__ void __launch_bounds__(256) kv_rows_kernel(const __grid_constant__ Kv
   const uint32_t cpv = t.head_bytes / 16, row = t.hkv * cpv, tpp = 256 / row;  // tokens per pass
   const uint32_t rem = threadIdx.x % row, tok0 = threadIdx.x / row;
   const uint32_t g = rem / cpv, j = rem - g * cpv;
-  const uint32_t ro = g / t.hc, ho = g - ro * t.hc, rn = g / t.hn, hn = g - rn * t.hn;
+  uint32_t ro = g / t.hc, ho = g - ro * t.hc;
+  if (t.use_map) { ro = t.map_rank[g]; ho = t.map_head[g]; }
+  const uint32_t rn = g / t.hn, hn = g - rn * t.hn;
   const uint8_t *sp = p.ptrs.src[ro] + ((uint64_t)(tok0 * t.hc + ho) * cpv + j) * 16;
   uint8_t *dp = p.ptrs.dst[rn] + ((uint64_t)(tok0 * t.hn + hn) * cpv + j) * 16;
   const uint64_t s_step = (uint64_t)tpp * t.hc * t.head_bytes, d_step = (uint64_t)tpp * t.hn * t.head_bytes;
@@ -905,7 +908,7 @@ bool kv_tma_supported(const KvTables &t, uint32_t *stages_out) {
   const uint64_t box = (uint64_t)t.block_tokens * g * hb;
   const uint64_t rows_old = (uint64_t)t.n_lk * t.nb_old * t.block_tokens;
   const uint64_t rows_new = (uint64_t)t.n_lk * t.nb_new * t.block_tokens;
-  if (hb % 16 || c > kKvTmaMaxRanks || d > kKvTmaMaxRanks) return false;
+  if (t.use_map || hb % 16 || c > kKvTmaMaxRanks || d > kKvTmaMaxRanks) return false;
   if ((hb % 4 == 0 ? hb / 4 : hb) > 256 || g > 256 || t.block_tokens > 256) return false;  // box extents
   if (box % 128 || t.hkv / g > kKvTmaMaxBoxes || tile > 96 * 1024) return false;
   if (rows_old >= (1ull << 31) || rows_new >= (1ull << 31)) return false;             // int32 coordinates
@@ -919,6 +922,7 @@ bool kv_tma_supported(const KvTables &t, uint32_t *stages_out) {
 bool kv_staged_supported(const KvTables &t, uint32_t *stages_out) {
   const uint64_t tile = (uint64_t)t.block_tokens * t.hkv * t.head_bytes;
   const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
+  if (t.use_map) return false;  // replicated heads: the default kernels handle the slot map
   if (t.head_bytes % 16 || tile > 64 * 1024 || blk_new >= (1u << 24) || t.hkv / t.hn > 255) return false;
   uint32_t stages = (uint32_t)((160 * 1024) / tile);
   if (stages > kMaxStages) stages = kMaxStages;

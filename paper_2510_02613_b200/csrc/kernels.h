@@ -43,12 +43,22 @@ struct SegTables {  // device pointers
   uint32_t n_units;
 };
 
+constexpr uint32_t kKvMapMax = 64;  // destination head slots a replicated split can have
+
 struct KvTables {  // device pointers + shape constants of the KV head re-split
   const uint32_t *pair_old, *pair_new;
   uint32_t n_pairs, n_lk;        // n_lk = 2 * n_layers
-  uint32_t block_tokens, hkv, hc, hn;
+  uint32_t block_tokens;
+  uint32_t hkv;                  // destination head slots per token: new ranks x heads per new rank
+                                 // (= the KV head count unless the new side replicates heads)
+  uint32_t hc, hn;               // heads per old / new rank
   uint32_t head_bytes;
   uint64_t nb_old, nb_new;
+  // With more ranks than KV heads on a side, slot j = new rank * hn + local head reads
+  // old rank map_rank[j], local head map_head[j]; otherwise slot j is global head j and
+  // lives at old rank j / hc, local head j % hc.
+  uint32_t use_map;
+  uint8_t map_rank[kKvMapMax], map_head[kKvMapMax];
 };
 
 struct BulkConfig {

@@ -174,8 +174,9 @@ void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &
 void plan_attn(const emoe_shape_t &sh, int c, int d, PhasePlan *pp) {
   const uint64_t D = sh.d_model, b = sh.elem_bytes, hd = sh.head_dim;
   const uint64_t row = D * b;
+  const uint32_t hkv = sh.n_kv_heads;
   auto q_bytes = [&](int T) { return (uint64_t)(sh.n_q_heads / T) * hd * row; };
-  auto kv_bytes = [&](int T) { return (uint64_t)(sh.n_kv_heads / T) * hd * row; };
+  auto kv_bytes = [&](int T) { return (uint64_t)kv_heads_per_rank(hkv, T) * hd * row; };
   auto layer_bytes = [&](int T) { return 2 * q_bytes(T) + 2 * kv_bytes(T); };
   const uint32_t L = sh.n_layers;
   pp->arena_old.assign(c, L * layer_bytes(c));
@@ -192,26 +193,45 @@ void plan_attn(const emoe_shape_t &sh, int c, int d, PhasePlan *pp) {
     }
     return;
   }
-  // q, k, v: intersect old and new row ranges of the logical matrix
-  for (int t = 0; t < 3; ++t) {
-    const uint64_t rows = (uint64_t)(t == 0 ? sh.n_q_heads : sh.n_kv_heads) * hd;
+  // q: intersect old and new row ranges of the logical matrix
+  {
+    const uint64_t rows = (uint64_t)sh.n_q_heads * hd;
     const uint64_t rc = rows / c, rd = rows / d;
-    auto piece = [&](int T) {
-      return t == 0 ? 0 : t == 1 ? q_bytes(T) : q_bytes(T) + kv_bytes(T);
-    };
     for (int ro = 0; ro < c; ++ro)
       for (int rn = 0; rn < d; ++rn) {
         const uint64_t lo = std::max(ro * rc, rn * rd), hi = std::min((ro + 1) * rc, (rn + 1) * rd);
         if (lo >= hi) continue;
         Segment s{};
-        s.src_off = piece(c) + (lo - ro * rc) * row;
+        s.src_off = (lo - ro * rc) * row;
         s.run_bytes = (hi - lo) * row;
         s.src_pitch = layer_bytes(c);
         s.n_runs = L;
         s.src_rank = (uint32_t)ro;
-        finish_segment(pp, s,
-                       {Dst{piece(d) + (lo - rn * rd) * row, layer_bytes(d), (uint32_t)rn, 0}});
+        finish_segment(pp, s, {Dst{(lo - rn * rd) * row, layer_bytes(d), (uint32_t)rn, 0}});
       }
+  }
+  // k, v: every new rank's heads, grouped into runs of heads that are consecutive on one
+  // old rank (with more ranks than KV heads a head has several holders: see kv_source_rank)
+  for (int t = 1; t < 3; ++t) {
+    auto piece = [&](int T) { return t == 1 ? q_bytes(T) : q_bytes(T) + kv_bytes(T); };
+    const uint32_t hn = kv_heads_per_rank(hkv, d);
+    for (int rn = 0; rn < d; ++rn) {
+      uint32_t hl = 0;
+      while (hl < hn) {
+        const uint32_t g0 = kv_first_head(hkv, d, rn) + hl;
+        const uint32_t ro = kv_source_rank(hkv, c, g0, rn);
+        uint32_t n = 1;
+        while (hl + n < hn && kv_source_rank(hkv, c, g0 + n, rn) == ro) ++n;
+        Segment s{};
+        s.src_off = piece(c) + (uint64_t)(g0 - kv_first_head(hkv, c, ro)) * hd * row;
+        s.run_bytes = (uint64_t)n * hd * row;
+        s.src_pitch = layer_bytes(c);
+        s.n_runs = L;
+        s.src_rank = ro;
+        finish_segment(pp, s, {Dst{piece(d) + (uint64_t)hl * hd * row, layer_bytes(d), (uint32_t)rn, 0}});
+        hl += n;
+      }
+    }
   }
   // o: intersect old and new column ranges; one strided segment per (layer, overlap)
   const uint64_t cols = (uint64_t)sh.n_q_heads * hd, cc = cols / c, cd = cols / d;
@@ -244,16 +264,34 @@ void plan_kv(const emoe_shape_t &sh, const emoe_config_t &o, const emoe_config_t
   kv.n_layers = sh.n_layers; kv.block_tokens = sh.kv_block_tokens; kv.hkv = sh.n_kv_heads;
   kv.head_bytes = vec; kv.nb_old = o.kv_num_blocks; kv.nb_new = n.kv_num_blocks;
   kv.head_split_changes = (o.tp != n.tp);
-  const uint64_t blk_old = B * (sh.n_kv_heads / o.tp) * vec, blk_new = B * (sh.n_kv_heads / n.tp) * vec;
+  kv.hc = kv_heads_per_rank(kv.hkv, kv.c);
+  kv.hn = kv_heads_per_rank(kv.hkv, kv.d);
+  kv.replicated = kv.c > kv.hkv || kv.d > kv.hkv;
+  kv.src_rank.clear();
+  kv.src_head.clear();
+  std::vector<char> read_slot((size_t)kv.c * kv.hc, 0);
+  for (uint32_t rn = 0; rn < kv.d; ++rn)
+    for (uint32_t hl = 0; hl < kv.hn; ++hl) {
+      const uint32_t g = kv_first_head(kv.hkv, kv.d, rn) + hl;
+      const uint32_t ro = kv_source_rank(kv.hkv, kv.c, g, rn);
+      const uint32_t ho = g - kv_first_head(kv.hkv, kv.c, ro);
+      kv.src_rank.push_back((uint8_t)ro);
+      kv.src_head.push_back((uint16_t)ho);
+      read_slot[(size_t)ro * kv.hc + ho] = 1;
+    }
+  uint64_t heads_read = 0;
+  for (char x : read_slot) heads_read += x;
+  const uint64_t blk_old = B * kv.hc * vec, blk_new = B * kv.hn * vec;
   pp->arena_old.assign(o.tp, L * 2 * o.kv_num_blocks * blk_old);
   pp->arena_new.assign(n.tp, L * 2 * n.kv_num_blocks * blk_new);
   const uint64_t n_pairs = pair_old.size();
-  const uint64_t logical_bytes = L * 2 * n_pairs * B * sh.n_kv_heads * vec;
+  const uint64_t per_head = L * 2 * n_pairs * B * vec;
 
   kv.pair_old = pair_old;  // kept in both cases: the fixed-scratch entry point reads them
   kv.pair_new = pair_new;
   if (kv.head_split_changes) {
-    pp->bytes_moved = pp->bytes_read = logical_bytes;
+    pp->bytes_moved = per_head * kv.d * kv.hn;  // every new rank's heads, replicas included
+    pp->bytes_read = per_head * heads_read;     // distinct (old rank, head) slots that are read
     return;
   }
   // head split kept: a block is one contiguous run per (layer, K|V); consecutive
@@ -278,6 +316,18 @@ void plan_kv(const emoe_shape_t &sh, const emoe_config_t &o, const emoe_config_t
 
 }  // namespace
 
+uint32_t kv_source_rank(uint32_t hkv, uint32_t c, uint32_t g, uint32_t r_new) {
+  const uint32_t h = kv_heads_per_rank(hkv, c);
+  auto holds = [&](uint32_t r) {
+    const uint32_t f = kv_first_head(hkv, c, r);
+    return f <= g && g < f + h;
+  };
+  if (r_new < c && holds(r_new)) return r_new;  // the same device keeps its copy
+  for (uint32_t r = 0; r < c; ++r)
+    if (holds(r)) return r;
+  return 0;  // not reached for valid degrees
+}
+
 emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
                               const emoe_config_t &n, HostPlan *hp) {
   if (sh.n_layers <= 0 || sh.n_routed <= 0 || sh.n_shared < 0 || sh.d_model <= 0 ||
@@ -291,8 +341,9 @@ emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
   st = read_placement(n, n_experts, &pn);
   if (st != EMOE_OK) return st;
   for (int tp : {o.tp, n.tp}) {
-    if (tp > sh.n_kv_heads) return EMOE_ERR_UNSUPPORTED;  // would need KV-head replication
-    if (sh.n_q_heads % tp || sh.n_kv_heads % tp) return EMOE_ERR_SHAPE;
+    if (sh.n_q_heads % tp) return EMOE_ERR_SHAPE;
+    // more ranks than KV heads: every head is held by tp / Hkv consecutive ranks
+    if (tp <= sh.n_kv_heads ? sh.n_kv_heads % tp : tp % sh.n_kv_heads) return EMOE_ERR_SHAPE;
   }
   std::vector<uint32_t> pair_old, pair_new;
   st = read_block_pairs(sh, o, n, &pair_old, &pair_new);
@@ -337,17 +388,21 @@ void export_segments(const HostPlan &hp, int phase, std::vector<emoe_segment_t> 
   }
   if (phase != EMOE_PHASE_KV || !hp.kv.head_split_changes) return;
   const KvPlan &kv = hp.kv;
-  const uint64_t hc = kv.hkv / kv.c, hn = kv.hkv / kv.d, B = kv.block_tokens, vec = kv.head_bytes;
+  const uint64_t hc = kv.hc, hn = kv.hn, B = kv.block_tokens, vec = kv.head_bytes;
   for (size_t i = 0; i < kv.pair_old.size(); ++i)
     for (uint64_t lk = 0; lk < (uint64_t)kv.n_layers * 2; ++lk)
-      for (uint32_t ro = 0; ro < kv.c; ++ro)
-        for (uint32_t rn = 0; rn < kv.d; ++rn) {
-          const uint64_t lo = std::max(ro * hc, rn * hn), hi = std::min((ro + 1) * hc, (rn + 1) * hn);
-          if (lo >= hi) continue;
-          out->push_back({((lk * kv.nb_old + kv.pair_old[i]) * B * hc + (lo - ro * hc)) * vec,
-                          ((lk * kv.nb_new + kv.pair_new[i]) * B * hn + (lo - rn * hn)) * vec,
-                          (hi - lo) * vec, hc * vec, hn * vec, (uint32_t)B, ro, rn, group++});
+      for (uint32_t rn = 0; rn < kv.d; ++rn) {
+        uint32_t hl = 0;
+        while (hl < hn) {  // runs of destination heads that are consecutive on one old rank
+          const uint32_t j = rn * (uint32_t)hn + hl, ro = kv.src_rank[j], ho = kv.src_head[j];
+          uint32_t n = 1;
+          while (hl + n < hn && kv.src_rank[j + n] == ro && kv.src_head[j + n] == ho + n) ++n;
+          out->push_back({((lk * kv.nb_old + kv.pair_old[i]) * B * hc + ho) * vec,
+                          ((lk * kv.nb_new + kv.pair_new[i]) * B * hn + hl) * vec,
+                          n * vec, hc * vec, hn * vec, (uint32_t)B, ro, rn, group++});
+          hl += n;
         }
+      }
 }
 
 }  // namespace emoe

@@ -50,7 +50,20 @@ struct KvPlan {
   uint64_t head_bytes = 0;                   // head_dim * elem_bytes
   uint64_t nb_old = 0, nb_new = 0;
   bool head_split_changes = false;
+  // Heads per rank on either side (1 when a side has more ranks than KV heads) and, for
+  // every destination head slot j = new rank * hn + local head, the old rank and local
+  // head it is read from.
+  uint32_t hc = 0, hn = 0;
+  std::vector<uint8_t> src_rank;
+  std::vector<uint16_t> src_head;
+  bool replicated = false;  // a side has more ranks than KV heads: the map is not g/hc, g%hc
 };
+
+// KV heads of a TP=T group (T <= Hkv: Hkv/T contiguous heads per rank; T > Hkv: one head per
+// rank, every head on T/Hkv consecutive ranks) and the old rank a new rank reads head g from.
+inline uint32_t kv_heads_per_rank(uint32_t hkv, uint32_t T) { return hkv >= T ? hkv / T : 1u; }
+inline uint32_t kv_first_head(uint32_t hkv, uint32_t T, uint32_t t) { return (uint32_t)((uint64_t)t * hkv / T); }
+uint32_t kv_source_rank(uint32_t hkv, uint32_t c, uint32_t g, uint32_t r_new);
 
 struct HostPlan {
   emoe_shape_t shape;

@@ -227,3 +227,20 @@ def test_maximum_rank_counts():
                 plan.set_tuning(kv_mode=kv_mode)
                 for phase in range(3):
                     check_phase_full(w, plan, phase)
+
+
+@pytest.mark.parametrize("c,d", [(2, 8), (8, 4), (4, 16), (16, 8), (8, 8)])
+def test_more_tp_ranks_than_kv_heads(c, d):
+    """Large-expert-count shape (4 KV heads, 32 q heads) at TP degrees above the KV head
+    count: every head is held by several ranks, attention k/v and the KV cache follow."""
+    wl = W.make_workload("c4_large", n_layers=1)
+    wl = R(wl, shape=R(wl.shape, d_ff=64, d_model=256), old=R(wl.old, tp=c), new=R(wl.new, tp=d))
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        for phase in (E.PHASE_ATTN, E.PHASE_KV):
+            check_phase_full(wl, plan, phase)
+        for kv_mode in (2, 3, 4):
+            plan.set_tuning(kv_mode=kv_mode, max_ctas=7)
+            check_phase_full(wl, plan, E.PHASE_KV)
+        st = plan.stats(E.PHASE_KV)
+        used = sum(-(-n // 16) for n in wl.old.seq_lens)
+        assert st["bytes_moved"] == 2 * used * 16 * max(4, d) * 128 * 2

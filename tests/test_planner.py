@@ -152,7 +152,10 @@ def test_validation_codes():
     assert _plan_code(sh, old, new) == 0
     assert _plan_code(R(sh, d_model=0), old, new) == 2                      # SHAPE
     assert _plan_code(sh, old, R(new, tp=3)) == 2                           # 3 does not divide 8
-    assert _plan_code(sh, old, R(new, tp=16)) == 9                          # TP > Hkv
+    assert _plan_code(sh, old, R(new, tp=16)) == 2                          # 16 does not divide the 8 q heads
+    wide = R(sh, n_q_heads=48)
+    assert _plan_code(wide, old, R(new, tp=16)) == 0                        # 8 KV heads on 16 ranks: 2 ranks per head
+    assert _plan_code(wide, old, R(new, tp=12)) == 2                        # 12 is no multiple of 8 KV heads
     assert _plan_code(sh, old, R(new, ep=65, placement=[[0]] * 65)) == 9    # too many ranks
     dup = [list(p) for p in new.placement]; dup[0] = [0, 0]
     assert _plan_code(sh, old, R(new, placement=dup)) == 3                  # duplicate in a rank

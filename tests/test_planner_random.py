@@ -3,6 +3,8 @@ TP pairs and block tables, replaying the exported segments with numpy copies mus
 the oracle on whole arenas, and the plan's byte counts must match the definitions."""
 from __future__ import annotations
 
+import math
+
 import numpy as np
 from hypothesis import HealthCheck, given, settings, strategies as st
 
@@ -33,11 +35,13 @@ def placements(draw, n_experts, max_ep=5):
 def cases(draw):
     hkv = draw(st.sampled_from([1, 2, 4, 6, 8]))
     group = draw(st.sampled_from([1, 2, 3]))
-    divs = [t for t in (1, 2, 3, 4, 6, 8) if hkv % t == 0]
+    # TP degrees: divisors of Hkv, and multiples of it (more ranks than KV heads)
+    divs = [t for t in (1, 2, 3, 4, 6, 8, 12, 16) if hkv % t == 0 or (t > hkv and t % hkv == 0)]
     c, d = draw(st.sampled_from(divs)), draw(st.sampled_from(divs))
     n_routed, n_shared = draw(st.integers(1, 7)), draw(st.integers(0, 2))
     sh = W.Shape(draw(st.integers(1, 3)), n_routed, n_shared, draw(st.sampled_from([3, 8, 16])),
-                 draw(st.sampled_from([1, 5, 8])), hkv * group, hkv, draw(st.sampled_from([1, 4, 8])),
+                 draw(st.sampled_from([1, 5, 8])), math.lcm(hkv * group, c, d), hkv,
+                 draw(st.sampled_from([1, 4, 8])),
                  draw(st.sampled_from([1, 3, 4])), draw(st.sampled_from([1, 2, 4])))
     B = sh.kv_block_tokens
     seq_lens = draw(st.lists(st.integers(0, 4 * B), min_size=0, max_size=4))
@@ -79,5 +83,6 @@ def test_drawn_plans_replay_to_the_oracle(wl):
             else:
                 sh = wl.shape
                 used = sum(-(-n // sh.kv_block_tokens) for n in wl.old.seq_lens)
+                heads = max(sh.n_kv_heads, wl.new.tp)    # replicas included
                 assert stt["bytes_moved"] == (sh.n_layers * 2 * used * sh.kv_block_tokens
-                                              * sh.n_kv_heads * sh.head_dim * sh.elem_bytes)
+                                              * heads * sh.head_dim * sh.elem_bytes)
