@@ -28,11 +28,11 @@ def lib() -> ctypes.CDLL:
         L.emoe_oracle_kv_arena_bytes.restype = i64
         L.emoe_oracle_kv_arena_bytes.argtypes = [i32] * 7
         L.emoe_oracle_reshard_experts.restype = i32
-        L.emoe_oracle_reshard_experts.argtypes = [i32, i64, i32, p, p, i32, p, p, p, p]
+        L.emoe_oracle_reshard_experts.argtypes = [i32, i64, i32, p, p, i32, p, p, p, p, i32]
         L.emoe_oracle_reshard_attn.restype = i32
         L.emoe_oracle_reshard_attn.argtypes = [i32] * 8 + [p, p]
         L.emoe_oracle_reshard_kv.restype = i32
-        L.emoe_oracle_reshard_kv.argtypes = [i32] * 11 + [p, p, p, p, p]
+        L.emoe_oracle_reshard_kv.argtypes = [i32] * 11 + [p, p, p, p, p, i32]
         _lib = L
     return _lib
 
@@ -77,8 +77,9 @@ def kv_arena_bytes(shape, tp: int, num_blocks: int) -> List[int]:
 # ---- the three phases ------------------------------------------------------------------
 
 def reshard_experts(shape, old_placement, new_placement, src: Sequence[np.ndarray],
-                    dst: Sequence[np.ndarray]) -> None:
-    """Writes the new expert arenas `dst` from the old arenas `src` (in place on dst)."""
+                    dst: Sequence[np.ndarray], fused_w13: bool = False) -> None:
+    """Writes the new expert arenas `dst` from the old arenas `src` (in place on dst).
+    fused_w13: per layer a [n_r][gate|up] tensor followed by a [n_r][down] tensor."""
     m = shape.d_model * shape.d_ff * shape.elem_bytes
     oo, oi = _csr(old_placement)
     no, ni = _csr(new_placement)
@@ -88,7 +89,7 @@ def reshard_experts(shape, old_placement, new_placement, src: Sequence[np.ndarra
         raise ValueError("expert arena sizes do not match the placements")
     rc = lib().emoe_oracle_reshard_experts(shape.n_layers, m, len(old_placement), _vp(oo), _vp(oi),
                                           len(new_placement), _vp(no), _vp(ni), _ptrs(src),
-                                          _ptrs(dst))
+                                          _ptrs(dst), int(bool(fused_w13)))
     if rc != 0:
         raise ValueError("oracle: an expert of the new placement is absent from the old one")
 
@@ -104,8 +105,9 @@ def reshard_attn(shape, tp_old: int, tp_new: int, src, dst) -> None:
         raise ValueError("oracle: TP degree does not divide the head counts")
 
 
-def reshard_kv(shape, old_cfg, new_cfg, src, dst) -> None:
-    """old_cfg / new_cfg carry tp, kv_num_blocks, seq_lens and block_table."""
+def reshard_kv(shape, old_cfg, new_cfg, src, dst, head_major: bool = False) -> None:
+    """old_cfg / new_cfg carry tp, kv_num_blocks, seq_lens and block_table.
+    head_major: blocks are [local head][token][hd] instead of [token][local head][hd]."""
     if ([a.size for a in src] != kv_arena_bytes(shape, old_cfg.tp, old_cfg.kv_num_blocks)
             or [a.size for a in dst] != kv_arena_bytes(shape, new_cfg.tp, new_cfg.kv_num_blocks)):
         raise ValueError("KV arena sizes do not match")
@@ -121,6 +123,7 @@ def reshard_kv(shape, old_cfg, new_cfg, src, dst) -> None:
     rc = lib().emoe_oracle_reshard_kv(shape.n_layers, shape.kv_block_tokens, shape.n_kv_heads,
                                      shape.head_dim, shape.elem_bytes, old_cfg.tp, new_cfg.tp,
                                      old_cfg.kv_num_blocks, new_cfg.kv_num_blocks, len(sl),
-                                     bo.shape[1], _vp(sl), _vp(bo), _vp(bn), _ptrs(src), _ptrs(dst))
+                                     bo.shape[1], _vp(sl), _vp(bo), _vp(bn), _ptrs(src), _ptrs(dst),
+                                     int(bool(head_major)))
     if rc != 0:
         raise ValueError("oracle: bad block table or TP degree")

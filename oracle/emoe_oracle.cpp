@@ -31,6 +31,12 @@
 //    rule as for replicated experts: the old rank with the same index if it
 //    holds the head, else the smallest old rank that does.
 //
+//  * layout variants (the paper only says experts are "large contiguous tensors" and
+//    KV blocks are paged, Sec. 4.1): fused_w13 stores, per layer, a [n_r][gate|up]
+//    tensor followed by a [n_r][down] tensor instead of three [n_r] tensors;
+//    head_major stores a KV block as [local head][token][hd] instead of
+//    [token][local head][hd].  Both are re-orderings of the same logical data.
+//
 // Pins: every function below is pinned by tests that do not use it to make
 // their expectation (numpy/torch indexing of logical tensors, hand-written
 // fixtures, identities and round trips); none is "parity unpinned".
@@ -105,10 +111,18 @@ int64_t emoe_oracle_kv_arena_bytes(int n_layers, int nb, int block_tokens, int h
 
 // Expert re-pack.  m = bytes of one expert matrix.  Returns 0, or -1 if an
 // expert of the new placement has no copy in the old one.
+// Offset of matrix (layer l, projection p, slot s) in the arena of a rank with n slots.
+// Plain layout: [L][3][n][m].  fused_w13: per layer [n][gate|up] (2m per slot), then [n][down].
+int64_t expert_offset(int fused_w13, int64_t l, int p, int64_t n, int64_t s, int64_t m) {
+  if (!fused_w13) return ((l * 3 + p) * n + s) * m;
+  const int64_t layer = l * 3 * n * m;
+  return p < 2 ? layer + s * 2 * m + p * m : layer + n * 2 * m + s * m;
+}
+
 int emoe_oracle_reshard_experts(int n_layers, int64_t m, int ep_old, const int32_t *old_off,
                                 const int32_t *old_ids, int ep_new, const int32_t *new_off,
                                 const int32_t *new_ids, const uint8_t *const *src,
-                                uint8_t *const *dst) {
+                                uint8_t *const *dst, int fused_w13) {
   Csr po{ep_old, old_off, old_ids}, pn{ep_new, new_off, new_ids};
   for (int rn = 0; rn < ep_new; ++rn) {
     const int64_t n_new = pn.count(rn);
@@ -118,8 +132,8 @@ int emoe_oracle_reshard_experts(int n_layers, int64_t m, int ep_old, const int32
           int ro, so;
           if (!find_source(po, pn.id(rn, sn), rn, &ro, &so)) return -1;
           const int64_t n_old = po.count(ro);
-          const int64_t off_new = (((int64_t)l * 3 + p) * n_new + sn) * m;
-          const int64_t off_old = (((int64_t)l * 3 + p) * n_old + so) * m;
+          const int64_t off_new = expert_offset(fused_w13, l, p, n_new, sn, m);
+          const int64_t off_old = expert_offset(fused_w13, l, p, n_old, so, m);
           std::memcpy(dst[rn] + off_new, src[ro] + off_old, (size_t)m);
         }
   }
@@ -183,7 +197,7 @@ int emoe_oracle_reshard_attn(int n_layers, int d_model, int hq, int hkv, int hd,
 int emoe_oracle_reshard_kv(int n_layers, int block_tokens, int hkv, int hd, int b, int c, int d,
                            int nb_old, int nb_new, int n_seqs, int max_blocks,
                            const int32_t *seq_lens, const int32_t *bt_old, const int32_t *bt_new,
-                           const uint8_t *const *src, uint8_t *const *dst) {
+                           const uint8_t *const *src, uint8_t *const *dst, int head_major) {
   if (!kv_tp_ok(hkv, c) || !kv_tp_ok(hkv, d)) return -1;
   const int64_t B = block_tokens, hc = kv_heads_per_rank(hkv, c), hdn = kv_heads_per_rank(hkv, d);
   const int64_t vec = (int64_t)hd * b;
@@ -201,8 +215,10 @@ int emoe_oracle_reshard_kv(int n_layers, int block_tokens, int hkv, int hd, int 
                 const int64_t g = kv_first_head(hkv, d, rn) + hn;   // global KV head
                 const int64_t ro = kv_source_rank(hkv, c, g, rn);
                 const int64_t ho = g - kv_first_head(hkv, c, ro);
-                const int64_t off_o = (((((int64_t)l * 2 + kv) * nb_old + po) * B + tok) * hc + ho) * vec;
-                const int64_t off_n = (((((int64_t)l * 2 + kv) * nb_new + pn) * B + tok) * hdn + hn) * vec;
+                // position of (token, local head) inside a block of H local heads
+                auto in_block = [&](int64_t H, int64_t h) { return head_major ? h * B + tok : tok * H + h; };
+                const int64_t off_o = ((((int64_t)l * 2 + kv) * nb_old + po) * B * hc + in_block(hc, ho)) * vec;
+                const int64_t off_n = ((((int64_t)l * 2 + kv) * nb_new + pn) * B * hdn + in_block(hdn, hn)) * vec;
                 std::memcpy(dst[rn] + off_n, src[ro] + off_o, (size_t)vec);
               }
     }

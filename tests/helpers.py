@@ -23,9 +23,19 @@ def logical_experts(shape, key=1):
     return rand_bytes(key, n).reshape(shape.n_layers, 3, shape.n_experts, m)
 
 
-def expert_arenas(logical, placement):
-    """Per-rank arena = the rank's experts gathered along the expert axis."""
-    return [np.ascontiguousarray(logical[:, :, list(p), :]).reshape(-1) for p in placement]
+def expert_arenas(logical, placement, fused_w13=False):
+    """Per-rank arena = the rank's experts gathered along the expert axis.  fused_w13:
+    per layer a [n][gate|up] tensor (built with numpy.concatenate) and then the [n][down] one."""
+    if not fused_w13:
+        return [np.ascontiguousarray(logical[:, :, list(p), :]).reshape(-1) for p in placement]
+    out = []
+    for p in placement:
+        mine = logical[:, :, list(p), :]                              # [L, 3, n, m]
+        w13 = np.concatenate([mine[:, 0], mine[:, 1]], axis=2)        # [L, n, 2m]
+        per_layer = [np.concatenate([w13[l].reshape(-1), mine[l, 2].reshape(-1)])
+                     for l in range(mine.shape[0])]
+        out.append(np.concatenate(per_layer) if per_layer else np.zeros(0, np.uint8))
+    return out
 
 
 # ---- attention -------------------------------------------------------------------------
@@ -92,8 +102,9 @@ def logical_kv(shape, cfg, key=3):
     return rand_bytes(key, n).reshape(shape.n_layers, 2, nblk, B, shape.n_kv_heads, vec)
 
 
-def kv_arenas(logical, shape, cfg, background=None):
-    """Scatters logical blocks into each rank's pool through the block table."""
+def kv_arenas(logical, shape, cfg, background=None, head_major=False):
+    """Scatters logical blocks into each rank's pool through the block table.  head_major:
+    a block is [local head][token][hd] (numpy.swapaxes of the token-major block)."""
     B = shape.kv_block_tokens
     L, vec = shape.n_layers, shape.head_dim * shape.elem_bytes
     hl = max(1, shape.n_kv_heads // cfg.tp)
@@ -107,5 +118,7 @@ def kv_arenas(logical, shape, cfg, background=None):
         else:
             pool = background[t].reshape(L, 2, cfg.kv_num_blocks, B, hl, vec).copy()
         pool[:, :, phys] = logical[:, :, :, :, kv_heads_of_rank(shape.n_kv_heads, cfg.tp, t)]
+        if head_major:
+            pool = np.ascontiguousarray(pool.swapaxes(3, 4))
         out.append(pool.reshape(-1))
     return out

@@ -59,6 +59,35 @@ def test_experts_equal_numpy_gather_of_logical_tensor(name, elem_bytes):
         assert np.array_equal(g, w), "rank %d" % r
 
 
+@pytest.mark.parametrize("name", sorted(PLACEMENTS))
+def test_experts_fused_w13_equals_numpy_concatenate(name):
+    """Fused gate|up layout: both sides built from the logical tensor with concatenate."""
+    sh = tiny_shape()
+    po, pn = (f() for f in PLACEMENTS[name])
+    logical = logical_experts(sh)
+    src = expert_arenas(logical, po, fused_w13=True)
+    want = expert_arenas(logical, pn, fused_w13=True)
+    assert [a.size for a in want] == oracle.expert_arena_bytes(sh, pn)
+    dst = filled([a.size for a in want])
+    oracle.reshard_experts(sh, po, pn, src, dst, fused_w13=True)
+    for r, (g, w) in enumerate(zip(dst, want)):
+        assert np.array_equal(g, w), "rank %d" % r
+    # and it is a different byte order from the plain layout whenever a rank has > 1 slot
+    plain = expert_arenas(logical, pn)
+    assert any(not np.array_equal(a, b) for a, b in zip(plain, want) if a.size)
+
+
+def test_experts_fused_w13_hand_written():
+    """One layer, one rank with slots [A, B] -> two ranks [B], [A]; matrices of 2 bytes.
+    Old arena: A.gate A.up B.gate B.up | A.down B.down."""
+    sh = tiny_shape(n_layers=1, n_routed=2, d_model=1, d_ff=1, elem_bytes=2)
+    src = [np.array([1, 1, 2, 2, 11, 11, 12, 12, 3, 3, 13, 13], np.uint8)]
+    dst = filled([6, 6])
+    oracle.reshard_experts(sh, [[0, 1]], [[1], [0]], src, dst, fused_w13=True)
+    assert list(dst[0]) == [11, 11, 12, 12, 13, 13]       # B: gate up | down
+    assert list(dst[1]) == [1, 1, 2, 2, 3, 3]             # A
+
+
 def test_experts_shared_experts_on_every_rank():
     sh = tiny_shape(n_routed=10, n_shared=2)
     po = W.with_shared(W.place_contiguous(10, 2), [10, 11])
@@ -288,6 +317,35 @@ def test_kv_more_ranks_than_heads_equals_numpy_scatter(c, d):
     oracle.reshard_kv(sh, old, new, src, dst)
     for t, (g, w) in enumerate(zip(dst, want)):
         assert np.array_equal(g, w), "rank %d" % t
+
+
+@pytest.mark.parametrize("c,d", [(1, 2), (2, 4), (4, 2), (2, 2), (4, 1), (2, 8), (8, 4)])
+def test_kv_head_major_equals_numpy_swapaxes(c, d):
+    """Head-major blocks: both layouts are the token-major pools with the token and head
+    axes swapped (numpy), so tokens still keep sequence, position and head identity."""
+    sh = tiny_shape(n_q_heads=8, n_kv_heads=4)
+    old, new = kv_cfgs(sh, c, d, [9, 4, 13, 1], 11, 14)
+    logical = logical_kv(sh, old)
+    src = kv_arenas(logical, sh, old, head_major=True)
+    want = kv_arenas(logical, sh, new, head_major=True)
+    dst = filled([a.size for a in want])
+    oracle.reshard_kv(sh, old, new, src, dst, head_major=True)
+    for t, (g, w) in enumerate(zip(dst, want)):
+        assert np.array_equal(g, w), "rank %d" % t
+
+
+def test_kv_head_major_hand_written():
+    """The two-head example of the token-major test, blocks stored head-major: old block
+    1 holds h0t0 h0t1 h1t0 h1t1."""
+    sh = tiny_shape(n_layers=1, n_kv_heads=2, head_dim=1, kv_block_tokens=2, elem_bytes=2)
+    old = W.ParallelConfig(1, 1, [[]], 2, [2], np.array([[1]], np.int32))
+    new = W.ParallelConfig(1, 2, [[]], 1, [2], np.array([[0]], np.int32))
+    K = [0] * 8 + [1, 2, 5, 6, 3, 4, 7, 8]
+    V = [0] * 8 + [21, 22, 25, 26, 23, 24, 27, 28]
+    dst = filled([8, 8])
+    oracle.reshard_kv(sh, old, new, [np.array(K + V, dtype=np.uint8)], dst, head_major=True)
+    assert list(dst[0]) == [1, 2, 5, 6, 21, 22, 25, 26]      # head 0: K t0,t1 then V t0,t1
+    assert list(dst[1]) == [3, 4, 7, 8, 23, 24, 27, 28]      # head 1
 
 
 def test_kv_replicated_head_source_is_own_rank_then_smallest():
