@@ -112,6 +112,12 @@ typedef struct {
 #define EMOE_PLAN_HOST_STEP 2u /* also prepare the pipelined form of emoe_reshard_step_host: */
                                /* chunk plans, two copy streams and their events           */
 
+/* Layout variants (the paper fixes neither; Sec. 4.1 only asks for contiguous per-device
+ * expert tensors and a paged KV cache).  They apply to BOTH sides of the step. */
+#define EMOE_LAYOUT_FUSED_W13 4u     /* expert arena per layer: [n_r][gate|up] (2m per slot),  */
+                                     /* then [n_r][down], instead of [3][n_r][m]               */
+#define EMOE_LAYOUT_KV_HEAD_MAJOR 8u /* KV block [Hkv/T][B][hd] instead of [B][Hkv/T][hd]     */
+
 /* phase / side selectors of the query helpers */
 #define EMOE_PHASE_EXPERTS 0
 #define EMOE_PHASE_ATTN 1
@@ -244,6 +250,11 @@ emoe_status_t emoe_reshard_step_host(const emoe_plan_t *plan, const void *const 
  * calls whose GPU work can overlap (different streams without an ordering
  * between them) race on it and must be serialised by the caller.  Nothing in
  * the array has to start at zero; each call overwrites the prefix it reads.
+ *
+ * Plans made with EMOE_LAYOUT_KV_HEAD_MAJOR are accepted while the TP degree
+ * is kept (whole blocks move); with a changed TP degree they are rejected
+ * with EMOE_ERR_UNSUPPORTED, since this entry point has only the token-major
+ * re-split kernel.
  *
  * The first call on each device looks up the array's device address
  * (one-time set-up, with that device current).  Make that first call outside

@@ -18,6 +18,8 @@ PHASE_EXPERTS, PHASE_ATTN, PHASE_KV = 0, 1, 2
 SIDE_OLD, SIDE_NEW = 0, 1
 PLAN_HOST_ONLY = 1
 PLAN_HOST_STEP = 2
+LAYOUT_FUSED_W13 = 4
+LAYOUT_KV_HEAD_MAJOR = 8
 MAX_RANKS = 64
 
 _i32, _u32, _u64, _vp = ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_void_p
@@ -205,7 +207,8 @@ def _stream_handle(stream) -> int:
 class Plan:
     """A scale-step plan: emoe_plan_create ... emoe_plan_destroy."""
 
-    def __init__(self, shape, old_cfg, new_cfg, host_only: bool = False, host_step: bool = False):
+    def __init__(self, shape, old_cfg, new_cfg, host_only: bool = False, host_step: bool = False,
+                 fused_w13: bool = False, kv_head_major: bool = False):
         self._h = _vp()
         keep: list = []
         sh = _Shape(shape.n_layers, shape.n_routed, shape.n_shared, shape.d_model, shape.d_ff,
@@ -214,7 +217,10 @@ class Plan:
         co, cn = _make_config(old_cfg, keep), _make_config(new_cfg, keep)
         _check(lib().emoe_plan_create(ctypes.byref(sh), ctypes.byref(co), ctypes.byref(cn),
                                       (PLAN_HOST_ONLY if host_only else 0)
-                                      | (PLAN_HOST_STEP if host_step else 0), ctypes.byref(self._h)))
+                                      | (PLAN_HOST_STEP if host_step else 0)
+                                      | (LAYOUT_FUSED_W13 if fused_w13 else 0)
+                                      | (LAYOUT_KV_HEAD_MAJOR if kv_head_major else 0),
+                                      ctypes.byref(self._h)))
         self.host_only = host_only
 
     # -- life cycle

@@ -305,7 +305,7 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
 // Chunk plans, streams and events of the pipelined host-buffer step.  Leaves p->hs null
 // (the step then runs serially) when a layer slice of some arena is not 16-byte aligned.
 emoe_status_t make_host_step(emoe_plan *p, const emoe_shape_t &shape, const emoe_config_t *old_cfg,
-                             const emoe_config_t *new_cfg) {
+                             const emoe_config_t *new_cfg, uint32_t layout_flags) {
   const int L = shape.n_layers;
   for (int ph = 0; ph < 3; ++ph) {
     for (uint64_t b : p->hp.phase[ph].arena_old) if ((b / L) % 16) return EMOE_OK;
@@ -318,10 +318,10 @@ emoe_status_t make_host_step(emoe_plan *p, const emoe_shape_t &shape, const emoe
   hs->n_chunks = n_full + (tail ? 1 : 0);
   emoe_shape_t sh = shape;
   sh.n_layers = hs->lc;
-  emoe_status_t st = create_plan(&sh, old_cfg, new_cfg, 0, &hs->chunk);
+  emoe_status_t st = create_plan(&sh, old_cfg, new_cfg, layout_flags, &hs->chunk);
   if (st == EMOE_OK && tail) {
     sh.n_layers = tail;
-    st = create_plan(&sh, old_cfg, new_cfg, 0, &hs->tail);
+    st = create_plan(&sh, old_cfg, new_cfg, layout_flags, &hs->tail);
   }
   cudaError_t e = cudaSuccess;
   if (st == EMOE_OK) e = cudaStreamCreateWithFlags(&hs->s_in, cudaStreamNonBlocking);
@@ -365,7 +365,7 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
   if (!p) return EMOE_ERR_OOM;
   emoe_status_t st;
   try {
-    st = build_host_plan(*shape, *old_cfg, *new_cfg, &p->hp);
+    st = build_host_plan(*shape, *old_cfg, *new_cfg, flags, &p->hp);
     if (st == EMOE_OK)
       for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
   } catch (const std::bad_alloc &) {
@@ -392,7 +392,8 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
       if (e3 == cudaSuccess) e3 = cudaMemset(p->d_status, 0, sizeof(int));
       st = cuda_status(e3);
     }
-    if (st == EMOE_OK && (flags & EMOE_PLAN_HOST_STEP)) st = make_host_step(p, *shape, old_cfg, new_cfg);
+    if (st == EMOE_OK && (flags & EMOE_PLAN_HOST_STEP)) st = make_host_step(p, *shape, old_cfg, new_cfg,
+                                  flags & (EMOE_LAYOUT_FUSED_W13 | EMOE_LAYOUT_KV_HEAD_MAJOR));
     if (st != EMOE_OK) { free_device(p); delete p; return st; }
   }
   *out = p;
@@ -485,6 +486,9 @@ emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *p, const void *const *sr
                                      void *stream) {
   if (!p || !src || !dst) return EMOE_ERR_INVALID_ARG;
   const KvPlan &kv = p->hp.kv;
+  // this entry point only has the token-major pair kernel: whole blocks (TP kept) are
+  // layout-agnostic, a head re-split of head-major blocks is not
+  if (kv.head_major && kv.c != kv.d) return EMOE_ERR_UNSUPPORTED;
   const std::vector<uint32_t> *pair_old = &kv.pair_old, *pair_new = &kv.pair_new;
   if (pair_old->size() > EMOE_STATIC_KV_MAX_PAIRS) return EMOE_ERR_TOO_LARGE;
   // the same argument checks as emoe_reshard_kv, but a host-only plan is welcome here

@@ -101,8 +101,9 @@ emoe_status_t read_block_pairs(const emoe_shape_t &sh, const emoe_config_t &o,
 // paged store pads every matrix to its allocation granularity).  remaps: if non-null,
 // a destination slot whose source sits on the same rank index is recorded there instead
 // of being copied (that device already holds the bytes).
+// fused_w13 (dense layout only): per layer a [n][gate|up] tensor, then the [n][down] one.
 void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &pn, uint64_t slab,
-                  std::vector<Remap> *remaps, PhasePlan *pp) {
+                  std::vector<Remap> *remaps, bool fused_w13, PhasePlan *pp) {
   const uint64_t m = (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes;
   const uint32_t runs = (uint32_t)sh.n_layers * 3;
   const int n_experts = sh.n_routed + sh.n_shared;
@@ -139,7 +140,9 @@ void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &
     const Move &a = moves[i];
     const uint64_t n_old = po.ids[a.rs].size(), n_new = pn.ids[a.rd].size();
     if (fan[{a.rs, a.ss}] > 1) {
-      multi[{a.rs, a.ss}].push_back({(uint64_t)a.sd * slab, n_new * slab, (uint32_t)a.rd, 0});
+      // fused layout: off = slot index, pitch = slot count; resolved to bytes below
+      if (fused_w13) multi[{a.rs, a.ss}].push_back({(uint64_t)a.sd, n_new, (uint32_t)a.rd, 0});
+      else multi[{a.rs, a.ss}].push_back({(uint64_t)a.sd * slab, n_new * slab, (uint32_t)a.rd, 0});
       ++i;
       continue;
     }
@@ -149,23 +152,51 @@ void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &
            fan[{moves[j].rs, moves[j].ss}] == 1)
       ++j;
     Segment s{};
-    s.src_off = (uint64_t)a.ss * slab;
-    s.run_bytes = (uint64_t)(j - i) * m;
-    s.src_pitch = n_old * slab;
-    s.n_runs = runs;
     s.src_rank = (uint32_t)a.rs;
-    finish_segment(pp, s, {Dst{(uint64_t)a.sd * slab, n_new * slab, (uint32_t)a.rd, 0}});
+    if (!fused_w13) {
+      s.src_off = (uint64_t)a.ss * slab;
+      s.run_bytes = (uint64_t)(j - i) * m;
+      s.src_pitch = n_old * slab;
+      s.n_runs = runs;
+      finish_segment(pp, s, {Dst{(uint64_t)a.sd * slab, n_new * slab, (uint32_t)a.rd, 0}});
+    } else {  // per layer: the slots' gate|up pairs, then their down matrices
+      s.n_runs = (uint32_t)sh.n_layers;
+      s.src_pitch = 3 * n_old * m;
+      s.src_off = (uint64_t)a.ss * 2 * m;
+      s.run_bytes = (uint64_t)(j - i) * 2 * m;
+      finish_segment(pp, s, {Dst{(uint64_t)a.sd * 2 * m, 3 * n_new * m, (uint32_t)a.rd, 0}});
+      s.src_off = n_old * 2 * m + (uint64_t)a.ss * m;
+      s.run_bytes = (uint64_t)(j - i) * m;
+      finish_segment(pp, s, {Dst{n_new * 2 * m + (uint64_t)a.sd * m, 3 * n_new * m, (uint32_t)a.rd, 0}});
+    }
     i = j;
   }
   // replicated sources: read once, write to every destination
   for (const auto &kv : multi) {
     Segment s{};
-    s.src_off = (uint64_t)kv.first.second * slab;
-    s.run_bytes = m;
-    s.src_pitch = po.ids[kv.first.first].size() * slab;
-    s.n_runs = runs;
     s.src_rank = (uint32_t)kv.first.first;
-    finish_segment(pp, s, kv.second);
+    const uint64_t n_old = po.ids[kv.first.first].size(), ss = (uint64_t)kv.first.second;
+    if (!fused_w13) {
+      s.src_off = ss * slab;
+      s.run_bytes = m;
+      s.src_pitch = n_old * slab;
+      s.n_runs = runs;
+      finish_segment(pp, s, kv.second);
+    } else {
+      std::vector<Dst> d13, d2;
+      for (const Dst &d : kv.second) {  // d.off = slot, d.pitch = slots of that rank
+        d13.push_back({d.off * 2 * m, 3 * d.pitch * m, d.rank, 0});
+        d2.push_back({d.pitch * 2 * m + d.off * m, 3 * d.pitch * m, d.rank, 0});
+      }
+      s.n_runs = (uint32_t)sh.n_layers;
+      s.src_pitch = 3 * n_old * m;
+      s.src_off = ss * 2 * m;
+      s.run_bytes = 2 * m;
+      finish_segment(pp, s, d13);
+      s.src_off = n_old * 2 * m + ss * m;
+      s.run_bytes = m;
+      finish_segment(pp, s, d2);
+    }
   }
 }
 
@@ -255,7 +286,8 @@ void plan_attn(const emoe_shape_t &sh, int c, int d, PhasePlan *pp) {
 // ---- KV ---------------------------------------------------------------------------------
 
 void plan_kv(const emoe_shape_t &sh, const emoe_config_t &o, const emoe_config_t &n,
-             std::vector<uint32_t> pair_old, std::vector<uint32_t> pair_new, HostPlan *hp) {
+             std::vector<uint32_t> pair_old, std::vector<uint32_t> pair_new, bool head_major,
+             HostPlan *hp) {
   PhasePlan *pp = &hp->phase[EMOE_PHASE_KV];
   KvPlan &kv = hp->kv;
   const uint64_t vec = (uint64_t)sh.head_dim * sh.elem_bytes, B = sh.kv_block_tokens;
@@ -289,6 +321,32 @@ void plan_kv(const emoe_shape_t &sh, const emoe_config_t &o, const emoe_config_t
 
   kv.pair_old = pair_old;  // kept in both cases: the fixed-scratch entry point reads them
   kv.pair_new = pair_new;
+  kv.head_major = head_major;
+  if (kv.head_split_changes && head_major) {
+    // head-major blocks: a head's tokens are contiguous, so every run of destination heads
+    // that sit consecutively on one old rank is one contiguous piece per (layer, K|V, block)
+    for (size_t i = 0; i < n_pairs; ++i)
+      for (uint32_t rn = 0; rn < kv.d; ++rn) {
+        uint32_t hl = 0;
+        while (hl < kv.hn) {
+          const uint32_t j = rn * kv.hn + hl, ro = kv.src_rank[j], ho = kv.src_head[j];
+          uint32_t cnt = 1;
+          while (hl + cnt < kv.hn && kv.src_rank[j + cnt] == ro && kv.src_head[j + cnt] == ho + cnt) ++cnt;
+          Segment s{};
+          s.src_off = pair_old[i] * blk_old + (uint64_t)ho * B * vec;
+          s.run_bytes = (uint64_t)cnt * B * vec;
+          s.src_pitch = o.kv_num_blocks * blk_old;
+          s.n_runs = (uint32_t)(L * 2);
+          s.src_rank = ro;
+          finish_segment(pp, s, {Dst{pair_new[i] * blk_new + (uint64_t)hl * B * vec,
+                                     n.kv_num_blocks * blk_new, rn, 0}});
+          hl += cnt;
+        }
+      }
+    pp->bytes_read = per_head * heads_read;  // distinct (old rank, head) slots that are read
+    kv.head_split_changes = false;           // the segment kernels do this phase
+    return;
+  }
   if (kv.head_split_changes) {
     pp->bytes_moved = per_head * kv.d * kv.hn;  // every new rank's heads, replicas included
     pp->bytes_read = per_head * heads_read;     // distinct (old rank, head) slots that are read
@@ -329,7 +387,7 @@ uint32_t kv_source_rank(uint32_t hkv, uint32_t c, uint32_t g, uint32_t r_new) {
 }
 
 emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
-                              const emoe_config_t &n, HostPlan *hp) {
+                              const emoe_config_t &n, uint32_t flags, HostPlan *hp) {
   if (sh.n_layers <= 0 || sh.n_routed <= 0 || sh.n_shared < 0 || sh.d_model <= 0 ||
       sh.d_ff <= 0 || sh.n_q_heads <= 0 || sh.n_kv_heads <= 0 || sh.head_dim <= 0 ||
       sh.kv_block_tokens <= 0 || sh.elem_bytes <= 0)
@@ -352,9 +410,9 @@ emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
   hp->shape = sh;
   hp->ep_old = o.ep; hp->ep_new = n.ep; hp->tp_old = o.tp; hp->tp_new = n.tp;
   plan_experts(sh, po, pn, (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes, nullptr,
-               &hp->phase[EMOE_PHASE_EXPERTS]);
+               (flags & EMOE_LAYOUT_FUSED_W13) != 0, &hp->phase[EMOE_PHASE_EXPERTS]);
   plan_attn(sh, o.tp, n.tp, &hp->phase[EMOE_PHASE_ATTN]);
-  plan_kv(sh, o, n, std::move(pair_old), std::move(pair_new), hp);
+  plan_kv(sh, o, n, std::move(pair_old), std::move(pair_new), (flags & EMOE_LAYOUT_KV_HEAD_MAJOR) != 0, hp);
   return EMOE_OK;
 }
 
@@ -370,7 +428,7 @@ emoe_status_t build_paged_expert_plan(const emoe_shape_t &sh, const emoe_config_
   if (st != EMOE_OK) return st;
   st = read_placement(n, sh.n_routed + sh.n_shared, &pn);
   if (st != EMOE_OK) return st;
-  plan_experts(sh, po, pn, slab, remaps, pp);
+  plan_experts(sh, po, pn, slab, remaps, false, pp);
   return EMOE_OK;
 }
 

@@ -56,6 +56,7 @@ struct KvPlan {
   uint32_t hc = 0, hn = 0;
   std::vector<uint8_t> src_rank;
   std::vector<uint16_t> src_head;
+  bool head_major = false;  // blocks are [local head][token][hd]
   bool replicated = false;  // a side has more ranks than KV heads: the map is not g/hc, g%hc
 };
 
@@ -73,8 +74,9 @@ struct HostPlan {
 };
 
 // Validates and plans.  Returns EMOE_OK or the first validation error.
+// flags: the EMOE_LAYOUT_* bits of emoe_plan_create.
 emoe_status_t build_host_plan(const emoe_shape_t &shape, const emoe_config_t &old_cfg,
-                              const emoe_config_t &new_cfg, HostPlan *out);
+                              const emoe_config_t &new_cfg, uint32_t flags, HostPlan *out);
 
 // A destination slot that keeps the bytes its rank already holds (paged expert store).
 struct Remap {

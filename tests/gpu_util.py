@@ -16,11 +16,18 @@ KINDS = {E.PHASE_EXPERTS: W.KIND_EXPERTS, E.PHASE_ATTN: W.KIND_ATTN, E.PHASE_KV:
 
 def oracle_phase(wl, phase, src, dst):
     if phase == E.PHASE_EXPERTS:
-        oracle.reshard_experts(wl.shape, wl.old.placement, wl.new.placement, src, dst)
+        oracle.reshard_experts(wl.shape, wl.old.placement, wl.new.placement, src, dst,
+                               fused_w13=wl.fused_w13)
     elif phase == E.PHASE_ATTN:
         oracle.reshard_attn(wl.shape, wl.old.tp, wl.new.tp, src, dst)
     else:
-        oracle.reshard_kv(wl.shape, wl.old, wl.new, src, dst)
+        oracle.reshard_kv(wl.shape, wl.old, wl.new, src, dst, head_major=wl.kv_head_major)
+
+
+def make_plan(wl, **kw):
+    """A plan with the workload's layout variants."""
+    return E.Plan(wl.shape, wl.old, wl.new, fused_w13=wl.fused_w13,
+                  kv_head_major=wl.kv_head_major, **kw)
 
 
 def run_phase(plan, phase, src, dst, stream=None):

@@ -244,3 +244,18 @@ def test_more_tp_ranks_than_kv_heads(c, d):
         st = plan.stats(E.PHASE_KV)
         used = sum(-(-n // 16) for n in wl.old.seq_lens)
         assert st["bytes_moved"] == 2 * used * 16 * max(4, d) * 128 * 2
+
+
+@pytest.mark.parametrize("name", ["c1_tiny", "c3_fine", "c4_large"])
+def test_layout_variants_one_layer(name):
+    """Fused gate|up expert tensors and head-major KV blocks at full width."""
+    from gpu_util import make_plan
+    wl = W.make_workload(name, n_layers=2 if name == "c1_tiny" else 1)
+    wl = R(wl, fused_w13=True, kv_head_major=True)
+    for w in (wl, wl.swapped()):
+        with make_plan(w) as plan:
+            for phase in (E.PHASE_EXPERTS, E.PHASE_KV):
+                check_phase_full(w, plan, phase)
+            plan.set_tuning(path=2, max_ctas=9)
+            for phase in (E.PHASE_EXPERTS, E.PHASE_KV):
+                check_phase_full(w, plan, phase)

@@ -7,7 +7,7 @@ import pytest
 from hypothesis import HealthCheck, given, settings
 
 import paper_2510_02613_b200 as E
-from gpu_util import check_phase_full
+from gpu_util import check_phase_full, make_plan
 from test_planner_random import cases
 
 pytestmark = pytest.mark.gpu
@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
           suppress_health_check=list(HealthCheck))
 @given(cases())
 def test_drawn_cases_match_the_oracle(wl):
-    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+    with make_plan(wl) as plan:
         for phase in range(3):
             check_phase_full(wl, plan, phase)
         for kv_mode in (2, 3, 4):

@@ -52,11 +52,12 @@ def arenas(sizes, key):
 
 def run_oracle(wl, phase, src, dst):
     if phase == E.PHASE_EXPERTS:
-        oracle.reshard_experts(wl.shape, wl.old.placement, wl.new.placement, src, dst)
+        oracle.reshard_experts(wl.shape, wl.old.placement, wl.new.placement, src, dst,
+                               fused_w13=wl.fused_w13)
     elif phase == E.PHASE_ATTN:
         oracle.reshard_attn(wl.shape, wl.old.tp, wl.new.tp, src, dst)
     else:
-        oracle.reshard_kv(wl.shape, wl.old, wl.new, src, dst)
+        oracle.reshard_kv(wl.shape, wl.old, wl.new, src, dst, head_major=wl.kv_head_major)
 
 
 def oracle_sizes(wl, phase):
@@ -210,4 +211,24 @@ def test_more_ranks_than_the_library_supports():
     for bad in (too_many_ep, too_many_tp):
         with pytest.raises(E.EmoeError) as ei:
             E.Plan(sh, ok, bad, host_only=True)
+        assert ei.value.code == 9
+
+
+def test_layout_variants_change_segments_not_sizes():
+    wl = small("c4_large")
+    with E.Plan(wl.shape, wl.old, wl.new, host_only=True) as plain, \
+            E.Plan(wl.shape, wl.old, wl.new, host_only=True, fused_w13=True, kv_head_major=True) as var:
+        for phase in range(3):
+            assert plain.arena_bytes(phase, E.SIDE_NEW) == var.arena_bytes(phase, E.SIDE_NEW)
+            assert plain.stats(phase)["bytes_moved"] == var.stats(phase)["bytes_moved"]
+        # fused gate|up: two runs per layer instead of three per (layer, projection)
+        a, b = plain.segments(E.PHASE_EXPERTS), var.segments(E.PHASE_EXPERTS)
+        assert int(a["n_runs"].max()) == 3 * wl.shape.n_layers and int(b["n_runs"].max()) == wl.shape.n_layers
+        # head-major KV: every piece is a whole head's tokens (B * hd * b bytes per head)
+        kv = var.segments(E.PHASE_KV)
+        assert set(int(x) for x in kv["run_bytes"]) == {wl.shape.kv_block_tokens * wl.shape.head_dim
+                                                       * wl.shape.elem_bytes}
+        # the allocation-free KV entry point has no head-major re-split
+        with pytest.raises(E.EmoeError) as ei:
+            var.reshard_kv_static([16] * 2, [16] * 4)
         assert ei.value.code == 9

@@ -57,13 +57,15 @@ def cases(draw):
     old = W.ParallelConfig(0, c, draw(placements(sh.n_experts)), max(nb_old, 1), seq_lens, bo)
     new = W.ParallelConfig(0, d, draw(placements(sh.n_experts)), max(nb_new, 1), seq_lens, bn)
     old.ep, new.ep = len(old.placement), len(new.placement)
-    return W.Workload("drawn", sh, old, new, seed)
+    return W.Workload("drawn", sh, old, new, seed, fused_w13=draw(st.booleans()),
+                      kv_head_major=draw(st.booleans()))
 
 
 @settings(max_examples=80, deadline=None, suppress_health_check=list(HealthCheck))
 @given(cases())
 def test_drawn_plans_replay_to_the_oracle(wl):
-    with E.Plan(wl.shape, wl.old, wl.new, host_only=True) as plan:
+    with E.Plan(wl.shape, wl.old, wl.new, host_only=True, fused_w13=wl.fused_w13,
+                kv_head_major=wl.kv_head_major) as plan:
         for phase in range(3):
             so, sn = oracle_sizes(wl, phase)
             assert plan.arena_bytes(phase, E.SIDE_OLD) == so

@@ -66,6 +66,8 @@ class Workload:
     seed: int
     notes: str = ""
     victim: Optional[dict] = field(default=None)   # C5: the concurrent GEMM's shape
+    fused_w13: bool = False        # layout variant: per layer [n][gate|up] then [n][down]
+    kv_head_major: bool = False    # layout variant: KV blocks [local head][token][hd]
 
     def with_layers(self, n_layers: int) -> "Workload":
         """Same workload cut to n_layers (layers are independent in every phase)."""
