@@ -406,6 +406,35 @@ typedef struct {
  * running concurrently on other host threads. */
 emoe_status_t emoe_plan_set_tuning(emoe_plan_t *plan, const emoe_tuning_t *tuning);
 
+/* ---- one rank per GPU: pull-based exchange --------------------------------
+ *
+ * With rank = GPU, every destination arena is written by the GPU that owns it
+ * and every segment has one source rank, so a scale step is ONE exchange: each
+ * GPU pulls what it needs from its peers' old arenas (the counterpart of the
+ * paper's P2P transfers, Sec. 4 and App. D) and copies the rest locally.  The
+ * kernels are the same; a remote source is simply a peer-mapped pointer.
+ *
+ * emoe_plan_set_local_rank: from now on the reshard calls of this plan write
+ * ONLY the destination arenas of new-rank index `rank` (-1: all, the
+ * default).  dst[] entries of other ranks and src[] entries of old ranks that
+ * this rank reads nothing from may then be NULL.  Every process builds the
+ * same plan from the same configurations and sets its own rank; the union of
+ * what the ranks write is the whole step.  Not for plans created with
+ * EMOE_PLAN_HOST_STEP.  Synchronises the device (descriptor tables are
+ * rebuilt). */
+emoe_status_t emoe_plan_set_local_rank(emoe_plan_t *plan, int32_t rank);
+
+/* Sharing an arena with the other processes of the node (CUDA IPC).
+ * emoe_ipc_export: handle_out receives EMOE_IPC_HANDLE_BYTES bytes naming the
+ * ALLOCATION that contains device_ptr, offset_out the pointer's offset in it.
+ * emoe_ipc_open (in another process, with its device current): maps that
+ * allocation and returns its base; the arena is at base + offset.
+ * emoe_ipc_close: unmaps it.  A process uses its own arenas directly. */
+#define EMOE_IPC_HANDLE_BYTES 64
+emoe_status_t emoe_ipc_export(const void *device_ptr, void *handle_out, uint64_t *offset_out);
+emoe_status_t emoe_ipc_open(const void *handle, void **base_out);
+emoe_status_t emoe_ipc_close(void *base);
+
 /* Static string for a status code. */
 const char *emoe_strerror(emoe_status_t status);
 

@@ -72,6 +72,7 @@ EXPORTS = ("emoe_plan_create", "emoe_reshard_experts", "emoe_reshard_attn", "emo
            "emoe_reshard_step_host", "emoe_plan_destroy", "emoe_plan_num_ranks",
            "emoe_plan_arena_bytes", "emoe_plan_stats", "emoe_plan_num_launches", "emoe_plan_segments",
            "emoe_plan_device_status", "emoe_plan_set_tuning", "emoe_strerror",
+           "emoe_plan_set_local_rank", "emoe_ipc_export", "emoe_ipc_open", "emoe_ipc_close",
            "emoe_vmm_create", "emoe_vmm_reshard", "emoe_vmm_dry_run", "emoe_vmm_num_ranks", "emoe_vmm_arena",
            "emoe_vmm_write", "emoe_vmm_read", "emoe_vmm_destroy")
 
@@ -123,6 +124,14 @@ def lib() -> ctypes.CDLL:
     L.emoe_plan_device_status.argtypes = [_vp, ctypes.POINTER(_i32)]
     L.emoe_plan_set_tuning.restype = _i32
     L.emoe_plan_set_tuning.argtypes = [_vp, ctypes.POINTER(_Tuning)]
+    L.emoe_plan_set_local_rank.restype = _i32
+    L.emoe_plan_set_local_rank.argtypes = [_vp, _i32]
+    L.emoe_ipc_export.restype = _i32
+    L.emoe_ipc_export.argtypes = [_vp, ctypes.c_char_p, ctypes.POINTER(_u64)]
+    L.emoe_ipc_open.restype = _i32
+    L.emoe_ipc_open.argtypes = [ctypes.c_char_p, ctypes.POINTER(_vp)]
+    L.emoe_ipc_close.restype = _i32
+    L.emoe_ipc_close.argtypes = [_vp]
     L.emoe_vmm_create.restype = _i32
     L.emoe_vmm_create.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Config), ctypes.POINTER(_vp)]
     L.emoe_vmm_reshard.restype = _i32
@@ -185,7 +194,9 @@ def _ptr_array(items: Sequence) -> ctypes.Array:
     """Device (or host) addresses from ints, torch tensors or numpy arrays."""
     vals = []
     for x in items:
-        if isinstance(x, int):
+        if x is None:
+            vals.append(0)
+        elif isinstance(x, int):
             vals.append(x)
         elif hasattr(x, "data_ptr"):
             vals.append(x.data_ptr())
@@ -287,6 +298,10 @@ class Plan:
                     unit_order)
         _check(lib().emoe_plan_set_tuning(self._h, ctypes.byref(t)))
 
+    def set_local_rank(self, rank: int) -> None:
+        """From now on write only the destination arenas of new-rank index `rank` (-1: all)."""
+        _check(lib().emoe_plan_set_local_rank(self._h, rank))
+
     # -- the hot path
     def _run(self, fn, src, dst, stream) -> None:
         _check(fn(self._h, _ptr_array(src), _ptr_array(dst), _stream_handle(stream)))
@@ -321,6 +336,28 @@ class Plan:
 
         _check(lib().emoe_reshard_step_host(self._h, pack(h_src), pack(h_dst), pack(d_src),
                                             pack(d_dst), _stream_handle(stream)))
+
+
+IPC_HANDLE_BYTES = 64
+
+
+def ipc_export(device_ptr: int):
+    """(handle bytes, offset) naming the allocation that holds device_ptr."""
+    buf = ctypes.create_string_buffer(IPC_HANDLE_BYTES)
+    off = _u64()
+    _check(lib().emoe_ipc_export(device_ptr, buf, ctypes.byref(off)))
+    return buf.raw, off.value
+
+
+def ipc_open(handle: bytes) -> int:
+    """Maps another process's allocation; returns its base address in this process."""
+    base = _vp()
+    _check(lib().emoe_ipc_open(handle, ctypes.byref(base)))
+    return base.value
+
+
+def ipc_close(base: int) -> None:
+    _check(lib().emoe_ipc_close(base))
 
 
 def _placement_config(placement, keep: list) -> _Config:

@@ -1,4 +1,5 @@
 // capi.cpp - the C ABI of libemoe.so: plan life cycle, argument checks, launches.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -56,6 +57,8 @@ struct emoe_plan {
   bool host_only = true;
   int device = -1, sm_count = 148;
   emoe_tuning_t tuning{};
+  int local_rank = -1;            // >= 0: only destinations of this new-rank index are written
+  bool reads_src[3][EMOE_MAX_RANKS];  // old ranks the (filtered) phase reads
   DevPhase dev[3];
   std::vector<uint32_t> pair_old, pair_new;  // block pairs in launch order (see kv_order)
   uint32_t *d_pair_old = nullptr, *d_pair_new = nullptr;
@@ -109,6 +112,7 @@ void build_tables(emoe_plan *p, int phase) {
   const PhasePlan &pp = p->hp.phase[phase];
   DevPhase &dp = p->dev[phase];
   dp.segs.clear(); dp.dsts.clear(); dp.bulk_units.clear(); dp.vec_units.clear();
+  for (bool &b : p->reads_src[phase]) b = false;
   const uint32_t T = bulk_tile(p);
 
   // KV with the head split kept: one segment per block pair and TP rank.  Visit them in
@@ -144,17 +148,26 @@ void build_tables(emoe_plan *p, int phase) {
     bool is_bulk = s0.align == 16 && s0.run_bytes >= kBulkMinRun && !all_vec;
     if (p->tuning.path == 1) is_bulk = false;
     if (p->tuning.path == 2) is_bulk = (s0.align == 16);
-    const uint32_t max_fan = is_bulk ? (uint32_t)kMaxFanout : s0.n_dst;
-    for (uint32_t k = 0; k < s0.n_dst; k += max_fan) {
+    // destinations this plan writes: all, or those of the local rank only
+    std::vector<Dst> mine;
+    for (uint32_t j = 0; j < s0.n_dst; ++j) {
+      const Dst &d = pp.dsts[s0.dst_first + j];
+      if (p->local_rank < 0 || (int)d.rank == p->local_rank) mine.push_back(d);
+    }
+    if (mine.empty()) continue;
+    p->reads_src[phase][s0.src_rank] = true;
+    const uint32_t n_mine = (uint32_t)mine.size();
+    const uint32_t max_fan = is_bulk ? (uint32_t)kMaxFanout : n_mine;
+    for (uint32_t k = 0; k < n_mine; k += max_fan) {
       DevSeg s{};
       s.src_off = s0.src_off; s.run_bytes = s0.run_bytes; s.src_pitch = s0.src_pitch;
       s.n_runs = s0.n_runs; s.src_rank = s0.src_rank; s.align = s0.align;
-      s.n_dst = s0.n_dst - k < max_fan ? s0.n_dst - k : max_fan;
+      s.n_dst = n_mine - k < max_fan ? n_mine - k : max_fan;
       s.dst_first = (uint32_t)dp.dsts.size();
-      const Dst &d0 = pp.dsts[s0.dst_first + k];
+      const Dst &d0 = mine[k];
       s.dst_off = d0.off; s.dst_pitch = d0.pitch; s.dst_rank = d0.rank;
       if (s.n_dst > 1)  // the one-destination case reads the inlined copy only
-        for (uint32_t j = 0; j < s.n_dst; ++j) dp.dsts.push_back(pp.dsts[s0.dst_first + k + j]);
+        for (uint32_t j = 0; j < s.n_dst; ++j) dp.dsts.push_back(mine[k + j]);
       const uint32_t idx = (uint32_t)dp.segs.size();
       dp.segs.push_back(s);
       if (is_bulk) add_units(&bulk, idx, s, T);
@@ -169,6 +182,10 @@ void build_tables(emoe_plan *p, int phase) {
 
   if (phase == EMOE_PHASE_KV) {  // block pairs of the head re-split, in launch order
     const KvPlan &kv = p->hp.kv;
+    if (kv.head_split_changes && !kv.pair_old.empty())
+      for (uint32_t rn = 0; rn < kv.d; ++rn)
+        if (p->local_rank < 0 || (int)rn == p->local_rank)
+          for (uint32_t hl = 0; hl < kv.hn; ++hl) p->reads_src[phase][kv.src_rank[rn * kv.hn + hl]] = true;
     std::vector<uint32_t> idx(kv.pair_old.size());
     for (uint32_t i = 0; i < idx.size(); ++i) idx[i] = i;
     if (kv_order(p) >= 2) {
@@ -231,18 +248,24 @@ emoe_status_t check_arenas(const emoe_plan *p, int phase, const void *const *src
   const PhasePlan &pp = p->hp.phase[phase];
   const int ns = ranks_of(p, phase, EMOE_SIDE_OLD), nd = ranks_of(p, phase, EMOE_SIDE_NEW);
   std::memset(out, 0, sizeof(*out));
+  // With a local rank set, only that rank's destination arena and the source arenas its
+  // work reads are needed; the other entries may be NULL and are never dereferenced.
+  const bool local = p->local_rank >= 0;
   for (int r = 0; r < ns; ++r) {
-    if (pp.arena_old[r] && !src[r]) return EMOE_ERR_INVALID_ARG;
+    const bool needed = local ? p->reads_src[phase][r] : pp.arena_old[r] != 0;
+    if (needed && !src[r]) return EMOE_ERR_INVALID_ARG;
     if ((uintptr_t)src[r] % 16) return EMOE_ERR_ALIGNMENT;
     out->src[r] = (const uint8_t *)src[r];
   }
   for (int r = 0; r < nd; ++r) {
-    if (pp.arena_new[r] && !dst[r]) return EMOE_ERR_INVALID_ARG;
+    const bool needed = pp.arena_new[r] != 0 && (!local || r == p->local_rank);
+    if (needed && !dst[r]) return EMOE_ERR_INVALID_ARG;
     if ((uintptr_t)dst[r] % 16) return EMOE_ERR_ALIGNMENT;
-    out->dst[r] = (uint8_t *)dst[r];
+    out->dst[r] = needed ? (uint8_t *)dst[r] : nullptr;
   }
   for (int a = 0; a < ns; ++a)
     for (int b = 0; b < nd; ++b) {
+      if (!src[a] || !out->dst[b]) continue;
       const uintptr_t s0 = (uintptr_t)src[a], s1 = s0 + pp.arena_old[a];
       const uintptr_t d0 = (uintptr_t)dst[b], d1 = d0 + pp.arena_new[b];
       if (s0 < d1 && d0 < s1) return EMOE_ERR_OVERLAP;
@@ -272,8 +295,10 @@ emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, 
 }
 
 // Shape constants of the KV head re-split as the kernels take them.
-KvTables kv_tables(const KvPlan &kv, const uint32_t *d_pair_old, const uint32_t *d_pair_new) {
+KvTables kv_tables(const KvPlan &kv, const uint32_t *d_pair_old, const uint32_t *d_pair_new,
+                   int local_rank = -1) {
   KvTables t{};
+  t.dst_only = local_rank >= 0 ? (uint32_t)local_rank : 0xffffffffu;
   t.pair_old = d_pair_old;
   t.pair_new = d_pair_new;
   t.n_pairs = (uint32_t)kv.pair_old.size();
@@ -476,7 +501,7 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *p, const void *const *src, void
   if (st != EMOE_OK) return st;
   if (!p->hp.kv.head_split_changes) return run_segments(p, EMOE_PHASE_KV, ptrs, (cudaStream_t)stream);
   const KvPlan &kv = p->hp.kv;
-  KvTables t = kv_tables(kv, p->d_pair_old, p->d_pair_new);
+  KvTables t = kv_tables(kv, p->d_pair_old, p->d_pair_new, p->local_rank);
   const int mode = p->tuning.kv_mode > 0 ? p->tuning.kv_mode : kDefaultKvMode;
   return cuda_status(launch_kv_copy(t, ptrs, mode, cta_budget(p), p->tuning.max_ctas <= 0, p->d_status,
                                     (cudaStream_t)stream));
@@ -727,6 +752,74 @@ emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
     }
   }
   return st;
+}
+
+emoe_status_t emoe_plan_set_local_rank(emoe_plan_t *p, int32_t rank) {
+  if (!p || rank < -1 || rank >= EMOE_MAX_RANKS) return EMOE_ERR_INVALID_ARG;
+  if (p->hs) return EMOE_ERR_UNSUPPORTED;  // the pipelined host step works on whole steps
+  p->local_rank = rank;
+  emoe_status_t st = EMOE_OK;
+  try {
+    for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
+  } catch (const std::bad_alloc &) {
+    return EMOE_ERR_OOM;
+  }
+  if (!p->host_only) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return EMOE_ERR_CUDA;
+    for (int ph = 0; st == EMOE_OK && ph < 3; ++ph) st = upload_phase(p, ph);
+  }
+  return st;
+}
+
+emoe_status_t emoe_ipc_export(const void *device_ptr, void *handle_out, uint64_t *offset_out) {
+  if (!device_ptr || !handle_out || !offset_out) return EMOE_ERR_INVALID_ARG;
+  // the handle names the whole allocation: report where inside it the pointer lies
+  using GetRangeFn = CUresult (*)(CUdeviceptr *, size_t *, CUdeviceptr);
+  static GetRangeFn get_range = [] {
+    void *f = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuMemGetAddressRange", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess) {
+      (void)cudaGetLastError();
+      f = nullptr;
+    }
+    return reinterpret_cast<GetRangeFn>(f);
+  }();
+  if (!get_range) return EMOE_ERR_UNSUPPORTED;
+  CUdeviceptr base = 0;
+  size_t size = 0;
+  if (get_range(&base, &size, (CUdeviceptr)(uintptr_t)device_ptr) != CUDA_SUCCESS) return EMOE_ERR_CUDA;
+  cudaIpcMemHandle_t h;
+  if (cudaIpcGetMemHandle(&h, reinterpret_cast<void *>(base)) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return EMOE_ERR_CUDA;
+  }
+  static_assert(sizeof(h) == EMOE_IPC_HANDLE_BYTES, "handle size");
+  std::memcpy(handle_out, &h, sizeof(h));
+  *offset_out = (uint64_t)((uintptr_t)device_ptr - (uintptr_t)base);
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_ipc_open(const void *handle, void **base_out) {
+  if (!handle || !base_out) return EMOE_ERR_INVALID_ARG;
+  cudaIpcMemHandle_t h;
+  std::memcpy(&h, handle, sizeof(h));
+  void *base = nullptr;
+  if (cudaIpcOpenMemHandle(&base, h, cudaIpcMemLazyEnablePeerAccess) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return EMOE_ERR_CUDA;
+  }
+  *base_out = base;
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_ipc_close(void *base) {
+  if (!base) return EMOE_OK;
+  if (cudaIpcCloseMemHandle(base) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return EMOE_ERR_CUDA;
+  }
+  return EMOE_OK;
 }
 
 const char *emoe_strerror(emoe_status_t s) {

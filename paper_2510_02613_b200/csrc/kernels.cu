@@ -451,14 +451,19 @@ __global__ void __launch_bounds__(256) kv_direct_kernel(const __grid_constant__ 
     for (uint32_t q0 = threadIdx.x; q0 < total; q0 += blockDim.x * 4) {
       V v[4];
       uint32_t tok[4], g[4], j[4];
+      bool live[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const uint32_t q = q0 + u * blockDim.x;
+        live[u] = false;
         if (q < total) {
           tok[u] = q / row;
           const uint32_t rem = q - tok[u] * row;
           g[u] = rem / cpv;
           j[u] = rem - g[u] * cpv;
+          live[u] = t.dst_only == 0xffffffffu || g[u] / t.hn == t.dst_only;
+        }
+        if (live[u]) {
           uint32_t ro = g[u] / t.hc, ho = g[u] - ro * t.hc;
           if (t.use_map) { ro = t.map_rank[g[u]]; ho = t.map_head[g[u]]; }
           v[u] = *reinterpret_cast<const V *>(
@@ -467,8 +472,7 @@ __global__ void __launch_bounds__(256) kv_direct_kernel(const __grid_constant__ 
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const uint32_t q = q0 + u * blockDim.x;
-        if (q < total) {
+        if (live[u]) {
           const uint32_t rn = g[u] / t.hn, hn = g[u] - rn * t.hn;
           *reinterpret_cast<V *>(s_dst[rn] + base_new +
                                  ((uint64_t)(tok[u] * t.hn + hn) * cpv + j[u]) * W) = v[u];
@@ -493,6 +497,7 @@ __global__ void __launch_bounds__(256) kv_rows_kernel(const __grid_constant__ Kv
   uint32_t ro = g / t.hc, ho = g - ro * t.hc;
   if (t.use_map) { ro = t.map_rank[g]; ho = t.map_head[g]; }
   const uint32_t rn = g / t.hn, hn = g - rn * t.hn;
+  if (t.dst_only != 0xffffffffu && rn != t.dst_only) return;  // another rank writes that block
   const uint8_t *sp = p.ptrs.src[ro] + ((uint64_t)(tok0 * t.hc + ho) * cpv + j) * 16;
   uint8_t *dp = p.ptrs.dst[rn] + ((uint64_t)(tok0 * t.hn + hn) * cpv + j) * 16;
   const uint64_t s_step = (uint64_t)tpp * t.hc * t.head_bytes, d_step = (uint64_t)tpp * t.hn * t.head_bytes;
@@ -908,7 +913,8 @@ bool kv_tma_supported(const KvTables &t, uint32_t *stages_out) {
   const uint64_t box = (uint64_t)t.block_tokens * g * hb;
   const uint64_t rows_old = (uint64_t)t.n_lk * t.nb_old * t.block_tokens;
   const uint64_t rows_new = (uint64_t)t.n_lk * t.nb_new * t.block_tokens;
-  if (t.use_map || hb % 16 || c > kKvTmaMaxRanks || d > kKvTmaMaxRanks) return false;
+  if (t.use_map || t.dst_only != 0xffffffffu || hb % 16 || c > kKvTmaMaxRanks || d > kKvTmaMaxRanks)
+    return false;
   if ((hb % 4 == 0 ? hb / 4 : hb) > 256 || g > 256 || t.block_tokens > 256) return false;  // box extents
   if (box % 128 || t.hkv / g > kKvTmaMaxBoxes || tile > 96 * 1024) return false;
   if (rows_old >= (1ull << 31) || rows_new >= (1ull << 31)) return false;             // int32 coordinates
@@ -922,7 +928,7 @@ bool kv_tma_supported(const KvTables &t, uint32_t *stages_out) {
 bool kv_staged_supported(const KvTables &t, uint32_t *stages_out) {
   const uint64_t tile = (uint64_t)t.block_tokens * t.hkv * t.head_bytes;
   const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
-  if (t.use_map) return false;  // replicated heads: the default kernels handle the slot map
+  if (t.use_map || t.dst_only != 0xffffffffu) return false;  // only the default kernels do these
   if (t.head_bytes % 16 || tile > 64 * 1024 || blk_new >= (1u << 24) || t.hkv / t.hn > 255) return false;
   uint32_t stages = (uint32_t)((160 * 1024) / tile);
   if (stages > kMaxStages) stages = kMaxStages;

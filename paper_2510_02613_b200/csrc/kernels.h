@@ -58,6 +58,7 @@ struct KvTables {  // device pointers + shape constants of the KV head re-split
   // old rank map_rank[j], local head map_head[j]; otherwise slot j is global head j and
   // lives at old rank j / hc, local head j % hc.
   uint32_t use_map;
+  uint32_t dst_only;             // write only this new rank's blocks (0xffffffff: all ranks)
   uint8_t map_rank[kKvMapMax], map_head[kKvMapMax];
 };
 
