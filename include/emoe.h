@@ -406,6 +406,20 @@ typedef struct {
  * running concurrently on other host threads. */
 emoe_status_t emoe_plan_set_tuning(emoe_plan_t *plan, const emoe_tuning_t *tuning);
 
+/* emoe_place_min_transfer - a placement for EP=ep_new that keeps as many experts
+ * where they are as balance allows (Sec. 5.2 "Expert Weights": the new placement
+ * balances the experts while moving as little as possible; the paper gives no
+ * algorithm).  Every expert 0..n_experts-1 is placed exactly once, rank sizes
+ * differ by at most one, slots within a rank are in id order, and the number of
+ * experts placed on a rank index that already holds a copy in old_cfg (ep,
+ * place_off, place_ids; other fields ignored) is the maximum any such placement
+ * reaches.  Experts that have to move fill the free slots in id order.
+ * new_off: [ep_new + 1], new_ids: [n_experts], caller-owned host arrays;
+ * n_kept (optional): the number of experts that stay.  Host only, no CUDA call. */
+emoe_status_t emoe_place_min_transfer(int32_t n_experts, const emoe_config_t *old_cfg,
+                                      int32_t ep_new, int32_t *new_off, int32_t *new_ids,
+                                      int32_t *n_kept);
+
 /* ---- one rank per GPU: pull-based exchange --------------------------------
  *
  * With rank = GPU, every destination arena is written by the GPU that owns it

@@ -127,3 +127,25 @@ def reshard_kv(shape, old_cfg, new_cfg, src, dst, head_major: bool = False) -> N
                                      int(bool(head_major)))
     if rc != 0:
         raise ValueError("oracle: bad block table or TP degree")
+
+
+# ---- placement chooser: brute force ----------------------------------------------------
+
+def max_kept_bruteforce(n_experts: int, old_placement, ep_new: int) -> int:
+    """The most experts any BALANCED placement for ep_new ranks (every expert once, rank
+    sizes differing by at most one) leaves on a rank index that already holds a copy
+    (Sec. 5.2 "Expert Weights": balance while moving as little as possible).  Exhaustive
+    enumeration of all ep_new ** n_experts assignments: tiny inputs only."""
+    import itertools
+    holds = [set(p) for p in old_placement]
+    lo, hi = n_experts // ep_new, -(-n_experts // ep_new)
+    best = -1
+    for assign in itertools.product(range(ep_new), repeat=n_experts):
+        counts = [0] * ep_new
+        for r in assign:
+            counts[r] += 1
+        if min(counts) < lo or max(counts) > hi:
+            continue
+        kept = sum(1 for e, r in enumerate(assign) if r < len(holds) and e in holds[r])
+        best = max(best, kept)
+    return best

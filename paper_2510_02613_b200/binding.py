@@ -72,7 +72,7 @@ EXPORTS = ("emoe_plan_create", "emoe_reshard_experts", "emoe_reshard_attn", "emo
            "emoe_reshard_step_host", "emoe_plan_destroy", "emoe_plan_num_ranks",
            "emoe_plan_arena_bytes", "emoe_plan_stats", "emoe_plan_num_launches", "emoe_plan_segments",
            "emoe_plan_device_status", "emoe_plan_set_tuning", "emoe_strerror",
-           "emoe_plan_set_local_rank", "emoe_ipc_export", "emoe_ipc_open", "emoe_ipc_close",
+           "emoe_place_min_transfer", "emoe_plan_set_local_rank", "emoe_ipc_export", "emoe_ipc_open", "emoe_ipc_close",
            "emoe_vmm_create", "emoe_vmm_reshard", "emoe_vmm_dry_run", "emoe_vmm_num_ranks", "emoe_vmm_arena",
            "emoe_vmm_write", "emoe_vmm_read", "emoe_vmm_destroy")
 
@@ -124,6 +124,8 @@ def lib() -> ctypes.CDLL:
     L.emoe_plan_device_status.argtypes = [_vp, ctypes.POINTER(_i32)]
     L.emoe_plan_set_tuning.restype = _i32
     L.emoe_plan_set_tuning.argtypes = [_vp, ctypes.POINTER(_Tuning)]
+    L.emoe_place_min_transfer.restype = _i32
+    L.emoe_place_min_transfer.argtypes = [_i32, ctypes.POINTER(_Config), _i32, _i32p, _i32p, _i32p]
     L.emoe_plan_set_local_rank.restype = _i32
     L.emoe_plan_set_local_rank.argtypes = [_vp, _i32]
     L.emoe_ipc_export.restype = _i32
@@ -369,6 +371,19 @@ def _placement_config(placement, keep: list) -> _Config:
     keep += [off, ids]
     p = lambda a: a.ctypes.data_as(_i32p)
     return _Config(len(placement), 1, p(off), p(ids), 0, 0, 0, None, None)
+
+
+def place_min_transfer(n_experts: int, old_placement, ep_new: int):
+    """(new placement, experts kept): balanced, every expert once, as many experts as
+    possible on a rank index that already holds them."""
+    keep: list = []
+    off = np.zeros(ep_new + 1, dtype=np.int32)
+    ids = np.zeros(n_experts, dtype=np.int32)
+    kept = _i32()
+    _check(lib().emoe_place_min_transfer(n_experts, ctypes.byref(_placement_config(old_placement, keep)),
+                                         ep_new, off.ctypes.data_as(_i32p), ids.ctypes.data_as(_i32p),
+                                         ctypes.byref(kept)))
+    return [[int(e) for e in ids[off[r]:off[r + 1]]] for r in range(ep_new)], kept.value
 
 
 def vmm_dry_run(shape, old_placement, new_placement, slab_bytes: int) -> dict:
