@@ -259,3 +259,22 @@ def test_layout_variants_one_layer(name):
             plan.set_tuning(path=2, max_ctas=9)
             for phase in (E.PHASE_EXPERTS, E.PHASE_KV):
                 check_phase_full(w, plan, phase)
+
+
+def test_scaling_sequence_with_chosen_placements():
+    """A sequence of scale steps in the paper's step pattern (+2 devices per step, then
+    back down), each new placement chosen by emoe_place_min_transfer from the previous
+    one; after every step the arenas must equal the oracle applied to the previous arenas."""
+    sh = W.Shape(2, 24, 0, 64, 96, 8, 8, 16, 4, 2)
+    empty = np.zeros((0, 0), np.int32)
+    placement = W.place_contiguous(24, 2)
+    cur = WD.alloc_filled(oracle.expert_arena_bytes(sh, placement), 123, W.KIND_EXPERTS)
+    for ep_new in (4, 6, 8, 6, 4, 2):
+        new_p, kept = E.place_min_transfer(24, placement, ep_new)
+        old = W.ParallelConfig(len(placement), 1, placement, 1, [], empty)
+        new = W.ParallelConfig(ep_new, 1, new_p, 1, [], empty)
+        wl = W.Workload("seq", sh, old, new, 123)
+        with E.Plan(sh, old, new) as plan:
+            _, nxt = check_phase_full(wl, plan, E.PHASE_EXPERTS, src=cur)
+        assert kept == min(len(placement), ep_new) * min(24 // len(placement), 24 // ep_new)
+        placement, cur = new_p, nxt
