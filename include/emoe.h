@@ -161,6 +161,10 @@ emoe_status_t emoe_plan_create(const emoe_shape_t *shape, const emoe_config_t *o
  * and no source arena may intersect a destination arena (out of place).
  * The call only enqueues work on the stream: it neither synchronises nor
  * allocates.  The pointer arrays are read before the call returns.
+ * Calls may be enqueued on any streams; at most 4 launches of the SAME phase of
+ * the SAME plan may be in flight on the GPU at once (they claim work through
+ * per-launch counters of which the plan has 4 per phase) - more must be
+ * ordered by the caller.  Calls on one stream are always fine.
  */
 emoe_status_t emoe_reshard_experts(const emoe_plan_t *plan, const void *const *src,
                                    void *const *dst, void *cuda_stream);
@@ -399,7 +403,8 @@ typedef struct {
   int32_t kv_order;        /* order in which mapped KV blocks are visited: 0 default,   */
                            /* 1 block-table order, 2 by old physical id, 3 by new id    */
   int32_t unit_order;      /* bulk work order: 0 default (run-major: one layer slab or  */
-                           /* KV pool at a time), 1 segment-major                       */
+                           /* KV pool at a time), 1 segment-major; +2: CTAs take units  */
+                           /* round-robin instead of claiming them from a counter       */
 } emoe_tuning_t;
 
 /* Replaces the plan's launch tuning.  Not thread-safe against reshard calls

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -20,6 +21,8 @@ namespace {
 constexpr uint32_t kUnitTiles = 8;
 constexpr uint32_t kDefaultBulkTile = 32768, kDefaultBulkStages = 6;
 constexpr uint32_t kDefaultHints = 0;
+constexpr int kCtrSlots = 4;        // launches of one phase of one plan that may be in flight at once
+constexpr int kStatusWords = 1 + 3 * kCtrSlots * 2;
 constexpr int kDefaultKvMode = 1;   // 1 direct, 2 staged through shared memory
 constexpr int kDefaultKvOrder = 1;  // 1 table order, 2 by old block id, 3 by new block id
 constexpr uint32_t kDefaultBulkCtas = 74;  // measured optimum on B200: half the SMs, deep rings
@@ -62,7 +65,9 @@ struct emoe_plan {
   DevPhase dev[3];
   std::vector<uint32_t> pair_old, pair_new;  // block pairs in launch order (see kv_order)
   uint32_t *d_pair_old = nullptr, *d_pair_new = nullptr;
-  int *d_status = nullptr;
+  int *d_status = nullptr;  // [0] status word; then kCtrSlots x 2 work-counter words per phase
+  mutable std::atomic<uint32_t> launch_seq[3];
+  emoe_plan() { for (auto &a : launch_seq) a.store(0); }
 };
 
 namespace {
@@ -174,7 +179,7 @@ void build_tables(emoe_plan *p, int phase) {
       else add_units(&vec, idx, s, kVecTile);
     }
   }
-  if (p->tuning.unit_order != 1)
+  if (p->tuning.unit_order % 2 == 0)
     std::stable_sort(bulk.begin(), bulk.end(),
                      [](const KeyedUnit &a, const KeyedUnit &b) { return a.run < b.run; });
   for (const KeyedUnit &k : bulk) dp.bulk_units.push_back(k.u);
@@ -286,8 +291,14 @@ emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, 
   const DevPhase &dp = p->dev[phase];
   const BulkConfig bc{bulk_tile(p), bulk_stages(p),
                       p->tuning.bulk_hints > 0 ? (uint32_t)p->tuning.bulk_hints - 1 : kDefaultHints};
+  // work counter of this launch: the phase's slots are used in turn
+  unsigned int *ctr = nullptr;
+  if (p->tuning.unit_order < 2) {
+    const uint32_t slot = p->launch_seq[phase].fetch_add(1) % kCtrSlots;
+    ctr = reinterpret_cast<unsigned int *>(p->d_status) + 1 + (phase * kCtrSlots + slot) * 2;
+  }
   cudaError_t e = launch_bulk_copy({dp.d_segs, dp.d_dsts, dp.d_bulk_units, (uint32_t)dp.bulk_units.size()},
-                                   ptrs, bc, bulk_budget(p), p->d_status, st);
+                                   ptrs, bc, bulk_budget(p), p->d_status, ctr, st);
   if (e != cudaSuccess) return cuda_status(e);
   e = launch_vec_copy({dp.d_segs, dp.d_dsts, dp.d_vec_units, (uint32_t)dp.vec_units.size()}, ptrs,
                       kVecTile, p->tuning.max_ctas > 0 ? cta_budget(p) * 8 : 0xffffffffu, st);
@@ -413,8 +424,8 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
       st = cuda_status(e2);
     }
     if (st == EMOE_OK) {
-      cudaError_t e3 = cudaMalloc((void **)&p->d_status, sizeof(int));
-      if (e3 == cudaSuccess) e3 = cudaMemset(p->d_status, 0, sizeof(int));
+      cudaError_t e3 = cudaMalloc((void **)&p->d_status, kStatusWords * sizeof(int));
+      if (e3 == cudaSuccess) e3 = cudaMemset(p->d_status, 0, kStatusWords * sizeof(int));
       st = cuda_status(e3);
     }
     if (st == EMOE_OK && (flags & EMOE_PLAN_HOST_STEP)) st = make_host_step(p, *shape, old_cfg, new_cfg,
@@ -446,8 +457,8 @@ emoe_status_t emoe::run_phase_once(const PhasePlan &pp, const RankPtrs &ptrs, cu
   rc = cuda_status(e);
   if (rc == EMOE_OK) rc = upload_phase(&tmp, 0);
   if (rc == EMOE_OK) {
-    e = cudaMalloc((void **)&tmp.d_status, sizeof(int));
-    if (e == cudaSuccess) e = cudaMemsetAsync(tmp.d_status, 0, sizeof(int), st);
+    e = cudaMalloc((void **)&tmp.d_status, kStatusWords * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemsetAsync(tmp.d_status, 0, kStatusWords * sizeof(int), st);
     rc = cuda_status(e);
   }
   if (rc == EMOE_OK) rc = run_segments(&tmp, 0, ptrs, st);
@@ -721,7 +732,7 @@ emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
   if (t->max_ctas < 0 || t->bulk_tile_bytes < 0 || t->bulk_stages < 0 || t->path < 0 ||
       t->path > 2 || t->kv_mode < 0 || t->kv_mode > 4 || t->bulk_hints < 0 ||
       t->bulk_hints > 4 || t->kv_order < 0 || t->kv_order > 3 || t->unit_order < 0 ||
-      t->unit_order > 1)
+      t->unit_order > 3)
     return EMOE_ERR_INVALID_ARG;
   if (t->bulk_tile_bytes && (t->bulk_tile_bytes % 128 || t->bulk_tile_bytes < 1024))
     return EMOE_ERR_INVALID_ARG;

@@ -139,6 +139,7 @@ struct BulkParams {
   uint32_t tile_bytes, stages;
   uint32_t hints;      // bit 0: loads evict-first in L2, bit 1: stores evict-first
   int *status;
+  unsigned int *ctr;   // {next unit to claim, CTAs finished}, both 0 between launches; null: static
   RankPtrs ptrs;
 };
 
@@ -178,16 +179,34 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
     const uint32_t G = gridDim.x, n = p.t.n_units;
     uint32_t it = 0;
     bool ok = true;
-    uint32_t u = blockIdx.x;                 // < n: the grid never exceeds the unit count
+    // Units: the first one is the CTA's own index; the following ones are claimed from a
+    // global counter (SMs do not all see the same bandwidth, and a static split ends with
+    // the slowest: +1..3 % measured), or taken round-robin when there is no counter.  A
+    // claim is made two units before its use, so its latency is hidden too.
+    const bool dyn = p.ctr != nullptr;
+    // raw claim -> unit index; n = no more units (n >= G: the grid never exceeds the unit count)
+    auto claimed = [&](unsigned int c) -> uint32_t { return c < n - G ? G + c : n; };
+    uint32_t u = blockIdx.x;
+    uint32_t u1, u2;
+    if (dyn) {
+      u1 = claimed(atomicAdd(&p.ctr[0], 1u));
+      u2 = claimed(atomicAdd(&p.ctr[0], 1u));
+    } else {
+      u1 = (uint64_t)u + G < n ? u + G : n;
+      u2 = (uint64_t)u + 2ull * G < n ? u + 2 * G : n;
+    }
     Unit un0 = p.t.units[u];
     DevSeg sg0 = p.t.segs[un0.seg];
     Unit un1 = un0;
-    if ((uint64_t)u + G < n) un1 = p.t.units[u + G];
-    for (; ok && u < n; u += G) {
+    if (u1 < n) un1 = p.t.units[u1];
+    while (ok && u < n) {
       DevSeg sg1 = sg0;
       Unit un2 = un1;
-      if ((uint64_t)u + G < n) sg1 = p.t.segs[un1.seg];
-      if ((uint64_t)u + 2ull * G < n) un2 = p.t.units[u + 2 * G];
+      if (u1 < n) sg1 = p.t.segs[un1.seg];
+      if (u2 < n) un2 = p.t.units[u2];
+      // the claim's result is first looked at when the unit indices rotate, at the loop's end
+      unsigned int raw3 = 0xffffffffu;
+      if (dyn && u2 < n) raw3 = atomicAdd(&p.ctr[0], 1u);
       const Unit &un = un0;
       const DevSeg &sg = sg0;
       const uint8_t *src_base = s_src[sg.src_rank] + sg.src_off;
@@ -247,6 +266,10 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
       un0 = un1;
       sg0 = sg1;
       un1 = un2;
+      u = u1;
+      u1 = u2;
+      if (dyn) u2 = u2 < n ? claimed(raw3) : n;
+      else u2 = (uint64_t)u2 + G < n ? u2 + G : n;
     }
     if (ok) {
       // end marker
@@ -266,6 +289,14 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
       for (uint32_t j = 1; j <= back; ++j) {
         const uint32_t i2 = it - j;
         (void)mbar_wait(smem_u32(&full[i2 % S]), (i2 / S) & 1);
+      }
+    }
+    if (dyn) {  // the last producer to finish leaves the counters at zero for the next launch
+      __threadfence();
+      if (atomicAdd(&p.ctr[1], 1u) == G - 1) {
+        p.ctr[0] = 0;
+        p.ctr[1] = 0;
+        __threadfence();
       }
     }
   } else if (tid == 32) {
@@ -829,12 +860,12 @@ cudaError_t kernels_init() {
 }
 
 cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, const BulkConfig &c,
-                             uint32_t grid, int *status, cudaStream_t stream) {
+                             uint32_t grid, int *status, unsigned int *ctr, cudaStream_t stream) {
   if (t.n_units == 0) return cudaSuccess;
   if (c.stages < 2 || c.stages > kMaxStages || c.tile_bytes % 128 != 0) return cudaErrorInvalidValue;
   const size_t smem = bulk_smem_bytes(c.tile_bytes, c.stages);
   if (bulk_smem_bytes(c.tile_bytes, c.stages) > bulk_smem_limit()) return cudaErrorInvalidValue;
-  BulkParams p{t, c.tile_bytes, c.stages, c.hints, status, ptrs};
+  BulkParams p{t, c.tile_bytes, c.stages, c.hints, status, ctr, ptrs};
   if (grid > t.n_units) grid = t.n_units;
   bulk_copy_kernel<<<grid, 64, smem, stream>>>(p);
   return cudaGetLastError();

@@ -69,8 +69,11 @@ struct BulkConfig {
 size_t bulk_smem_bytes(uint32_t tile_bytes, uint32_t stages);
 size_t bulk_smem_limit();
 // Bulk path: cp.async.bulk global -> shared -> global through an mbarrier ring.
+// ctr: two zero-initialised words in device memory through which the CTAs of ONE launch
+// claim units (they leave them at zero); launches that may run at the same time need
+// different words.  null: units are dealt round-robin.
 cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, const BulkConfig &c,
-                             uint32_t grid, int *status, cudaStream_t stream);
+                             uint32_t grid, int *status, unsigned int *ctr, cudaStream_t stream);
 // Vector path: a warp per tile, 16-byte (or narrower, per segment alignment) loads and stores.
 cudaError_t launch_vec_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
                             uint32_t grid, cudaStream_t stream);

@@ -48,7 +48,8 @@ TUNINGS = [dict(path=1), dict(path=2), dict(bulk_tile_bytes=8192, bulk_stages=3)
            dict(kv_mode=1), dict(kv_mode=2), dict(kv_mode=2, max_ctas=3), dict(kv_order=2),
            dict(kv_order=3, kv_mode=2), dict(kv_order=1, unit_order=1),
            dict(kv_order=3, bulk_tile_bytes=16384), dict(kv_mode=3), dict(kv_mode=3, max_ctas=5),
-           dict(kv_mode=3, kv_order=3), dict(kv_mode=4)]
+           dict(kv_mode=3, kv_order=3), dict(kv_mode=4), dict(unit_order=2, path=2),
+           dict(unit_order=3, path=2, max_ctas=5), dict(path=2, max_ctas=1)]
 
 
 @pytest.mark.parametrize("tuning", TUNINGS, ids=lambda t: "-".join("%s%s" % kv for kv in t.items()))
