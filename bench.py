@@ -36,8 +36,8 @@ FALLBACK_PEAK_GBS = 6650.0
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under
 # profiles/ (workload -> read + written bytes), or None while no capture covers it
 NCU_TRAFFIC = {
-    # expert launch of a 2-layer cut: 2.0766 GB read + 2.0316 GB written; x12 for 24 layers
-    "c2_mid": 12 * (2076600000 + 2031598000),
+    # expert launch of a 2-layer cut: 2.0763 GB read + 2.0264 GB written; x12 for 24 layers
+    "c2_mid": 12 * (2076335000 + 2026361000),
 }
 
 
