@@ -148,6 +148,7 @@ void build_tables(emoe_plan *p, int phase) {
                         bulk_bytes + vec_bytes < kSmallPhaseBytes);
 
   std::vector<KeyedUnit> bulk, vec;
+  bulk.reserve((size_t)(bulk_bytes / ((uint64_t)T * kUnitTiles)) + pp.segs.size() * 4);
   for (uint32_t oi : order) {
     const Segment &s0 = pp.segs[oi];
     bool is_bulk = s0.align == 16 && s0.run_bytes >= kBulkMinRun && !all_vec;
@@ -179,10 +180,20 @@ void build_tables(emoe_plan *p, int phase) {
       else add_units(&vec, idx, s, kVecTile);
     }
   }
-  if (p->tuning.unit_order % 2 == 0)
-    std::stable_sort(bulk.begin(), bulk.end(),
-                     [](const KeyedUnit &a, const KeyedUnit &b) { return a.run < b.run; });
-  for (const KeyedUnit &k : bulk) dp.bulk_units.push_back(k.u);
+  dp.bulk_units.resize(bulk.size());
+  if (p->tuning.unit_order % 2 == 0) {
+    // stable counting sort by run (hundreds of thousands of units: a comparison sort
+    // would cost more host time than the copy takes on the device)
+    uint32_t max_run = 0;
+    for (const KeyedUnit &k : bulk) max_run = std::max(max_run, k.run);
+    std::vector<uint32_t> start((size_t)max_run + 2, 0);
+    for (const KeyedUnit &k : bulk) start[k.run + 1]++;
+    for (size_t i = 1; i < start.size(); ++i) start[i] += start[i - 1];
+    for (const KeyedUnit &k : bulk) dp.bulk_units[start[k.run]++] = k.u;
+  } else {
+    for (size_t i = 0; i < bulk.size(); ++i) dp.bulk_units[i] = bulk[i].u;
+  }
+  dp.vec_units.reserve(vec.size());
   for (const KeyedUnit &k : vec) dp.vec_units.push_back(k.u);
 
   if (phase == EMOE_PHASE_KV) {  // block pairs of the head re-split, in launch order
