@@ -209,7 +209,7 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *plan, const void *const *src,
  * copied back as the staging arena held them.
  *
  * A plan created with EMOE_PLAN_HOST_STEP runs the step as a pipeline over
- * chunks of layers (layers are independent in every phase): copy-in of one
+ * up to 32 chunks of layers (layers are independent in every phase): copy-in of one
  * chunk, the kernels of the previous one and copy-out of the one before
  * overlap on the plan's own two copy streams, so both directions of the host
  * link are busy at once.  Work still starts after what cuda_stream held before

@@ -360,7 +360,9 @@ emoe_status_t make_host_step(emoe_plan *p, const emoe_shape_t &shape, const emoe
   }
   HostStep *hs = new (std::nothrow) HostStep();
   if (!hs) return EMOE_ERR_OOM;
-  hs->lc = (L + 7) / 8;  // about eight chunks: copy-in, kernels and copy-out overlap chunk by chunk
+  // up to 32 chunks (single layers for most models): the pipeline's fill and drain - the
+  // first copy-in and the last copy-out, which nothing overlaps - shrink with the chunk
+  hs->lc = (L + 31) / 32;
   const int n_full = L / hs->lc, tail = L % hs->lc;
   hs->n_chunks = n_full + (tail ? 1 : 0);
   emoe_shape_t sh = shape;

@@ -184,8 +184,8 @@ def test_step_on_host_buffers_matches_oracle(host_step):
 
 
 def test_pipelined_host_step_with_a_ragged_last_chunk():
-    """11 layers: chunks of 2 layers and a tail chunk of 1."""
-    wl = W.make_workload("c1_tiny", n_layers=11)
+    """35 layers: chunks of 2 layers and a tail chunk of 1."""
+    wl = W.make_workload("c1_tiny", n_layers=35)
     wl = R(wl, shape=R(wl.shape, d_ff=64))
     _step_on_host_buffers(wl, True)
     _step_on_host_buffers(wl.swapped(), True)
