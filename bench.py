@@ -35,10 +35,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAK_GBS = 6650.0
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under
 # profiles/ (workload -> read + written bytes), or None while no capture covers it
-NCU_TRAFFIC = {
-    # expert launch of a 2-layer cut: 2.0763 GB read + 2.0264 GB written; x12 for 24 layers
-    "c2_mid": 12 * (2076335000 + 2026361000),
-}
+NCU_TRAFFIC = {}
 
 
 def measured_peak():
@@ -116,14 +113,12 @@ def setup(name, torch, E, W, WD, n_layers=None):
 
 
 def one_step(plan, src, dst, stream):
-    plan.reshard_experts(src[0], dst[0], stream)
-    plan.reshard_attn(src[1], dst[1], stream)
-    plan.reshard_kv(src[2], dst[2], stream)
+    plan.reshard_step(src, dst, stream)
 
 
 def time_steps(torch, plan, src, dst, steps, warmup, stream, barrier=None):
-    """Returns (total ms over `steps` steps, per-phase mean ms).  Events are recorded on
-    the stream the kernels are launched on."""
+    """Total ms over `steps` whole steps (emoe_reshard_step, back to back), events recorded
+    on the stream the kernels are launched on."""
     with torch.cuda.stream(stream):
         for _ in range(warmup):
             one_step(plan, src, dst, stream)
@@ -131,6 +126,19 @@ def time_steps(torch, plan, src, dst, steps, warmup, stream, barrier=None):
         if barrier:
             barrier()
         torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            one_step(plan, src, dst, stream)
+        e1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def time_phases(torch, plan, src, dst, steps, stream):
+    """Mean ms of each phase run on its own (the per-phase entry points), for the report."""
+    with torch.cuda.stream(stream):
         ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
         for i in range(steps):
             ev[i][0].record(stream)
@@ -141,10 +149,7 @@ def time_steps(torch, plan, src, dst, steps, warmup, stream, barrier=None):
             plan.reshard_kv(src[2], dst[2], stream)
             ev[i][3].record(stream)
         stream.synchronize()
-        torch.cuda.synchronize()
-    total = ev[0][0].elapsed_time(ev[-1][3])
-    phase = [statistics.mean(e[k].elapsed_time(e[k + 1]) for e in ev) for k in range(3)]
-    return total, phase
+    return [statistics.mean(e[k].elapsed_time(e[k + 1]) for e in ev) for k in range(3)]
 
 
 def time_graph_steps(torch, plan, src, dst, steps, warmup, stream):
@@ -187,6 +192,7 @@ def config_report(E, plan, wl, total_ms, phase_ms, steps, peak, plan_ms):
                        if phase_ms[k] > 0 else None,
                        "bytes_moved": st[k]["bytes_moved"], "segments": st[k]["n_segments"],
                        "launches": plan.num_launches(k)} for k, n in enumerate(names)},
+        "launches_per_step": plan.num_launches(E.PHASE_STEP),
     }
 
 
@@ -466,26 +472,37 @@ def main():
     wl, plan, src, dst, plan_ms = setup(args.workload, torch, E, W, WD, n_layers=args.layers)
     sampler = ClockSampler(local)
     sampler.start()
-    total_ms, phase_ms = time_steps(torch, plan, src, dst, args.steps, args.warmup, stream, barrier)
+    total_ms = time_steps(torch, plan, src, dst, args.steps, args.warmup, stream, barrier)
     clocks = sampler.stop()
+    phase_ms = time_phases(torch, plan, src, dst, max(3, min(args.steps, 20)), stream)
     total_ms = replicas.job_time_ms(total_ms, dist, device="cuda")   # max over ranks
     rep = config_report(E, plan, wl, total_ms, phase_ms, args.steps, peak, plan_ms)
     if plan.device_status() != 0:
         raise SystemExit("device status word set: a bounded wait expired")
     ms = total_ms / args.steps
     value = replicas.job_throughput_gbs(rep["bytes_moved"], world, ms)
-    launches = sum(plan.num_launches(ph) for ph in range(3)) * args.steps
+    per_step = plan.num_launches(E.PHASE_STEP)
+    launches = per_step * args.steps
 
-    # roofline of the dominant kernel: the expert re-pack's bulk-copy launch
-    st0 = plan.stats(E.PHASE_EXPERTS)
-    alg_bytes = st0["bytes_moved"] + st0["bytes_read"]
-    achieved = alg_bytes / (phase_ms[0] * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "bulk_copy_kernel (expert re-pack)",
+    # roofline of the dominant kernel, the bulk-copy launch.  When the whole step is that one
+    # launch (TP kept: every segment of every phase is a long run), its duration is the step
+    # time of the timed region; otherwise the expert phase run on its own stands in.
+    st_all = [plan.stats(ph) for ph in range(3)]
+    if per_step == 1:
+        alg_bytes = sum(x["bytes_moved"] + x["bytes_read"] for x in st_all)
+        launch_ms, what = ms, "bulk_copy_kernel (whole step: experts + attention + KV in one launch)"
+    else:
+        alg_bytes = st_all[0]["bytes_moved"] + st_all[0]["bytes_read"]
+        small = alg_bytes < (512 << 20)     # small phases are routed to the vector kernel whole
+        launch_ms = phase_ms[0]
+        what = ("vec_copy_kernel" if small else "bulk_copy_kernel") + " (expert re-pack, timed as its own call)"
+    achieved = alg_bytes / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": what,
                 "achieved": round(achieved, 1), "peak": peak, "peak_kind": "of " + peak_kind,
                 "unit": UNIT, "frac": round(achieved / peak, 4),
                 "algorithmic_bytes_per_launch": alg_bytes,
-                "launch_ms": round(phase_ms[0], 4),
-                "traffic": NCU_TRAFFIC.get(wl.name)}
+                "launch_ms": round(launch_ms, 4),
+                "traffic": NCU_TRAFFIC.get(wl.name) if per_step == 1 and args.layers is None else None}
 
     line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 4),
@@ -536,7 +553,8 @@ def main():
                 continue
             wl2, plan2, src2, dst2, pms = setup(name, torch, E, W, WD)
             k = max(5, args.steps // 2) if name != "c1_tiny" else 200
-            tot, ph = time_steps(torch, plan2, src2, dst2, k, 3, stream)
+            tot = time_steps(torch, plan2, src2, dst2, k, 3, stream)
+            ph = time_phases(torch, plan2, src2, dst2, max(3, min(k, 20)), stream)
             r = config_report(E, plan2, wl2, tot, ph, k, peak, pms)
             if name == "c1_tiny":    # launch-bound: also as a CUDA-graph replay
                 g_ms = time_graph_steps(torch, plan2, src2, dst2, k, 3, stream)

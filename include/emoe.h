@@ -122,6 +122,7 @@ typedef struct {
 #define EMOE_PHASE_EXPERTS 0
 #define EMOE_PHASE_ATTN 1
 #define EMOE_PHASE_KV 2
+#define EMOE_PHASE_STEP 3 /* emoe_plan_num_launches only: one emoe_reshard_step call */
 #define EMOE_SIDE_OLD 0
 #define EMOE_SIDE_NEW 1
 
@@ -193,6 +194,21 @@ emoe_status_t emoe_reshard_attn(const emoe_plan_t *plan, const void *const *src,
  */
 emoe_status_t emoe_reshard_kv(const emoe_plan_t *plan, const void *const *src,
                               void *const *dst, void *cuda_stream);
+
+/*
+ * emoe_reshard_step - the whole scale step (Sec. 5.2: experts, attention
+ * weights and KV cache are reconfigured together): the three phases of
+ * emoe_reshard_experts / _attn / _kv with the same results, enqueued as ONE
+ * set of launches.  The phases touch disjoint arenas, so their copy segments
+ * share a launch (no ramp-up and tail per phase); only a KV head re-split keeps
+ * its own kernel.
+ *
+ * src / dst: indexed by EMOE_PHASE_EXPERTS / _ATTN / _KV, each a HOST array of
+ * DEVICE pointers as for the per-phase call.  All arguments of all phases are
+ * checked before anything is enqueued.  Otherwise as emoe_reshard_experts.
+ */
+emoe_status_t emoe_reshard_step(const emoe_plan_t *plan, const void *const *const src[3],
+                                void *const *const dst[3], void *cuda_stream);
 
 /*
  * emoe_reshard_step_host - one whole scale step on HOST buffers: copies

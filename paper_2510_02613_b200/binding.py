@@ -15,6 +15,7 @@ import numpy as np
 from . import build as _build
 
 PHASE_EXPERTS, PHASE_ATTN, PHASE_KV = 0, 1, 2
+PHASE_STEP = 3   # num_launches only: one reshard_step call
 SIDE_OLD, SIDE_NEW = 0, 1
 PLAN_HOST_ONLY = 1
 PLAN_HOST_STEP = 2
@@ -68,7 +69,7 @@ SEGMENT_DTYPE = np.dtype([("src_off", "<u8"), ("dst_off", "<u8"), ("run_bytes", 
                           ("src_rank", "<u4"), ("dst_rank", "<u4"), ("group", "<u4")])
 
 EXPORTS = ("emoe_plan_create", "emoe_reshard_experts", "emoe_reshard_attn", "emoe_reshard_kv",
-           "emoe_reshard_kv_static",
+           "emoe_reshard_kv_static", "emoe_reshard_step",
            "emoe_reshard_step_host", "emoe_plan_destroy", "emoe_plan_num_ranks",
            "emoe_plan_arena_bytes", "emoe_plan_stats", "emoe_plan_num_launches", "emoe_plan_segments",
            "emoe_plan_device_status", "emoe_plan_set_tuning", "emoe_strerror",
@@ -105,6 +106,8 @@ def lib() -> ctypes.CDLL:
         f = getattr(L, name)
         f.restype = _i32
         f.argtypes = [_vp, PP, PP, _vp]
+    L.emoe_reshard_step.restype = _i32
+    L.emoe_reshard_step.argtypes = [_vp, ctypes.POINTER(PP), ctypes.POINTER(PP), _vp]
     L.emoe_reshard_step_host.restype = _i32
     L.emoe_reshard_step_host.argtypes = [_vp, ctypes.POINTER(PP), ctypes.POINTER(PP),
                                          ctypes.POINTER(PP), ctypes.POINTER(PP), _vp]
@@ -325,6 +328,14 @@ class Plan:
         calls on the device, so calls that may overlap on the GPU must be serialised.
         Make the first call on a device outside stream capture."""
         self._run(lib().emoe_reshard_kv_static, src, dst, stream)
+
+    def reshard_step(self, src, dst, stream=None) -> None:
+        """All three phases as one set of launches.  src / dst: three lists (experts, attn,
+        kv) of per-rank device buffers."""
+        PP = ctypes.POINTER(_vp)
+        arrs = [_ptr_array(g) for g in list(src) + list(dst)]
+        pack = lambda a: (PP * 3)(*[ctypes.cast(x, PP) for x in a])
+        _check(lib().emoe_reshard_step(self._h, pack(arrs[:3]), pack(arrs[3:]), _stream_handle(stream)))
 
     def reshard_step_host(self, h_src, h_dst, d_src, d_dst, stream=None) -> None:
         """Each argument: three lists (experts, attn, kv) of per-rank buffers."""

@@ -22,7 +22,8 @@ constexpr uint32_t kUnitTiles = 8;
 constexpr uint32_t kDefaultBulkTile = 32768, kDefaultBulkStages = 6;
 constexpr uint32_t kDefaultHints = 0;
 constexpr int kCtrSlots = 4;        // launches of one phase of one plan that may be in flight at once
-constexpr int kStatusWords = 1 + 3 * kCtrSlots * 2;
+constexpr int kTableSets = 4;        // experts, attn, kv, and the three merged for one whole step
+constexpr int kStatusWords = 1 + kTableSets * kCtrSlots * 2;
 constexpr int kDefaultKvMode = 1;   // 1 direct, 2 staged through shared memory
 constexpr int kDefaultKvOrder = 1;  // 1 table order, 2 by old block id, 3 by new block id
 constexpr uint32_t kDefaultBulkCtas = 74;  // measured optimum on B200: half the SMs, deep rings
@@ -62,11 +63,13 @@ struct emoe_plan {
   emoe_tuning_t tuning{};
   int local_rank = -1;            // >= 0: only destinations of this new-rank index are written
   bool reads_src[3][EMOE_MAX_RANKS];  // old ranks the (filtered) phase reads
-  DevPhase dev[3];
+  DevPhase dev[kTableSets];       // [3]: all three phases as one launch set (see build_merged)
+  uint32_t src_base[3] = {0, 0, 0}, dst_base[3] = {0, 0, 0};  // rank offsets of a phase in the merged set
+  bool merged = false;
   std::vector<uint32_t> pair_old, pair_new;  // block pairs in launch order (see kv_order)
   uint32_t *d_pair_old = nullptr, *d_pair_new = nullptr;
   int *d_status = nullptr;  // [0] status word; then kCtrSlots x 2 work-counter words per phase
-  mutable std::atomic<uint32_t> launch_seq[3];
+  mutable std::atomic<uint32_t> launch_seq[kTableSets];
   emoe_plan() { for (auto &a : launch_seq) a.store(0); }
 };
 
@@ -214,6 +217,40 @@ void build_tables(emoe_plan *p, int phase) {
       p->pair_old[i] = kv.pair_old[idx[i]];
       p->pair_new[i] = kv.pair_new[idx[i]];
     }
+  }
+}
+
+// One launch set for the whole step: the three phases are independent of one another, so
+// their segments can share a launch.  Ranks of the phases are renumbered into one pointer
+// table (experts first, then attention, then KV); if they do not fit, the step falls back
+// to phase-by-phase launches.
+void build_merged(emoe_plan *p) {
+  DevPhase &all = p->dev[3];
+  all.segs.clear(); all.dsts.clear(); all.bulk_units.clear(); all.vec_units.clear();
+  uint32_t ns = 0, nd = 0;
+  for (int ph = 0; ph < 3; ++ph) {
+    p->src_base[ph] = ns;
+    p->dst_base[ph] = nd;
+    ns += (uint32_t)p->hp.phase[ph].arena_old.size();
+    nd += (uint32_t)p->hp.phase[ph].arena_new.size();
+  }
+  p->merged = ns <= EMOE_MAX_RANKS && nd <= EMOE_MAX_RANKS;
+  if (!p->merged) return;
+  for (int ph = 0; ph < 3; ++ph) {
+    const DevPhase &dp = p->dev[ph];
+    const uint32_t seg0 = (uint32_t)all.segs.size(), dst0 = (uint32_t)all.dsts.size();
+    for (DevSeg s : dp.segs) {
+      s.src_rank += p->src_base[ph];
+      s.dst_rank += p->dst_base[ph];
+      s.dst_first += dst0;
+      all.segs.push_back(s);
+    }
+    for (Dst d : dp.dsts) {
+      d.rank += p->dst_base[ph];
+      all.dsts.push_back(d);
+    }
+    for (Unit u : dp.bulk_units) { u.seg += seg0; all.bulk_units.push_back(u); }
+    for (Unit u : dp.vec_units) { u.seg += seg0; all.vec_units.push_back(u); }
   }
 }
 
@@ -417,6 +454,7 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
     st = build_host_plan(*shape, *old_cfg, *new_cfg, flags, &p->hp);
     if (st == EMOE_OK)
       for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
+      build_merged(p);
   } catch (const std::bad_alloc &) {
     st = EMOE_ERR_OOM;
   }
@@ -430,7 +468,7 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
       e = g_init_err;
     }
     st = cuda_status(e);
-    for (int ph = 0; st == EMOE_OK && ph < 3; ++ph) st = upload_phase(p, ph);
+    for (int ph = 0; st == EMOE_OK && ph < kTableSets; ++ph) st = upload_phase(p, ph);
     if (st == EMOE_OK && p->hp.kv.head_split_changes) {
       cudaError_t e2 = upload(p->pair_old, &p->d_pair_old);
       if (e2 == cudaSuccess) e2 = upload(p->pair_new, &p->d_pair_new);
@@ -531,6 +569,38 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *p, const void *const *src, void
                                     (cudaStream_t)stream));
 }
 
+emoe_status_t emoe_reshard_step(const emoe_plan_t *p, const void *const *const src[3],
+                                void *const *const dst[3], void *stream) {
+  if (!p || !src || !dst) return EMOE_ERR_INVALID_ARG;
+  RankPtrs ph_ptrs[3];
+  for (int ph = 0; ph < 3; ++ph) {  // every argument is checked before anything is enqueued
+    if (!src[ph] || !dst[ph]) return EMOE_ERR_INVALID_ARG;
+    const emoe_status_t st = check_arenas(p, ph, src[ph], dst[ph], &ph_ptrs[ph]);
+    if (st != EMOE_OK) return st;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  const KvPlan &kv = p->hp.kv;
+  emoe_status_t rc = EMOE_OK;
+  if (p->merged) {
+    RankPtrs all;
+    std::memset(&all, 0, sizeof(all));
+    for (int ph = 0; ph < 3; ++ph) {
+      for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_OLD); ++r) all.src[p->src_base[ph] + r] = ph_ptrs[ph].src[r];
+      for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_NEW); ++r) all.dst[p->dst_base[ph] + r] = ph_ptrs[ph].dst[r];
+    }
+    rc = run_segments(p, 3, all, st);
+  } else {
+    for (int ph = 0; rc == EMOE_OK && ph < 3; ++ph) rc = run_segments(p, ph, ph_ptrs[ph], st);
+  }
+  if (rc == EMOE_OK && kv.head_split_changes) {
+    KvTables t = kv_tables(kv, p->d_pair_old, p->d_pair_new, p->local_rank);
+    const int mode = p->tuning.kv_mode > 0 ? p->tuning.kv_mode : kDefaultKvMode;
+    rc = cuda_status(launch_kv_copy(t, ph_ptrs[2], mode, cta_budget(p), p->tuning.max_ctas <= 0,
+                                    p->d_status, st));
+  }
+  return rc;
+}
+
 emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *p, const void *const *src, void *const *dst,
                                      void *stream) {
   if (!p || !src || !dst) return EMOE_ERR_INVALID_ARG;
@@ -610,9 +680,9 @@ emoe_status_t step_host_pipelined(const emoe_plan *p, const void *const *const h
     e = cudaEventRecord(hs->ev_in[ci], hs->s_in);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(st, hs->ev_in[ci], 0);
     if (e != cudaSuccess) return cuda_status(e);
-    emoe_status_t rc = emoe_reshard_experts(sub, sp[0], dp[0], st);
-    if (rc == EMOE_OK) rc = emoe_reshard_attn(sub, sp[1], dp[1], st);
-    if (rc == EMOE_OK) rc = emoe_reshard_kv(sub, sp[2], dp[2], st);
+    const void *const *sps[3] = {sp[0], sp[1], sp[2]};
+    void *const *dps[3] = {dp[0], dp[1], dp[2]};
+    const emoe_status_t rc = emoe_reshard_step(sub, sps, dps, st);
     if (rc != EMOE_OK) return rc;
     e = cudaEventRecord(hs->ev_k[ci], st);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(hs->s_out, hs->ev_k[ci], 0);
@@ -701,7 +771,19 @@ emoe_status_t emoe_plan_stats(const emoe_plan_t *p, int phase, uint64_t *bytes_m
 }
 
 emoe_status_t emoe_plan_num_launches(const emoe_plan_t *p, int phase, int32_t *n) {
-  if (!p || !n || phase < 0 || phase > 2) return EMOE_ERR_INVALID_ARG;
+  if (!p || !n || phase < 0 || phase > EMOE_PHASE_STEP) return EMOE_ERR_INVALID_ARG;
+  if (phase == EMOE_PHASE_STEP) {  // launches of one emoe_reshard_step call
+    const int kv_pairs = p->hp.kv.head_split_changes && !p->hp.kv.pair_old.empty() ? 1 : 0;
+    int k = 0;
+    if (p->merged) {
+      k = (p->dev[3].bulk_units.empty() ? 0 : 1) + (p->dev[3].vec_units.empty() ? 0 : 1);
+    } else {
+      for (int ph = 0; ph < 3; ++ph)
+        k += (p->dev[ph].bulk_units.empty() ? 0 : 1) + (p->dev[ph].vec_units.empty() ? 0 : 1);
+    }
+    *n = k + kv_pairs;
+    return EMOE_OK;
+  }
   if (phase == EMOE_PHASE_KV && p->hp.kv.head_split_changes) {
     *n = p->hp.kv.pair_old.empty() ? 0 : 1;
     return EMOE_OK;
@@ -763,12 +845,13 @@ emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
   emoe_status_t st = EMOE_OK;
   try {
     for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
+    build_merged(p);
   } catch (const std::bad_alloc &) {
     return EMOE_ERR_OOM;
   }
   if (!p->host_only) {
     if (cudaDeviceSynchronize() != cudaSuccess) return EMOE_ERR_CUDA;
-    for (int ph = 0; st == EMOE_OK && ph < 3; ++ph) st = upload_phase(p, ph);
+    for (int ph = 0; st == EMOE_OK && ph < kTableSets; ++ph) st = upload_phase(p, ph);
     if (st == EMOE_OK && p->hp.kv.head_split_changes) {
       cudaError_t e2 = upload(p->pair_old, &p->d_pair_old);
       if (e2 == cudaSuccess) e2 = upload(p->pair_new, &p->d_pair_new);
@@ -785,12 +868,13 @@ emoe_status_t emoe_plan_set_local_rank(emoe_plan_t *p, int32_t rank) {
   emoe_status_t st = EMOE_OK;
   try {
     for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
+    build_merged(p);
   } catch (const std::bad_alloc &) {
     return EMOE_ERR_OOM;
   }
   if (!p->host_only) {
     if (cudaDeviceSynchronize() != cudaSuccess) return EMOE_ERR_CUDA;
-    for (int ph = 0; st == EMOE_OK && ph < 3; ++ph) st = upload_phase(p, ph);
+    for (int ph = 0; st == EMOE_OK && ph < kTableSets; ++ph) st = upload_phase(p, ph);
   }
   return st;
 }

@@ -77,3 +77,24 @@ def check_phase_layers(wl, plan, phase, src, dst, layers):
                 bad = np.flatnonzero(g != w)
                 raise AssertionError("%s phase %d layer %d rank %d: %d bytes differ, first at %d"
                                      % (wl.name, phase, l, r, bad.size, bad[0]))
+
+
+def check_step_full(wl, plan):
+    """emoe_reshard_step: all three phases in one call, whole arenas against the oracle."""
+    src, dst, want = [], [], []
+    for phase in range(3):
+        so, sn = plan.arena_bytes(phase, E.SIDE_OLD), plan.arena_bytes(phase, E.SIDE_NEW)
+        src.append(WD.alloc_filled(so, wl.seed, KINDS[phase]))
+        dst.append(WD.alloc_const(sn))
+    plan.reshard_step(src, dst)
+    torch.cuda.synchronize()
+    for phase in range(3):
+        w = [np.full(t.numel(), WD.FILL_BYTE, np.uint8) for t in dst[phase]]
+        oracle_phase(wl, phase, [t.cpu().numpy() for t in src[phase]], w)
+        for r, (g, x) in enumerate(zip(dst[phase], w)):
+            g = g.cpu().numpy()
+            if not np.array_equal(g, x):
+                bad = np.flatnonzero(g != x)
+                raise AssertionError("%s step, phase %d rank %d: %d bytes differ, first at %d"
+                                     % (wl.name, phase, r, bad.size, bad[0]))
+    assert plan.device_status() == 0

@@ -12,7 +12,7 @@ import oracle
 import paper_2510_02613_b200 as E
 import workloads as W
 from workloads import device as WD
-from gpu_util import KINDS, check_phase_full, check_phase_layers, run_phase
+from gpu_util import KINDS, check_phase_full, check_phase_layers, check_step_full, run_phase
 
 pytestmark = pytest.mark.gpu
 R = dataclasses.replace
@@ -31,6 +31,8 @@ def test_c1_tiny_all_phases(inverse):
     with E.Plan(wl.shape, wl.old, wl.new) as plan:
         for phase in range(3):
             check_phase_full(wl, plan, phase)
+        check_step_full(wl, plan)
+        assert plan.num_launches(E.PHASE_STEP) == 2     # one vector launch + the KV re-split
 
 
 @pytest.mark.parametrize("name", ["c2_mid", "c3_fine", "c4_large"])
@@ -40,6 +42,9 @@ def test_one_layer_cut_all_phases(name):
     with E.Plan(wl.shape, wl.old, wl.new) as plan:
         for phase in range(3):
             check_phase_full(wl, plan, phase)
+        check_step_full(wl, plan)
+        plan.set_tuning(path=2, max_ctas=20)
+        check_step_full(wl, plan)
 
 
 TUNINGS = [dict(path=1), dict(path=2), dict(bulk_tile_bytes=8192, bulk_stages=3),
@@ -92,6 +97,7 @@ def test_odd_shapes_and_alignments(dims):
             for kv_mode in (1, 2, 3, 4):   # every KV kernel (each falls back where it cannot run)
                 plan.set_tuning(kv_mode=kv_mode, kv_order=3)
                 check_phase_full(w, plan, E.PHASE_KV)
+            check_step_full(w, plan)
 
 
 def test_replicas_with_different_contents_pick_the_documented_source():
@@ -228,6 +234,7 @@ def test_maximum_rank_counts():
                 plan.set_tuning(kv_mode=kv_mode)
                 for phase in range(3):
                     check_phase_full(w, plan, phase)
+            check_step_full(w, plan)   # 64 + 63 + .. ranks do not fit one launch set: falls back
 
 
 @pytest.mark.parametrize("c,d", [(2, 8), (8, 4), (4, 16), (16, 8), (8, 8)])

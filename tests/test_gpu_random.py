@@ -7,7 +7,7 @@ import pytest
 from hypothesis import HealthCheck, given, settings
 
 import paper_2510_02613_b200 as E
-from gpu_util import check_phase_full, make_plan
+from gpu_util import check_phase_full, check_step_full, make_plan
 from test_planner_random import cases
 
 pytestmark = pytest.mark.gpu
@@ -26,3 +26,6 @@ def test_drawn_cases_match_the_oracle(wl):
         plan.set_tuning(path=2, max_ctas=2)
         for phase in range(3):
             check_phase_full(wl, plan, phase)
+        check_step_full(wl, plan)
+        plan.set_tuning()
+        check_step_full(wl, plan)
