@@ -35,7 +35,11 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAK_GBS = 6650.0
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under
 # profiles/ (workload -> read + written bytes), or None while no capture covers it
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # whole step of a 2-layer cut (bulk launch 2.6139 + 2.5671 GB, the attention shard's vector
+    # launch 0.0677 + 0.0236 GB; at full size both are one bulk launch): x12 for 24 layers
+    "c2_mid": 12 * (2613877000 + 2567138000 + 67747000 + 23625000),
+}
 
 
 def measured_peak():
@@ -469,6 +473,8 @@ def main():
     peak, peak_kind = measured_peak()
     stream = torch.cuda.Stream()
 
+    tiny = W.make_workload("c1_tiny")        # loads the CUDA module, so that plan times below are the planner's
+    E.Plan(tiny.shape, tiny.old, tiny.new).close()
     wl, plan, src, dst, plan_ms = setup(args.workload, torch, E, W, WD, n_layers=args.layers)
     sampler = ClockSampler(local)
     sampler.start()
