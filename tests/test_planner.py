@@ -232,3 +232,21 @@ def test_layout_variants_change_segments_not_sizes():
         with pytest.raises(E.EmoeError) as ei:
             var.reshard_kv_static([16] * 2, [16] * 4)
         assert ei.value.code == 9
+
+
+def test_header_is_plain_c_and_usable_from_a_c_program(tmp_path):
+    """Compiles tests/c_abi_smoke.c as C99 against include/emoe.h, links it with libemoe.so
+    and runs it (host-only plan: no GPU needed)."""
+    import shutil
+    import subprocess
+    if not shutil.which("gcc"):
+        pytest.skip("no gcc")
+    lib = E.library_path()
+    E.lib()
+    exe = str(tmp_path / "c_abi_smoke")
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"),
+                           os.path.join(ROOT, "tests", "c_abi_smoke.c"), "-o", exe, lib,
+                           "-Wl,-rpath," + os.path.dirname(lib)])
+    out = subprocess.run([exe], capture_output=True, text=True)
+    assert out.returncode == 0, (out.returncode, out.stdout, out.stderr)
+    assert "c abi ok" in out.stdout
