@@ -199,20 +199,29 @@ def test_pipelined_host_step_with_a_ragged_last_chunk():
 
 @pytest.mark.parametrize("name", ["c2_mid", "c3_fine", "c4_large"])
 def test_full_size_configs_sampled_layers(name):
-    """The benchmark's launch configuration at full size; first, middle and last layer
-    compared in full with the oracle (layers are independent in every phase)."""
+    """The benchmark's launch configuration at full size - the whole step through
+    emoe_reshard_step with all arenas resident; first, middle and last layer compared in
+    full with the oracle (layers are independent in every phase)."""
     wl = W.make_workload(name)
     L = wl.shape.n_layers
+    torch.cuda.empty_cache()
     with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        src = [WD.alloc_filled(plan.arena_bytes(ph, E.SIDE_OLD), wl.seed, KINDS[ph]) for ph in range(3)]
+        dst = [WD.alloc_const(plan.arena_bytes(ph, E.SIDE_NEW)) for ph in range(3)]
+        plan.reshard_step(src, dst)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
         for phase in range(3):
-            src = WD.alloc_filled(plan.arena_bytes(phase, E.SIDE_OLD), wl.seed, KINDS[phase])
-            dst = WD.alloc_const(plan.arena_bytes(phase, E.SIDE_NEW))
-            run_phase(plan, phase, src, dst)
+            check_phase_layers(wl, plan, phase, src[phase], dst[phase], [0, L // 2, L - 1])
+        # and the per-phase entry points write the same bytes
+        for phase in (E.PHASE_ATTN, E.PHASE_KV):
+            again = WD.alloc_const(plan.arena_bytes(phase, E.SIDE_NEW))
+            run_phase(plan, phase, src[phase], again)
             torch.cuda.synchronize()
-            assert plan.device_status() == 0
-            check_phase_layers(wl, plan, phase, src, dst, [0, L // 2, L - 1])
-            del src, dst
-            torch.cuda.empty_cache()
+            assert all(torch.equal(a, b) for a, b in zip(again, dst[phase]))
+            del again
+        del src, dst
+    torch.cuda.empty_cache()
 
 
 def test_maximum_rank_counts():
