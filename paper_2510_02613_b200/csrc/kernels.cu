@@ -562,14 +562,17 @@ __global__ void __launch_bounds__(256) kv_rows_kernel(const __grid_constant__ Kv
   }
 }
 
-// Staged variant: the fused gather-transpose through shared memory.  One producer
-// thread brings the c contiguous pieces of a logical block (one per old rank, each
-// [token][local head][head_dim]) into a stage of a shared-memory ring with
-// cp.async.bulk; 256 consumer threads then read the stage in NEW-layout order and
-// write each new rank's block with coalesced 16-byte stores.  The stage -> destination
-// mapping is the same for every tile, so it is tabulated once per CTA (no division in
-// the steady state); per tile only the two block base offsets change.
+// Staged variant: the fused gather-transpose through shared memory, with the copy engine on
+// both sides.  One producer thread brings the c contiguous pieces of a logical block (one
+// per old rank, each [token][local head][head_dim]) into a stage of an input ring with
+// cp.async.bulk; 256 consumer threads transpose the stage inside shared memory into an
+// output stage laid out as the d new blocks ([token][new local head][head_dim] each); one
+// of them then issues one cp.async.bulk store per new rank.  No global load or store goes
+// through the load/store units.  The input -> output piece mapping is the same for every
+// tile, so it is tabulated once per CTA (no division in the steady state).
 constexpr uint32_t kKvConsumers = 256;
+constexpr uint32_t kKvOutStages = 2;
+constexpr uint32_t kKvStagedCtasPerSm = 2;  // the per-tile chain of waits and barriers is long: overlap two CTAs
 
 struct KvStagedParams {
   KvTables t;
@@ -578,19 +581,25 @@ struct KvStagedParams {
   RankPtrs ptrs;
 };
 
-__global__ void __launch_bounds__(kKvConsumers + 32, 1)
+__device__ __forceinline__ void consumers_sync() {
+  asm volatile("bar.sync 1, %0;" ::"n"(kKvConsumers) : "memory");
+}
+
+__global__ void __launch_bounds__(kKvConsumers + 32, kKvStagedCtasPerSm)
 kv_staged_kernel(const __grid_constant__ KvStagedParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const KvTables &t = p.t;
   const uint32_t S = p.stages, T = p.tile_bytes;
-  uint8_t *data = smem;
-  uint2 *table = reinterpret_cast<uint2 *>(smem + (size_t)S * T);
-  uint64_t *base_new_of = reinterpret_cast<uint64_t *>(table + p.n_pieces);  // per stage
+  uint8_t *data = smem;                                   // input ring: S stages, old layout
+  uint8_t *out = smem + (size_t)S * T;                    // output ring: kKvOutStages, new layout
+  uint32_t *table = reinterpret_cast<uint32_t *>(out + (size_t)kKvOutStages * T);
+  uint64_t *base_new_of = reinterpret_cast<uint64_t *>(table + 2 * ((p.n_pieces + 1) / 2));  // per stage
   uint64_t *full = base_new_of + S;
   uint64_t *empty = full + S;
   __shared__ const uint8_t *s_src[EMOE_MAX_RANKS];
   __shared__ uint8_t *s_dst[EMOE_MAX_RANKS];
   __shared__ volatile int s_abort;
+  __shared__ volatile int s_go;  // consumer 0 -> all consumers: 1 tile ready, 0 leave
   constexpr uint64_t kEnd = ~0ull;
 
   const uint32_t tid = threadIdx.x;
@@ -598,7 +607,7 @@ kv_staged_kernel(const __grid_constant__ KvStagedParams p) {
     s_src[tid] = p.ptrs.src[tid];
     s_dst[tid] = p.ptrs.dst[tid];
   }
-  // stage offset and destination (rank, offset in block) of every 16-byte piece, new-layout order
+  // input-stage offset of every 16-byte piece of the output stage (new-layout order)
   {
     const uint32_t cpv = t.head_bytes / 16, row_new = t.hn * cpv, ppr = t.block_tokens * row_new;
     for (uint32_t q = tid; q < p.n_pieces; q += blockDim.x) {
@@ -606,14 +615,14 @@ kv_staged_kernel(const __grid_constant__ KvStagedParams p) {
       const uint32_t tok = r / row_new, rem = r - tok * row_new;
       const uint32_t hl = rem / cpv, j = rem - hl * cpv;
       const uint32_t g = rn * t.hn + hl, ro = g / t.hc, ho = g - ro * t.hc;
-      table[q] = make_uint2(ro * p.chunk_bytes + ((tok * t.hc + ho) * cpv + j) * 16, (rn << 24) | (r * 16));
+      table[q] = ro * p.chunk_bytes + ((tok * t.hc + ho) * cpv + j) * 16;
     }
   }
   if (tid == 0) {
     s_abort = 0;
     for (uint32_t s = 0; s < S; ++s) {
       mbar_init(smem_u32(&full[s]), 1);
-      mbar_init(smem_u32(&empty[s]), kKvConsumers / 32);
+      mbar_init(smem_u32(&empty[s]), 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async_smem();
@@ -621,9 +630,9 @@ kv_staged_kernel(const __grid_constant__ KvStagedParams p) {
   __syncthreads();
 
   const uint64_t blk_old = (uint64_t)p.chunk_bytes;
-  const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
+  const uint32_t blk_new = t.block_tokens * t.hn * t.head_bytes;
   const uint64_t n_tiles = (uint64_t)t.n_pairs * t.n_lk;
-  const uint32_t c = t.hkv / t.hc;
+  const uint32_t c = t.hkv / t.hc, d = t.hkv / t.hn;
 
   if (tid == kKvConsumers) {
     // ---------------- producer ----------------
@@ -675,42 +684,55 @@ kv_staged_kernel(const __grid_constant__ KvStagedParams p) {
     }
   } else if (tid < kKvConsumers) {
     // ---------------- consumers ----------------
+    // Consumer 0 does every wait (bounded) and tells the others through s_go, so that all
+    // 256 leave the loop in the same iteration and no named barrier is left short.
     const uint32_t n = p.n_pieces;
     for (uint32_t it = 0;; ++it) {
-      const uint32_t st = it % S, round = it / S;
-      if (!mbar_wait(smem_u32(&full[st]), round & 1)) {
-        s_abort = 1;
-        atomicExch(p.status, (int)EMOE_ERR_DEVICE_TIMEOUT);
-        break;
+      const uint32_t st = it % S, round = it / S, os = it % kKvOutStages;
+      if (tid == 0) {
+        int go = 1;
+        if (!mbar_wait(smem_u32(&full[st]), round & 1)) {
+          s_abort = 1;
+          atomicExch(p.status, (int)EMOE_ERR_DEVICE_TIMEOUT);
+          go = 0;
+        } else if (base_new_of[st] == kEnd) {
+          go = 0;
+        }
+        // the stores issued kKvOutStages tiles ago have finished reading this output stage
+        bulk_wait_read<kKvOutStages - 1>();
+        s_go = go;
       }
-      const uint64_t base_new = base_new_of[st];
-      if (base_new == kEnd) break;
+      consumers_sync();
+      if (!s_go) break;
       const uint8_t *stage = data + (size_t)st * T;
+      uint8_t *ostage = out + (size_t)os * T;
       for (uint32_t q0 = tid; q0 < n; q0 += kKvConsumers * 4) {
         uint4 v[4];
-        uint32_t where[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const uint32_t q = q0 + u * kKvConsumers;
-          if (q < n) {
-            const uint2 e = table[q];
-            v[u] = *reinterpret_cast<const uint4 *>(stage + e.x);
-            where[u] = e.y;
-          }
+          if (q < n) v[u] = *reinterpret_cast<const uint4 *>(stage + table[q]);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const uint32_t q = q0 + u * kKvConsumers;
-          if (q < n)
-            *reinterpret_cast<uint4 *>(s_dst[where[u] >> 24] + base_new + (where[u] & 0xFFFFFFu)) = v[u];
+          if (q < n) *reinterpret_cast<uint4 *>(ostage + (size_t)q * 16) = v[u];
         }
       }
-      __syncwarp();
-      if ((tid & 31) == 0) mbar_arrive(smem_u32(&empty[st]));
+      fence_proxy_async_smem();   // the transposed stage becomes visible to the copy engine
+      consumers_sync();           // ... and everyone is done with the input stage
+      if (tid == 0) {
+        const uint64_t base_new = base_new_of[st];
+        const uint32_t sp = smem_u32(ostage);
+        for (uint32_t rn = 0; rn < d; ++rn)
+          bulk_store(s_dst[rn] + base_new, sp + rn * blk_new, blk_new);
+        bulk_commit();
+        mbar_arrive(smem_u32(&empty[st]));
+      }
     }
+    if (tid == 0) bulk_wait_read<0>();
   }
 }
-
 
 // Tensor-map variant: the copy engine does the gather-transpose.  Every arena is
 // described to TMA as a 3-D tensor [token rows][local heads][head bytes]; a box of
@@ -882,7 +904,8 @@ cudaError_t launch_vec_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t t
 
 namespace {
 size_t kv_staged_smem(uint32_t tile_bytes, uint32_t stages) {
-  return (size_t)stages * tile_bytes + (size_t)(tile_bytes / 16) * sizeof(uint2) +
+  const size_t pieces = tile_bytes / 16;
+  return (size_t)(stages + kKvOutStages) * tile_bytes + 2 * ((pieces + 1) / 2) * sizeof(uint32_t) +
          (size_t)stages * 3 * sizeof(uint64_t);
 }
 }  // namespace
@@ -960,8 +983,9 @@ bool kv_staged_supported(const KvTables &t, uint32_t *stages_out) {
   const uint64_t tile = (uint64_t)t.block_tokens * t.hkv * t.head_bytes;
   const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
   if (t.use_map || t.dst_only != 0xffffffffu) return false;  // only the default kernels do these
-  if (t.head_bytes % 16 || tile > 64 * 1024 || blk_new >= (1u << 24) || t.hkv / t.hn > 255) return false;
-  uint32_t stages = (uint32_t)((160 * 1024) / tile);
+  if (t.head_bytes % 16 || tile > 24 * 1024 || blk_new >= (1u << 24) || t.hkv / t.hn > 255) return false;
+  uint32_t stages = (uint32_t)((100 * 1024) / tile);            // two CTAs per SM
+  stages = stages > kKvOutStages ? stages - kKvOutStages : 0;   // the output ring takes two
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) return false;
   if (stages_out) *stages_out = stages;
@@ -1002,6 +1026,9 @@ cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, ui
   if (mode == 2 && status && kv_staged_supported(t, &stages)) {
     const uint32_t tile = t.block_tokens * t.hkv * hb;
     KvStagedParams sp{t, stages, tile, tile / 16, t.block_tokens * t.hc * hb, status, ptrs};
+    // two CTAs per budgeted SM; with no budget, 1.5 per SM measured best (6.6 TB/s on the
+    // large-expert-count shape against 6.0 with 2 and 5.6 with 1)
+    grid = unbounded ? grid * 3 / 2 : grid * kKvStagedCtasPerSm;
     if (grid > n_tiles) grid = (uint32_t)n_tiles;
     kv_staged_kernel<<<grid, kKvConsumers + 32, kv_staged_smem(tile, stages), stream>>>(sp);
     return cudaGetLastError();
