@@ -238,6 +238,48 @@ def cpu_baseline_sample(wl, src_layer_getter, budget_s=12.0, max_layers=64):
             "projected_step_ms": round(spent / layers * 1e3 * wl.shape.n_layers, 1)}
 
 
+def cpu_baseline_all_cores(wl, src_layer_getter, max_threads=16):
+    """The same oracle, still one thread per call, run on different layers at once (layers
+    are independent): what the host manages with all its cores, so that the single-thread
+    figure is not the only yardstick.  One pass: one layer per thread."""
+    import concurrent.futures as cf
+    import oracle
+    wl1 = wl.with_layers(1)
+    sh = wl1.shape
+    n = max(1, min(max_threads, os.cpu_count() or 1, wl.shape.n_layers))
+    try:
+        import psutil
+        per_layer = sum(oracle.expert_arena_bytes(sh, wl.new.placement)) * 2.6
+        n = max(1, min(n, int(psutil.virtual_memory().available * 0.5 // max(per_layer, 1))))
+    except Exception:
+        pass
+    sizes_new = [oracle.expert_arena_bytes(sh, wl.new.placement),
+                 oracle.attn_arena_bytes(sh, wl.new.tp),
+                 oracle.kv_arena_bytes(sh, wl.new.tp, wl.new.kv_num_blocks)]
+    used = sum(-(-x // sh.kv_block_tokens) for x in wl.old.seq_lens)
+    kv_moved = 2 * used * sh.kv_block_tokens * max(sh.n_kv_heads, wl.new.tp) * sh.head_dim * sh.elem_bytes
+    moved_per_layer = sum(sizes_new[0]) + sum(sizes_new[1]) + kv_moved
+    work = []
+    for i in range(n):
+        src = src_layer_getter(i)
+        dst = [[np.full(k, 0xCD, np.uint8) for k in s] for s in sizes_new]
+        work.append((src, dst))
+
+    def run(item):
+        src, dst = item
+        oracle.reshard_experts(sh, wl.old.placement, wl.new.placement, src[0], dst[0])
+        oracle.reshard_attn(sh, wl.old.tp, wl.new.tp, src[1], dst[1])
+        oracle.reshard_kv(sh, wl.old, wl.new, src[2], dst[2])
+
+    with cf.ThreadPoolExecutor(n) as ex:
+        t0 = time.perf_counter()
+        list(ex.map(run, work))
+        spent = time.perf_counter() - t0
+    return {"value": round(2 * moved_per_layer * n / spent / 1e9, 3), "unit": UNIT, "cores": n,
+            "kind": "oracle", "sample": "%d layers of %s at once, one oracle thread each; %.2f s"
+                                        % (n, wl.name, spent)}
+
+
 def device_layer_getter(torch, src, n_layers):
     def get(l):
         out = []
@@ -540,8 +582,12 @@ def main():
         except Exception as e:  # report, never hide
             line["e2e"] = {"value": None, "unit": UNIT, "error": repr(e)[:200]}
         # CPU baseline: the oracle on sampled layers of the same arenas
-        line["cpu_baseline"] = cpu_baseline_sample(
-            wl, device_layer_getter(torch, src, wl.shape.n_layers))
+        getter = device_layer_getter(torch, src, wl.shape.n_layers)
+        line["cpu_baseline"] = cpu_baseline_sample(wl, getter)
+        try:
+            line["cpu_baseline_all_cores"] = cpu_baseline_all_cores(wl, getter)
+        except Exception as e:  # report, never hide
+            line["cpu_baseline_all_cores"] = {"value": None, "error": repr(e)[:200]}
     elif world > 1:
         line["e2e"] = {"value": None, "unit": UNIT, "note": "measured at --gpus 1 only"}
 
