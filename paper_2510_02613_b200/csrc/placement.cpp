@@ -1,8 +1,8 @@
 // placement.cpp - a new expert placement that keeps as many experts where they are as a
 // balanced placement allows.
 //
-// The paper's plan "balances expert load while minimizing data transfer" (Sec. 5.2
-// "Expert Weights") but gives no algorithm.  Here: every expert is placed exactly once,
+// The paper wants the new placement balanced and cheap to reach (Sec. 5.2 "Expert
+// Weights") but gives no algorithm.  Here: every expert is placed exactly once,
 // rank sizes differ by at most one, and the number of experts that stay on a rank index
 // that already holds a copy is maximal.  That is a bipartite b-matching (rank capacities,
 // one unit per expert, plus a shared pool for the E mod EP ranks that take one expert
