@@ -123,6 +123,7 @@ def one_step(plan, src, dst, stream):
 def time_steps(torch, plan, src, dst, steps, warmup, stream, barrier=None):
     """Total ms over `steps` whole steps (emoe_reshard_step, back to back), events recorded
     on the stream the kernels are launched on."""
+    torch.cuda.synchronize()   # the arenas were filled on the default stream
     with torch.cuda.stream(stream):
         for _ in range(warmup):
             one_step(plan, src, dst, stream)
@@ -305,6 +306,7 @@ def host_layer_getter(wl, W, WD, sizes_old_per_layer):
 
 def run_e2e(torch, plan, src, dst, steps, stream):
     """src/dst: device arenas (reused as staging).  Host buffers are pinned copies."""
+    torch.cuda.synchronize()
     h_src = [[t.cpu().pin_memory() for t in g] for g in src]
     h_dst = [[torch.empty(t.numel(), dtype=torch.uint8).pin_memory() for t in g] for g in dst]
     h2d = sum(t.numel() for g in h_src for t in g)

@@ -171,6 +171,7 @@ def _step_on_host_buffers(wl, host_step):
             w = [np.full(n, WD.FILL_BYTE, np.uint8) for n in sn]
             oracle_phase(wl, phase, [t.numpy() for t in hs], w)
             want.append(w)
+        torch.cuda.synchronize()      # staging arenas were filled on the default stream
         s = torch.cuda.Stream()
         for _ in range(2):      # twice: the pipelined form reuses the plan's events
             for g in h_dst:
@@ -295,3 +296,61 @@ def test_scaling_sequence_with_chosen_placements():
             _, nxt = check_phase_full(wl, plan, E.PHASE_EXPERTS, src=cur)
         assert kept == min(len(placement), ep_new) * min(24 // len(placement), 24 // ep_new)
         placement, cur = new_p, nxt
+
+
+def test_step_captured_in_a_cuda_graph_replays_correctly():
+    """The reshard calls only enqueue kernels, so a step can be captured once and replayed;
+    every replay must write the oracle's bytes (the destination is re-filled in between)."""
+    from gpu_util import oracle_phase
+    wl = W.make_workload("c1_tiny")
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        src = [WD.alloc_filled(plan.arena_bytes(ph, E.SIDE_OLD), wl.seed, KINDS[ph]) for ph in range(3)]
+        dst = [WD.alloc_const(plan.arena_bytes(ph, E.SIDE_NEW)) for ph in range(3)]
+        want = []
+        for ph in range(3):
+            w = [np.full(t.numel(), WD.FILL_BYTE, np.uint8) for t in dst[ph]]
+            oracle_phase(wl, ph, [t.cpu().numpy() for t in src[ph]], w)
+            want.append(w)
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            plan.reshard_step(src, dst, stream)           # warm-up outside the capture
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                plan.reshard_step(src, dst, stream)
+            for _ in range(3):
+                for g in dst:
+                    for t in g:
+                        t.fill_(WD.FILL_BYTE)
+                graph.replay()
+                graph.replay()                            # back to back: same work counters
+                stream.synchronize()
+                for ph in range(3):
+                    for t, w in zip(dst[ph], want[ph]):
+                        assert np.array_equal(t.cpu().numpy(), w)
+        assert plan.device_status() == 0
+    # and a bulk-kernel step (forced), whose launches claim work through the plan's counters
+    wl = W.make_workload("c2_mid", n_layers=1)
+    wl = R(wl, shape=R(wl.shape, d_ff=128))
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        plan.set_tuning(path=2)
+        src = [WD.alloc_filled(plan.arena_bytes(ph, E.SIDE_OLD), wl.seed, KINDS[ph]) for ph in range(3)]
+        dst = [WD.alloc_const(plan.arena_bytes(ph, E.SIDE_NEW)) for ph in range(3)]
+        torch.cuda.synchronize()      # the arenas were filled on the default stream
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            plan.reshard_step(src, dst, stream)
+            stream.synchronize()
+            ref = [[t.clone() for t in g] for g in dst]
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                plan.reshard_step(src, dst, stream)
+            for g in dst:
+                for t in g:
+                    t.fill_(WD.FILL_BYTE)
+            for _ in range(6):                            # more replays than counter slots
+                graph.replay()
+            stream.synchronize()
+            for ph in range(3):
+                assert all(torch.equal(a, b) for a, b in zip(dst[ph], ref[ph]))
+        check_step_full(wl, plan)
