@@ -85,27 +85,24 @@ int kv_order(const emoe_plan *p) {
   return p->tuning.kv_order > 0 ? p->tuning.kv_order : kDefaultKvOrder;
 }
 
-struct KeyedUnit {
-  uint32_t run;  // first run the unit touches
-  Unit u;
-};
-
-// Cuts one segment into units of at most kUnitTiles tiles.  A unit of a long-run
-// segment (run >= tile) stays inside one run, so that units can be ordered by run.
-void add_units(std::vector<KeyedUnit> *units, uint32_t seg, const DevSeg &s, uint32_t T) {
+// Cuts one segment into units of at most kUnitTiles tiles and hands each to f(first run
+// the unit touches, unit).  A unit of a long-run segment (run >= tile) stays inside one run,
+// so that units can be ordered by run.
+template <typename F>
+void for_each_unit(uint32_t seg, const DevSeg &s, uint32_t T, F &&f) {
   if (s.run_bytes >= T) {
     const uint32_t tpr = (uint32_t)((s.run_bytes + T - 1) / T);
     for (uint32_t run = 0; run < s.n_runs; ++run)
       for (uint32_t t = 0; t < tpr; t += kUnitTiles) {
         const uint32_t n = tpr - t < kUnitTiles ? tpr - t : kUnitTiles;
-        units->push_back({run, {seg, run * tpr + t, n, 0}});
+        f(run, Unit{seg, run * tpr + t, n, 0});
       }
   } else {
     const uint32_t rpt = (uint32_t)(T / s.run_bytes);
     const uint32_t n_tiles = (s.n_runs + rpt - 1) / rpt;
     for (uint32_t t = 0; t < n_tiles; t += kUnitTiles) {
       const uint32_t n = n_tiles - t < kUnitTiles ? n_tiles - t : kUnitTiles;
-      units->push_back({t * rpt, {seg, t, n, 0}});
+      f(t * rpt, Unit{seg, t, n, 0});
     }
   }
 }
@@ -150,22 +147,22 @@ void build_tables(emoe_plan *p, int phase) {
                        ((vec_bytes > 0 && bulk_bytes < kMergeBulkBelow) ||
                         bulk_bytes + vec_bytes < kSmallPhaseBytes);
 
-  std::vector<KeyedUnit> bulk, vec;
-  bulk.reserve((size_t)(bulk_bytes / ((uint64_t)T * kUnitTiles)) + pp.segs.size() * 4);
+  std::vector<uint32_t> bulk_segs;  // indices into dp.segs of the segments the bulk kernel takes
+  Dst mine[EMOE_MAX_RANKS];
   for (uint32_t oi : order) {
     const Segment &s0 = pp.segs[oi];
     bool is_bulk = s0.align == 16 && s0.run_bytes >= kBulkMinRun && !all_vec;
     if (p->tuning.path == 1) is_bulk = false;
     if (p->tuning.path == 2) is_bulk = (s0.align == 16);
-    // destinations this plan writes: all, or those of the local rank only
-    std::vector<Dst> mine;
+    // destinations this plan writes: all, or those of the local rank only (a source has at
+    // most one destination per rank, so EMOE_MAX_RANKS entries suffice)
+    uint32_t n_mine = 0;
     for (uint32_t j = 0; j < s0.n_dst; ++j) {
       const Dst &d = pp.dsts[s0.dst_first + j];
-      if (p->local_rank < 0 || (int)d.rank == p->local_rank) mine.push_back(d);
+      if ((p->local_rank < 0 || (int)d.rank == p->local_rank) && n_mine < EMOE_MAX_RANKS) mine[n_mine++] = d;
     }
-    if (mine.empty()) continue;
+    if (n_mine == 0) continue;
     p->reads_src[phase][s0.src_rank] = true;
-    const uint32_t n_mine = (uint32_t)mine.size();
     const uint32_t max_fan = is_bulk ? (uint32_t)kMaxFanout : n_mine;
     for (uint32_t k = 0; k < n_mine; k += max_fan) {
       DevSeg s{};
@@ -179,26 +176,27 @@ void build_tables(emoe_plan *p, int phase) {
         for (uint32_t j = 0; j < s.n_dst; ++j) dp.dsts.push_back(mine[k + j]);
       const uint32_t idx = (uint32_t)dp.segs.size();
       dp.segs.push_back(s);
-      if (is_bulk) add_units(&bulk, idx, s, T);
-      else add_units(&vec, idx, s, kVecTile);
+      if (is_bulk) bulk_segs.push_back(idx);
+      else for_each_unit(idx, s, kVecTile, [&](uint32_t, const Unit &u) { dp.vec_units.push_back(u); });
     }
   }
-  dp.bulk_units.resize(bulk.size());
+  // Bulk units in run-major order without a sort: count the units of every run, turn the
+  // counts into start positions, then place (hundreds of thousands of units: anything
+  // slower costs more host time than the copy takes on the device).
   if (p->tuning.unit_order % 2 == 0) {
-    // stable counting sort by run (hundreds of thousands of units: a comparison sort
-    // would cost more host time than the copy takes on the device)
     uint32_t max_run = 0;
-    for (const KeyedUnit &k : bulk) max_run = std::max(max_run, k.run);
+    for (uint32_t idx : bulk_segs) max_run = std::max(max_run, dp.segs[idx].n_runs);
     std::vector<uint32_t> start((size_t)max_run + 2, 0);
-    for (const KeyedUnit &k : bulk) start[k.run + 1]++;
+    for (uint32_t idx : bulk_segs)
+      for_each_unit(idx, dp.segs[idx], T, [&](uint32_t run, const Unit &) { start[run + 1]++; });
     for (size_t i = 1; i < start.size(); ++i) start[i] += start[i - 1];
-    for (const KeyedUnit &k : bulk) dp.bulk_units[start[k.run]++] = k.u;
+    dp.bulk_units.resize(start.back());
+    for (uint32_t idx : bulk_segs)
+      for_each_unit(idx, dp.segs[idx], T, [&](uint32_t run, const Unit &u) { dp.bulk_units[start[run]++] = u; });
   } else {
-    for (size_t i = 0; i < bulk.size(); ++i) dp.bulk_units[i] = bulk[i].u;
+    for (uint32_t idx : bulk_segs)
+      for_each_unit(idx, dp.segs[idx], T, [&](uint32_t, const Unit &u) { dp.bulk_units.push_back(u); });
   }
-  dp.vec_units.reserve(vec.size());
-  for (const KeyedUnit &k : vec) dp.vec_units.push_back(k.u);
-
   if (phase == EMOE_PHASE_KV) {  // block pairs of the head re-split, in launch order
     const KvPlan &kv = p->hp.kv;
     if (kv.head_split_changes && !kv.pair_old.empty())
@@ -236,21 +234,30 @@ void build_merged(emoe_plan *p) {
   }
   p->merged = ns <= EMOE_MAX_RANKS && nd <= EMOE_MAX_RANKS;
   if (!p->merged) return;
+  size_t n_seg = 0, n_dst = 0, n_bulk = 0, n_vec = 0;
+  for (int ph = 0; ph < 3; ++ph) {
+    n_seg += p->dev[ph].segs.size(); n_dst += p->dev[ph].dsts.size();
+    n_bulk += p->dev[ph].bulk_units.size(); n_vec += p->dev[ph].vec_units.size();
+  }
+  all.segs.resize(n_seg); all.dsts.resize(n_dst); all.bulk_units.resize(n_bulk); all.vec_units.resize(n_vec);
+  size_t i_seg = 0, i_dst = 0, i_bulk = 0, i_vec = 0;
   for (int ph = 0; ph < 3; ++ph) {
     const DevPhase &dp = p->dev[ph];
-    const uint32_t seg0 = (uint32_t)all.segs.size(), dst0 = (uint32_t)all.dsts.size();
-    for (DevSeg s : dp.segs) {
+    const uint32_t seg0 = (uint32_t)i_seg, dst0 = (uint32_t)i_dst;
+    for (const DevSeg &s0 : dp.segs) {
+      DevSeg &s = all.segs[i_seg++];
+      s = s0;
       s.src_rank += p->src_base[ph];
       s.dst_rank += p->dst_base[ph];
       s.dst_first += dst0;
-      all.segs.push_back(s);
     }
-    for (Dst d : dp.dsts) {
+    for (const Dst &d0 : dp.dsts) {
+      Dst &d = all.dsts[i_dst++];
+      d = d0;
       d.rank += p->dst_base[ph];
-      all.dsts.push_back(d);
     }
-    for (Unit u : dp.bulk_units) { u.seg += seg0; all.bulk_units.push_back(u); }
-    for (Unit u : dp.vec_units) { u.seg += seg0; all.vec_units.push_back(u); }
+    for (const Unit &u0 : dp.bulk_units) { Unit &u = all.bulk_units[i_bulk++]; u = u0; u.seg += seg0; }
+    for (const Unit &u0 : dp.vec_units) { Unit &u = all.vec_units[i_vec++]; u = u0; u.seg += seg0; }
   }
 }
 
@@ -452,9 +459,10 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
   emoe_status_t st;
   try {
     st = build_host_plan(*shape, *old_cfg, *new_cfg, flags, &p->hp);
-    if (st == EMOE_OK)
+    if (st == EMOE_OK) {
       for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
       build_merged(p);
+    }
   } catch (const std::bad_alloc &) {
     st = EMOE_ERR_OOM;
   }
