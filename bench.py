@@ -508,11 +508,18 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the re-layout has no CPU path")
+    local = local % torch.cuda.device_count()
     torch.cuda.set_device(local)
     dist = None
+    # control plane only (barrier, max of the step times): NCCL, or gloo when several ranks
+    # have to share one GPU (EMOE_BENCH_BACKEND=gloo, for checking the N > 1 flow on one device)
+    backend = os.environ.get("EMOE_BENCH_BACKEND", "nccl")
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend)
     barrier = (lambda: dist.barrier()) if dist else None
     peak, peak_kind = measured_peak()
     stream = torch.cuda.Stream()
@@ -525,7 +532,7 @@ def main():
     total_ms = time_steps(torch, plan, src, dst, args.steps, args.warmup, stream, barrier)
     clocks = sampler.stop()
     phase_ms = time_phases(torch, plan, src, dst, max(3, min(args.steps, 20)), stream)
-    total_ms = replicas.job_time_ms(total_ms, dist, device="cuda")   # max over ranks
+    total_ms = replicas.job_time_ms(total_ms, dist, device="cuda" if backend == "nccl" else "cpu")  # max over ranks
     rep = config_report(E, plan, wl, total_ms, phase_ms, args.steps, peak, plan_ms)
     if plan.device_status() != 0:
         raise SystemExit("device status word set: a bounded wait expired")
