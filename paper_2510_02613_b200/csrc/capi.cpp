@@ -8,6 +8,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <thread>
 #include <vector>
 
 #include "internal.h"
@@ -261,6 +262,27 @@ void build_merged(emoe_plan *p) {
   }
 }
 
+// Tables of the three phases (independent of one another: built on three threads when the
+// plan is large enough to pay for them) and the merged set.  Throws std::bad_alloc.
+void build_all_tables(emoe_plan *p) {
+  uint64_t work = 0;
+  for (int ph = 0; ph < 3; ++ph) work += p->hp.phase[ph].segs.size() + p->hp.phase[ph].bytes_moved / (1u << 20);
+  if (work < 4096) {  // small plan: threads would cost more than they save
+    for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
+  } else {
+    bool failed[3] = {false, false, false};
+    std::thread th[2];
+    for (int ph = 1; ph < 3; ++ph)
+      th[ph - 1] = std::thread([p, ph, &failed] {
+        try { build_tables(p, ph); } catch (...) { failed[ph] = true; }
+      });
+    try { build_tables(p, 0); } catch (...) { failed[0] = true; }
+    for (std::thread &t : th) t.join();
+    if (failed[0] || failed[1] || failed[2]) throw std::bad_alloc();
+  }
+  build_merged(p);
+}
+
 template <typename T>
 cudaError_t upload(const std::vector<T> &v, T **d) {
   if (*d) { cudaFree(*d); *d = nullptr; }
@@ -460,8 +482,7 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
   try {
     st = build_host_plan(*shape, *old_cfg, *new_cfg, flags, &p->hp);
     if (st == EMOE_OK) {
-      for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
-      build_merged(p);
+      build_all_tables(p);
     }
   } catch (const std::bad_alloc &) {
     st = EMOE_ERR_OOM;
@@ -852,8 +873,7 @@ emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
   p->tuning = *t;
   emoe_status_t st = EMOE_OK;
   try {
-    for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
-    build_merged(p);
+    build_all_tables(p);
   } catch (const std::bad_alloc &) {
     return EMOE_ERR_OOM;
   }
@@ -875,8 +895,7 @@ emoe_status_t emoe_plan_set_local_rank(emoe_plan_t *p, int32_t rank) {
   p->local_rank = rank;
   emoe_status_t st = EMOE_OK;
   try {
-    for (int ph = 0; ph < 3; ++ph) build_tables(p, ph);
-    build_merged(p);
+    build_all_tables(p);
   } catch (const std::bad_alloc &) {
     return EMOE_ERR_OOM;
   }
