@@ -191,6 +191,13 @@ emoe_status_t emoe_reshard_attn(const emoe_plan_t *plan, const void *const *src,
  * rank g/(Hkv/d), block bt_new[s][j], local head g%(Hkv/d).  Whole blocks
  * move; destination blocks that no sequence maps are not written.
  * src: [tp_old] device pointers, dst: [tp_new]; otherwise as above.
+ *
+ * Migrating while serving goes on (the paper scales without stopping the old
+ * instance, Sec. 4): run the step once for the whole cache, let serving append
+ * tokens meanwhile, then run a second, small plan that lists only the blocks
+ * written since - each as a "sequence" of one block (seq_len = B, one table
+ * entry) - before switching over.  A plan is a pure function of the tables it
+ * is given, so any subset of blocks can be re-copied this way.
  */
 emoe_status_t emoe_reshard_kv(const emoe_plan_t *plan, const void *const *src,
                               void *const *dst, void *cuda_stream);

@@ -354,3 +354,52 @@ def test_step_captured_in_a_cuda_graph_replays_correctly():
             for ph in range(3):
                 assert all(torch.equal(a, b) for a, b in zip(dst[ph], ref[ph]))
         check_step_full(wl, plan)
+
+
+def test_kv_delta_plan_recopies_blocks_written_during_the_migration():
+    """Scale while serving: migrate the whole KV cache, let "serving" append tokens to the
+    last block of every sequence and claim one more block, then re-copy only those blocks
+    with a delta plan (every dirty block a one-block sequence).  The result must equal the
+    oracle run on the final cache in one go."""
+    from gpu_util import oracle_phase
+    wl = W.make_workload("c4_large", n_layers=2)
+    B = wl.shape.kv_block_tokens
+    # leave room for one more block per sequence in both pools
+    n_seq = len(wl.old.seq_lens)
+    nb_old, nb_new = wl.old.kv_num_blocks + n_seq, wl.new.kv_num_blocks + n_seq
+    seq0 = [n - (n % B or B) + 3 for n in wl.old.seq_lens]          # last block partly filled
+    def tables(seq_lens):
+        return (W.make_block_table(31, seq_lens, B, nb_old), W.make_block_table(32, seq_lens, B, nb_new))
+    grown = [n + B for n in seq0]                                    # one more block each
+    bo1, bn1 = tables(grown)                                         # final tables; the early ones are their prefix
+    nblk0 = [-(-n // B) for n in seq0]
+    bo0 = np.full_like(bo1, -1); bn0 = np.full_like(bn1, -1)
+    for s_, k in enumerate(nblk0):
+        bo0[s_, :k] = bo1[s_, :k]; bn0[s_, :k] = bn1[s_, :k]
+    early = R(wl, old=R(wl.old, kv_num_blocks=nb_old, seq_lens=seq0, block_table=bo0),
+              new=R(wl.new, kv_num_blocks=nb_new, seq_lens=seq0, block_table=bn0))
+    final = R(wl, old=R(wl.old, kv_num_blocks=nb_old, seq_lens=grown, block_table=bo1),
+              new=R(wl.new, kv_num_blocks=nb_new, seq_lens=grown, block_table=bn1))
+    # dirty blocks: the last block of the early state and the new block, per sequence
+    d_old = np.array([[bo1[s_, k - 1]] for s_, k in enumerate(nblk0)] + [[bo1[s_, k]] for s_, k in enumerate(nblk0)], np.int32)
+    d_new = np.array([[bn1[s_, k - 1]] for s_, k in enumerate(nblk0)] + [[bn1[s_, k]] for s_, k in enumerate(nblk0)], np.int32)
+    delta = R(wl, old=R(wl.old, kv_num_blocks=nb_old, seq_lens=[B] * len(d_old), block_table=d_old),
+              new=R(wl.new, kv_num_blocks=nb_new, seq_lens=[B] * len(d_new), block_table=d_new))
+    with E.Plan(early.shape, early.old, early.new) as p_all, E.Plan(delta.shape, delta.old, delta.new) as p_delta:
+        src = WD.alloc_filled(p_all.arena_bytes(E.PHASE_KV, E.SIDE_OLD), wl.seed, W.KIND_KV)
+        dst = WD.alloc_const(p_all.arena_bytes(E.PHASE_KV, E.SIDE_NEW))
+        p_all.reshard_kv(src, dst)
+        # serving writes: new contents for every dirty block of every layer and K|V
+        L, hl = wl.shape.n_layers, wl.shape.n_kv_heads // wl.old.tp
+        blk = B * hl * wl.shape.head_dim * wl.shape.elem_bytes
+        for t in src:
+            pool = t.view(L * 2, nb_old, blk)
+            pool[:, torch.from_numpy(d_old[:, 0].astype(np.int64)).cuda()] += 1
+        p_delta.reshard_kv(src, dst)
+        torch.cuda.synchronize()
+        want = [np.full(t.numel(), WD.FILL_BYTE, np.uint8) for t in dst]
+        oracle_phase(final, E.PHASE_KV, [t.cpu().numpy() for t in src], want)
+        for r, (g, w) in enumerate(zip(dst, want)):
+            assert np.array_equal(g.cpu().numpy(), w), "rank %d" % r
+        moved = p_delta.stats(E.PHASE_KV)["bytes_moved"]
+        assert moved * 8 < p_all.stats(E.PHASE_KV)["bytes_moved"]      # the delta is small
