@@ -403,3 +403,17 @@ def test_kv_delta_plan_recopies_blocks_written_during_the_migration():
             assert np.array_equal(g.cpu().numpy(), w), "rank %d" % r
         moved = p_delta.stats(E.PHASE_KV)["bytes_moved"]
         assert moved * 8 < p_all.stats(E.PHASE_KV)["bytes_moved"]      # the delta is small
+
+
+def test_fp8_weights_with_block_scales_as_two_plans():
+    """FP8 expert weights (elem_bytes = 1) and their per-128x128-block fp32 scale tensors
+    move with the same placement through two plans: one for the weights, one whose
+    "matrix" is the scale tensor of an expert ([d_ff/128][d_model/128] floats)."""
+    base = W.make_workload("c3_fine", n_layers=1)
+    weights = R(base, shape=R(base.shape, elem_bytes=1))
+    scales = R(base, shape=R(base.shape, d_model=base.shape.d_model // 128,
+                             d_ff=base.shape.d_ff // 128, elem_bytes=4))
+    assert scales.shape.d_model * scales.shape.d_ff * 4 == 16 * 11 * 4
+    for wl in (weights, scales):
+        with E.Plan(wl.shape, wl.old, wl.new) as plan:
+            check_phase_full(wl, plan, E.PHASE_EXPERTS)
