@@ -36,7 +36,13 @@ constexpr uint64_t kSmallPhaseBytes = 256ull << 20;
 struct DevPhase {
   std::vector<DevSeg> segs;  // routed copy of the host segments (fan-out split to kMaxFanout)
   std::vector<Dst> dsts;
-  std::vector<Unit> bulk_units, vec_units;
+  std::vector<Unit> bulk_units, vec_units;   // bulk_units: general case only (see `regular`)
+  uint64_t n_bulk = 0;                        // bulk units of the phase
+  // Regular phase: its bulk unit table is expanded on the device from these (bulk segment
+  // indices, offset of each one's units inside a run, runs per segment, units per run).
+  bool regular = false;
+  std::vector<uint32_t> gen_seg, gen_pre;
+  uint32_t gen_runs = 0, gen_upr = 0;
   DevSeg *d_segs = nullptr;
   Dst *d_dsts = nullptr;
   Unit *d_bulk_units = nullptr, *d_vec_units = nullptr;
@@ -67,6 +73,8 @@ struct emoe_plan {
   DevPhase dev[kTableSets];       // [3]: all three phases as one launch set (see build_merged)
   uint32_t src_base[3] = {0, 0, 0}, dst_base[3] = {0, 0, 0};  // rank offsets of a phase in the merged set
   bool merged = false;
+  uint32_t merged_seg0[3] = {0, 0, 0};        // first segment / first bulk unit of a phase in the merged set
+  uint64_t merged_unit0[3] = {0, 0, 0};
   std::vector<uint32_t> pair_old, pair_new;  // block pairs in launch order (see kv_order)
   uint32_t *d_pair_old = nullptr, *d_pair_new = nullptr;
   int *d_status = nullptr;  // [0] status word; then kCtrSlots x 2 work-counter words per phase
@@ -108,6 +116,26 @@ void for_each_unit(uint32_t seg, const DevSeg &s, uint32_t T, F &&f) {
   }
 }
 
+// The general case: the bulk unit table written on the host, run-major without a sort
+// (count the units of every run, turn the counts into start positions, then place).
+void expand_units_on_host(DevPhase *dp, const std::vector<uint32_t> &bulk_segs, uint32_t T, bool run_major) {
+  dp->bulk_units.clear();
+  if (run_major) {
+    uint32_t max_run = 0;
+    for (uint32_t idx : bulk_segs) max_run = std::max(max_run, dp->segs[idx].n_runs);
+    std::vector<uint32_t> start((size_t)max_run + 2, 0);
+    for (uint32_t idx : bulk_segs)
+      for_each_unit(idx, dp->segs[idx], T, [&](uint32_t run, const Unit &) { start[run + 1]++; });
+    for (size_t i = 1; i < start.size(); ++i) start[i] += start[i - 1];
+    dp->bulk_units.resize(start.back());
+    for (uint32_t idx : bulk_segs)
+      for_each_unit(idx, dp->segs[idx], T, [&](uint32_t run, const Unit &u) { dp->bulk_units[start[run]++] = u; });
+  } else {
+    for (uint32_t idx : bulk_segs)
+      for_each_unit(idx, dp->segs[idx], T, [&](uint32_t, const Unit &u) { dp->bulk_units.push_back(u); });
+  }
+}
+
 // Routes every host segment to the bulk or the vector kernel and cuts it into units.
 //
 // Launch order of the bulk units is run-major: all segments' run 0, then all segments'
@@ -118,6 +146,8 @@ void build_tables(emoe_plan *p, int phase) {
   const PhasePlan &pp = p->hp.phase[phase];
   DevPhase &dp = p->dev[phase];
   dp.segs.clear(); dp.dsts.clear(); dp.bulk_units.clear(); dp.vec_units.clear();
+  dp.gen_seg.clear(); dp.gen_pre.clear();
+  dp.regular = false; dp.n_bulk = 0; dp.gen_runs = dp.gen_upr = 0;
   for (bool &b : p->reads_src[phase]) b = false;
   const uint32_t T = bulk_tile(p);
 
@@ -181,22 +211,34 @@ void build_tables(emoe_plan *p, int phase) {
       else for_each_unit(idx, s, kVecTile, [&](uint32_t, const Unit &u) { dp.vec_units.push_back(u); });
     }
   }
-  // Bulk units in run-major order without a sort: count the units of every run, turn the
-  // counts into start positions, then place (hundreds of thousands of units: anything
-  // slower costs more host time than the copy takes on the device).
-  if (p->tuning.unit_order % 2 == 0) {
-    uint32_t max_run = 0;
-    for (uint32_t idx : bulk_segs) max_run = std::max(max_run, dp.segs[idx].n_runs);
-    std::vector<uint32_t> start((size_t)max_run + 2, 0);
-    for (uint32_t idx : bulk_segs)
-      for_each_unit(idx, dp.segs[idx], T, [&](uint32_t run, const Unit &) { start[run + 1]++; });
-    for (size_t i = 1; i < start.size(); ++i) start[i] += start[i - 1];
-    dp.bulk_units.resize(start.back());
-    for (uint32_t idx : bulk_segs)
-      for_each_unit(idx, dp.segs[idx], T, [&](uint32_t run, const Unit &u) { dp.bulk_units[start[run]++] = u; });
-  } else {
-    for (uint32_t idx : bulk_segs)
-      for_each_unit(idx, dp.segs[idx], T, [&](uint32_t, const Unit &u) { dp.bulk_units.push_back(u); });
+  // Bulk units in run-major order.  Regular phase (every bulk segment has the same number
+  // of runs, each at least a tile long - all bench phases): only each segment's offset inside
+  // a run is computed here, the table itself is written by a kernel at upload time.
+  bool regular = p->tuning.unit_order % 2 == 0 && !bulk_segs.empty();
+  for (uint32_t idx : bulk_segs)
+    regular = regular && dp.segs[idx].run_bytes >= T && dp.segs[idx].n_runs == dp.segs[bulk_segs[0]].n_runs;
+  if (regular) {
+    uint64_t upr = 0;
+    dp.gen_pre.reserve(bulk_segs.size());
+    for (uint32_t idx : bulk_segs) {
+      dp.gen_pre.push_back((uint32_t)upr);
+      const uint64_t tpr = (dp.segs[idx].run_bytes + T - 1) / T;
+      upr += (tpr + kUnitTiles - 1) / kUnitTiles;
+    }
+    dp.gen_runs = dp.segs[bulk_segs[0]].n_runs;
+    regular = upr * dp.gen_runs < 0xffffffffull;
+    if (regular) {
+      dp.regular = true;
+      dp.gen_seg = bulk_segs;
+      dp.gen_upr = (uint32_t)upr;
+      dp.n_bulk = upr * dp.gen_runs;
+    } else {
+      dp.gen_pre.clear();
+    }
+  }
+  if (!dp.regular) {
+    expand_units_on_host(&dp, bulk_segs, T, p->tuning.unit_order % 2 == 0);
+    dp.n_bulk = dp.bulk_units.size();
   }
   if (phase == EMOE_PHASE_KV) {  // block pairs of the head re-split, in launch order
     const KvPlan &kv = p->hp.kv;
@@ -235,12 +277,27 @@ void build_merged(emoe_plan *p) {
   }
   p->merged = ns <= EMOE_MAX_RANKS && nd <= EMOE_MAX_RANKS;
   if (!p->merged) return;
-  size_t n_seg = 0, n_dst = 0, n_bulk = 0, n_vec = 0;
+  all.gen_seg.clear(); all.gen_pre.clear();
+  all.regular = false; all.n_bulk = 0;
+  // the merged bulk table is written on the device too if every phase's is
+  bool regular = true;
+  for (int ph = 0; ph < 3; ++ph) regular = regular && (p->dev[ph].n_bulk == 0 || p->dev[ph].regular);
+  size_t n_seg = 0, n_dst = 0, n_vec = 0;
+  uint64_t n_bulk = 0;
   for (int ph = 0; ph < 3; ++ph) {
-    n_seg += p->dev[ph].segs.size(); n_dst += p->dev[ph].dsts.size();
-    n_bulk += p->dev[ph].bulk_units.size(); n_vec += p->dev[ph].vec_units.size();
+    DevPhase &dp = p->dev[ph];
+    p->merged_seg0[ph] = (uint32_t)n_seg;
+    p->merged_unit0[ph] = n_bulk;
+    if (!regular && dp.regular && dp.bulk_units.empty())   // its units are needed on the host after all
+      expand_units_on_host(&dp, dp.gen_seg, bulk_tile(p), true);
+    n_seg += dp.segs.size(); n_dst += dp.dsts.size();
+    n_bulk += dp.n_bulk; n_vec += dp.vec_units.size();
   }
-  all.segs.resize(n_seg); all.dsts.resize(n_dst); all.bulk_units.resize(n_bulk); all.vec_units.resize(n_vec);
+  if (n_bulk >= 0xffffffffull) { p->merged = false; return; }
+  all.regular = regular && n_bulk > 0;
+  all.n_bulk = n_bulk;
+  all.segs.resize(n_seg); all.dsts.resize(n_dst); all.vec_units.resize(n_vec);
+  if (!all.regular) all.bulk_units.resize(n_bulk);
   size_t i_seg = 0, i_dst = 0, i_bulk = 0, i_vec = 0;
   for (int ph = 0; ph < 3; ++ph) {
     const DevPhase &dp = p->dev[ph];
@@ -257,7 +314,8 @@ void build_merged(emoe_plan *p) {
       d = d0;
       d.rank += p->dst_base[ph];
     }
-    for (const Unit &u0 : dp.bulk_units) { Unit &u = all.bulk_units[i_bulk++]; u = u0; u.seg += seg0; }
+    if (!all.regular)
+      for (const Unit &u0 : dp.bulk_units) { Unit &u = all.bulk_units[i_bulk++]; u = u0; u.seg += seg0; }
     for (const Unit &u0 : dp.vec_units) { Unit &u = all.vec_units[i_vec++]; u = u0; u.seg += seg0; }
   }
 }
@@ -298,13 +356,43 @@ emoe_status_t cuda_status(cudaError_t e) {
   return e == cudaErrorMemoryAllocation ? EMOE_ERR_OOM : EMOE_ERR_CUDA;
 }
 
+// Expands the regular unit table of phase `src_ph` into `out` on the device.
+cudaError_t gen_units(const emoe_plan *p, int src_ph, const DevSeg *d_segs, uint32_t seg_offset, Unit *out) {
+  const DevPhase &dp = p->dev[src_ph];
+  uint32_t *d_idx = nullptr, *d_pre = nullptr;
+  const size_t bytes = dp.gen_seg.size() * sizeof(uint32_t);
+  cudaError_t e = cudaMalloc((void **)&d_idx, bytes);
+  if (e == cudaSuccess) e = cudaMalloc((void **)&d_pre, bytes);
+  if (e == cudaSuccess) e = cudaMemcpy(d_idx, dp.gen_seg.data(), bytes, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(d_pre, dp.gen_pre.data(), bytes, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess)
+    e = launch_gen_units(d_segs, d_idx, d_pre, (uint32_t)dp.gen_seg.size(), dp.gen_runs, dp.gen_upr,
+                         bulk_tile(p), kUnitTiles, seg_offset, out, nullptr);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(nullptr);
+  cudaFree(d_idx);
+  cudaFree(d_pre);
+  return e;
+}
+
 emoe_status_t upload_phase(emoe_plan *p, int phase) {
   DevPhase &dp = p->dev[phase];
   cudaError_t e;
   if ((e = upload(dp.segs, &dp.d_segs)) != cudaSuccess) return cuda_status(e);
   if ((e = upload(dp.dsts, &dp.d_dsts)) != cudaSuccess) return cuda_status(e);
-  if ((e = upload(dp.bulk_units, &dp.d_bulk_units)) != cudaSuccess) return cuda_status(e);
   if ((e = upload(dp.vec_units, &dp.d_vec_units)) != cudaSuccess) return cuda_status(e);
+  if (!dp.regular) {
+    if ((e = upload(dp.bulk_units, &dp.d_bulk_units)) != cudaSuccess) return cuda_status(e);
+    return EMOE_OK;
+  }
+  // regular: the table is written by a kernel (for the merged set, phase by phase)
+  if (dp.d_bulk_units) { cudaFree(dp.d_bulk_units); dp.d_bulk_units = nullptr; }
+  if ((e = cudaMalloc((void **)&dp.d_bulk_units, dp.n_bulk * sizeof(Unit))) != cudaSuccess) return cuda_status(e);
+  if (phase < 3) return cuda_status(gen_units(p, phase, dp.d_segs, 0, dp.d_bulk_units));
+  for (int q = 0; q < 3; ++q)
+    if (p->dev[q].n_bulk) {
+      e = gen_units(p, q, dp.d_segs, p->merged_seg0[q], dp.d_bulk_units + p->merged_unit0[q]);
+      if (e != cudaSuccess) return cuda_status(e);
+    }
   return EMOE_OK;
 }
 
@@ -374,7 +462,7 @@ emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, 
     const uint32_t slot = p->launch_seq[phase].fetch_add(1) % kCtrSlots;
     ctr = reinterpret_cast<unsigned int *>(p->d_status) + 1 + (phase * kCtrSlots + slot) * 2;
   }
-  cudaError_t e = launch_bulk_copy({dp.d_segs, dp.d_dsts, dp.d_bulk_units, (uint32_t)dp.bulk_units.size()},
+  cudaError_t e = launch_bulk_copy({dp.d_segs, dp.d_dsts, dp.d_bulk_units, (uint32_t)dp.n_bulk},
                                    ptrs, bc, bulk_budget(p), p->d_status, ctr, st);
   if (e != cudaSuccess) return cuda_status(e);
   e = launch_vec_copy({dp.d_segs, dp.d_dsts, dp.d_vec_units, (uint32_t)dp.vec_units.size()}, ptrs,
@@ -805,10 +893,10 @@ emoe_status_t emoe_plan_num_launches(const emoe_plan_t *p, int phase, int32_t *n
     const int kv_pairs = p->hp.kv.head_split_changes && !p->hp.kv.pair_old.empty() ? 1 : 0;
     int k = 0;
     if (p->merged) {
-      k = (p->dev[3].bulk_units.empty() ? 0 : 1) + (p->dev[3].vec_units.empty() ? 0 : 1);
+      k = (p->dev[3].n_bulk ? 1 : 0) + (p->dev[3].vec_units.empty() ? 0 : 1);
     } else {
       for (int ph = 0; ph < 3; ++ph)
-        k += (p->dev[ph].bulk_units.empty() ? 0 : 1) + (p->dev[ph].vec_units.empty() ? 0 : 1);
+        k += (p->dev[ph].n_bulk ? 1 : 0) + (p->dev[ph].vec_units.empty() ? 0 : 1);
     }
     *n = k + kv_pairs;
     return EMOE_OK;
@@ -817,7 +905,7 @@ emoe_status_t emoe_plan_num_launches(const emoe_plan_t *p, int phase, int32_t *n
     *n = p->hp.kv.pair_old.empty() ? 0 : 1;
     return EMOE_OK;
   }
-  *n = (p->dev[phase].bulk_units.empty() ? 0 : 1) + (p->dev[phase].vec_units.empty() ? 0 : 1);
+  *n = (p->dev[phase].n_bulk ? 1 : 0) + (p->dev[phase].vec_units.empty() ? 0 : 1);
   return EMOE_OK;
 }
 

@@ -1056,6 +1056,41 @@ cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, ui
   return cudaGetLastError();
 }
 
+// ---- unit tables expanded on the device ---------------------------------------------------
+//
+// A phase whose bulk segments all have the same number of runs, each run at least a tile
+// long, has a regular unit table: run-major, and inside a run segment after segment.  The
+// host then only sends, per segment, where its units start inside a run; one thread per
+// (segment, run) writes that segment's units of that run.
+
+namespace {
+__global__ void gen_units_kernel(const DevSeg *segs, const uint32_t *seg_idx, const uint32_t *seg_pre,
+                                 uint32_t n_segs, uint32_t n_runs, uint32_t units_per_run,
+                                 uint32_t tile_bytes, uint32_t unit_tiles, uint32_t seg_offset,
+                                 Unit *out) {
+  const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (uint64_t)n_segs * n_runs) return;
+  const uint32_t k = (uint32_t)(i % n_segs), run = (uint32_t)(i / n_segs);
+  const uint32_t seg = seg_idx[k] + seg_offset;
+  const uint64_t run_bytes = segs[seg].run_bytes;
+  const uint32_t tpr = (uint32_t)((run_bytes + tile_bytes - 1) / tile_bytes);
+  Unit *o = out + (uint64_t)run * units_per_run + seg_pre[k];
+  for (uint32_t t = 0; t < tpr; t += unit_tiles, ++o)
+    *o = Unit{seg, run * tpr + t, tpr - t < unit_tiles ? tpr - t : unit_tiles, 0};
+}
+}  // namespace
+
+cudaError_t launch_gen_units(const DevSeg *segs, const uint32_t *seg_idx, const uint32_t *seg_pre,
+                             uint32_t n_segs, uint32_t n_runs, uint32_t units_per_run,
+                             uint32_t tile_bytes, uint32_t unit_tiles, uint32_t seg_offset, Unit *out,
+                             cudaStream_t stream) {
+  const uint64_t n = (uint64_t)n_segs * n_runs;
+  if (n == 0) return cudaSuccess;
+  gen_units_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(
+      segs, seg_idx, seg_pre, n_segs, n_runs, units_per_run, tile_bytes, unit_tiles, seg_offset, out);
+  return cudaGetLastError();
+}
+
 // ---- KV re-split without any allocation ---------------------------------------------------
 //
 // For callers that cannot call cudaMalloc (all of HBM already owned by a memory daemon,
