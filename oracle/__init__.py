@@ -33,6 +33,10 @@ def lib() -> ctypes.CDLL:
         L.emoe_oracle_reshard_attn.argtypes = [i32] * 8 + [p, p]
         L.emoe_oracle_reshard_kv.restype = i32
         L.emoe_oracle_reshard_kv.argtypes = [i32] * 11 + [p, p, p, p, p, i32]
+        L.emoe_oracle_inplace_slots.restype = i32
+        L.emoe_oracle_inplace_slots.argtypes = [i32, p, p, i32, p, p, p, p]
+        L.emoe_oracle_reshard_experts_inplace.restype = i32
+        L.emoe_oracle_reshard_experts_inplace.argtypes = [i32, i64, i32, p, p, i32, p, p, p, p, p]
         _lib = L
     return _lib
 
@@ -127,6 +131,60 @@ def reshard_kv(shape, old_cfg, new_cfg, src, dst, head_major: bool = False) -> N
                                      int(bool(head_major)))
     if rc != 0:
         raise ValueError("oracle: bad block table or TP degree")
+
+
+# ---- in-place expert step on capacity-strided arenas ------------------------------------
+
+_INPLACE_ERRORS = {-1: "a wanted expert has no copy in the old slot tables",
+                   -2: "a rank has fewer free slots than arrivals",
+                   -3: "the capacity of a rank that stays differs between the two sides",
+                   -4: "an expert is wanted twice on one rank"}
+
+
+def inplace_slots(old_slots, want, cap_new) -> List[List[int]]:
+    """New slot tables of the in-place expert step.  old_slots: per old rank a list of
+    expert ids or -1 (free), its length being the rank's capacity; want: per new rank the
+    experts it must hold afterwards; cap_new: capacity per new rank (unchanged for a rank
+    that exists on both sides).  Kept experts keep their slot, arrivals take - in the order
+    listed - the lowest slot that was free before the step, leaving experts free theirs."""
+    oo, oi = _csr(old_slots)
+    wo, wi = _csr(want)
+    cap = np.ascontiguousarray(cap_new, dtype=np.int32)
+    out = np.full(int(cap.sum()), -7, dtype=np.int32)
+    rc = lib().emoe_oracle_inplace_slots(len(old_slots), _vp(oo), _vp(oi), len(want), _vp(cap),
+                                         _vp(wo), _vp(wi), _vp(out))
+    if rc != 0:
+        raise ValueError("oracle: " + _INPLACE_ERRORS.get(rc, str(rc)))
+    res, b = [], 0
+    for c in cap:
+        res.append([int(x) for x in out[b:b + c]])
+        b += int(c)
+    return res
+
+
+def inplace_arena_bytes(shape, caps) -> List[int]:
+    m = shape.d_model * shape.d_ff * shape.elem_bytes
+    return [lib().emoe_oracle_expert_arena_bytes(shape.n_layers, int(c), m) for c in caps]
+
+
+def reshard_experts_inplace(shape, old_slots, want, cap_new, arenas: Sequence[np.ndarray]):
+    """Runs the in-place step on `arenas` (max(old ranks, new ranks) arrays, arena r being
+    [L][3][cap_r][m]); only arrivals are written.  Returns the new slot tables."""
+    new_slots = inplace_slots(old_slots, want, cap_new)
+    caps = [len(t) for t in old_slots] + [int(c) for c in list(cap_new)[len(old_slots):]]
+    if [a.size for a in arenas] != inplace_arena_bytes(shape, caps):
+        raise ValueError("arena sizes do not match the capacities")
+    m = shape.d_model * shape.d_ff * shape.elem_bytes
+    oo, oi = _csr(old_slots)
+    wo, wi = _csr(want)
+    cap = np.ascontiguousarray(cap_new, dtype=np.int32)
+    flat = np.array([e for t in new_slots for e in t], dtype=np.int32)
+    rc = lib().emoe_oracle_reshard_experts_inplace(shape.n_layers, m, len(old_slots), _vp(oo), _vp(oi),
+                                                  len(want), _vp(cap), _vp(wo), _vp(wi), _vp(flat),
+                                                  _ptrs(arenas))
+    if rc != 0:
+        raise ValueError("oracle: " + _INPLACE_ERRORS.get(rc, str(rc)))
+    return new_slots
 
 
 # ---- placement chooser: brute force ----------------------------------------------------

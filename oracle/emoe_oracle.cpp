@@ -17,11 +17,11 @@
 //    uneven and replicated placements are allowed (Sec. 2.1).
 //  * attention: TP shards the attention operations (Sec. 2.1); with TP fixed
 //    the shards carry over unchanged (Sec. 5.2 "Attention Weights"); changing
-//    TP is the paper's future work (Sec. 9), read here in the usual way:
-//    q/k/v split by head along stored rows, o split by head along stored
-//    columns.
+//    TP is the paper's future work (App. C "Limitations and Future Work"),
+//    read here in the usual way: q/k/v split by head along stored rows, o
+//    split by head along stored columns.
 //  * KV cache: follows TP (Sec. 4.1, Sec. 5.2 "KV Cache"); "reshaping KV
-//    caches" under a TP change (Sec. 9) is read as a contiguous split of the
+//    caches" under a TP change (App. C) is read as a contiguous split of the
 //    KV heads, block tables translating physical block ids.
 //
 //  * more TP ranks than KV heads (grouped-query attention; the paper is silent):
@@ -36,6 +36,16 @@
 //    tensor followed by a [n_r][down] tensor instead of three [n_r] tensors;
 //    head_major stores a KV block as [local head][token][hd] instead of
 //    [token][local head][hd].  Both are re-orderings of the same logical data.
+//
+//  * in-place expert step (Sec. 4.1 "Virtual Expert Management", Sec. 5.2 "Expert
+//    Weights", App. D.5, App. E): a device that stays keeps the experts it already
+//    holds where they are and only arrivals are transferred.  Read here for a dense
+//    arena with spare capacity, [L][3][cap_r][m] with a slot table (expert id or -1
+//    per slot): an expert wanted again keeps its slot; an arrival takes the lowest
+//    slot that was FREE BEFORE the step (the old instance keeps serving from the old
+//    experts until the switch-over, Sec. 5.2 "Coordinator Performs Instance
+//    Switchover", so their bytes are not overwritten); a slot whose expert leaves is
+//    marked free for later steps and its bytes stay.
 //
 // Pins: every function below is pinned by tests that do not use it to make
 // their expectation (numpy/torch indexing of logical tensors, hand-written
@@ -223,6 +233,86 @@ int emoe_oracle_reshard_kv(int n_layers, int block_tokens, int hkv, int hd, int 
               }
     }
   }
+  return 0;
+}
+
+// ---- in-place expert step on capacity-strided arenas ---------------------------------
+//
+// Slot tables are CSR: rank r has slots ids[off[r] .. off[r+1]), each an expert id or -1.
+// cap_new[r] is the capacity of new rank r; a rank that exists on both sides keeps its
+// arena, so its capacity must not change.  want_off / want_ids: the experts every new rank
+// must hold afterwards (order matters only for which free slot an arrival gets).
+// Return codes: 0 ok, -1 a wanted expert has no copy in the old tables, -2 a rank has
+// fewer free slots than arrivals, -3 a staying rank's capacity differs, -4 a wanted
+// expert is listed twice for one rank.
+
+// New slot tables (slot_new: sum(cap_new) entries, rank after rank).
+int emoe_oracle_inplace_slots(int ep_old, const int32_t *off_old, const int32_t *ids_old, int ep_new,
+                              const int32_t *cap_new, const int32_t *want_off,
+                              const int32_t *want_ids, int32_t *slot_new) {
+  int64_t base = 0;
+  for (int r = 0; r < ep_new; ++r) {
+    const int cap = cap_new[r];
+    int32_t *mine = slot_new + base;
+    base += cap;
+    const bool stays = r < ep_old;
+    if (stays && off_old[r + 1] - off_old[r] != cap) return -3;
+    // 1. start from the old table; remember which slots were free before the step
+    for (int s = 0; s < cap; ++s) mine[s] = stays ? ids_old[off_old[r] + s] : -1;
+    // 2. experts that are not wanted any more leave (their slot is free from the NEXT step on)
+    for (int s = 0; s < cap; ++s) {
+      if (mine[s] < 0) continue;
+      bool wanted = false;
+      for (int i = want_off[r]; i < want_off[r + 1]; ++i) wanted = wanted || want_ids[i] == mine[s];
+      if (!wanted) mine[s] = -2;  // leaving: neither an expert nor available to an arrival
+    }
+    // 3. arrivals, in the order they are listed, take the lowest slot that was free before
+    for (int i = want_off[r]; i < want_off[r + 1]; ++i) {
+      const int32_t e = want_ids[i];
+      for (int k = want_off[r]; k < i; ++k)
+        if (want_ids[k] == e) return -4;
+      bool held = false;
+      for (int s = 0; s < cap; ++s) held = held || mine[s] == e;
+      if (held) continue;
+      int s = 0;
+      while (s < cap && mine[s] != -1) ++s;
+      if (s == cap) return -2;
+      mine[s] = e;
+    }
+    for (int s = 0; s < cap; ++s)
+      if (mine[s] == -2) mine[s] = -1;
+  }
+  return 0;
+}
+
+// The step itself.  arenas: max(ep_old, ep_new) pointers; arena r is [L][3][cap_r][m] with
+// cap_r = old capacity for r < ep_old, cap_new[r] otherwise.  Only arrivals are written.
+int emoe_oracle_reshard_experts_inplace(int n_layers, int64_t m, int ep_old, const int32_t *off_old,
+                                        const int32_t *ids_old, int ep_new, const int32_t *cap_new,
+                                        const int32_t *want_off, const int32_t *want_ids,
+                                        const int32_t *slot_new, uint8_t *const *arenas) {
+  int64_t base = 0;
+  for (int rn = 0; rn < ep_new; ++rn) {
+    const int64_t cap = cap_new[rn];
+    for (int sn = 0; sn < cap; ++sn) {
+      const int32_t e = slot_new[base + sn];
+      if (e < 0) continue;
+      if (rn < ep_old && ids_old[off_old[rn] + sn] == e) continue;  // kept where it is
+      // arrival: smallest (rank, slot) that held e before the step
+      int ro = -1, so = -1;
+      for (int r = 0; r < ep_old && ro < 0; ++r)
+        for (int s = 0; s < off_old[r + 1] - off_old[r]; ++s)
+          if (ids_old[off_old[r] + s] == e) { ro = r; so = s; break; }
+      if (ro < 0) return -1;
+      const int64_t cap_o = off_old[ro + 1] - off_old[ro];
+      for (int l = 0; l < n_layers; ++l)
+        for (int p = 0; p < 3; ++p)
+          std::memcpy(arenas[rn] + (((int64_t)l * 3 + p) * cap + sn) * m,
+                      arenas[ro] + (((int64_t)l * 3 + p) * cap_o + so) * m, (size_t)m);
+    }
+    base += cap;
+  }
+  (void)want_off; (void)want_ids;
   return 0;
 }
 

@@ -450,3 +450,172 @@ def test_published_step_bytes_of_the_five_configs():
         got = (sum(oracle.expert_arena_bytes(sh, wl.new.placement))
                + sum(oracle.attn_arena_bytes(sh, wl.new.tp)) + kv_moved)
         assert got == total, name
+
+
+# ============================================================ in-place expert step ======
+
+def slot_arenas(logical, slots, key):
+    """Arena [L, 3, cap, m] of every rank: occupied slots hold their expert's logical
+    matrices (numpy indexing), free slots hold bytes of their own (so that a write to a
+    slot that must stay untouched is seen)."""
+    L, _, _, m = logical.shape
+    out = []
+    for r, table in enumerate(slots):
+        a = rand_bytes((key, r), L * 3 * len(table) * m).reshape(L, 3, len(table), m).copy()
+        for s, e in enumerate(table):
+            if e >= 0:
+                a[:, :, s] = logical[:, :, e]
+        out.append(a.reshape(-1))
+    return out
+
+
+INPLACE_CASES = {
+    # old slot tables, wanted experts per new rank, capacity of the new ranks
+    "grow_2_3": ([[0, 1, 2, -1, -1], [3, 4, 5, -1, -1]], [[0, 1], [3, 4], [2, 5]], [5, 5, 3]),
+    "grow_with_swaps": ([[0, 1, 2, -1, -1, -1], [3, 4, 5, -1, -1, -1]],
+                        [[5, 0, 4], [1, 3], [2, 0, 3]], [6, 6, 4]),
+    "shrink_3_2": ([[0, 1, -1, -1], [2, 3, -1, -1], [4, 5, -1]], [[0, 1, 4, 2], [3, 5, 2]], [4, 4]),
+    "holes_first": ([[-1, 0, -1, 1], [-1, -1, 2, 3]], [[3, 2, 0], [1, 3]], [4, 4]),
+    "replicated": ([[0, 1, -1, -1], [1, 2, -1, -1]], [[0, 2, 1], [0, 1], [1, 2, 0]], [4, 4, 3]),
+    "nothing_moves": ([[0, 1, -1], [2, -1, 3]], [[1, 0], [3, 2]], [3, 3]),
+}
+
+
+@pytest.mark.parametrize("name", sorted(INPLACE_CASES))
+def test_inplace_step_against_numpy_indexing_of_the_logical_tensor(name):
+    """After the step every occupied slot of every rank holds logical[:, :, expert]; a kept
+    expert is in the slot it had; every other byte - free slots, slots of experts that
+    left - is exactly what it was."""
+    old, want, cap_new = INPLACE_CASES[name]
+    n_exp = 1 + max(e for t in old for e in t)
+    sh = tiny_shape(n_routed=n_exp, n_layers=2)
+    m = sh.d_model * sh.d_ff * sh.elem_bytes
+    logical = logical_experts(sh, key=11)
+    arenas = slot_arenas(logical, old, 12)
+    for r in range(len(old), len(want)):          # added devices: fresh arenas
+        arenas.append(rand_bytes((13, r), sh.n_layers * 3 * cap_new[r] * m))
+    before = [a.copy() for a in arenas]
+    new = oracle.reshard_experts_inplace(sh, old, want, cap_new, arenas)
+    assert len(new) == len(want)
+    for r, table in enumerate(new):
+        assert len(table) == cap_new[r]
+        assert sorted(e for e in table if e >= 0) == sorted(want[r])
+        got = arenas[r].reshape(sh.n_layers, 3, cap_new[r], m)
+        was = before[r].reshape(sh.n_layers, 3, cap_new[r], m)
+        for s, e in enumerate(table):
+            if e >= 0:
+                assert np.array_equal(got[:, :, s], logical[:, :, e]), (r, s, e)
+                if r < len(old) and e in old[r]:
+                    assert old[r][s] == e                       # kept where it was
+                else:
+                    assert r >= len(old) or old[r][s] == -1     # arrivals use old-free slots only
+            else:
+                assert np.array_equal(got[:, :, s], was[:, :, s]), (r, s)   # untouched
+    for r in range(len(want), len(old)):          # removed devices are not written
+        assert np.array_equal(arenas[r], before[r])
+
+
+def test_inplace_arrivals_take_lowest_free_slots_in_listed_order():
+    old = [[7, -1, 3, -1, -1]]
+    # 9 and 8 have no source here; the table itself does not need one
+    assert oracle.inplace_slots(old, [[3, 9, 8]], [5]) == [[-1, 9, 3, 8, -1]]
+    assert oracle.inplace_slots(old, [[8, 9, 3]], [5]) == [[-1, 8, 3, 9, -1]]
+    assert oracle.inplace_slots(old, [[7, 3]], [5]) == old
+    assert oracle.inplace_slots(old, [[]], [5]) == [[-1] * 5]
+
+
+def test_inplace_refuses_what_the_capacity_cannot_hold():
+    with pytest.raises(ValueError, match="free slots"):
+        oracle.inplace_slots([[0, 1, -1]], [[2, 3]], [3])      # one free slot, two arrivals
+    with pytest.raises(ValueError, match="capacity"):
+        oracle.inplace_slots([[0, 1, -1]], [[0]], [4])         # a staying rank cannot grow
+    with pytest.raises(ValueError, match="twice"):
+        oracle.inplace_slots([[0, 1, -1]], [[0, 0]], [3])
+    sh = tiny_shape(n_routed=3, n_layers=1)
+    m = sh.d_model * sh.d_ff * sh.elem_bytes
+    with pytest.raises(ValueError, match="no copy"):
+        oracle.reshard_experts_inplace(sh, [[0, -1]], [[0, 2]], [2], [np.zeros(3 * 2 * m, np.uint8)])
+
+
+def test_inplace_source_is_the_smallest_rank_and_slot():
+    """Replicas with different contents: the arrival must carry the bytes of the smallest
+    (rank, slot) that held the expert before the step."""
+    sh = tiny_shape(n_layers=1, n_routed=2, d_model=2, d_ff=2, elem_bytes=1)
+    m = 4
+    old = [[-1, 1, 0], [1, -1, -1]]
+    tag = lambda r, s: 10 * r + s + 1
+    arenas = [np.repeat(np.array([[tag(r, s) for s in range(3)]] * 3, np.uint8).reshape(-1), m)
+              for r in range(2)]
+    arenas.append(np.zeros(3 * 2 * m, np.uint8))
+    new = oracle.reshard_experts_inplace(sh, old, [[0, 1], [1, 0], [1, 0]], [3, 3, 2], arenas)
+    assert new == [[-1, 1, 0], [1, 0, -1], [1, 0]]
+    a1 = arenas[1].reshape(3, 3, m)
+    assert set(a1[:, 1].reshape(-1)) == {tag(0, 2)}          # expert 0 came from rank 0 slot 2
+    a2 = arenas[2].reshape(3, 2, m)
+    assert set(a2[:, 0].reshape(-1)) == {tag(0, 1)}          # expert 1: rank 0 slot 1, not rank 1 slot 0
+    assert set(a2[:, 1].reshape(-1)) == {tag(0, 2)}
+
+
+def test_inplace_chain_reuses_slots_freed_by_the_previous_step():
+    """A slot freed in one step is available to arrivals of the NEXT step; compacted to the
+    wanted order, every step agrees with the out-of-place expert re-pack."""
+    sh = tiny_shape(n_routed=8, n_layers=2)
+    m = sh.d_model * sh.d_ff * sh.elem_bytes
+    logical = logical_experts(sh, key=21)
+    slots = [[0, 1, 2, 3, -1, -1], [4, 5, 6, 7, -1, -1]]
+    arenas = slot_arenas(logical, slots, 22)
+    steps = [([[0, 1, 4, 5], [6, 7, 2, 3]], [6, 6]),           # two arrivals each way
+             ([[0, 1, 4, 5, 3], [6, 7, 2]], [6, 6]),           # 3 comes back into a slot freed before
+             ([[0, 1], [6, 7], [2, 3, 4, 5]], [6, 6, 4]),      # grow
+             ([[0, 1, 2, 3, 4, 5], [6, 7]], [6, 6])]           # shrink again
+    for want, cap in steps:
+        while len(arenas) < len(want):
+            arenas.append(rand_bytes((23, len(arenas)), sh.n_layers * 3 * cap[len(arenas)] * m))
+        slots = oracle.reshard_experts_inplace(sh, slots, want, cap, arenas[:max(len(slots), len(want))])
+        arenas = arenas[:len(want)]
+        for r, table in enumerate(slots):
+            got = arenas[r].reshape(sh.n_layers, 3, len(table), m)
+            order = [table.index(e) for e in want[r]]
+            compact = np.ascontiguousarray(got[:, :, order]).reshape(-1)
+            assert np.array_equal(compact, expert_arenas(logical, [want[r]])[0])
+    assert slots == [[0, 1, 2, 3, 4, 5], [-1, -1, 6, 7, -1, -1]]      # worked out by hand
+
+
+@pytest.mark.parametrize("case", ["up", "down"])
+def test_inplace_paper_scenario_fixture(case):
+    """The paper's scale-up / scale-down scenario in its in-place form against hand-written
+    slot tables and a hand-written list of the only transfers the step may make."""
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "paper_scale_inplace.txt"))
+            if l.strip() and not l.startswith("#")]
+    want_slots = {int(r[2]): [int(x) for x in r[3:]] for r in rows if r[0] == "slots" and r[1] == case}
+    copies = [tuple(int(x) for x in r[2:]) for r in rows if r[0] == "copy" and r[1] == case]
+    if case == "up":
+        old = [[3 * r, 3 * r + 1, 3 * r + 2, -1] for r in range(4)]
+        want, cap = [[0, 1], [3, 2], [6, 5], [9, 8], [4, 7, 1], [10, 11]], [4] * 6
+    else:
+        old = [[0, 1, -1, -1], [3, -1, -1, 2], [6, 7, -1, 5], [9, 10, 11, 8]]
+        want, cap = [[0, 1, 6, 7], [3, 2, 9, 5]], [4, 4]
+    sh = tiny_shape(n_layers=2, d_model=2, d_ff=2, elem_bytes=2)
+    m = 8
+    n_dev = max(len(old), len(want))
+    tag = lambda r, s, l, p: 1 + ((r * 4 + s) * 3 + p) * 2 + l      # every slab its own byte value
+    arenas = []
+    for r in range(n_dev):
+        a = np.zeros((2, 3, 4, m), np.uint8)
+        for l in range(2):
+            for p in range(3):
+                for s in range(4):
+                    a[l, p, s] = tag(r, s, l, p)
+        arenas.append(a.reshape(-1))
+    new = oracle.reshard_experts_inplace(sh, old, want, cap, arenas)
+    assert new == [want_slots[r] for r in range(len(want))]
+    written = {(rn, sn): (ro, so) for rn, sn, e, ro, so in copies}
+    for rn, sn, e, ro, so in copies:
+        assert new[rn][sn] == e and old[ro][so] == e
+    for r in range(n_dev):
+        got = arenas[r].reshape(2, 3, 4, m)
+        for s in range(4):
+            ro, so = written.get((r, s), (r, s))                  # everything else is untouched
+            for l in range(2):
+                for p in range(3):
+                    assert set(got[l, p, s]) == {tag(ro, so, l, p)}, (r, s)
