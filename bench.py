@@ -33,13 +33,89 @@ METRIC = "reshard_gbs"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAK_GBS = 6650.0
-# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under
-# profiles/ (workload -> read + written bytes), or None while no capture covers it
-NCU_TRAFFIC = {
-    # whole step of a 2-layer cut (bulk launch 2.6139 + 2.5671 GB, the attention shard's vector
-    # launch 0.0677 + 0.0236 GB; at full size both are one bulk launch): x12 for 24 layers
-    "c2_mid": 12 * (2613877000 + 2567138000 + 67747000 + 23625000),
-}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic.json")
+KERNEL_SOURCES = [os.path.join(ROOT, "paper_2510_02613_b200", "csrc", f)
+                  for f in ("kernels.cu", "kernels.h", "capi.cpp", "planner.cpp", "planner.h")]
+
+
+def kernel_sources_sha() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
+def load_traffic():
+    """DRAM bytes per kernel from the ncu captures recorded in profiles/traffic.json (small
+    cuts of the workloads; see --record-traffic).  Returns {} when the kernel sources have
+    changed since the counters were taken: stale counters are not reported."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            t = json.load(f)
+    except Exception:
+        return {}
+    if t.get("kernel_sources_sha256") != kernel_sources_sha():
+        return {}
+    return t.get("captures", {})
+
+
+def traffic_per_launch(traffic, wl_name, kernel, full_layers):
+    """Read + written DRAM bytes of one launch of `kernel` at full size (kernel None: of all
+    kernels of one step): the capture's bytes scaled by layers (every layer has identical
+    units, so traffic grows in proportion)."""
+    cap = traffic.get(wl_name)
+    if not cap:
+        return None
+    ks = cap.get("kernels", {})
+    pick = list(ks.values()) if kernel is None else [ks[kernel]] if kernel in ks else []
+    if not pick:
+        return None
+    per = sum((k["dram_bytes_read"] + k["dram_bytes_write"]) / max(k["launches"], 1) for k in pick)
+    return int(per * full_layers / cap["layers"])
+
+
+def record_traffic(args):
+    """Parses an `ncu --page raw --csv` dump of a capture of `bench.py --only-main --workload W
+    --layers N` and stores the kernels' DRAM byte counters in profiles/traffic.json."""
+    import csv
+    rows = list(csv.reader(open(args.record_traffic, newline="")))
+    head = next(i for i, r in enumerate(rows) if "Kernel Name" in r)
+    cols = {n: i for i, n in enumerate(rows[head])}
+    units = rows[head + 1]
+    scale = {"byte": 1, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9, "Tbyte": 1e12}
+    kernels = {}
+    for r in rows[head + 2:]:
+        if len(r) <= cols["Kernel Name"]:
+            continue
+        name = r[cols["Kernel Name"]].split("(")[0].split("<")[0].split("::")[-1].strip()
+        k = kernels.setdefault(name, {"launches": 0, "dram_bytes_read": 0.0, "dram_bytes_write": 0.0,
+                                      "duration_us": 0.0})
+        k["launches"] += 1
+        for key, col in (("dram_bytes_read", "dram__bytes_read.sum"), ("dram_bytes_write", "dram__bytes_write.sum")):
+            k[key] += float(r[cols[col]].replace(",", "")) * scale[units[cols[col]]]
+        if "gpu__time_duration.sum" in cols:
+            c = cols["gpu__time_duration.sum"]
+            k["duration_us"] += float(r[c].replace(",", "")) * {"ns": 1e-3, "us": 1, "ms": 1e3, "s": 1e6}.get(units[c], 1)
+    try:
+        with open(TRAFFIC_FILE) as f:
+            t = json.load(f)
+    except Exception:
+        t = {}
+    sha = kernel_sources_sha()
+    if t.get("kernel_sources_sha256") != sha:
+        t = {"kernel_sources_sha256": sha, "captures": {}}
+    t["note"] = ("DRAM counters (dram__bytes_read.sum / dram__bytes_write.sum, summed over the captured "
+                 "launches) of small cuts of the workloads; bench.py scales them by layers and drops them "
+                 "when the kernel sources no longer hash to kernel_sources_sha256")
+    t["captures"][args.workload] = {"layers": args.layers, "command": args.traffic_command or "",
+                                    "kernels": {n: {k: (int(v) if k != "duration_us" else round(v, 1))
+                                                    for k, v in d.items()} for n, d in kernels.items()}}
+    with open(TRAFFIC_FILE, "w") as f:
+        json.dump(t, f, indent=1, sort_keys=True)
+        f.write("\n")
+    print(json.dumps(t["captures"][args.workload]))
 
 
 def measured_peak():
@@ -120,9 +196,11 @@ def one_step(plan, src, dst, stream):
     plan.reshard_step(src, dst, stream)
 
 
-def time_steps(torch, plan, src, dst, steps, warmup, stream, barrier=None):
-    """Total ms over `steps` whole steps (emoe_reshard_step, back to back), events recorded
-    on the stream the kernels are launched on."""
+def time_steps(torch, plan, src, dst, steps, warmup, stream, barrier=None, per_step=True):
+    """(total ms over `steps` whole steps, per-step ms list).  The steps run back to back
+    (emoe_reshard_step) between two events on the stream the kernels are launched on; with
+    per_step an event is also recorded between consecutive steps, so that the spread over
+    the region can be reported (median / min / max) beside the mean the total gives."""
     torch.cuda.synchronize()   # the arenas were filled on the default stream
     with torch.cuda.stream(stream):
         for _ in range(warmup):
@@ -131,14 +209,24 @@ def time_steps(torch, plan, src, dst, steps, warmup, stream, barrier=None):
         if barrier:
             barrier()
         torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(steps):
+        n_ev = steps + 1 if per_step else 2
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_ev)]
+        ev[0].record(stream)
+        for i in range(steps):
             one_step(plan, src, dst, stream)
-        e1.record(stream)
+            if per_step or i == steps - 1:
+                ev[i + 1 if per_step else 1].record(stream)
         stream.synchronize()
         torch.cuda.synchronize()
-    return e0.elapsed_time(e1)
+    each = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)] if per_step else []
+    return ev[0].elapsed_time(ev[-1]), each
+
+
+def step_spread(each):
+    if not each:
+        return None
+    return {"median_ms": round(statistics.median(each), 4), "min_ms": round(min(each), 4),
+            "max_ms": round(max(each), 4), "n": len(each)}
 
 
 def time_phases(torch, plan, src, dst, steps, stream):
@@ -178,7 +266,54 @@ def time_graph_steps(torch, plan, src, dst, steps, warmup, stream):
     return e0.elapsed_time(e1) / steps
 
 
-def config_report(E, plan, wl, total_ms, phase_ms, steps, peak, plan_ms):
+KERNEL_OF = {"ring_units": "bulk_copy_kernel", "vector_units": "vec_copy_kernel", "kv_tiles": "kv_rows_kernel"}
+
+
+def kernels_of(work):
+    """Names of the kernels a launch set consists of, from emoe_plan_launch_work."""
+    return [KERNEL_OF[k] for k in ("ring_units", "vector_units", "kv_tiles") if work[k]]
+
+
+def roofline_block(kernel, alg_bytes, ms, peak, peak_kind, traffic):
+    achieved = alg_bytes / (ms * 1e-3) / 1e9
+    return {"bound": "hbm", "kernel": kernel, "achieved": round(achieved, 1), "peak": peak,
+            "peak_kind": "of " + peak_kind, "unit": UNIT, "frac": round(achieved / peak, 4),
+            "frac_of_nominal_8000": round(achieved / NOMINAL_HBM_GBS, 4),
+            "algorithmic_bytes_per_launch": alg_bytes, "launch_ms": round(ms, 4), "traffic": traffic}
+
+
+def config_rooflines(E, plan, wl, step_ms, phase_ms, peak, peak_kind, traffic, full_layers, cut):
+    """One roofline block for the whole step and one per kernel.  Algorithmic bytes of a launch =
+    bytes_read + bytes_moved of what it covers (a source that feeds k destinations is read
+    once).  A kernel's duration: the step's, when the step is that one launch; otherwise the
+    phase that consists of that kernel alone, run through its own entry point (in a step the
+    launch sets overlap, so their durations cannot be told apart there)."""
+    st = [plan.stats(ph) for ph in range(3)]
+    alg = [x["bytes_moved"] + x["bytes_read"] for x in st]
+    work = plan.launch_work(E.PHASE_STEP)
+    names = kernels_of(work)
+    fused = plan.num_launches(E.PHASE_STEP) < len(names)     # vector work and KV tiles share a kernel
+    tr = (lambda k: None) if cut else (lambda k: traffic_per_launch(traffic, wl.name, k, full_layers))
+    out = {"step": roofline_block(" + ".join(names) + (" (vector and KV work in one kernel)" if fused else ""),
+                                  sum(alg), step_ms, peak, peak_kind, tr(None)),
+           "kernels": []}
+    if len(names) == 1:
+        out["kernels"].append(dict(out["step"], kernel=names[0], timed_as="the whole step (one launch)"))
+        return out
+    for ph, pname in enumerate(("experts", "attn", "kv")):
+        w = plan.launch_work(ph)
+        k = kernels_of(w)
+        if len(k) != 1 or phase_ms[ph] <= 0:
+            continue
+        b = roofline_block(k[0], alg[ph], phase_ms[ph], peak, peak_kind,
+                           tr(k[0]) if k[0] == "bulk_copy_kernel" and work["ring_units"] == w["ring_units"] else None)
+        b["timed_as"] = "the %s phase through its own entry point" % pname
+        out["kernels"].append(b)
+    return out
+
+
+def config_report(E, plan, wl, total_ms, each, phase_ms, steps, peak, peak_kind, plan_ms, traffic,
+                  cut=False):
     st = [plan.stats(ph) for ph in range(3)]
     moved = sum(s["bytes_moved"] for s in st)
     read = sum(s["bytes_read"] for s in st)
@@ -187,7 +322,7 @@ def config_report(E, plan, wl, total_ms, phase_ms, steps, peak, plan_ms):
     names = ["experts", "attn", "kv"]
     return {
         "workload": wl.name, "reconfig": wl.notes, "bytes_moved": moved, "bytes_read": read,
-        "scale_step_ms": round(ms, 4), "reshard_gbs": round(gbs, 1),
+        "scale_step_ms": round(ms, 4), "step_spread": step_spread(each), "reshard_gbs": round(gbs, 1),
         "pct_of_nominal_8000": round(100 * gbs / NOMINAL_HBM_GBS, 2),
         "pct_of_measured_peak": round(100 * gbs / peak, 2),
         "algorithmic_min_gbs": round((moved + read) / (ms * 1e-3) / 1e9, 1),
@@ -198,6 +333,8 @@ def config_report(E, plan, wl, total_ms, phase_ms, steps, peak, plan_ms):
                        "bytes_moved": st[k]["bytes_moved"], "segments": st[k]["n_segments"],
                        "launches": plan.num_launches(k)} for k, n in enumerate(names)},
         "launches_per_step": plan.num_launches(E.PHASE_STEP),
+        "roofline": config_rooflines(E, plan, wl, ms, phase_ms, peak, peak_kind, traffic,
+                                     wl.shape.n_layers, cut),
     }
 
 
@@ -325,22 +462,34 @@ def run_e2e(torch, plan, src, dst, steps, stream):
 
 # ---- C5: reshard on a low-priority stream beside a grouped expert GEMM -------------------
 
-def run_overlap(torch, E, plan, wl, src, dst, peak, budgets=(0, 96, 48, 24)):
+OVERLAP_POINTS = (
+    dict(), dict(max_ctas=96), dict(max_ctas=48), dict(max_ctas=24),
+    dict(bw_limit_gbs=5500), dict(bw_limit_gbs=4500), dict(bw_limit_gbs=3500), dict(bw_limit_gbs=2500),
+    dict(bw_limit_gbs=1500), dict(bw_limit_gbs=3500, bulk_stages=3), dict(bw_limit_gbs=3500, bulk_hints=2),
+    dict(max_ctas=48, bw_limit_gbs=2500), dict(max_ctas=37, bulk_stages=3, bw_limit_gbs=2500),
+)
+
+
+def run_overlap(torch, E, plan, wl, src, dst, peak, victim, points=OVERLAP_POINTS, verify=True):
     """Victim: 8 active experts x 256 tokens (top-8 routing: every active expert sees all
     tokens), gate/up/down bf16 batched GEMMs (torch.bmm, a measurement fixture, not part
-    of the library) on a high-priority stream, weights taken from the old expert arena of
-    rank 0, the layer cycling per step."""
-    v = wl.victim
+    of the library) on a high-priority stream, CUDA-graph replayed; the reshard runs on a
+    least-priority stream.  Weights are taken from the old expert arena of rank 0 when the
+    shapes agree (the layer cycling per step), else from a buffer of their own.  Every
+    point of `points` is one launch tuning: the trade-off curve victim slowdown against
+    reshard bandwidth."""
+    v = victim
     A, T, D, F = v["active_experts"], v["tokens"], v["d_model"], v["d_ff"]
     L = wl.shape.n_layers
-    arena = src[0][0].view(torch.bfloat16)
-    n_slots = len(wl.old.placement[0])
-    m = D * F
-    slab = arena.view(L, 3, n_slots, m)
-    lo, hi = torch.cuda.Stream.priority_range()[1], torch.cuda.Stream.priority_range()[0]
-    lo, hi = max(lo, hi), min(lo, hi)          # numerically larger = lower priority
-    s_main = torch.cuda.Stream(priority=hi)
-    s_low = torch.cuda.Stream(priority=lo)
+    if D == wl.shape.d_model and F == wl.shape.d_ff and len(wl.old.placement[0]) >= A:
+        slab = src[0][0].view(torch.bfloat16).view(L, 3, len(wl.old.placement[0]), D * F)
+        n_l = L
+    else:
+        n_l = 4        # 4 x 138 MB of weights: larger than L2
+        slab = (torch.randn(n_l, 3, A, D * F, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+    least, greatest = torch.cuda.Stream.priority_range()
+    s_main = torch.cuda.Stream(priority=greatest)
+    s_low = torch.cuda.Stream(priority=least)
     x = (torch.randn(A, T, D, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
     n_graph_steps = 8
 
@@ -353,12 +502,12 @@ def run_overlap(torch, E, plan, wl, src, dst, peak, budgets=(0, 96, 48, 24)):
 
     with torch.cuda.stream(s_main):
         for l in range(3):
-            gemm_step(l)
+            gemm_step(l % n_l)
         s_main.synchronize()
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=s_main):
             for i in range(n_graph_steps):
-                gemm_step(i % L)
+                gemm_step(i % n_l)
     torch.cuda.synchronize()
 
     def gemm_loop(n_replays):
@@ -375,16 +524,25 @@ def run_overlap(torch, E, plan, wl, src, dst, peak, budgets=(0, 96, 48, 24)):
     torch.cuda.synchronize()
     alone_us = statistics.median(evs[i].elapsed_time(evs[i + 1]) for i in range(5, 40)) \
         / n_graph_steps * 1e3
-    moved = sum(plan.stats(ph)["bytes_moved"] for ph in range(3))
+    st = [plan.stats(ph) for ph in range(3)]
+    moved = sum(x_["bytes_moved"] for x_ in st)
+    alg = sum(x_["bytes_moved"] + x_["bytes_read"] for x_ in st)
+    weight_bytes = 3 * A * D * F * 2
+    victim_gbs = weight_bytes / alone_us / 1e3
     out = {"victim": "torch.bmm grouped expert GEMM, %d experts x %d tokens, d_model %d, d_ff %d"
-                     % (A, T, D, F), "victim_alone_us_per_step": round(alone_us, 2), "runs": []}
-    for budget in budgets:
-        plan.set_tuning(max_ctas=budget)
+                     % (A, T, D, F), "victim_alone_us_per_step": round(alone_us, 2),
+           "victim_weight_bytes_per_step": weight_bytes, "victim_alone_gbs": round(victim_gbs, 1),
+           "runs": []}
+    hbm_total = None
+    for tuning in points:
+        plan.set_tuning(**tuning)
         # reshard alone on the low-priority stream
         r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         one_step(plan, src, dst, s_low); s_low.synchronize()
         r0.record(s_low); one_step(plan, src, dst, s_low); r1.record(s_low); s_low.synchronize()
         alone_ms = r0.elapsed_time(r1)
+        if hbm_total is None:
+            hbm_total = alg / alone_ms / 1e6       # what the unconstrained reshard gets out of HBM
         # overlapped: enough victim replays to cover the reshard
         n_rep = int(alone_ms * 1e3 / (alone_us * n_graph_steps) * 2.5) + 20
         torch.cuda.synchronize()
@@ -395,21 +553,54 @@ def run_overlap(torch, E, plan, wl, src, dst, peak, budgets=(0, 96, 48, 24)):
         torch.cuda.synchronize()
         both_ms = r0.elapsed_time(r1)
         # victim replays that ended while the reshard was still running
-        t_end = both_ms
         inside = [evs[i].elapsed_time(evs[i + 1]) for i in range(n_rep)
-                  if r0.elapsed_time(evs[i + 1]) < t_end and r0.elapsed_time(evs[i]) > 0]
+                  if r0.elapsed_time(evs[i + 1]) < both_ms and r0.elapsed_time(evs[i]) > 0]
         during_us = (statistics.mean(inside) / n_graph_steps * 1e3) if inside else None
+        alg_gbs = alg / both_ms / 1e6
+        # if the two only competed for HBM bytes, the victim would keep what the reshard leaves
+        left = max(hbm_total - alg_gbs, 1.0)
         out["runs"].append({
-            "max_ctas": budget or "default",
+            "tuning": tuning or "default",
             "reshard_alone_ms": round(alone_ms, 3),
             "reshard_alone_gbs": round(2 * moved / alone_ms / 1e6, 1),
             "reshard_overlapped_ms": round(both_ms, 3),
             "reshard_overlapped_gbs": round(2 * moved / both_ms / 1e6, 1),
+            "reshard_overlapped_hbm_gbs": round(alg_gbs, 1),
             "victim_us_per_step_during": round(during_us, 2) if during_us else None,
             "victim_slowdown": round(during_us / alone_us, 3) if during_us else None,
+            "slowdown_if_only_hbm_bytes_were_shared": round(max(1.0, victim_gbs / left), 3),
             "victim_replays_inside": len(inside)})
+    out["hbm_gbs_of_unconstrained_reshard"] = round(hbm_total, 1)
+    ok = [r for r in out["runs"] if r["victim_slowdown"] and r["victim_slowdown"] <= 1.5]
+    best = max(ok, key=lambda r: r["reshard_overlapped_gbs"]) if ok else None
+    out["best_with_victim_within_1p5x"] = ({"tuning": best["tuning"], "victim_slowdown": best["victim_slowdown"],
+                                            "reshard_overlapped_gbs": best["reshard_overlapped_gbs"]}
+                                           if best else None)
     plan.set_tuning()
+    if verify:
+        # harness check, outside every timed part: layer 0 of what the LAST overlapped run wrote,
+        # against the CPU oracle run on that layer alone (layers are independent)
+        out["overlapped_output_matches_oracle_layer0"] = verify_layer(torch, E, plan, wl, src, dst, 0)
     return out
+
+
+def verify_layer(torch, E, plan, wl, src, dst, layer):
+    import oracle
+    wl1 = wl.with_layers(1)
+    L = wl.shape.n_layers
+    ok = True
+    for ph in range(3):
+        h_src = [t[layer * (t.numel() // L):(layer + 1) * (t.numel() // L)].cpu().numpy() for t in src[ph]]
+        got = [t[layer * (t.numel() // L):(layer + 1) * (t.numel() // L)].cpu().numpy() for t in dst[ph]]
+        want = [g.copy() for g in got]       # bytes the step does not write must stay as they are
+        if ph == 0:
+            oracle.reshard_experts(wl1.shape, wl.old.placement, wl.new.placement, h_src, want)
+        elif ph == 1:
+            oracle.reshard_attn(wl1.shape, wl.old.tp, wl.new.tp, h_src, want)
+        else:
+            oracle.reshard_kv(wl1.shape, wl.old, wl.new, h_src, want)
+        ok = ok and all(np.array_equal(g, w) for g, w in zip(got, want))
+    return bool(ok)
 
 
 # ---- paged expert store: the expert phase as a page re-map plus copies of arrivals -------
@@ -480,7 +671,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c2_mid")
     ap.add_argument("--impl", default="emoe", choices=["emoe", "reference"])
@@ -490,8 +681,17 @@ def main():
     ap.add_argument("--layers", type=int, default=None,
                     help="cut the workload to this many layers (for small profiler captures "
                          "only: the result is then not the named configuration)")
+    ap.add_argument("--steps-only", action="store_true",
+                    help="with --only-main: run nothing but the warm-up and the timed steps (for profiler captures)")
+    ap.add_argument("--record-traffic", default=None, metavar="NCU_RAW_CSV",
+                    help="do not run: parse `ncu -i X.ncu-rep --page raw --csv` of a capture of "
+                         "`bench.py --only-main --steps-only --workload W --layers N` into profiles/traffic.json")
+    ap.add_argument("--traffic-command", default=None, help="the capture's command line, stored with --record-traffic")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "emoe" else args.warmup
+    if args.record_traffic:
+        record_traffic(args)
+        return
 
     if args.impl == "reference":
         run_reference(args)
@@ -527,13 +727,18 @@ def main():
     tiny = W.make_workload("c1_tiny")        # loads the CUDA module, so that plan times below are the planner's
     E.Plan(tiny.shape, tiny.old, tiny.new).close()
     wl, plan, src, dst, plan_ms = setup(args.workload, torch, E, W, WD, n_layers=args.layers)
+    traffic = load_traffic()
     sampler = ClockSampler(local)
     sampler.start()
-    total_ms = time_steps(torch, plan, src, dst, args.steps, args.warmup, stream, barrier)
+    total_ms, each = time_steps(torch, plan, src, dst, args.steps, args.warmup, stream, barrier)
     clocks = sampler.stop()
-    phase_ms = time_phases(torch, plan, src, dst, max(3, min(args.steps, 20)), stream)
+    if args.steps_only:
+        phase_ms = [0.0, 0.0, 0.0]
+    else:
+        phase_ms = time_phases(torch, plan, src, dst, max(3, min(args.steps, 20)), stream)
     total_ms = replicas.job_time_ms(total_ms, dist, device="cuda" if backend == "nccl" else "cpu")  # max over ranks
-    rep = config_report(E, plan, wl, total_ms, phase_ms, args.steps, peak, plan_ms)
+    rep = config_report(E, plan, wl, total_ms, each, phase_ms, args.steps, peak, peak_kind, plan_ms, traffic,
+                        cut=args.layers is not None)
     if plan.device_status() != 0:
         raise SystemExit("device status word set: a bounded wait expired")
     ms = total_ms / args.steps
@@ -541,25 +746,11 @@ def main():
     per_step = plan.num_launches(E.PHASE_STEP)
     launches = per_step * args.steps
 
-    # roofline of the dominant kernel, the bulk-copy launch.  When the whole step is that one
-    # launch (TP kept: every segment of every phase is a long run), its duration is the step
-    # time of the timed region; otherwise the expert phase run on its own stands in.
-    st_all = [plan.stats(ph) for ph in range(3)]
-    if per_step == 1:
-        alg_bytes = sum(x["bytes_moved"] + x["bytes_read"] for x in st_all)
-        launch_ms, what = ms, "bulk_copy_kernel (whole step: experts + attention + KV in one launch)"
-    else:
-        alg_bytes = st_all[0]["bytes_moved"] + st_all[0]["bytes_read"]
-        small = alg_bytes < (512 << 20)     # small phases are routed to the vector kernel whole
-        launch_ms = phase_ms[0]
-        what = ("vec_copy_kernel" if small else "bulk_copy_kernel") + " (expert re-pack, timed as its own call)"
-    achieved = alg_bytes / (launch_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": what,
-                "achieved": round(achieved, 1), "peak": peak, "peak_kind": "of " + peak_kind,
-                "unit": UNIT, "frac": round(achieved / peak, 4),
-                "algorithmic_bytes_per_launch": alg_bytes,
-                "launch_ms": round(launch_ms, 4),
-                "traffic": NCU_TRAFFIC.get(wl.name) if per_step == 1 and args.layers is None else None}
+    # roofline of the dominant kernel, the ring-copy launch: the whole step when the step is
+    # that one launch (TP kept: every segment of every phase is a long run), otherwise the
+    # kernel block timed through the expert phase's own entry point
+    blocks = rep["roofline"]["kernels"]
+    roofline = next((b for b in blocks if b["kernel"] == "bulk_copy_kernel"), None) or rep["roofline"]["step"]
 
     line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 4),
@@ -569,10 +760,11 @@ def main():
                        else "%s cut to %d layers" % (wl.name, args.layers),
                        "reconfig": wl.notes, "parallelism": "replicas",
                        "l2": "inputs_larger_than_l2", "value_convention": "2 x bytes moved / time",
-                       "scale_step_ms": rep["scale_step_ms"],
+                       "scale_step_ms": rep["scale_step_ms"], "step_spread": rep["step_spread"],
                        "pct_of_nominal_8000": rep["pct_of_nominal_8000"],
                        "pct_of_measured_peak": rep["pct_of_measured_peak"]},
             "clocks": clocks, "gpu_launches": launches, "roofline": roofline,
+            "roofline_step": rep["roofline"]["step"],
             "phases": rep["phases"], "planner_ms": rep["planner_ms"]}
 
     if rank == 0 and not args.only_main:
@@ -613,16 +805,22 @@ def main():
                 others[name] = rep
                 continue
             wl2, plan2, src2, dst2, pms = setup(name, torch, E, W, WD)
-            k = max(5, args.steps // 2) if name != "c1_tiny" else 200
-            tot = time_steps(torch, plan2, src2, dst2, k, 3, stream)
-            ph = time_phases(torch, plan2, src2, dst2, max(3, min(k, 20)), stream)
-            r = config_report(E, plan2, wl2, tot, ph, k, peak, pms)
+            # at least 100 steps and about a second of timed region each; the tiny config is
+            # timed without per-step events (an event costs a tenth of its step)
+            k = {"c1_tiny": 2000}.get(name, max(100, args.steps // 2))
+            tot, each2 = time_steps(torch, plan2, src2, dst2, k, 3, stream, per_step=name != "c1_tiny")
+            ph = time_phases(torch, plan2, src2, dst2, 20, stream)
+            r = config_report(E, plan2, wl2, tot, each2, ph, k, peak, peak_kind, pms, traffic)
             if name == "c1_tiny":    # launch-bound: also as a CUDA-graph replay
                 g_ms = time_graph_steps(torch, plan2, src2, dst2, k, 3, stream)
                 r["cuda_graph"] = {"scale_step_ms": round(g_ms, 4),
                                    "reshard_gbs": round(2 * r["bytes_moved"] / g_ms / 1e6, 1)}
             if name == "c5_overlap":
-                r["overlap"] = run_overlap(torch, E, plan2, wl2, src2, dst2, peak)
+                r["overlap"] = run_overlap(torch, E, plan2, wl2, src2, dst2, peak, wl2.victim)
+            if name == "c4_large":   # the same victim beside the TP-changing reshard
+                r["overlap"] = run_overlap(torch, E, plan2, wl2, src2, dst2, peak,
+                                           W.make_workload("c5_overlap").victim,
+                                           points=(dict(), dict(bw_limit_gbs=4500), dict(bw_limit_gbs=2500)))
             others[name] = r
             del src2, dst2
             plan2.close()

@@ -10,9 +10,10 @@
  * its experts as one contiguous tensor (Sec. 4.1 "Virtual Expert
  * Management", App. D.5).  The paper keeps TP fixed and remaps pages instead
  * of copying; it names the copy-based reshaping as the naive alternative
- * (Sec. 4.1) and TP change with KV reshaping as future work (Sec. 9).  This
- * library implements that copy-based, TP-changing re-layout on ONE GPU,
- * where every "rank" is a distinct region ("arena") of that GPU's memory.
+ * (Sec. 4.1) and TP change with KV reshaping as future work (App. C
+ * "Limitations and Future Work").  This library implements that copy-based,
+ * TP-changing re-layout on ONE GPU, where every "rank" is a distinct region
+ * ("arena") of that GPU's memory.
  *
  * All sizes and offsets are in BYTES unless a name says otherwise.  The
  * library never interprets element values; `elem_bytes` only scales sizes.
@@ -173,7 +174,7 @@ emoe_status_t emoe_reshard_experts(const emoe_plan_t *plan, const void *const *s
 /*
  * emoe_reshard_attn - attention q/k/v/o re-slice TP=c -> TP=d (Sec. 2.1:
  * TP shards the attention operations; Sec. 5.2 "Attention Weights" is the
- * c == d case, a whole-tensor copy onto added devices; Sec. 9 names c != d
+ * c == d case, a whole-tensor copy onto added devices; App. C names c != d
  * as future work).  q/k/v are split by stored rows (heads), o by stored
  * columns (heads).  src: [tp_old] device pointers, dst: [tp_new]; otherwise
  * as emoe_reshard_experts.
@@ -183,7 +184,7 @@ emoe_status_t emoe_reshard_attn(const emoe_plan_t *plan, const void *const *src,
 
 /*
  * emoe_reshard_kv - paged KV cache head re-split and re-paging (Sec. 5.2
- * "KV Cache" is the c == d, same-table case; Sec. 9 "reshaping KV caches").
+ * "KV Cache" is the c == d, same-table case; App. C "reshaping KV caches").
  *
  * For every sequence s, block index j < ceil(seq_len/B), layer, K|V, token
  * slot and global KV head g, head_dim elements move from old rank
@@ -291,6 +292,59 @@ emoe_status_t emoe_reshard_step_host(const emoe_plan_t *plan, const void *const 
 emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *plan, const void *const *src,
                                      void *const *dst, void *cuda_stream);
 
+/* ---- in-place expert step: only arrivals move -------------------------------
+ *
+ * The paper's expert step leaves what a device already holds where it is and
+ * transfers only the experts that arrive (Sec. 4.1 "Virtual Expert
+ * Management", Sec. 5.2 "Expert Weights", App. D.5; App. E for scale-down).
+ * This is that step for DENSE arenas with spare capacity - no page re-mapping:
+ *
+ *   arena of device r:  [L][3 (gate, up, down)][cap_r][m bytes],
+ *   slot table of device r: cap_r entries, an expert id or -1 (free).
+ *
+ * An expert that device r holds and still wants keeps its slot and is not
+ * touched.  An arrival is copied from the smallest (device, slot) that held it
+ * before the step into the lowest slot of r that was FREE BEFORE the step,
+ * arrivals being served in the order want_ids lists them.  A slot whose expert
+ * is no longer wanted becomes free in the new table, but its bytes stay: the
+ * old instance keeps serving from them until the switch-over (Sec. 5.2), and
+ * only a later step may reuse the slot.  So no byte that anything still reads
+ * is ever overwritten, and source and destination may be the same arena.
+ *
+ * emoe_plan_create_inplace
+ *   slot_off_old [ep_old+1], slot_ids_old: CSR slot tables before the step
+ *     (capacity of device r = slot_off_old[r+1] - slot_off_old[r]).
+ *   cap_new [ep_new]: capacities after the step; for r < ep_old it must equal the
+ *     old capacity (the device keeps its arena), for an added device it is free.
+ *   want_off [ep_new+1], want_ids: the experts every device must hold afterwards.
+ *   flags: 0 or EMOE_PLAN_HOST_ONLY.
+ *   Errors: EMOE_ERR_PLACEMENT (id out of range, an expert twice in one table or
+ *   one want list, a wanted expert nobody holds), EMOE_ERR_TOO_LARGE (a device
+ *   has fewer slots free before the step than arrivals), EMOE_ERR_INVALID_ARG
+ *   (a staying device's capacity differs), EMOE_ERR_UNSUPPORTED (too many ranks).
+ *   The plan answers emoe_plan_stats / _arena_bytes / _num_launches / _segments for
+ *   EMOE_PHASE_EXPERTS (bytes_moved = arrivals only; arena sizes by capacity) and
+ *   takes emoe_plan_set_tuning / _set_local_rank; it has no attention or KV phase
+ *   and the out-of-place reshard calls reject it with EMOE_ERR_INVALID_ARG.
+ *
+ * emoe_plan_slot_table: the slot table of `rank` after the step (up to `cap`
+ *   entries into `out`, the table's length into *n_slots).
+ *
+ * emoe_reshard_experts_inplace: arenas = HOST array of max(ep_old, ep_new)
+ *   DEVICE pointers, arena r serving as source (r < ep_old) and as destination
+ *   (r < ep_new).  16-byte aligned; arenas of different devices must not
+ *   intersect.  Enqueues on cuda_stream only, like emoe_reshard_experts.
+ */
+emoe_status_t emoe_plan_create_inplace(const emoe_shape_t *shape, int32_t ep_old,
+                                       const int32_t *slot_off_old, const int32_t *slot_ids_old,
+                                       int32_t ep_new, const int32_t *cap_new,
+                                       const int32_t *want_off, const int32_t *want_ids,
+                                       uint32_t flags, emoe_plan_t **out);
+emoe_status_t emoe_plan_slot_table(const emoe_plan_t *plan, int32_t rank, int32_t *out, int32_t cap,
+                                   int32_t *n_slots);
+emoe_status_t emoe_reshard_experts_inplace(const emoe_plan_t *plan, void *const *arenas,
+                                           void *cuda_stream);
+
 /* ---- paged expert store: re-layout by re-mapping pages ---------------------
  *
  * The paper's own expert mechanism (Sec. 4.1 "Virtual Expert Management",
@@ -388,6 +442,14 @@ emoe_status_t emoe_plan_stats(const emoe_plan_t *plan, int phase, uint64_t *byte
 /* Kernel launches one reshard call of this phase enqueues with the current tuning. */
 emoe_status_t emoe_plan_num_launches(const emoe_plan_t *plan, int phase, int32_t *n);
 
+/* Work items one reshard call of this phase (or EMOE_PHASE_STEP: one emoe_reshard_step
+ * call) hands to each kind of kernel with the current tuning: units of the ring kernel
+ * (cp.async.bulk through shared memory), units of the vector kernel, tiles of the KV head
+ * re-split (0 when the head split is kept: whole blocks then move as ring or vector units).
+ * NULL outputs are skipped.  For reports: which kernels a launch set consists of. */
+emoe_status_t emoe_plan_launch_work(const emoe_plan_t *plan, int phase, uint64_t *ring_units,
+                                    uint64_t *vector_units, uint64_t *kv_tiles);
+
 /* One coalesced copy descriptor, as exported for inspection and host-side
  * replay: n_runs runs of run_bytes each; run i reads
  * src[src_rank] + src_off + i*src_pitch and writes
@@ -410,6 +472,11 @@ emoe_status_t emoe_plan_segments(const emoe_plan_t *plan, int phase, emoe_segmen
  * the caller has synchronised the stream(s) the plan ran on. */
 emoe_status_t emoe_plan_device_status(const emoe_plan_t *plan, int32_t *status);
 
+/* Clears the status word after an EMOE_ERR_DEVICE_TIMEOUT has been read; the plan is
+ * usable again (the launch that timed out has left its destination undefined).  Call it
+ * with none of the plan's launches in flight. */
+emoe_status_t emoe_plan_clear_device_status(emoe_plan_t *plan);
+
 /* Launch tuning.  Fields set to 0 keep the library default. */
 typedef struct {
   int32_t max_ctas;        /* upper bound on CTAs per launch (SM budget when the    */
@@ -428,6 +495,20 @@ typedef struct {
   int32_t unit_order;      /* bulk work order: 0 default (run-major: one layer slab or  */
                            /* KV pool at a time), 1 segment-major; +2: CTAs take units  */
                            /* round-robin instead of claiming them from a counter       */
+  int32_t wait_limit_us;   /* bound of every device-side wait in microseconds (default  */
+                           /* 4 s).  -1: a wait that is not already satisfied when it   */
+                           /* is first polled expires at once - for exercising the      */
+                           /* time-out path; such a launch returns normally, sets the   */
+                           /* status word and leaves its destination undefined          */
+  int32_t bw_limit_gbs;    /* bandwidth limit of the ring kernel in GB/s of bytes read  */
+                           /* plus bytes written (its CTAs space their loads so that    */
+                           /* the launch as a whole stays near it); 0 = none.  For a    */
+                           /* reshard that shares HBM with a live kernel                */
+  int32_t bulk_min_run;    /* 16-byte-aligned runs of at least this many bytes go to    */
+                           /* the ring kernel (default 16384; a multiple of 16)         */
+  int32_t serial;          /* emoe_reshard_step: 1 = its launch sets run one after the  */
+                           /* other on the caller's stream; 2 = also keep the vector    */
+                           /* work and the KV head re-split in separate kernels         */
 } emoe_tuning_t;
 
 /* Replaces the plan's launch tuning.  Not thread-safe against reshard calls

@@ -54,7 +54,8 @@ class _Segment(ctypes.Structure):
 class _Tuning(ctypes.Structure):
     _fields_ = [("max_ctas", _i32), ("bulk_tile_bytes", _i32), ("bulk_stages", _i32),
                 ("path", _i32), ("kv_mode", _i32), ("bulk_hints", _i32), ("kv_order", _i32),
-                ("unit_order", _i32)]
+                ("unit_order", _i32), ("wait_limit_us", _i32), ("bw_limit_gbs", _i32),
+                ("bulk_min_run", _i32), ("serial", _i32)]
 
 
 class _VmmStats(ctypes.Structure):
@@ -69,10 +70,13 @@ SEGMENT_DTYPE = np.dtype([("src_off", "<u8"), ("dst_off", "<u8"), ("run_bytes", 
                           ("src_rank", "<u4"), ("dst_rank", "<u4"), ("group", "<u4")])
 
 EXPORTS = ("emoe_plan_create", "emoe_reshard_experts", "emoe_reshard_attn", "emoe_reshard_kv",
-           "emoe_reshard_kv_static", "emoe_reshard_step",
+           "emoe_reshard_kv_static", "emoe_reshard_step", "emoe_plan_create_inplace",
+           "emoe_plan_slot_table", "emoe_reshard_experts_inplace",
            "emoe_reshard_step_host", "emoe_plan_destroy", "emoe_plan_num_ranks",
-           "emoe_plan_arena_bytes", "emoe_plan_stats", "emoe_plan_num_launches", "emoe_plan_segments",
-           "emoe_plan_device_status", "emoe_plan_set_tuning", "emoe_strerror",
+           "emoe_plan_arena_bytes", "emoe_plan_stats", "emoe_plan_num_launches", "emoe_plan_launch_work",
+           "emoe_plan_segments",
+           "emoe_plan_device_status", "emoe_plan_clear_device_status", "emoe_plan_set_tuning",
+           "emoe_strerror",
            "emoe_place_min_transfer", "emoe_plan_set_local_rank", "emoe_ipc_export", "emoe_ipc_open", "emoe_ipc_close",
            "emoe_vmm_create", "emoe_vmm_reshard", "emoe_vmm_dry_run", "emoe_vmm_num_ranks", "emoe_vmm_arena",
            "emoe_vmm_write", "emoe_vmm_read", "emoe_vmm_destroy")
@@ -91,11 +95,11 @@ def lib() -> ctypes.CDLL:
         return _lib
     path = _build.OUT
     if _build.is_stale():
-        try:
-            _build.build()
-        except Exception as e:  # no nvcc on this machine: use the shipped binary if there is one
-            if not os.path.exists(path):
-                raise RuntimeError("libemoe.so is missing and could not be built: %s" % e) from e
+        if _build.have_nvcc():
+            _build.build()      # a failed compile raises: a stale binary is never used in its place
+        elif not os.path.exists(path):
+            raise RuntimeError("libemoe.so is missing and there is no nvcc to build it with")
+        # no nvcc on this machine: the shipped binary is all there is
     L = ctypes.CDLL(path)
     PP = ctypes.POINTER(_vp)
     L.emoe_plan_create.restype = _i32
@@ -106,6 +110,13 @@ def lib() -> ctypes.CDLL:
         f = getattr(L, name)
         f.restype = _i32
         f.argtypes = [_vp, PP, PP, _vp]
+    L.emoe_plan_create_inplace.restype = _i32
+    L.emoe_plan_create_inplace.argtypes = [ctypes.POINTER(_Shape), _i32, _i32p, _i32p, _i32, _i32p, _i32p,
+                                           _i32p, _u32, ctypes.POINTER(_vp)]
+    L.emoe_plan_slot_table.restype = _i32
+    L.emoe_plan_slot_table.argtypes = [_vp, _i32, _i32p, _i32, _i32p]
+    L.emoe_reshard_experts_inplace.restype = _i32
+    L.emoe_reshard_experts_inplace.argtypes = [_vp, PP, _vp]
     L.emoe_reshard_step.restype = _i32
     L.emoe_reshard_step.argtypes = [_vp, ctypes.POINTER(PP), ctypes.POINTER(PP), _vp]
     L.emoe_reshard_step_host.restype = _i32
@@ -121,10 +132,14 @@ def lib() -> ctypes.CDLL:
     L.emoe_plan_stats.argtypes = [_vp, _i32] + [ctypes.POINTER(_u64)] * 3
     L.emoe_plan_num_launches.restype = _i32
     L.emoe_plan_num_launches.argtypes = [_vp, _i32, ctypes.POINTER(_i32)]
+    L.emoe_plan_launch_work.restype = _i32
+    L.emoe_plan_launch_work.argtypes = [_vp, _i32] + [ctypes.POINTER(_u64)] * 3
     L.emoe_plan_segments.restype = _i32
     L.emoe_plan_segments.argtypes = [_vp, _i32, _vp, _u64, ctypes.POINTER(_u64)]
     L.emoe_plan_device_status.restype = _i32
     L.emoe_plan_device_status.argtypes = [_vp, ctypes.POINTER(_i32)]
+    L.emoe_plan_clear_device_status.restype = _i32
+    L.emoe_plan_clear_device_status.argtypes = [_vp]
     L.emoe_plan_set_tuning.restype = _i32
     L.emoe_plan_set_tuning.argtypes = [_vp, ctypes.POINTER(_Tuning)]
     L.emoe_place_min_transfer.restype = _i32
@@ -282,6 +297,13 @@ class Plan:
         _check(lib().emoe_plan_num_launches(self._h, phase, ctypes.byref(n)))
         return n.value
 
+    def launch_work(self, phase: int) -> dict:
+        """Work items per kind of kernel for one call of this phase (PHASE_STEP: a whole step)."""
+        a, b, c = _u64(), _u64(), _u64()
+        _check(lib().emoe_plan_launch_work(self._h, phase, ctypes.byref(a), ctypes.byref(b),
+                                           ctypes.byref(c)))
+        return dict(ring_units=a.value, vector_units=b.value, kv_tiles=c.value)
+
     def segments(self, phase: int) -> np.ndarray:
         n = _u64()
         _check(lib().emoe_plan_segments(self._h, phase, None, 0, ctypes.byref(n)))
@@ -296,11 +318,15 @@ class Plan:
         _check(lib().emoe_plan_device_status(self._h, ctypes.byref(s)))
         return s.value
 
+    def clear_device_status(self) -> None:
+        _check(lib().emoe_plan_clear_device_status(self._h))
+
     def set_tuning(self, max_ctas: int = 0, bulk_tile_bytes: int = 0, bulk_stages: int = 0,
                    path: int = 0, kv_mode: int = 0, bulk_hints: int = 0, kv_order: int = 0,
-                   unit_order: int = 0) -> None:
+                   unit_order: int = 0, wait_limit_us: int = 0, bw_limit_gbs: int = 0,
+                   bulk_min_run: int = 0, serial: int = 0) -> None:
         t = _Tuning(max_ctas, bulk_tile_bytes, bulk_stages, path, kv_mode, bulk_hints, kv_order,
-                    unit_order)
+                    unit_order, wait_limit_us, bw_limit_gbs, bulk_min_run, serial)
         _check(lib().emoe_plan_set_tuning(self._h, ctypes.byref(t)))
 
     def set_local_rank(self, rank: int) -> None:
@@ -349,6 +375,49 @@ class Plan:
 
         _check(lib().emoe_reshard_step_host(self._h, pack(h_src), pack(h_dst), pack(d_src),
                                             pack(d_dst), _stream_handle(stream)))
+
+
+class InplacePlan(Plan):
+    """The expert step on capacity-strided arenas: emoe_plan_create_inplace.  old_slots: per
+    old device a list of expert ids or -1 (free), as long as the device's capacity; want:
+    per new device the experts it must hold; cap_new: capacity per new device."""
+
+    def __init__(self, shape, old_slots, want, cap_new, host_only: bool = False):
+        self._h = _vp()
+        sh = _Shape(shape.n_layers, shape.n_routed, shape.n_shared, shape.d_model, shape.d_ff,
+                    shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.kv_block_tokens,
+                    shape.elem_bytes)
+
+        def csr(lists):
+            off = np.zeros(len(lists) + 1, dtype=np.int32)
+            off[1:] = np.cumsum([len(x) for x in lists])
+            ids = _i32arr([e for x in lists for e in x])
+            return off, (ids if ids.size else np.zeros(1, dtype=np.int32))
+
+        oo, oi = csr(old_slots)
+        wo, wi = csr(want)
+        cap = _i32arr(cap_new)
+        p = lambda a: a.ctypes.data_as(_i32p)
+        _check(lib().emoe_plan_create_inplace(ctypes.byref(sh), len(old_slots), p(oo), p(oi), len(want),
+                                              p(cap), p(wo), p(wi), PLAN_HOST_ONLY if host_only else 0,
+                                              ctypes.byref(self._h)))
+        self.host_only = host_only
+        self.n_ranks = len(want)
+        self.caps = [len(t) for t in old_slots] + [int(c) for c in list(cap_new)[len(old_slots):]]
+
+    def slot_tables(self):
+        out = []
+        for r in range(self.n_ranks):
+            n = _i32()
+            _check(lib().emoe_plan_slot_table(self._h, r, None, 0, ctypes.byref(n)))
+            t = np.zeros(max(n.value, 1), dtype=np.int32)
+            _check(lib().emoe_plan_slot_table(self._h, r, t.ctypes.data_as(_i32p), n.value, ctypes.byref(n)))
+            out.append([int(x) for x in t[:n.value]])
+        return out
+
+    def reshard(self, arenas, stream=None) -> None:
+        """arenas: one device buffer per device index, max(old devices, new devices) of them."""
+        _check(lib().emoe_reshard_experts_inplace(self._h, _ptr_array(arenas), _stream_handle(stream)))
 
 
 IPC_HANDLE_BYTES = 64

@@ -19,6 +19,14 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found: libemoe.so cannot be built")
 
 
+def have_nvcc() -> bool:
+    try:
+        _nvcc()
+        return True
+    except RuntimeError:
+        return False
+
+
 def is_stale() -> bool:
     if not os.path.exists(OUT):
         return True

@@ -30,6 +30,7 @@ constexpr int kDefaultKvOrder = 1;  // 1 table order, 2 by old block id, 3 by ne
 constexpr uint32_t kDefaultBulkCtas = 74;  // measured optimum on B200: half the SMs, deep rings
 constexpr uint32_t kVecTile = 16384;
 constexpr uint64_t kBulkMinRun = 16384;  // shorter runs go to the vector kernel
+constexpr unsigned long long kDefaultWaitNs = 4000000000ull;  // bound of a device-side wait: 4 s
 constexpr uint64_t kMergeBulkBelow = 1ull << 30;   // see build_tables
 constexpr uint64_t kSmallPhaseBytes = 256ull << 20;
 
@@ -68,6 +69,8 @@ struct emoe_plan {
   bool host_only = true;
   int device = -1, sm_count = 148;
   emoe_tuning_t tuning{};
+  bool inplace = false;           // expert step on capacity-strided arenas (emoe_plan_create_inplace)
+  std::vector<std::vector<int32_t>> slot_new;   // ... its slot tables after the step
   int local_rank = -1;            // >= 0: only destinations of this new-rank index are written
   bool reads_src[3][EMOE_MAX_RANKS];  // old ranks the (filtered) phase reads
   DevPhase dev[kTableSets];       // [3]: all three phases as one launch set (see build_merged)
@@ -79,6 +82,13 @@ struct emoe_plan {
   uint32_t *d_pair_old = nullptr, *d_pair_new = nullptr;
   int *d_status = nullptr;  // [0] status word; then kCtrSlots x 2 work-counter words per phase
   mutable std::atomic<uint32_t> launch_seq[kTableSets];
+  // A whole step with two launch sets runs them side by side: the second set goes to a
+  // stream of the plan's own, forked from and joined to the caller's stream with events.
+  // side[0] has the least priority, side[1] the greatest; the one nearer the caller's
+  // stream is used.  The mutex orders the record / wait pairs of concurrent callers.
+  cudaStream_t side[2] = {nullptr, nullptr};
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  mutable std::mutex fork_mu;
   emoe_plan() { for (auto &a : launch_seq) a.store(0); }
 };
 
@@ -89,6 +99,19 @@ uint32_t bulk_tile(const emoe_plan *p) {
 }
 uint32_t bulk_stages(const emoe_plan *p) {
   return p->tuning.bulk_stages > 0 ? (uint32_t)p->tuning.bulk_stages : kDefaultBulkStages;
+}
+uint64_t bulk_min_run(const emoe_plan *p) {
+  return p->tuning.bulk_min_run > 0 ? (uint64_t)p->tuning.bulk_min_run : kBulkMinRun;
+}
+// Bound of the device-side waits in ns; 0 = a wait that is not satisfied at once fails.
+unsigned long long wait_ns(const emoe_plan *p) {
+  if (p->tuning.wait_limit_us < 0) return 0;
+  return p->tuning.wait_limit_us > 0 ? (unsigned long long)p->tuning.wait_limit_us * 1000ull : kDefaultWaitNs;
+}
+int kv_mode(const emoe_plan *p) { return p->tuning.kv_mode > 0 ? p->tuning.kv_mode : kDefaultKvMode; }
+// The KV head re-split shares a launch with the vector work when it uses the direct copy.
+bool fused_kv(const emoe_plan *p, const KvTables &t) {
+  return (kv_mode(p) == 1 || kv_mode(p) == 4) && p->tuning.serial < 2 && vec_kv_supported(t);
 }
 int kv_order(const emoe_plan *p) {
   return p->tuning.kv_order > 0 ? p->tuning.kv_order : kDefaultKvOrder;
@@ -172,7 +195,7 @@ void build_tables(emoe_plan *p, int phase) {
   uint64_t bulk_bytes = 0, vec_bytes = 0;
   for (const Segment &s0 : pp.segs) {
     const uint64_t b = (uint64_t)s0.n_runs * s0.run_bytes * s0.n_dst;
-    if (s0.align == 16 && s0.run_bytes >= kBulkMinRun) bulk_bytes += b; else vec_bytes += b;
+    if (s0.align == 16 && s0.run_bytes >= bulk_min_run(p)) bulk_bytes += b; else vec_bytes += b;
   }
   const bool all_vec = p->tuning.path == 0 &&
                        ((vec_bytes > 0 && bulk_bytes < kMergeBulkBelow) ||
@@ -182,7 +205,7 @@ void build_tables(emoe_plan *p, int phase) {
   Dst mine[EMOE_MAX_RANKS];
   for (uint32_t oi : order) {
     const Segment &s0 = pp.segs[oi];
-    bool is_bulk = s0.align == 16 && s0.run_bytes >= kBulkMinRun && !all_vec;
+    bool is_bulk = s0.align == 16 && s0.run_bytes >= bulk_min_run(p) && !all_vec;
     if (p->tuning.path == 1) is_bulk = false;
     if (p->tuning.path == 2) is_bulk = (s0.align == 16);
     // destinations this plan writes: all, or those of the local rank only (a source has at
@@ -403,6 +426,10 @@ void free_device(emoe_plan *p) {
   }
   cudaFree(p->d_pair_old); cudaFree(p->d_pair_new); cudaFree(p->d_status);
   p->d_pair_old = p->d_pair_new = nullptr; p->d_status = nullptr;
+  for (cudaStream_t &sd : p->side) { if (sd) cudaStreamDestroy(sd); sd = nullptr; }
+  if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+  if (p->ev_join) cudaEventDestroy(p->ev_join);
+  p->ev_fork = p->ev_join = nullptr;
 }
 
 int ranks_of(const emoe_plan *p, int phase, int side) {
@@ -413,7 +440,7 @@ int ranks_of(const emoe_plan *p, int phase, int side) {
 // Host-side argument checks of a reshard call; fills the by-value pointer table.
 emoe_status_t check_arenas(const emoe_plan *p, int phase, const void *const *src, void *const *dst,
                            RankPtrs *out) {
-  if (!p || !src || !dst) return EMOE_ERR_INVALID_ARG;
+  if (!p || !src || !dst || p->inplace) return EMOE_ERR_INVALID_ARG;
   if (p->host_only) return EMOE_ERR_CUDA;
   const PhasePlan &pp = p->hp.phase[phase];
   const int ns = ranks_of(p, phase, EMOE_SIDE_OLD), nd = ranks_of(p, phase, EMOE_SIDE_NEW);
@@ -452,22 +479,53 @@ uint32_t cta_budget(const emoe_plan *p) {
   return p->tuning.max_ctas > 0 ? (uint32_t)p->tuning.max_ctas : (uint32_t)p->sm_count;
 }
 
-emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, cudaStream_t st) {
-  const DevPhase &dp = p->dev[phase];
-  const BulkConfig bc{bulk_tile(p), bulk_stages(p),
-                      p->tuning.bulk_hints > 0 ? (uint32_t)p->tuning.bulk_hints - 1 : kDefaultHints};
-  // work counter of this launch: the phase's slots are used in turn
+// Launch configuration of the bulk kernel for a launch of `grid` CTAs.
+BulkConfig bulk_config(const emoe_plan *p, uint32_t grid) {
+  BulkConfig bc{bulk_tile(p), bulk_stages(p),
+                p->tuning.bulk_hints > 0 ? (uint32_t)p->tuning.bulk_hints - 1 : kDefaultHints, 0, wait_ns(p)};
+  if (p->tuning.bw_limit_gbs > 0 && grid > 0) {
+    // The limit counts bytes read plus bytes written, so loads get half of it; spread over
+    // the CTAs of the launch that is one tile per CTA every tile * grid / (limit / 2) ns.
+    const double ns = 2.0 * bc.tile_bytes * grid / (double)p->tuning.bw_limit_gbs;
+    bc.pace_ns = ns < 1.0 ? 1u : ns > 1e6 ? 1000000u : (uint32_t)ns;
+  }
+  return bc;
+}
+
+// The bulk launch of a table set.  Its work counter: the set's slots are used in turn; a
+// launch that is being captured into a graph gets none (its CTAs take units round-robin),
+// because a graph would keep its slot for as long as it lives.
+emoe_status_t run_bulk(const emoe_plan *p, int set, const RankPtrs &ptrs, cudaStream_t st) {
+  const DevPhase &dp = p->dev[set];
+  if (dp.n_bulk == 0) return EMOE_OK;
   unsigned int *ctr = nullptr;
   if (p->tuning.unit_order < 2) {
-    const uint32_t slot = p->launch_seq[phase].fetch_add(1) % kCtrSlots;
-    ctr = reinterpret_cast<unsigned int *>(p->d_status) + 1 + (phase * kCtrSlots + slot) * 2;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) { (void)cudaGetLastError(); cs = cudaStreamCaptureStatusNone; }
+    if (cs == cudaStreamCaptureStatusNone) {
+      const uint32_t slot = p->launch_seq[set].fetch_add(1) % kCtrSlots;
+      ctr = reinterpret_cast<unsigned int *>(p->d_status) + 1 + (set * kCtrSlots + slot) * 2;
+    }
   }
-  cudaError_t e = launch_bulk_copy({dp.d_segs, dp.d_dsts, dp.d_bulk_units, (uint32_t)dp.n_bulk},
-                                   ptrs, bc, bulk_budget(p), p->d_status, ctr, st);
-  if (e != cudaSuccess) return cuda_status(e);
-  e = launch_vec_copy({dp.d_segs, dp.d_dsts, dp.d_vec_units, (uint32_t)dp.vec_units.size()}, ptrs,
-                      kVecTile, p->tuning.max_ctas > 0 ? cta_budget(p) * 8 : 0xffffffffu, st);
-  return cuda_status(e);
+  uint32_t grid = bulk_budget(p);
+  if (grid > dp.n_bulk) grid = (uint32_t)dp.n_bulk;
+  return cuda_status(launch_bulk_copy({dp.d_segs, dp.d_dsts, dp.d_bulk_units, (uint32_t)dp.n_bulk}, ptrs,
+                                      bulk_config(p, grid), grid, p->d_status, ctr, st));
+}
+
+uint32_t vec_grid(const emoe_plan *p) {
+  return p->tuning.max_ctas > 0 ? cta_budget(p) * 8 : 0xffffffffu;
+}
+
+emoe_status_t run_vec(const emoe_plan *p, int set, const RankPtrs &ptrs, cudaStream_t st) {
+  const DevPhase &dp = p->dev[set];
+  return cuda_status(launch_vec_copy({dp.d_segs, dp.d_dsts, dp.d_vec_units, (uint32_t)dp.vec_units.size()},
+                                     ptrs, kVecTile, vec_grid(p), st));
+}
+
+emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, cudaStream_t st) {
+  const emoe_status_t rc = run_bulk(p, phase, ptrs, st);
+  return rc != EMOE_OK ? rc : run_vec(p, phase, ptrs, st);
 }
 
 // Shape constants of the KV head re-split as the kernels take them.
@@ -494,9 +552,6 @@ KvTables kv_tables(const KvPlan &kv, const uint32_t *d_pair_old, const uint32_t 
     }
   return t;
 }
-
-std::once_flag g_init_once;
-cudaError_t g_init_err = cudaSuccess;
 
 void destroy_host_step(HostStep *hs);
 
@@ -561,6 +616,34 @@ void destroy_host_step(HostStep *hs) {
   delete hs;
 }
 
+// Device side of a new plan: descriptor tables, status word and work counters, the side
+// streams of the whole step.  On failure everything is freed again.
+emoe_status_t finish_device_plan(emoe_plan *p) {
+  cudaError_t e = cudaGetDevice(&p->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
+  if (e == cudaSuccess) e = kernels_init();   // per device: the plan's device is current
+  emoe_status_t st = cuda_status(e);
+  for (int ph = 0; st == EMOE_OK && ph < kTableSets; ++ph) st = upload_phase(p, ph);
+  if (st == EMOE_OK && p->hp.kv.head_split_changes) {
+    cudaError_t e2 = upload(p->pair_old, &p->d_pair_old);
+    if (e2 == cudaSuccess) e2 = upload(p->pair_new, &p->d_pair_new);
+    st = cuda_status(e2);
+  }
+  if (st == EMOE_OK) {
+    cudaError_t e3 = cudaMalloc((void **)&p->d_status, kStatusWords * sizeof(int));
+    if (e3 == cudaSuccess) e3 = cudaMemset(p->d_status, 0, kStatusWords * sizeof(int));
+    int least = 0, greatest = 0;
+    if (e3 == cudaSuccess) e3 = cudaDeviceGetStreamPriorityRange(&least, &greatest);
+    if (e3 == cudaSuccess) e3 = cudaStreamCreateWithPriority(&p->side[0], cudaStreamNonBlocking, least);
+    if (e3 == cudaSuccess) e3 = cudaStreamCreateWithPriority(&p->side[1], cudaStreamNonBlocking, greatest);
+    if (e3 == cudaSuccess) e3 = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
+    if (e3 == cudaSuccess) e3 = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
+    st = cuda_status(e3);
+  }
+  if (st != EMOE_OK) free_device(p);
+  return st;
+}
+
 emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
                           const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out) {
   if (!shape || !old_cfg || !new_cfg || !out) return EMOE_ERR_INVALID_ARG;
@@ -578,27 +661,13 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
   if (st != EMOE_OK) { delete p; return st; }
   p->host_only = (flags & EMOE_PLAN_HOST_ONLY) != 0;
   if (!p->host_only) {
-    cudaError_t e = cudaGetDevice(&p->device);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
-    if (e == cudaSuccess) {
-      std::call_once(g_init_once, [] { g_init_err = kernels_init(); });
-      e = g_init_err;
+    st = finish_device_plan(p);
+    if (st == EMOE_OK && (flags & EMOE_PLAN_HOST_STEP)) {
+      st = make_host_step(p, *shape, old_cfg, new_cfg,
+                          flags & (EMOE_LAYOUT_FUSED_W13 | EMOE_LAYOUT_KV_HEAD_MAJOR));
+      if (st != EMOE_OK) free_device(p);
     }
-    st = cuda_status(e);
-    for (int ph = 0; st == EMOE_OK && ph < kTableSets; ++ph) st = upload_phase(p, ph);
-    if (st == EMOE_OK && p->hp.kv.head_split_changes) {
-      cudaError_t e2 = upload(p->pair_old, &p->d_pair_old);
-      if (e2 == cudaSuccess) e2 = upload(p->pair_new, &p->d_pair_new);
-      st = cuda_status(e2);
-    }
-    if (st == EMOE_OK) {
-      cudaError_t e3 = cudaMalloc((void **)&p->d_status, kStatusWords * sizeof(int));
-      if (e3 == cudaSuccess) e3 = cudaMemset(p->d_status, 0, kStatusWords * sizeof(int));
-      st = cuda_status(e3);
-    }
-    if (st == EMOE_OK && (flags & EMOE_PLAN_HOST_STEP)) st = make_host_step(p, *shape, old_cfg, new_cfg,
-                                  flags & (EMOE_LAYOUT_FUSED_W13 | EMOE_LAYOUT_KV_HEAD_MAJOR));
-    if (st != EMOE_OK) { free_device(p); delete p; return st; }
+    if (st != EMOE_OK) { delete p; return st; }
   }
   *out = p;
   return EMOE_OK;
@@ -618,10 +687,7 @@ emoe_status_t emoe::run_phase_once(const PhasePlan &pp, const RankPtrs &ptrs, cu
   }
   cudaError_t e = cudaGetDevice(&tmp.device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&tmp.sm_count, cudaDevAttrMultiProcessorCount, tmp.device);
-  if (e == cudaSuccess) {
-    std::call_once(g_init_once, [] { g_init_err = kernels_init(); });
-    e = g_init_err;
-  }
+  if (e == cudaSuccess) e = kernels_init();
   rc = cuda_status(e);
   if (rc == EMOE_OK) rc = upload_phase(&tmp, 0);
   if (rc == EMOE_OK) {
@@ -681,14 +747,14 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *p, const void *const *src, void
   if (!p->hp.kv.head_split_changes) return run_segments(p, EMOE_PHASE_KV, ptrs, (cudaStream_t)stream);
   const KvPlan &kv = p->hp.kv;
   KvTables t = kv_tables(kv, p->d_pair_old, p->d_pair_new, p->local_rank);
-  const int mode = p->tuning.kv_mode > 0 ? p->tuning.kv_mode : kDefaultKvMode;
+  const int mode = kv_mode(p);
   return cuda_status(launch_kv_copy(t, ptrs, mode, cta_budget(p), p->tuning.max_ctas <= 0, p->d_status,
-                                    (cudaStream_t)stream));
+                                    wait_ns(p), (cudaStream_t)stream));
 }
 
 emoe_status_t emoe_reshard_step(const emoe_plan_t *p, const void *const *const src[3],
                                 void *const *const dst[3], void *stream) {
-  if (!p || !src || !dst) return EMOE_ERR_INVALID_ARG;
+  if (!p || !src || !dst || p->inplace) return EMOE_ERR_INVALID_ARG;
   RankPtrs ph_ptrs[3];
   for (int ph = 0; ph < 3; ++ph) {  // every argument is checked before anything is enqueued
     if (!src[ph] || !dst[ph]) return EMOE_ERR_INVALID_ARG;
@@ -698,56 +764,168 @@ emoe_status_t emoe_reshard_step(const emoe_plan_t *p, const void *const *const s
   cudaStream_t st = (cudaStream_t)stream;
   const KvPlan &kv = p->hp.kv;
   emoe_status_t rc = EMOE_OK;
-  if (p->merged) {
-    RankPtrs all;
-    std::memset(&all, 0, sizeof(all));
-    for (int ph = 0; ph < 3; ++ph) {
-      for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_OLD); ++r) all.src[p->src_base[ph] + r] = ph_ptrs[ph].src[r];
-      for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_NEW); ++r) all.dst[p->dst_base[ph] + r] = ph_ptrs[ph].dst[r];
-    }
-    rc = run_segments(p, 3, all, st);
-  } else {
+  if (!p->merged) {  // too many ranks for one pointer table: phase by phase
     for (int ph = 0; rc == EMOE_OK && ph < 3; ++ph) rc = run_segments(p, ph, ph_ptrs[ph], st);
+    if (rc == EMOE_OK && kv.head_split_changes) {
+      KvTables t = kv_tables(kv, p->d_pair_old, p->d_pair_new, p->local_rank);
+      rc = cuda_status(launch_kv_copy(t, ph_ptrs[2], kv_mode(p), cta_budget(p), p->tuning.max_ctas <= 0,
+                                      p->d_status, wait_ns(p), st));
+    }
+    return rc;
   }
-  if (rc == EMOE_OK && kv.head_split_changes) {
+  RankPtrs all;
+  std::memset(&all, 0, sizeof(all));
+  for (int ph = 0; ph < 3; ++ph) {
+    for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_OLD); ++r) all.src[p->src_base[ph] + r] = ph_ptrs[ph].src[r];
+    for (int r = 0; r < ranks_of(p, ph, EMOE_SIDE_NEW); ++r) all.dst[p->dst_base[ph] + r] = ph_ptrs[ph].dst[r];
+  }
+  // Up to two launch sets: the ring kernel (long runs of all three phases), and the
+  // register-copy work - short and strided runs plus the KV head re-split, as ONE kernel
+  // when the re-split uses the direct copy (the default).  With both present the second
+  // set runs beside the first on a stream of the plan's own, so that neither waits for
+  // the other's ramp-up and tail.
+  const DevPhase &dp = p->dev[3];
+  const bool kv_work = kv.head_split_changes && !kv.pair_old.empty();
+  const bool has_bulk = dp.n_bulk > 0, has_small = !dp.vec_units.empty() || kv_work;
+  const bool fork = has_bulk && has_small && p->tuning.serial == 0 && p->side[0];
+  cudaStream_t st2 = st;
+  std::unique_lock<std::mutex> lock(p->fork_mu, std::defer_lock);
+  if (fork) {
+    int prio = 0, least = 0, greatest = 0;
+    cudaError_t e = cudaStreamGetPriority(st, &prio);
+    if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&least, &greatest);
+    if (e != cudaSuccess) return cuda_status(e);
+    st2 = (prio - greatest) < (least - prio) ? p->side[1] : p->side[0];
+    lock.lock();
+    e = cudaEventRecord(p->ev_fork, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st2, p->ev_fork, 0);
+    if (e != cudaSuccess) return cuda_status(e);
+  }
+  rc = run_bulk(p, 3, all, st);
+  if (rc == EMOE_OK && has_small) {
     KvTables t = kv_tables(kv, p->d_pair_old, p->d_pair_new, p->local_rank);
-    const int mode = p->tuning.kv_mode > 0 ? p->tuning.kv_mode : kDefaultKvMode;
-    rc = cuda_status(launch_kv_copy(t, ph_ptrs[2], mode, cta_budget(p), p->tuning.max_ctas <= 0,
-                                    p->d_status, st));
+    if (kv_work && fused_kv(p, t)) {
+      rc = cuda_status(launch_vec_kv_copy({dp.d_segs, dp.d_dsts, dp.d_vec_units, (uint32_t)dp.vec_units.size()},
+                                          all, kVecTile, t, ph_ptrs[2],
+                                          p->tuning.max_ctas > 0 ? cta_budget(p) * 8 : 0,
+                                          p->tuning.max_ctas <= 0, st2));
+    } else {
+      rc = run_vec(p, 3, all, st2);
+      if (rc == EMOE_OK && kv_work)
+        rc = cuda_status(launch_kv_copy(t, ph_ptrs[2], kv_mode(p), cta_budget(p), p->tuning.max_ctas <= 0,
+                                        p->d_status, wait_ns(p), st2));
+    }
+  }
+  if (fork) {  // joined even after an error, so that the caller's stream never loses the side work
+    cudaError_t e = cudaEventRecord(p->ev_join, st2);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, p->ev_join, 0);
+    if (rc == EMOE_OK) rc = cuda_status(e);
   }
   return rc;
 }
 
+emoe_status_t emoe_plan_create_inplace(const emoe_shape_t *shape, int32_t ep_old,
+                                       const int32_t *slot_off_old, const int32_t *slot_ids_old,
+                                       int32_t ep_new, const int32_t *cap_new, const int32_t *want_off,
+                                       const int32_t *want_ids, uint32_t flags, emoe_plan_t **out) {
+  if (!shape || !out || (flags & ~EMOE_PLAN_HOST_ONLY)) return EMOE_ERR_INVALID_ARG;
+  emoe_plan *p = new (std::nothrow) emoe_plan();
+  if (!p) return EMOE_ERR_OOM;
+  emoe_status_t st;
+  try {
+    st = build_inplace_expert_plan(*shape, ep_old, slot_off_old, slot_ids_old, ep_new, cap_new, want_off,
+                                   want_ids, &p->hp.phase[EMOE_PHASE_EXPERTS], &p->slot_new);
+    if (st == EMOE_OK) {
+      p->inplace = true;
+      p->hp.shape = *shape;
+      p->hp.ep_old = ep_old; p->hp.ep_new = ep_new;
+      p->hp.tp_old = p->hp.tp_new = 0;       // no attention or KV phase in this kind of plan
+      build_all_tables(p);
+    }
+  } catch (const std::bad_alloc &) {
+    st = EMOE_ERR_OOM;
+  }
+  if (st != EMOE_OK) { delete p; return st; }
+  p->host_only = (flags & EMOE_PLAN_HOST_ONLY) != 0;
+  if (!p->host_only && (st = finish_device_plan(p)) != EMOE_OK) { delete p; return st; }
+  *out = p;
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_plan_slot_table(const emoe_plan_t *p, int32_t rank, int32_t *out, int32_t cap,
+                                   int32_t *n_slots) {
+  if (!p || !p->inplace || rank < 0 || rank >= (int)p->slot_new.size() || (cap > 0 && !out))
+    return EMOE_ERR_INVALID_ARG;
+  const std::vector<int32_t> &t = p->slot_new[rank];
+  if (n_slots) *n_slots = (int32_t)t.size();
+  for (int32_t i = 0; i < cap && i < (int32_t)t.size(); ++i) out[i] = t[i];
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_reshard_experts_inplace(const emoe_plan_t *p, void *const *arenas, void *stream) {
+  if (!p || !arenas || !p->inplace) return EMOE_ERR_INVALID_ARG;
+  if (p->host_only) return EMOE_ERR_CUDA;
+  const PhasePlan &pp = p->hp.phase[EMOE_PHASE_EXPERTS];
+  const int ns = p->hp.ep_old, nd = p->hp.ep_new, n = ns > nd ? ns : nd;
+  RankPtrs ptrs;
+  std::memset(&ptrs, 0, sizeof(ptrs));
+  uint64_t bytes[EMOE_MAX_RANKS];
+  const bool local = p->local_rank >= 0;
+  for (int r = 0; r < n; ++r) {
+    bytes[r] = r < ns ? pp.arena_old[r] : pp.arena_new[r];
+    // with a local rank set only that rank's arena and the arenas it reads are needed
+    const bool needed = local ? (r == p->local_rank || (r < ns && p->reads_src[EMOE_PHASE_EXPERTS][r]))
+                              : bytes[r] != 0;
+    if (needed && !arenas[r]) return EMOE_ERR_INVALID_ARG;
+    if ((uintptr_t)arenas[r] % 16) return EMOE_ERR_ALIGNMENT;
+    if (!needed || !arenas[r]) { bytes[r] = 0; continue; }
+    if (r < ns) ptrs.src[r] = (const uint8_t *)arenas[r];
+    if (r < nd) ptrs.dst[r] = (uint8_t *)arenas[r];
+  }
+  for (int a = 0; a < n; ++a)        // different devices' arenas must not intersect
+    for (int b = a + 1; b < n; ++b) {
+      const uintptr_t a0 = (uintptr_t)arenas[a], a1 = a0 + bytes[a];
+      const uintptr_t b0 = (uintptr_t)arenas[b], b1 = b0 + bytes[b];
+      if (bytes[a] && bytes[b] && a0 < b1 && b0 < a1) return EMOE_ERR_OVERLAP;
+    }
+  return run_segments(p, EMOE_PHASE_EXPERTS, ptrs, (cudaStream_t)stream);
+}
+
 emoe_status_t emoe_reshard_kv_static(const emoe_plan_t *p, const void *const *src, void *const *dst,
                                      void *stream) {
-  if (!p || !src || !dst) return EMOE_ERR_INVALID_ARG;
+  if (!p || !src || !dst || p->inplace) return EMOE_ERR_INVALID_ARG;
   const KvPlan &kv = p->hp.kv;
   // this entry point only has the token-major pair kernel: whole blocks (TP kept) are
   // layout-agnostic, a head re-split of head-major blocks is not
   if (kv.head_major && kv.c != kv.d) return EMOE_ERR_UNSUPPORTED;
   const std::vector<uint32_t> *pair_old = &kv.pair_old, *pair_new = &kv.pair_new;
   if (pair_old->size() > EMOE_STATIC_KV_MAX_PAIRS) return EMOE_ERR_TOO_LARGE;
-  // the same argument checks as emoe_reshard_kv, but a host-only plan is welcome here
+  // the same argument checks as emoe_reshard_kv, but a host-only plan is welcome here.  With
+  // a local rank set only that rank's destination and the old ranks it reads are needed.
   const PhasePlan &pp = p->hp.phase[EMOE_PHASE_KV];
+  const bool local = p->local_rank >= 0;
   RankPtrs ptrs;
   std::memset(&ptrs, 0, sizeof(ptrs));
   for (int r = 0; r < p->hp.tp_old; ++r) {
-    if (pp.arena_old[r] && !src[r]) return EMOE_ERR_INVALID_ARG;
+    const bool needed = local ? p->reads_src[EMOE_PHASE_KV][r] : pp.arena_old[r] != 0;
+    if (needed && !src[r]) return EMOE_ERR_INVALID_ARG;
     if ((uintptr_t)src[r] % 16) return EMOE_ERR_ALIGNMENT;
     ptrs.src[r] = (const uint8_t *)src[r];
   }
   for (int r = 0; r < p->hp.tp_new; ++r) {
-    if (pp.arena_new[r] && !dst[r]) return EMOE_ERR_INVALID_ARG;
+    const bool needed = pp.arena_new[r] != 0 && (!local || r == p->local_rank);
+    if (needed && !dst[r]) return EMOE_ERR_INVALID_ARG;
     if ((uintptr_t)dst[r] % 16) return EMOE_ERR_ALIGNMENT;
-    ptrs.dst[r] = (uint8_t *)dst[r];
+    ptrs.dst[r] = needed ? (uint8_t *)dst[r] : nullptr;
   }
   for (int a = 0; a < p->hp.tp_old; ++a)
     for (int b = 0; b < p->hp.tp_new; ++b) {
+      if (!ptrs.src[a] || !ptrs.dst[b]) continue;
       const uintptr_t s0 = (uintptr_t)src[a], s1 = s0 + pp.arena_old[a];
       const uintptr_t d0 = (uintptr_t)dst[b], d1 = d0 + pp.arena_new[b];
       if (s0 < d1 && d0 < s1) return EMOE_ERR_OVERLAP;
     }
-  KvTables t = kv_tables(kv, nullptr, nullptr);
+  KvTables t = kv_tables(kv, nullptr, nullptr, p->local_rank);
   return launch_kv_copy_static(t, pair_old->data(), pair_new->data(), ptrs, (cudaStream_t)stream);
 }
 
@@ -827,7 +1005,7 @@ extern "C" {
 emoe_status_t emoe_reshard_step_host(const emoe_plan_t *p, const void *const *const h_src[3],
                                      void *const *const h_dst[3], void *const *const d_src[3],
                                      void *const *const d_dst[3], void *stream) {
-  if (!p || !h_src || !h_dst || !d_src || !d_dst) return EMOE_ERR_INVALID_ARG;
+  if (!p || !h_src || !h_dst || !d_src || !d_dst || p->inplace) return EMOE_ERR_INVALID_ARG;
   if (p->host_only) return EMOE_ERR_CUDA;
   cudaStream_t st = (cudaStream_t)stream;
   if (p->hs) return step_host_pipelined(p, h_src, h_dst, d_src, d_dst, st);
@@ -893,12 +1071,17 @@ emoe_status_t emoe_plan_num_launches(const emoe_plan_t *p, int phase, int32_t *n
     const int kv_pairs = p->hp.kv.head_split_changes && !p->hp.kv.pair_old.empty() ? 1 : 0;
     int k = 0;
     if (p->merged) {
-      k = (p->dev[3].n_bulk ? 1 : 0) + (p->dev[3].vec_units.empty() ? 0 : 1);
+      const int vec = p->dev[3].vec_units.empty() ? 0 : 1;
+      k = (p->dev[3].n_bulk ? 1 : 0);
+      // the vector work and a direct KV head re-split share one kernel
+      const KvTables t = kv_tables(p->hp.kv, nullptr, nullptr, p->local_rank);
+      k += kv_pairs && fused_kv(p, t) ? 1 : vec + kv_pairs;
     } else {
       for (int ph = 0; ph < 3; ++ph)
         k += (p->dev[ph].n_bulk ? 1 : 0) + (p->dev[ph].vec_units.empty() ? 0 : 1);
+      k += kv_pairs;
     }
-    *n = k + kv_pairs;
+    *n = k;
     return EMOE_OK;
   }
   if (phase == EMOE_PHASE_KV && p->hp.kv.head_split_changes) {
@@ -906,6 +1089,23 @@ emoe_status_t emoe_plan_num_launches(const emoe_plan_t *p, int phase, int32_t *n
     return EMOE_OK;
   }
   *n = (p->dev[phase].n_bulk ? 1 : 0) + (p->dev[phase].vec_units.empty() ? 0 : 1);
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_plan_launch_work(const emoe_plan_t *p, int phase, uint64_t *ring_units,
+                                    uint64_t *vector_units, uint64_t *kv_tiles) {
+  if (!p || phase < 0 || phase > EMOE_PHASE_STEP) return EMOE_ERR_INVALID_ARG;
+  const bool kv_here = (phase == EMOE_PHASE_KV || phase == EMOE_PHASE_STEP) && p->hp.kv.head_split_changes;
+  uint64_t ring = 0, vec = 0;
+  if (phase == EMOE_PHASE_STEP && !p->merged) {
+    for (int ph = 0; ph < 3; ++ph) { ring += p->dev[ph].n_bulk; vec += p->dev[ph].vec_units.size(); }
+  } else {
+    ring = p->dev[phase].n_bulk;
+    vec = p->dev[phase].vec_units.size();
+  }
+  if (ring_units) *ring_units = ring;
+  if (vector_units) *vector_units = vec;
+  if (kv_tiles) *kv_tiles = kv_here ? (uint64_t)p->hp.kv.pair_old.size() * p->hp.kv.n_layers * 2 : 0;
   return EMOE_OK;
 }
 
@@ -939,15 +1139,30 @@ emoe_status_t emoe_plan_device_status(const emoe_plan_t *p, int32_t *status) {
   return EMOE_OK;
 }
 
+emoe_status_t emoe_plan_clear_device_status(emoe_plan_t *p) {
+  if (!p) return EMOE_ERR_INVALID_ARG;
+  if (p->host_only) return EMOE_ERR_CUDA;
+  if (cudaMemset(p->d_status, 0, sizeof(int)) != cudaSuccess) return cuda_status(cudaGetLastError());
+  if (p->hs)
+    for (emoe_plan *sub : {p->hs->chunk, p->hs->tail})
+      if (sub) {
+        const emoe_status_t rc = emoe_plan_clear_device_status(sub);
+        if (rc != EMOE_OK) return rc;
+      }
+  return EMOE_OK;
+}
+
 emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
   if (!p || !t) return EMOE_ERR_INVALID_ARG;
   if (t->max_ctas < 0 || t->bulk_tile_bytes < 0 || t->bulk_stages < 0 || t->path < 0 ||
       t->path > 2 || t->kv_mode < 0 || t->kv_mode > 4 || t->bulk_hints < 0 ||
       t->bulk_hints > 4 || t->kv_order < 0 || t->kv_order > 3 || t->unit_order < 0 ||
-      t->unit_order > 3)
+      t->unit_order > 3 || t->wait_limit_us < -1 || t->bw_limit_gbs < 0 || t->bulk_min_run < 0 ||
+      t->serial < 0 || t->serial > 2)
     return EMOE_ERR_INVALID_ARG;
   if (t->bulk_tile_bytes && (t->bulk_tile_bytes % 128 || t->bulk_tile_bytes < 1024))
     return EMOE_ERR_INVALID_ARG;
+  if (t->bulk_min_run && t->bulk_min_run % 16) return EMOE_ERR_INVALID_ARG;
   const uint32_t tile = t->bulk_tile_bytes ? t->bulk_tile_bytes : kDefaultBulkTile;
   const uint32_t stages = t->bulk_stages ? t->bulk_stages : kDefaultBulkStages;
   if (stages < 2 || stages > 16 || bulk_smem_bytes(tile, stages) > bulk_smem_limit())

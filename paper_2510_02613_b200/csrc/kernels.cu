@@ -25,7 +25,13 @@ namespace emoe {
 namespace {
 
 constexpr uint32_t kMaxStages = 16;
-constexpr unsigned long long kWaitLimitNs = 4000000000ull;  // 4 s per wait
+constexpr int kMaxDevices = 64;
+// Dynamic shared memory the bulk kernel may ask for: the 227 KiB a CTA can have, less room
+// for the kernel's static shared memory (two pointer tables of EMOE_MAX_RANKS entries).
+constexpr size_t kBulkSmemLimit = 224 * 1024;
+// Bound of the waits that let copies already in flight land after a wait has expired
+// (those copies always complete; the bound only keeps the loop finite).
+constexpr unsigned long long kDrainLimitNs = 4000000000ull;
 
 // ---- PTX wrappers -----------------------------------------------------------------------
 
@@ -58,15 +64,33 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within kWaitLimitNs.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Non-blocking form: has the phase completed right now?
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within limit_ns, or if the CTA's
+// other role has given up meanwhile (*abort set).
+// limit_ns == 0: a wait that is not satisfied the moment it is asked fails at once
+// (try_wait may itself suspend the thread for a while, so this case uses test_wait).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns,
+                                          const volatile int *abort = nullptr) {
+  if (limit_ns == 0) return mbar_test_wait(bar, parity);
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
+    if (abort && *abort) return false;
+    if (globaltimer_ns() - t0 > limit_ns) return false;
   }
 }
 __device__ __forceinline__ uint64_t policy_evict_first() {
@@ -138,6 +162,8 @@ struct BulkParams {
   SegTables t;
   uint32_t tile_bytes, stages;
   uint32_t hints;      // bit 0: loads evict-first in L2, bit 1: stores evict-first
+  uint32_t pace_ns;    // least time between a CTA's full-tile loads (0: unpaced): bandwidth limit
+  unsigned long long wait_ns;  // bound of every wait (0: fail at once if not already satisfied)
   int *status;
   unsigned int *ctr;   // {next unit to claim, CTAs finished}, both 0 between launches; null: static
   RankPtrs ptrs;
@@ -179,6 +205,7 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
     const uint32_t G = gridDim.x, n = p.t.n_units;
     uint32_t it = 0;
     bool ok = true;
+    unsigned long long t_next = 0;  // earliest start of the next load when the launch is paced
     // Units: the first one is the CTA's own index; the following ones are claimed from a
     // global counter (SMs do not all see the same bandwidth, and a static split ends with
     // the slowest: +1..3 % measured), or taken round-robin when there is no counter.  A
@@ -218,7 +245,10 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
       uint32_t ch = long_run ? un.first_tile % tpr : 0u;                    // chunk in run
       for (uint32_t k = 0; k < un.n_tiles; ++k, ++it) {
         const uint32_t st = it % S, round = it / S;
-        if (round > 0 && !mbar_wait(smem_u32(&empty[st]), (round - 1) & 1)) { ok = false; break; }
+        if (round > 0 && !mbar_wait(smem_u32(&empty[st]), (round - 1) & 1, p.wait_ns, &s_abort)) {
+          ok = false;
+          break;
+        }
         if (s_abort) { ok = false; break; }
         uint32_t rows, row_bytes;
         uint64_t in_run;
@@ -246,16 +276,32 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
         ti.n_dst = sg.n_dst;
         ti.n_rows = rows;
         ti.row_bytes = row_bytes;
+        if (p.pace_ns) {
+          // bandwidth limit: a CTA's loads are spaced pace_ns per full tile apart (a short
+          // tile earns a proportionally short gap); time not used is not saved up beyond
+          // two tiles.  The sleep is at most one gap long.
+          const unsigned long long burst = 2ull * p.pace_ns;
+          unsigned long long now = globaltimer_ns();
+          for (int spin = 0; now < t_next && spin < (1 << 16); ++spin) {
+            __nanosleep(t_next - now < 1000 ? (unsigned)(t_next - now) : 1000u);
+            now = globaltimer_ns();
+          }
+          if (t_next + burst < now) t_next = now - burst;
+          t_next += (unsigned long long)p.pace_ns * (rows * row_bytes) / T;
+        }
         const uint32_t bar = smem_u32(&full[st]);
         mbar_arrive_expect_tx(bar, rows * row_bytes);
         const uint8_t *sp = src_base + (uint64_t)run * sg.src_pitch + in_run;
         const uint32_t dp = smem_u32(data + (size_t)st * T);
+        // rows that follow one another without a gap in the source are one load
+        uint32_t n_ld = rows, ld_bytes = row_bytes;
+        if (rows > 1 && sg.src_pitch == row_bytes) { n_ld = 1; ld_bytes = rows * row_bytes; }
         if (hint) {
-          for (uint32_t r = 0; r < rows; ++r)
-            bulk_load_hint(dp + r * row_bytes, sp + (uint64_t)r * sg.src_pitch, row_bytes, bar, pol);
+          for (uint32_t r = 0; r < n_ld; ++r)
+            bulk_load_hint(dp + r * ld_bytes, sp + (uint64_t)r * sg.src_pitch, ld_bytes, bar, pol);
         } else {
-          for (uint32_t r = 0; r < rows; ++r)
-            bulk_load(dp + r * row_bytes, sp + (uint64_t)r * sg.src_pitch, row_bytes, bar);
+          for (uint32_t r = 0; r < n_ld; ++r)
+            bulk_load(dp + r * ld_bytes, sp + (uint64_t)r * sg.src_pitch, ld_bytes, bar);
         }
         if (long_run) {
           if (++ch == tpr) { ch = 0; ++run; }
@@ -274,7 +320,7 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
     if (ok) {
       // end marker
       const uint32_t st = it % S, round = it / S;
-      if (round == 0 || mbar_wait(smem_u32(&empty[st]), (round - 1) & 1)) {
+      if (round == 0 || mbar_wait(smem_u32(&empty[st]), (round - 1) & 1, p.wait_ns, &s_abort)) {
         info[st].n_rows = 0;
         mbar_arrive(smem_u32(&full[st]));
       } else {
@@ -288,7 +334,7 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
       const uint32_t back = it < S ? it : S;
       for (uint32_t j = 1; j <= back; ++j) {
         const uint32_t i2 = it - j;
-        (void)mbar_wait(smem_u32(&full[i2 % S]), (i2 / S) & 1);
+        (void)mbar_wait(smem_u32(&full[i2 % S]), (i2 / S) & 1, kDrainLimitNs);
       }
     }
     if (dyn) {  // the last producer to finish leaves the counters at zero for the next launch
@@ -309,7 +355,7 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
     const bool hint = (p.hints & 2u) != 0;
     for (uint32_t it = 0;; ++it) {
       const uint32_t st = it % S, round = it / S;
-      if (!mbar_wait(smem_u32(&full[st]), round & 1)) {
+      if (!mbar_wait(smem_u32(&full[st]), round & 1, p.wait_ns, &s_abort)) {
         s_abort = 1;
         atomicExch(p.status, (int)EMOE_ERR_DEVICE_TIMEOUT);
         break;
@@ -321,11 +367,14 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
       for (uint32_t d = 0; d < ti.n_dst; ++d) {
         uint8_t *dp = reinterpret_cast<uint8_t *>(ti.dst_ptr[d]);
         const uint64_t pitch = ti.dst_pitch[d];
+        // rows that follow one another without a gap in the destination are one store
+        uint32_t n_st = rows, sb = rb;
+        if (rows > 1 && pitch == rb) { n_st = 1; sb = rows * rb; }
         if (hint) {
-          for (uint32_t r = 0; r < rows; ++r)
-            bulk_store_hint(dp + (uint64_t)r * pitch, sp + r * rb, rb, pol);
+          for (uint32_t r = 0; r < n_st; ++r)
+            bulk_store_hint(dp + (uint64_t)r * pitch, sp + r * sb, sb, pol);
         } else {
-          for (uint32_t r = 0; r < rows; ++r) bulk_store(dp + (uint64_t)r * pitch, sp + r * rb, rb);
+          for (uint32_t r = 0; r < n_st; ++r) bulk_store(dp + (uint64_t)r * pitch, sp + r * sb, sb);
         }
       }
       bulk_commit();
@@ -338,12 +387,151 @@ __global__ void __launch_bounds__(64, 1) bulk_copy_kernel(const __grid_constant_
   }
 }
 
+// ---- KV head re-split -------------------------------------------------------------------
+
+struct KvParams {
+  KvTables t;
+  RankPtrs ptrs;
+};
+
+// Direct variant: thread q of a tile owns piece q of the LOGICAL block
+// [token][global head][piece]; it reads the piece from the old rank that holds the
+// head and writes it to the new rank that will.  Reads of a warp cover whole token
+// rows of the old layout, writes whole head vectors of the new one.
+// The CTA copies tiles first, first + stride, ... (a tile = one (layer, K|V, block pair)).
+template <typename V>
+__device__ __forceinline__ void kv_direct_tiles(const KvTables &t, const RankPtrs &ptrs, uint64_t first,
+                                                uint64_t stride) {
+  constexpr uint32_t W = sizeof(V);
+  const uint32_t cpv = t.head_bytes / W;     // pieces per head vector
+  const uint32_t row = t.hkv * cpv;          // pieces per logical token row
+  const uint32_t total = t.block_tokens * row;
+  const uint64_t blk_old = (uint64_t)t.block_tokens * t.hc * t.head_bytes;
+  const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
+  const uint64_t n_tiles = (uint64_t)t.n_pairs * t.n_lk;
+  for (uint64_t tile = first; tile < n_tiles; tile += stride) {
+    const uint32_t lk = (uint32_t)(tile / t.n_pairs), pr = (uint32_t)(tile % t.n_pairs);
+    const uint64_t base_old = ((uint64_t)lk * t.nb_old + t.pair_old[pr]) * blk_old;
+    const uint64_t base_new = ((uint64_t)lk * t.nb_new + t.pair_new[pr]) * blk_new;
+    for (uint32_t q0 = threadIdx.x; q0 < total; q0 += blockDim.x * 4) {
+      V v[4];
+      uint32_t tok[4], g[4], j[4];
+      bool live[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t q = q0 + u * blockDim.x;
+        live[u] = false;
+        if (q < total) {
+          tok[u] = q / row;
+          const uint32_t rem = q - tok[u] * row;
+          g[u] = rem / cpv;
+          j[u] = rem - g[u] * cpv;
+          live[u] = t.dst_only == 0xffffffffu || g[u] / t.hn == t.dst_only;
+        }
+        if (live[u]) {
+          uint32_t ro = g[u] / t.hc, ho = g[u] - ro * t.hc;
+          if (t.use_map) { ro = t.map_rank[g[u]]; ho = t.map_head[g[u]]; }
+          v[u] = *reinterpret_cast<const V *>(
+              ptrs.src[ro] + base_old + ((uint64_t)(tok[u] * t.hc + ho) * cpv + j[u]) * W);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (live[u]) {
+          const uint32_t rn = g[u] / t.hn, hn = g[u] - rn * t.hn;
+          *reinterpret_cast<V *>(ptrs.dst[rn] + base_new +
+                                 ((uint64_t)(tok[u] * t.hn + hn) * cpv + j[u]) * W) = v[u];
+        }
+      }
+    }
+  }
+}
+
+template <typename V>
+__global__ void __launch_bounds__(256) kv_direct_kernel(const __grid_constant__ KvParams p) {
+  kv_direct_tiles<V>(p.t, p.ptrs, blockIdx.x, gridDim.x);
+}
+
+// Row-mapped variant of the direct kernel for the usual case that a CTA's 256 threads
+// cover whole logical token rows (256 % pieces-per-row == 0): a thread then keeps the same
+// (head, piece) for every token it touches, so its source / destination rank and in-block
+// offsets are fixed for the whole kernel and a tile costs two base offsets, U loads and U
+// stores.  The block ids of the next tile are fetched while the current one is in flight.
+template <int U>
+__device__ __forceinline__ void kv_rows_tiles(const KvTables &t, const RankPtrs &ptrs, uint64_t first,
+                                              uint64_t stride) {
+  const uint32_t cpv = t.head_bytes / 16, row = t.hkv * cpv, tpp = 256 / row;  // tokens per pass
+  const uint32_t rem = threadIdx.x % row, tok0 = threadIdx.x / row;
+  const uint32_t g = rem / cpv, j = rem - g * cpv;
+  uint32_t ro = g / t.hc, ho = g - ro * t.hc;
+  if (t.use_map) { ro = t.map_rank[g]; ho = t.map_head[g]; }
+  const uint32_t rn = g / t.hn, hn = g - rn * t.hn;
+  if (t.dst_only != 0xffffffffu && rn != t.dst_only) return;  // another rank writes that block
+  const uint8_t *sp = ptrs.src[ro] + ((uint64_t)(tok0 * t.hc + ho) * cpv + j) * 16;
+  uint8_t *dp = ptrs.dst[rn] + ((uint64_t)(tok0 * t.hn + hn) * cpv + j) * 16;
+  const uint64_t s_step = (uint64_t)tpp * t.hc * t.head_bytes, d_step = (uint64_t)tpp * t.hn * t.head_bytes;
+  const uint64_t blk_old = (uint64_t)t.block_tokens * t.hc * t.head_bytes;
+  const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
+  const uint64_t n_tiles = (uint64_t)t.n_pairs * t.n_lk;
+  uint64_t tile = first;
+  if (tile >= n_tiles) return;
+  uint32_t lk = (uint32_t)(tile / t.n_pairs), pr = (uint32_t)(tile - (uint64_t)lk * t.n_pairs);
+  uint32_t po = t.pair_old[pr], pn = t.pair_new[pr];
+  for (;;) {
+    const uint64_t tile2 = tile + stride;
+    uint32_t lk2 = lk, po2 = po, pn2 = pn;
+    if (tile2 < n_tiles) {
+      lk2 = (uint32_t)(tile2 / t.n_pairs);
+      const uint32_t pr2 = (uint32_t)(tile2 - (uint64_t)lk2 * t.n_pairs);
+      po2 = t.pair_old[pr2];
+      pn2 = t.pair_new[pr2];
+    }
+    const uint8_t *s = sp + ((uint64_t)lk * t.nb_old + po) * blk_old;
+    uint8_t *d = dp + ((uint64_t)lk * t.nb_new + pn) * blk_new;
+    uint4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (tok0 + u * tpp < t.block_tokens) v[u] = *reinterpret_cast<const uint4 *>(s + u * s_step);
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (tok0 + u * tpp < t.block_tokens) *reinterpret_cast<uint4 *>(d + u * d_step) = v[u];
+    if (tile2 >= n_tiles) break;
+    tile = tile2; lk = lk2; po = po2; pn = pn2;
+  }
+}
+
+template <int U>
+__global__ void __launch_bounds__(256) kv_rows_kernel(const __grid_constant__ KvParams p) {
+  kv_rows_tiles<U>(p.t, p.ptrs, blockIdx.x, gridDim.x);
+}
+
+// Passes the row-mapped copy needs for a block (0: the shape does not fit it).
+__host__ __device__ inline uint32_t kv_rows_passes(const KvTables &t) {
+  if (t.head_bytes % 16) return 0;
+  const uint32_t row = t.hkv * (t.head_bytes / 16);
+  if (row == 0 || row > 256 || 256 % row) return 0;
+  return (t.block_tokens + 256 / row - 1) / (256 / row);
+}
+
 // ---- vector path ------------------------------------------------------------------------
 
 struct VecParams {
   SegTables t;
   uint32_t tile_bytes;
   RankPtrs ptrs;
+};
+
+// The vector kernel with the tiles of a KV head re-split appended to its work: CTAs
+// [0, vec_ctas) walk the segment units, the others the KV tiles.  One launch then covers
+// a whole TP-changing step whose phases are too small for a launch each.
+struct VecKvParams {
+  SegTables t;
+  uint32_t tile_bytes;
+  uint32_t vec_ctas;     // CTAs that take segment units
+  uint32_t kv_passes;    // row-mapped copy: passes per block (1, 2, 4, 8); 0: the direct copy
+  RankPtrs ptrs;         // segment arenas
+  KvTables kv;
+  RankPtrs kv_ptrs;      // KV arenas
 };
 
 // One warp copies one tile to one destination: `rows` rows of cpr pieces, a pitch apart
@@ -390,18 +578,20 @@ __device__ __forceinline__ void warp_copy_tile(const uint8_t *sp, uint64_t src_p
 }
 
 // A CTA takes one unit at a time (its segment is parked in shared memory), a warp one tile.
-__global__ void __launch_bounds__(256, 4) vec_copy_kernel(const __grid_constant__ VecParams p) {
+// The CTA walks units first, first + stride, ...
+__device__ __forceinline__ void vec_copy_units(const SegTables &t, const RankPtrs &ptrs, uint32_t T,
+                                               uint32_t first, uint32_t stride) {
   __shared__ DevSeg s_sg;
   __shared__ Unit s_un;
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-  const uint32_t T = p.tile_bytes;
-  for (uint32_t u = blockIdx.x; u < p.t.n_units; u += gridDim.x) {
+  for (uint64_t u64 = first; u64 < t.n_units; u64 += stride) {
+    const uint32_t u = (uint32_t)u64;
     __syncthreads();  // everyone is done with the previous unit's segment
-    if (threadIdx.x == 0) s_un = p.t.units[u];
+    if (threadIdx.x == 0) s_un = t.units[u];
     if (threadIdx.x < 4) {
-      const uint32_t seg = p.t.units[u].seg;
+      const uint32_t seg = t.units[u].seg;
       reinterpret_cast<uint4 *>(&s_sg)[threadIdx.x] =
-          reinterpret_cast<const uint4 *>(&p.t.segs[seg])[threadIdx.x];
+          reinterpret_cast<const uint4 *>(&t.segs[seg])[threadIdx.x];
     }
     __syncthreads();
     const uint64_t run_bytes = s_sg.run_bytes;
@@ -425,16 +615,16 @@ __global__ void __launch_bounds__(256, 4) vec_copy_kernel(const __grid_constant_
         row_bytes = (uint32_t)run_bytes;
       }
       const uint64_t src_pitch = s_sg.src_pitch;
-      const uint8_t *sp = p.ptrs.src[s_sg.src_rank] + s_sg.src_off + (uint64_t)run * src_pitch + in_run;
+      const uint8_t *sp = ptrs.src[s_sg.src_rank] + s_sg.src_off + (uint64_t)run * src_pitch + in_run;
       const uint32_t n_dst = s_sg.n_dst, align = s_sg.align;
       for (uint32_t d = 0; d < n_dst; ++d) {
         uint64_t d_off = s_sg.dst_off, d_pitch = s_sg.dst_pitch;
         uint32_t d_rank = s_sg.dst_rank;
         if (n_dst > 1) {
-          const Dst dd = p.t.dsts[s_sg.dst_first + d];
+          const Dst dd = t.dsts[s_sg.dst_first + d];
           d_off = dd.off; d_pitch = dd.pitch; d_rank = dd.rank;
         }
-        uint8_t *dp = p.ptrs.dst[d_rank] + d_off + (uint64_t)run * d_pitch + in_run;
+        uint8_t *dp = ptrs.dst[d_rank] + d_off + (uint64_t)run * d_pitch + in_run;
         switch (align) {
           case 16: warp_copy_tile<uint4>(sp, src_pitch, dp, d_pitch, rows, row_bytes / 16, lane); break;
           case 8: warp_copy_tile<uint2>(sp, src_pitch, dp, d_pitch, rows, row_bytes / 8, lane); break;
@@ -447,118 +637,22 @@ __global__ void __launch_bounds__(256, 4) vec_copy_kernel(const __grid_constant_
   }
 }
 
-// ---- KV head re-split -------------------------------------------------------------------
-
-struct KvParams {
-  KvTables t;
-  RankPtrs ptrs;
-};
-
-// Direct variant: thread q of a tile owns piece q of the LOGICAL block
-// [token][global head][piece]; it reads the piece from the old rank that holds the
-// head and writes it to the new rank that will.  Reads of a warp cover whole token
-// rows of the old layout, writes whole head vectors of the new one.
-template <typename V>
-__global__ void __launch_bounds__(256) kv_direct_kernel(const __grid_constant__ KvParams p) {
-  __shared__ const uint8_t *s_src[EMOE_MAX_RANKS];
-  __shared__ uint8_t *s_dst[EMOE_MAX_RANKS];
-  if (threadIdx.x < EMOE_MAX_RANKS) {
-    s_src[threadIdx.x] = p.ptrs.src[threadIdx.x];
-    s_dst[threadIdx.x] = p.ptrs.dst[threadIdx.x];
-  }
-  __syncthreads();
-  constexpr uint32_t W = sizeof(V);
-  const KvTables &t = p.t;
-  const uint32_t cpv = t.head_bytes / W;     // pieces per head vector
-  const uint32_t row = t.hkv * cpv;          // pieces per logical token row
-  const uint32_t total = t.block_tokens * row;
-  const uint64_t blk_old = (uint64_t)t.block_tokens * t.hc * t.head_bytes;
-  const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
-  const uint64_t n_tiles = (uint64_t)t.n_pairs * t.n_lk;
-  for (uint64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-    const uint32_t lk = (uint32_t)(tile / t.n_pairs), pr = (uint32_t)(tile % t.n_pairs);
-    const uint64_t base_old = ((uint64_t)lk * t.nb_old + t.pair_old[pr]) * blk_old;
-    const uint64_t base_new = ((uint64_t)lk * t.nb_new + t.pair_new[pr]) * blk_new;
-    for (uint32_t q0 = threadIdx.x; q0 < total; q0 += blockDim.x * 4) {
-      V v[4];
-      uint32_t tok[4], g[4], j[4];
-      bool live[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const uint32_t q = q0 + u * blockDim.x;
-        live[u] = false;
-        if (q < total) {
-          tok[u] = q / row;
-          const uint32_t rem = q - tok[u] * row;
-          g[u] = rem / cpv;
-          j[u] = rem - g[u] * cpv;
-          live[u] = t.dst_only == 0xffffffffu || g[u] / t.hn == t.dst_only;
-        }
-        if (live[u]) {
-          uint32_t ro = g[u] / t.hc, ho = g[u] - ro * t.hc;
-          if (t.use_map) { ro = t.map_rank[g[u]]; ho = t.map_head[g[u]]; }
-          v[u] = *reinterpret_cast<const V *>(
-              s_src[ro] + base_old + ((uint64_t)(tok[u] * t.hc + ho) * cpv + j[u]) * W);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (live[u]) {
-          const uint32_t rn = g[u] / t.hn, hn = g[u] - rn * t.hn;
-          *reinterpret_cast<V *>(s_dst[rn] + base_new +
-                                 ((uint64_t)(tok[u] * t.hn + hn) * cpv + j[u]) * W) = v[u];
-        }
-      }
-    }
-  }
+__global__ void __launch_bounds__(256, 4) vec_copy_kernel(const __grid_constant__ VecParams p) {
+  vec_copy_units(p.t, p.ptrs, p.tile_bytes, blockIdx.x, gridDim.x);
 }
 
-
-// Row-mapped variant of the direct kernel for the usual case that a CTA's 256 threads
-// cover whole logical token rows (256 % pieces-per-row == 0): a thread then keeps the same
-// (head, piece) for every token it touches, so its source / destination rank and in-block
-// offsets are fixed for the whole kernel and a tile costs two base offsets, U loads and U
-// stores.  The block ids of the next tile are fetched while the current one is in flight.
-template <int U>
-__global__ void __launch_bounds__(256) kv_rows_kernel(const __grid_constant__ KvParams p) {
-  const KvTables &t = p.t;
-  const uint32_t cpv = t.head_bytes / 16, row = t.hkv * cpv, tpp = 256 / row;  // tokens per pass
-  const uint32_t rem = threadIdx.x % row, tok0 = threadIdx.x / row;
-  const uint32_t g = rem / cpv, j = rem - g * cpv;
-  uint32_t ro = g / t.hc, ho = g - ro * t.hc;
-  if (t.use_map) { ro = t.map_rank[g]; ho = t.map_head[g]; }
-  const uint32_t rn = g / t.hn, hn = g - rn * t.hn;
-  if (t.dst_only != 0xffffffffu && rn != t.dst_only) return;  // another rank writes that block
-  const uint8_t *sp = p.ptrs.src[ro] + ((uint64_t)(tok0 * t.hc + ho) * cpv + j) * 16;
-  uint8_t *dp = p.ptrs.dst[rn] + ((uint64_t)(tok0 * t.hn + hn) * cpv + j) * 16;
-  const uint64_t s_step = (uint64_t)tpp * t.hc * t.head_bytes, d_step = (uint64_t)tpp * t.hn * t.head_bytes;
-  const uint64_t blk_old = (uint64_t)t.block_tokens * t.hc * t.head_bytes;
-  const uint64_t blk_new = (uint64_t)t.block_tokens * t.hn * t.head_bytes;
-  const uint64_t n_tiles = (uint64_t)t.n_pairs * t.n_lk;
-  uint64_t tile = blockIdx.x;
-  if (tile >= n_tiles) return;
-  uint32_t lk = (uint32_t)(tile / t.n_pairs), pr = (uint32_t)(tile - (uint64_t)lk * t.n_pairs);
-  uint32_t po = t.pair_old[pr], pn = t.pair_new[pr];
-  for (;;) {
-    const uint64_t tile2 = tile + gridDim.x;
-    uint32_t lk2 = lk, po2 = po, pn2 = pn;
-    if (tile2 < n_tiles) {
-      lk2 = (uint32_t)(tile2 / t.n_pairs);
-      const uint32_t pr2 = (uint32_t)(tile2 - (uint64_t)lk2 * t.n_pairs);
-      po2 = t.pair_old[pr2];
-      pn2 = t.pair_new[pr2];
-    }
-    const uint8_t *s = sp + ((uint64_t)lk * t.nb_old + po) * blk_old;
-    uint8_t *d = dp + ((uint64_t)lk * t.nb_new + pn) * blk_new;
-    uint4 v[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u)
-      if (tok0 + u * tpp < t.block_tokens) v[u] = *reinterpret_cast<const uint4 *>(s + u * s_step);
-#pragma unroll
-    for (int u = 0; u < U; ++u)
-      if (tok0 + u * tpp < t.block_tokens) *reinterpret_cast<uint4 *>(d + u * d_step) = v[u];
-    if (tile2 >= n_tiles) break;
-    tile = tile2; lk = lk2; po = po2; pn = pn2;
+__global__ void __launch_bounds__(256, 4) vec_kv_kernel(const __grid_constant__ VecKvParams p) {
+  if (blockIdx.x < p.vec_ctas) {
+    vec_copy_units(p.t, p.ptrs, p.tile_bytes, blockIdx.x, p.vec_ctas);
+    return;
+  }
+  const uint64_t first = blockIdx.x - p.vec_ctas, stride = gridDim.x - p.vec_ctas;
+  switch (p.kv_passes) {
+    case 1: kv_rows_tiles<1>(p.kv, p.kv_ptrs, first, stride); break;
+    case 2: kv_rows_tiles<2>(p.kv, p.kv_ptrs, first, stride); break;
+    case 4: kv_rows_tiles<4>(p.kv, p.kv_ptrs, first, stride); break;
+    case 8: kv_rows_tiles<8>(p.kv, p.kv_ptrs, first, stride); break;
+    default: kv_direct_tiles<uint4>(p.kv, p.kv_ptrs, first, stride); break;
   }
 }
 
@@ -577,6 +671,7 @@ constexpr uint32_t kKvStagedCtasPerSm = 2;  // the per-tile chain of waits and b
 struct KvStagedParams {
   KvTables t;
   uint32_t stages, tile_bytes, n_pieces, chunk_bytes;  // chunk = one old rank's share of a block
+  unsigned long long wait_ns;
   int *status;
   RankPtrs ptrs;
 };
@@ -652,7 +747,7 @@ kv_staged_kernel(const __grid_constant__ KvStagedParams p) {
         pn2 = t.pair_new[pr2];
       }
       const uint32_t st = it % S, round = it / S;
-      if (round > 0 && !mbar_wait(smem_u32(&empty[st]), (round - 1) & 1)) { ok = false; break; }
+      if (round > 0 && !mbar_wait(smem_u32(&empty[st]), (round - 1) & 1, p.wait_ns, &s_abort)) { ok = false; break; }
       if (s_abort) { ok = false; break; }
       base_new_of[st] = ((uint64_t)lk * t.nb_new + pn) * blk_new;
       const uint64_t base_old = ((uint64_t)lk * t.nb_old + po) * blk_old;
@@ -665,7 +760,7 @@ kv_staged_kernel(const __grid_constant__ KvStagedParams p) {
     }
     if (ok) {  // end marker
       const uint32_t st = it % S, round = it / S;
-      if (round == 0 || mbar_wait(smem_u32(&empty[st]), (round - 1) & 1)) {
+      if (round == 0 || mbar_wait(smem_u32(&empty[st]), (round - 1) & 1, p.wait_ns, &s_abort)) {
         base_new_of[st] = kEnd;
         mbar_arrive(smem_u32(&full[st]));
       } else {
@@ -679,7 +774,7 @@ kv_staged_kernel(const __grid_constant__ KvStagedParams p) {
       const uint32_t back = it < S ? it : S;
       for (uint32_t j = 1; j <= back; ++j) {
         const uint32_t i2 = it - j;
-        (void)mbar_wait(smem_u32(&full[i2 % S]), (i2 / S) & 1);
+        (void)mbar_wait(smem_u32(&full[i2 % S]), (i2 / S) & 1, kDrainLimitNs);
       }
     }
   } else if (tid < kKvConsumers) {
@@ -691,7 +786,7 @@ kv_staged_kernel(const __grid_constant__ KvStagedParams p) {
       const uint32_t st = it % S, round = it / S, os = it % kKvOutStages;
       if (tid == 0) {
         int go = 1;
-        if (!mbar_wait(smem_u32(&full[st]), round & 1)) {
+        if (!mbar_wait(smem_u32(&full[st]), round & 1, p.wait_ns, &s_abort)) {
           s_abort = 1;
           atomicExch(p.status, (int)EMOE_ERR_DEVICE_TIMEOUT);
           go = 0;
@@ -745,6 +840,7 @@ constexpr uint32_t kKvTmaMaxBoxes = 64;
 struct KvTmaParams {
   KvTables t;
   uint32_t stages, tile_bytes, box_bytes, n_box, g;
+  unsigned long long wait_ns;
   int *status;
   CUtensorMap src[kKvTmaMaxRanks], dst[kKvTmaMaxRanks];
 };
@@ -800,7 +896,7 @@ __global__ void __launch_bounds__(64, 1) kv_tma_kernel(const __grid_constant__ K
         pn2 = t.pair_new[pr2];
       }
       const uint32_t st = it % S, round = it / S;
-      if (round > 0 && !mbar_wait(smem_u32(&empty[st]), (round - 1) & 1)) { ok = false; break; }
+      if (round > 0 && !mbar_wait(smem_u32(&empty[st]), (round - 1) & 1, p.wait_ns, &s_abort)) { ok = false; break; }
       if (s_abort) { ok = false; break; }
       // first token row of the block in the old / new arena tensors (< 2^31, checked on the host)
       const int32_t tok_old = (int32_t)(((uint64_t)lk * t.nb_old + po) * t.block_tokens);
@@ -814,7 +910,7 @@ __global__ void __launch_bounds__(64, 1) kv_tma_kernel(const __grid_constant__ K
     }
     if (ok) {  // end marker
       const uint32_t st = it % S, round = it / S;
-      if (round == 0 || mbar_wait(smem_u32(&empty[st]), (round - 1) & 1)) {
+      if (round == 0 || mbar_wait(smem_u32(&empty[st]), (round - 1) & 1, p.wait_ns, &s_abort)) {
         tok_new_of[st] = -1;
         mbar_arrive(smem_u32(&full[st]));
       } else {
@@ -828,14 +924,14 @@ __global__ void __launch_bounds__(64, 1) kv_tma_kernel(const __grid_constant__ K
       const uint32_t back = it < S ? it : S;
       for (uint32_t j = 1; j <= back; ++j) {
         const uint32_t i2 = it - j;
-        (void)mbar_wait(smem_u32(&full[i2 % S]), (i2 / S) & 1);
+        (void)mbar_wait(smem_u32(&full[i2 % S]), (i2 / S) & 1, kDrainLimitNs);
       }
     }
   } else if (tid == 32) {
     // ---------------- consumer ----------------
     for (uint32_t it = 0;; ++it) {
       const uint32_t st = it % S, round = it / S;
-      if (!mbar_wait(smem_u32(&full[st]), round & 1)) {
+      if (!mbar_wait(smem_u32(&full[st]), round & 1, p.wait_ns, &s_abort)) {
         s_abort = 1;
         atomicExch(p.status, (int)EMOE_ERR_DEVICE_TIMEOUT);
         break;
@@ -863,22 +959,28 @@ size_t bulk_smem_bytes(uint32_t tile_bytes, uint32_t stages) {
   return (size_t)stages * tile_bytes + stages * (sizeof(TileInfo) + 2 * sizeof(uint64_t));
 }
 
-size_t bulk_smem_limit() {
-  cudaFuncAttributes a{};
-  if (cudaFuncGetAttributes(&a, bulk_copy_kernel) != cudaSuccess) {
-    (void)cudaGetLastError();
-    return 200 * 1024;
-  }
-  return 227 * 1024 - a.sharedSizeBytes;
-}
+size_t bulk_smem_limit() { return kBulkSmemLimit; }
 
+// Dynamic shared memory opt-in of the ring kernels.  The attribute belongs to the device
+// that is current when it is set, so this runs once per device ordinal.
 cudaError_t kernels_init() {
-  cudaError_t e = cudaFuncSetAttribute(bulk_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)bulk_smem_limit());
+  static std::mutex mu;
+  static bool done[kMaxDevices] = {};
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  if (done[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(bulk_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)kBulkSmemLimit);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(kv_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(kv_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  e = cudaFuncSetAttribute(kv_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e != cudaSuccess) return e;
+  done[dev] = true;
+  return cudaSuccess;
 }
 
 cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, const BulkConfig &c,
@@ -886,8 +988,8 @@ cudaError_t launch_bulk_copy(const SegTables &t, const RankPtrs &ptrs, const Bul
   if (t.n_units == 0) return cudaSuccess;
   if (c.stages < 2 || c.stages > kMaxStages || c.tile_bytes % 128 != 0) return cudaErrorInvalidValue;
   const size_t smem = bulk_smem_bytes(c.tile_bytes, c.stages);
-  if (bulk_smem_bytes(c.tile_bytes, c.stages) > bulk_smem_limit()) return cudaErrorInvalidValue;
-  BulkParams p{t, c.tile_bytes, c.stages, c.hints, status, ctr, ptrs};
+  if (smem > kBulkSmemLimit) return cudaErrorInvalidValue;
+  BulkParams p{t, c.tile_bytes, c.stages, c.hints, c.pace_ns, c.wait_ns, status, ctr, ptrs};
   if (grid > t.n_units) grid = t.n_units;
   bulk_copy_kernel<<<grid, 64, smem, stream>>>(p);
   return cudaGetLastError();
@@ -899,6 +1001,43 @@ cudaError_t launch_vec_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t t
   VecParams p{t, tile_bytes, ptrs};
   if (grid > t.n_units) grid = t.n_units;
   vec_copy_kernel<<<grid, 256, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+bool vec_kv_supported(const KvTables &kv) { return kv.head_bytes % 16 == 0; }
+
+cudaError_t launch_vec_kv_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
+                               const KvTables &kv, const RankPtrs &kv_ptrs, uint32_t grid,
+                               bool unbounded, cudaStream_t stream) {
+  const uint64_t n_tiles = (uint64_t)kv.n_pairs * kv.n_lk;
+  if (n_tiles == 0) return launch_vec_copy(t, ptrs, tile_bytes, unbounded ? 0xffffffffu : grid, stream);
+  if (t.n_units == 0 && n_tiles == 0) return cudaSuccess;
+  VecKvParams p{};
+  p.t = t;
+  p.tile_bytes = tile_bytes;
+  p.ptrs = ptrs;
+  p.kv = kv;
+  p.kv_ptrs = kv_ptrs;
+  const uint32_t passes = kv_rows_passes(kv);
+  p.kv_passes = passes == 1 ? 1 : passes == 2 ? 2 : passes >= 3 && passes <= 4 ? 4 :
+                passes >= 5 && passes <= 8 ? 8 : 0;
+  // no budget: one CTA per segment unit and one per KV tile (the hardware scheduler balances
+  // them); with a budget the CTAs are split in proportion to the two kinds of work
+  uint64_t vec_ctas, kv_ctas;
+  if (unbounded) {
+    vec_ctas = t.n_units;
+    kv_ctas = n_tiles;
+  } else {
+    if (grid < 2) grid = 2;
+    vec_ctas = t.n_units == 0 ? 0 : (uint64_t)grid * t.n_units / (t.n_units + n_tiles);
+    if (t.n_units && vec_ctas == 0) vec_ctas = 1;
+    if (vec_ctas > t.n_units) vec_ctas = t.n_units;
+    kv_ctas = grid - vec_ctas;
+    if (kv_ctas > n_tiles) kv_ctas = n_tiles;
+  }
+  if (vec_ctas + kv_ctas > 0x7fffffffull) kv_ctas = 0x7fffffffull - vec_ctas;
+  p.vec_ctas = (uint32_t)vec_ctas;
+  vec_kv_kernel<<<(uint32_t)(vec_ctas + kv_ctas), 256, 0, stream>>>(p);
   return cudaGetLastError();
 }
 
@@ -993,7 +1132,8 @@ bool kv_staged_supported(const KvTables &t, uint32_t *stages_out) {
 }
 
 cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, uint32_t grid,
-                           bool unbounded, int *status, cudaStream_t stream) {
+                           bool unbounded, int *status, unsigned long long wait_ns,
+                           cudaStream_t stream) {
   const uint64_t n_tiles = (uint64_t)t.n_pairs * t.n_lk;
   if (n_tiles == 0) return cudaSuccess;
   KvParams p{t, ptrs};
@@ -1008,6 +1148,7 @@ cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, ui
     tp.box_bytes = t.block_tokens * g * hb;
     tp.n_box = t.hkv / g;
     tp.g = g;
+    tp.wait_ns = wait_ns;
     tp.status = status;
     bool ok = true;
     for (uint32_t r = 0; ok && r < c; ++r)
@@ -1025,7 +1166,7 @@ cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, ui
   }
   if (mode == 2 && status && kv_staged_supported(t, &stages)) {
     const uint32_t tile = t.block_tokens * t.hkv * hb;
-    KvStagedParams sp{t, stages, tile, tile / 16, t.block_tokens * t.hc * hb, status, ptrs};
+    KvStagedParams sp{t, stages, tile, tile / 16, t.block_tokens * t.hc * hb, wait_ns, status, ptrs};
     // two CTAs per budgeted SM; with no budget, 1.5 per SM measured best (6.6 TB/s on the
     // large-expert-count shape against 6.0 with 2 and 5.6 with 1)
     grid = unbounded ? grid * 3 / 2 : grid * kKvStagedCtasPerSm;
@@ -1039,10 +1180,9 @@ cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, ui
   const uint64_t want = unbounded ? n_tiles : (uint64_t)grid * 8;
   grid = (uint32_t)(want < n_tiles ? want : n_tiles);
   if (n_tiles > 0x7fffffffull && unbounded) grid = 0x7fffffffu;
-  if (mode != 4 && hb % 16 == 0) {
+  if (mode != 4) {
     // whole token rows per CTA pass, and few enough passes: the row-mapped kernel
-    const uint32_t row = t.hkv * (hb / 16);
-    const uint32_t passes = row <= 256 && 256 % row == 0 ? (t.block_tokens + 256 / row - 1) / (256 / row) : 0;
+    const uint32_t passes = kv_rows_passes(t);
     if (passes == 1) { kv_rows_kernel<1><<<grid, 256, 0, stream>>>(p); return cudaGetLastError(); }
     if (passes == 2) { kv_rows_kernel<2><<<grid, 256, 0, stream>>>(p); return cudaGetLastError(); }
     if (passes >= 3 && passes <= 4) { kv_rows_kernel<4><<<grid, 256, 0, stream>>>(p); return cudaGetLastError(); }
@@ -1102,7 +1242,6 @@ cudaError_t launch_gen_units(const DevSeg *segs, const uint32_t *seg_idx, const 
 static __device__ __align__(256) uint32_t g_kv_static_pairs[2 * EMOE_STATIC_KV_MAX_PAIRS];
 
 namespace {
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mu;
 uint32_t *g_static_ptr[kMaxDevices] = {};
 int g_static_sms[kMaxDevices] = {};
@@ -1148,7 +1287,7 @@ emoe_status_t launch_kv_copy_static(const KvTables &shape_only, const uint32_t *
   KvTables t = shape_only;
   t.pair_old = d_old;
   t.pair_new = d_new;
-  const cudaError_t e = launch_kv_copy(t, ptrs, 1, (uint32_t)sms, false, nullptr, stream);
+  const cudaError_t e = launch_kv_copy(t, ptrs, 1, (uint32_t)sms, false, nullptr, 0, stream);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
     return EMOE_ERR_CUDA;

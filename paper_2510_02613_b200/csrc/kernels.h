@@ -64,6 +64,8 @@ struct KvTables {  // device pointers + shape constants of the KV head re-split
 
 struct BulkConfig {
   uint32_t tile_bytes, stages, hints;
+  uint32_t pace_ns;             // least time between a CTA's full-tile loads; 0 = unpaced
+  unsigned long long wait_ns;   // bound of every device-side wait
 };
 // Dynamic shared memory the bulk kernel needs / may use at most.
 size_t bulk_smem_bytes(uint32_t tile_bytes, uint32_t stages);
@@ -85,7 +87,14 @@ constexpr uint32_t kKvTmaMaxRanks = 12;  // tensor maps travel in the kernel par
 bool kv_staged_supported(const KvTables &t, uint32_t *stages_out);
 bool kv_tma_supported(const KvTables &t, uint32_t *stages_out);
 cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, uint32_t grid,
-                           bool unbounded, int *status, cudaStream_t stream);
+                           bool unbounded, int *status, unsigned long long wait_ns,
+                           cudaStream_t stream);
+// The vector path and the direct KV head re-split in ONE launch (head vectors must be
+// multiples of 16 bytes: vec_kv_supported).  grid / unbounded as for launch_kv_copy.
+bool vec_kv_supported(const KvTables &kv);
+cudaError_t launch_vec_kv_copy(const SegTables &t, const RankPtrs &ptrs, uint32_t tile_bytes,
+                               const KvTables &kv, const RankPtrs &kv_ptrs, uint32_t grid,
+                               bool unbounded, cudaStream_t stream);
 
 // KV head re-split with its block-pair list in a fixed __device__ array of the library
 // image (no allocation).  pair_old / pair_new: host arrays of n_pairs ids.  Returns
@@ -102,7 +111,8 @@ cudaError_t launch_gen_units(const DevSeg *segs, const uint32_t *seg_idx, const 
                              uint32_t tile_bytes, uint32_t unit_tiles, uint32_t seg_offset, Unit *out,
                              cudaStream_t stream);
 
-// One-time per-process kernel attribute setup (dynamic shared memory opt-in).
+// Kernel attribute setup (dynamic shared memory opt-in) for the CURRENT device; cheap after
+// the first call on a device.
 cudaError_t kernels_init();
 
 }  // namespace emoe

@@ -97,48 +97,23 @@ emoe_status_t read_block_pairs(const emoe_shape_t &sh, const emoe_config_t &o,
 
 // ---- experts ----------------------------------------------------------------------------
 
-// slab: distance between consecutive slots of an arena (= m for the dense layout; the
-// paged store pads every matrix to its allocation granularity).  remaps: if non-null,
-// a destination slot whose source sits on the same rank index is recorded there instead
-// of being copied (that device already holds the bytes).
-// fused_w13 (dense layout only): per layer a [n][gate|up] tensor, then the [n][down] one.
-void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &pn, uint64_t slab,
-                  std::vector<Remap> *remaps, bool fused_w13, PhasePlan *pp) {
+struct ExpertMove { int rs, ss, rd, sd; };
+
+// Moves -> segments.  slots_old / slots_new: slots per arena (the slot stride of a layer slab).
+// Single-destination sources: runs of consecutive slots on both sides merge (dense layout
+// only); a source with several destinations becomes one segment that is read once.
+void emit_expert_moves(const emoe_shape_t &sh, const std::vector<uint64_t> &slots_old,
+                       const std::vector<uint64_t> &slots_new, uint64_t slab,
+                       const std::vector<ExpertMove> &moves, std::map<std::pair<int, int>, int> &fan,
+                       bool fused_w13, PhasePlan *pp) {
   const uint64_t m = (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes;
   const uint32_t runs = (uint32_t)sh.n_layers * 3;
-  const int n_experts = sh.n_routed + sh.n_shared;
-  for (int r = 0; r < po.ep; ++r) pp->arena_old.push_back(runs * po.ids[r].size() * slab);
-  for (int r = 0; r < pn.ep; ++r) pp->arena_new.push_back(runs * pn.ids[r].size() * slab);
-
-  // every old copy of every expert, in (rank, slot) order
-  std::vector<std::vector<std::pair<int, int>>> copies(n_experts);
-  for (int r = 0; r < po.ep; ++r)
-    for (int s = 0; s < (int)po.ids[r].size(); ++s) copies[po.ids[r][s]].push_back({r, s});
-
-  // source of every destination slot: the copy on the same rank index, else the first
-  struct Move { int rs, ss, rd, sd; };
-  std::vector<Move> moves;
-  std::map<std::pair<int, int>, int> fan;  // (src rank, src slot) -> number of destinations
-  for (int rd = 0; rd < pn.ep; ++rd)
-    for (int sd = 0; sd < (int)pn.ids[rd].size(); ++sd) {
-      const auto &c = copies[pn.ids[rd][sd]];
-      std::pair<int, int> src = c.front();
-      for (const auto &x : c)
-        if (x.first == rd) { src = x; break; }
-      if (remaps && src.first == rd) {
-        remaps->push_back({(uint32_t)src.first, (uint32_t)src.second, (uint32_t)rd, (uint32_t)sd});
-        continue;
-      }
-      moves.push_back({src.first, src.second, rd, sd});
-      fan[src]++;
-    }
-
   // single-destination sources: merge runs of consecutive slots on both sides (dense layout only)
   std::map<std::pair<int, int>, std::vector<Dst>> multi;
   size_t i = 0;
   while (i < moves.size()) {
-    const Move &a = moves[i];
-    const uint64_t n_old = po.ids[a.rs].size(), n_new = pn.ids[a.rd].size();
+    const ExpertMove &a = moves[i];
+    const uint64_t n_old = slots_old[a.rs], n_new = slots_new[a.rd];
     if (fan[{a.rs, a.ss}] > 1) {
       // fused layout: off = slot index, pitch = slot count; resolved to bytes below
       if (fused_w13) multi[{a.rs, a.ss}].push_back({(uint64_t)a.sd, n_new, (uint32_t)a.rd, 0});
@@ -175,7 +150,7 @@ void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &
   for (const auto &kv : multi) {
     Segment s{};
     s.src_rank = (uint32_t)kv.first.first;
-    const uint64_t n_old = po.ids[kv.first.first].size(), ss = (uint64_t)kv.first.second;
+    const uint64_t n_old = slots_old[kv.first.first], ss = (uint64_t)kv.first.second;
     if (!fused_w13) {
       s.src_off = ss * slab;
       s.run_bytes = m;
@@ -198,6 +173,48 @@ void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &
       finish_segment(pp, s, d2);
     }
   }
+}
+
+
+// slab: distance between consecutive slots of an arena (= m for the dense layout; the
+// paged store pads every matrix to its allocation granularity).  remaps: if non-null,
+// a destination slot whose source sits on the same rank index is recorded there instead
+// of being copied (that device already holds the bytes).
+// fused_w13 (dense layout only): per layer a [n][gate|up] tensor, then the [n][down] one.
+void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &pn, uint64_t slab,
+                  std::vector<Remap> *remaps, bool fused_w13, PhasePlan *pp) {
+  const uint64_t m = (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes;
+  const uint32_t runs = (uint32_t)sh.n_layers * 3;
+  const int n_experts = sh.n_routed + sh.n_shared;
+  for (int r = 0; r < po.ep; ++r) pp->arena_old.push_back(runs * po.ids[r].size() * slab);
+  for (int r = 0; r < pn.ep; ++r) pp->arena_new.push_back(runs * pn.ids[r].size() * slab);
+
+  // every old copy of every expert, in (rank, slot) order
+  std::vector<std::vector<std::pair<int, int>>> copies(n_experts);
+  for (int r = 0; r < po.ep; ++r)
+    for (int s = 0; s < (int)po.ids[r].size(); ++s) copies[po.ids[r][s]].push_back({r, s});
+
+  // source of every destination slot: the copy on the same rank index, else the first
+  std::vector<ExpertMove> moves;
+  std::vector<uint64_t> slots_old, slots_new;
+  for (int r = 0; r < po.ep; ++r) slots_old.push_back(po.ids[r].size());
+  for (int r = 0; r < pn.ep; ++r) slots_new.push_back(pn.ids[r].size());
+  std::map<std::pair<int, int>, int> fan;  // (src rank, src slot) -> number of destinations
+  for (int rd = 0; rd < pn.ep; ++rd)
+    for (int sd = 0; sd < (int)pn.ids[rd].size(); ++sd) {
+      const auto &c = copies[pn.ids[rd][sd]];
+      std::pair<int, int> src = c.front();
+      for (const auto &x : c)
+        if (x.first == rd) { src = x; break; }
+      if (remaps && src.first == rd) {
+        remaps->push_back({(uint32_t)src.first, (uint32_t)src.second, (uint32_t)rd, (uint32_t)sd});
+        continue;
+      }
+      moves.push_back({src.first, src.second, rd, sd});
+      fan[src]++;
+    }
+
+  emit_expert_moves(sh, slots_old, slots_new, slab, moves, fan, fused_w13, pp);
 }
 
 // ---- attention --------------------------------------------------------------------------
@@ -429,6 +446,80 @@ emoe_status_t build_paged_expert_plan(const emoe_shape_t &sh, const emoe_config_
   st = read_placement(n, sh.n_routed + sh.n_shared, &pn);
   if (st != EMOE_OK) return st;
   plan_experts(sh, po, pn, slab, remaps, false, pp);
+  return EMOE_OK;
+}
+
+emoe_status_t build_inplace_expert_plan(const emoe_shape_t &sh, int ep_old, const int32_t *off_old,
+                                        const int32_t *ids_old, int ep_new, const int32_t *cap_new,
+                                        const int32_t *want_off, const int32_t *want_ids,
+                                        PhasePlan *pp, std::vector<std::vector<int32_t>> *slot_new) {
+  if (sh.n_layers <= 0 || sh.n_routed <= 0 || sh.n_shared < 0 || sh.d_model <= 0 || sh.d_ff <= 0 ||
+      sh.elem_bytes <= 0)
+    return EMOE_ERR_SHAPE;
+  if (ep_old < 1 || ep_new < 1 || !off_old || !ids_old || !cap_new || !want_off || !want_ids)
+    return EMOE_ERR_INVALID_ARG;
+  if (ep_old > EMOE_MAX_RANKS || ep_new > EMOE_MAX_RANKS) return EMOE_ERR_UNSUPPORTED;
+  const int n_experts = sh.n_routed + sh.n_shared;
+  if (off_old[0] != 0 || want_off[0] != 0) return EMOE_ERR_PLACEMENT;
+  // old tables: ids in range or -1, an expert at most once per rank
+  std::vector<std::pair<int, int>> first_copy(n_experts, {-1, -1});   // smallest (rank, slot)
+  for (int r = 0; r < ep_old; ++r) {
+    if (off_old[r + 1] < off_old[r]) return EMOE_ERR_PLACEMENT;
+    std::vector<char> seen(n_experts, 0);
+    for (int i = off_old[r]; i < off_old[r + 1]; ++i) {
+      const int32_t e = ids_old[i];
+      if (e == -1) continue;
+      if (e < 0 || e >= n_experts || seen[e]) return EMOE_ERR_PLACEMENT;
+      seen[e] = 1;
+      if (first_copy[e].first < 0) first_copy[e] = {r, i - off_old[r]};
+    }
+  }
+  const uint64_t m = (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes;
+  const uint32_t runs = (uint32_t)sh.n_layers * 3;
+  std::vector<uint64_t> slots_old, slots_new;
+  for (int r = 0; r < ep_old; ++r) {
+    slots_old.push_back((uint64_t)(off_old[r + 1] - off_old[r]));
+    pp->arena_old.push_back(runs * slots_old.back() * m);
+  }
+  slot_new->assign(ep_new, {});
+  std::vector<ExpertMove> moves;
+  std::map<std::pair<int, int>, int> fan;
+  for (int r = 0; r < ep_new; ++r) {
+    if (cap_new[r] < 0 || want_off[r + 1] < want_off[r]) return EMOE_ERR_INVALID_ARG;
+    const bool stays = r < ep_old;
+    if (stays && (uint64_t)cap_new[r] != slots_old[r]) return EMOE_ERR_INVALID_ARG;  // same arena
+    slots_new.push_back((uint64_t)cap_new[r]);
+    pp->arena_new.push_back(runs * slots_new.back() * m);
+    std::vector<int32_t> &mine = (*slot_new)[r];
+    mine.assign(cap_new[r], -1);
+    std::vector<char> free_before(cap_new[r], 1), wanted(n_experts, 0);
+    for (int i = want_off[r]; i < want_off[r + 1]; ++i) {
+      const int32_t e = want_ids[i];
+      if (e < 0 || e >= n_experts || wanted[e]) return EMOE_ERR_PLACEMENT;
+      if (first_copy[e].first < 0) return EMOE_ERR_PLACEMENT;   // nobody holds it: it would be lost
+      wanted[e] = 1;
+    }
+    std::vector<char> held(n_experts, 0);
+    if (stays)
+      for (int s = 0; s < cap_new[r]; ++s) {
+        const int32_t e = ids_old[off_old[r] + s];
+        if (e < 0) continue;
+        free_before[s] = 0;                     // occupied before the step: never overwritten by it
+        if (wanted[e]) { mine[s] = e; held[e] = 1; }
+      }
+    int next_free = 0;
+    for (int i = want_off[r]; i < want_off[r + 1]; ++i) {
+      const int32_t e = want_ids[i];
+      if (held[e]) continue;
+      while (next_free < cap_new[r] && !free_before[next_free]) ++next_free;
+      if (next_free == cap_new[r]) return EMOE_ERR_TOO_LARGE;
+      mine[next_free] = e;
+      moves.push_back({first_copy[e].first, first_copy[e].second, r, next_free});
+      fan[first_copy[e]]++;
+      ++next_free;
+    }
+  }
+  emit_expert_moves(sh, slots_old, slots_new, m, moves, fan, false, pp);
   return EMOE_OK;
 }
 

@@ -32,7 +32,10 @@ def test_c1_tiny_all_phases(inverse):
         for phase in range(3):
             check_phase_full(wl, plan, phase)
         check_step_full(wl, plan)
-        assert plan.num_launches(E.PHASE_STEP) == 2     # one vector launch + the KV re-split
+        assert plan.num_launches(E.PHASE_STEP) == 1     # vector work and KV re-split share a kernel
+        plan.set_tuning(serial=2)
+        assert plan.num_launches(E.PHASE_STEP) == 2     # ... unless told to keep them apart
+        check_step_full(wl, plan)
 
 
 @pytest.mark.parametrize("name", ["c2_mid", "c3_fine", "c4_large"])
@@ -54,7 +57,10 @@ TUNINGS = [dict(path=1), dict(path=2), dict(bulk_tile_bytes=8192, bulk_stages=3)
            dict(kv_order=3, kv_mode=2), dict(kv_order=1, unit_order=1),
            dict(kv_order=3, bulk_tile_bytes=16384), dict(kv_mode=3), dict(kv_mode=3, max_ctas=5),
            dict(kv_mode=3, kv_order=3), dict(kv_mode=4), dict(unit_order=2, path=2),
-           dict(unit_order=3, path=2, max_ctas=5), dict(path=2, max_ctas=1)]
+           dict(unit_order=3, path=2, max_ctas=5), dict(path=2, max_ctas=1),
+           dict(serial=1, path=2), dict(serial=2), dict(bw_limit_gbs=300, path=2),
+           dict(bw_limit_gbs=4000, path=2, max_ctas=16), dict(bulk_min_run=256, path=2),
+           dict(bulk_min_run=1024), dict(wait_limit_us=2000000, path=2)]
 
 
 @pytest.mark.parametrize("tuning", TUNINGS, ids=lambda t: "-".join("%s%s" % kv for kv in t.items()))
@@ -67,6 +73,7 @@ def test_tunings_do_not_change_the_result(tuning):
             plan.set_tuning(**tuning)
             for phase in range(3):
                 check_phase_full(wl, plan, phase)
+            check_step_full(wl, plan)
 
 
 ODD = [
@@ -199,10 +206,10 @@ def test_pipelined_host_step_with_a_ragged_last_chunk():
 
 
 @pytest.mark.parametrize("name", ["c2_mid", "c3_fine", "c4_large"])
-def test_full_size_configs_sampled_layers(name):
+def test_full_size_configs_every_layer(name):
     """The benchmark's launch configuration at full size - the whole step through
-    emoe_reshard_step with all arenas resident; first, middle and last layer compared in
-    full with the oracle (layers are independent in every phase)."""
+    emoe_reshard_step with all arenas resident; EVERY layer compared in full with the
+    oracle (layers are independent in every phase, so the oracle takes them one by one)."""
     wl = W.make_workload(name)
     L = wl.shape.n_layers
     torch.cuda.empty_cache()
@@ -213,7 +220,7 @@ def test_full_size_configs_sampled_layers(name):
         torch.cuda.synchronize()
         assert plan.device_status() == 0
         for phase in range(3):
-            check_phase_layers(wl, plan, phase, src[phase], dst[phase], [0, L // 2, L - 1])
+            check_phase_layers(wl, plan, phase, src[phase], dst[phase], range(L))
         # and the per-phase entry points write the same bytes
         for phase in (E.PHASE_ATTN, E.PHASE_KV):
             again = WD.alloc_const(plan.arena_bytes(phase, E.SIDE_NEW))
@@ -223,6 +230,118 @@ def test_full_size_configs_sampled_layers(name):
             del again
         del src, dst
     torch.cuda.empty_cache()
+
+
+def _victim_graph(wl, expert_arena, stream, n_layers):
+    """The overlap case's concurrent kernel: a grouped expert GEMM (torch.bmm, a fixture of
+    the test and of the benchmark, not part of the library) reading expert weights of old
+    rank 0, captured as a CUDA graph on `stream`."""
+    v = wl.victim
+    A, T, D, F = v["active_experts"], v["tokens"], v["d_model"], v["d_ff"]
+    slab = expert_arena.view(torch.bfloat16).view(n_layers, 3, len(wl.old.placement[0]), D * F)
+    x = (torch.randn(A, T, D, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+
+    def gemm_step(l):
+        wg, wu = slab[l, 0, :A].view(A, D, F), slab[l, 1, :A].view(A, D, F)
+        wd = slab[l, 2, :A].view(A, F, D)
+        return torch.bmm(torch.bmm(x, wg) * torch.bmm(x, wu), wd)
+
+    with torch.cuda.stream(stream):
+        for l in range(n_layers):
+            gemm_step(l)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(4):
+                gemm_step(i % n_layers)
+    torch.cuda.synchronize()
+    return graph
+
+
+@pytest.mark.parametrize("name", ["c5_overlap", "c4_large"])
+def test_overlap_config_is_bit_exact_beside_a_live_gemm(name):
+    """The overlap configuration: the reshard on a least-priority stream while a grouped
+    expert GEMM keeps running on a high-priority stream, for the default CTA budget and
+    for 96 / 48 / 24 CTAs and a bandwidth limit.  Whole destination arenas against the
+    oracle every time; the GEMM must really have overlapped the reshard."""
+    n_layers = 2
+    wl = W.make_workload(name, n_layers=n_layers)
+    if wl.victim is None:
+        wl = R(wl, victim=W.make_workload("c5_overlap").victim)
+        wl = R(wl, victim=dict(wl.victim, d_ff=wl.shape.d_ff))
+    least, greatest = torch.cuda.Stream.priority_range()
+    s_low, s_high = torch.cuda.Stream(priority=least), torch.cuda.Stream(priority=greatest)
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        src = [WD.alloc_filled(plan.arena_bytes(ph, E.SIDE_OLD), wl.seed, KINDS[ph]) for ph in range(3)]
+        dst = [WD.alloc_const(plan.arena_bytes(ph, E.SIDE_NEW)) for ph in range(3)]
+        want = []
+        for ph in range(3):
+            w = [np.full(t.numel(), WD.FILL_BYTE, np.uint8) for t in dst[ph]]
+            from gpu_util import oracle_phase
+            oracle_phase(wl, ph, [t.cpu().numpy() for t in src[ph]], w)
+            want.append(w)
+        graph = _victim_graph(wl, src[0][0], s_high, n_layers)
+        for tuning in (dict(), dict(max_ctas=96), dict(max_ctas=48), dict(max_ctas=24),
+                       dict(bw_limit_gbs=3000), dict(max_ctas=48, bw_limit_gbs=1500, bulk_stages=3)):
+            plan.set_tuning(**tuning)
+            for g in dst:
+                for t in g:
+                    t.fill_(WD.FILL_BYTE)
+            torch.cuda.synchronize()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            with torch.cuda.stream(s_high):
+                ev[0].record(s_high)
+                for _ in range(10):
+                    graph.replay()
+            ev[2].record(s_low)
+            plan.reshard_step(src, dst, s_low)
+            ev[3].record(s_low)
+            with torch.cuda.stream(s_high):
+                for _ in range(60):
+                    graph.replay()
+                ev[1].record(s_high)
+            torch.cuda.synchronize()
+            # the reshard started before the GEMM loop ended and ended after it had started
+            assert ev[0].elapsed_time(ev[3]) > 0 and ev[2].elapsed_time(ev[1]) > 0, tuning
+            assert plan.device_status() == 0
+            for ph in range(3):
+                for r, (t, w) in enumerate(zip(dst[ph], want[ph])):
+                    assert np.array_equal(t.cpu().numpy(), w), (tuning, ph, r)
+
+
+def test_expired_device_wait_is_reported_and_the_plan_recovers():
+    """Every device-side wait is bounded.  wait_limit_us = -1 makes the first wait that is not
+    already satisfied expire: the kernel must return by itself, the call and the following
+    synchronise must succeed, the status word must read EMOE_ERR_DEVICE_TIMEOUT (the output
+    of that launch is undefined and is not looked at), and after the word has been cleared
+    the same plan - and a fresh one - must be bit-exact again."""
+    wl = W.make_workload("c1_tiny")
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        plan.set_tuning(path=2, wait_limit_us=-1)           # forced onto the ring kernel
+        so, sn = plan.arena_bytes(E.PHASE_EXPERTS, E.SIDE_OLD), plan.arena_bytes(E.PHASE_EXPERTS, E.SIDE_NEW)
+        src = WD.alloc_filled(so, wl.seed, W.KIND_EXPERTS)
+        dst = WD.alloc_const(sn)
+        plan.reshard_experts(src, dst)
+        torch.cuda.synchronize()                            # returns: no trap, no endless spin
+        assert plan.device_status() == 10
+        plan.clear_device_status()
+        assert plan.device_status() == 0
+        plan.set_tuning(path=2)                             # default bound again
+        for phase in range(3):
+            check_phase_full(wl, plan, phase)
+        # the staged and the tensor-map KV kernels have the same bounded waits
+        for kv_mode in (2, 3):
+            plan.set_tuning(kv_mode=kv_mode, wait_limit_us=-1)
+            ko, kn = plan.arena_bytes(E.PHASE_KV, E.SIDE_OLD), plan.arena_bytes(E.PHASE_KV, E.SIDE_NEW)
+            ks, kd = WD.alloc_filled(ko, wl.seed, W.KIND_KV), WD.alloc_const(kn)
+            plan.reshard_kv(ks, kd)
+            torch.cuda.synchronize()
+            assert plan.device_status() == 10
+            plan.clear_device_status()
+            plan.set_tuning(kv_mode=kv_mode)
+            check_phase_full(wl, plan, E.PHASE_KV)
+    with E.Plan(wl.shape, wl.old, wl.new) as fresh:
+        check_step_full(wl, fresh)
 
 
 def test_maximum_rank_counts():

@@ -250,3 +250,29 @@ def test_header_is_plain_c_and_usable_from_a_c_program(tmp_path):
     out = subprocess.run([exe], capture_output=True, text=True)
     assert out.returncode == 0, (out.returncode, out.stdout, out.stderr)
     assert "c abi ok" in out.stdout
+
+
+def test_host_only_plan_and_its_tuning_make_no_cuda_call():
+    """A host-only plan - creation, tuning, local rank, queries - must work in a process
+    that cannot see any CUDA device at all."""
+    import subprocess
+    import sys
+    code = r"""
+import paper_2510_02613_b200 as E, workloads as W
+wl = W.make_workload("c4_large", n_layers=1)
+with E.Plan(wl.shape, wl.old, wl.new, host_only=True) as p:
+    p.set_tuning(max_ctas=24, bulk_tile_bytes=16384, bulk_stages=8, bw_limit_gbs=1000)
+    p.set_tuning(bulk_min_run=1024)
+    p.set_local_rank(1)
+    assert p.num_launches(E.PHASE_STEP) >= 1
+    try:
+        p.set_tuning(bulk_tile_bytes=65536, bulk_stages=16)   # does not fit shared memory
+    except E.EmoeError as e:
+        assert e.code == 1
+    else:
+        raise SystemExit("oversized ring accepted")
+print("ok")
+"""
+    env = dict(os.environ, CUDA_VISIBLE_DEVICES="", PYTHONPATH=ROOT)
+    out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, cwd=ROOT)
+    assert out.returncode == 0 and out.stdout.strip() == "ok", out.stderr[-2000:]

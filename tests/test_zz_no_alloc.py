@@ -4,10 +4,11 @@ that cannot afford the implicit synchronisation of cudaMalloc.  Such a caller ma
 host-only plan (no CUDA call) and uses this entry point, whose only scratch is a fixed
 array inside the library image.
 
-The check: through the C ABI, on two calls in a row that share that array, the output
-must be byte-identical to emoe_reshard_kv (the tolerance of every parity test here is
-zero: this is byte movement).  Collected last on purpose (file name), and written so
-that it passes alone in a fresh process as well as after the other tests."""
+The check: through the C ABI, on calls in a row that share that array, the output must
+be byte-identical to emoe_reshard_kv AND to the CPU oracle (the tolerance of every
+parity test here is zero: this is byte movement), and the calls must leave the amount
+of free device memory unchanged.  Collected last on purpose (file name), and written
+so that it passes alone in a fresh process as well as after the other tests."""
 from __future__ import annotations
 
 import dataclasses
@@ -16,6 +17,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2510_02613_b200 as E
 import workloads as W
 from workloads import device as WD
@@ -33,12 +35,22 @@ def _reference_and_static(wl):
         got = WD.alloc_const(sn)
         plan.reshard_kv(src, want)
         torch.cuda.synchronize()
+        host_plan.reshard_kv_static(src, got)       # the first call on the device does the set-up
+        torch.cuda.synchronize()
+        for g in got:
+            g.fill_(WD.FILL_BYTE)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         host_plan.reshard_kv_static(src, got)
         torch.cuda.synchronize()
-        for r, (g, w) in enumerate(zip(got, want)):
+        assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the free device memory"
+        expect = [np.full(n, WD.FILL_BYTE, np.uint8) for n in sn]
+        oracle.reshard_kv(wl.shape, wl.old, wl.new, [t.cpu().numpy() for t in src], expect)
+        for r, (g, w, x) in enumerate(zip(got, want, expect)):
+            assert np.array_equal(g.cpu().numpy(), x), "%s: rank %d differs from the oracle" % (wl.name, r)
             assert torch.equal(g, w), "%s: rank %d differs from emoe_reshard_kv" % (wl.name, r)
         # something was actually moved
-        assert any(bool((w != WD.FILL_BYTE).any()) for w in want)
+        assert any(bool((x != WD.FILL_BYTE).any()) for x in expect)
 
 
 def test_static_entry_matches_reshard_kv_on_two_calls_in_a_row():
@@ -51,6 +63,26 @@ def test_static_entry_matches_reshard_kv_on_two_calls_in_a_row():
     _reference_and_static(small)
     # call 3: the inverse direction of call 1 (TP4 -> TP2)
     _reference_and_static(big.swapped())
+    # call 4: more TP ranks than KV heads (4 heads, TP2 -> TP8: every head on two new ranks)
+    many = dataclasses.replace(big, new=dataclasses.replace(big.new, tp=8))
+    _reference_and_static(many)
+
+
+def test_static_entry_with_a_local_rank_writes_that_rank_only():
+    """One rank per GPU: a plan restricted to new-rank index r writes only that rank's
+    blocks; the other destination pointers may be NULL."""
+    wl = W.make_workload("c4_large", n_layers=1)
+    sizes_new = oracle.kv_arena_bytes(wl.shape, wl.new.tp, wl.new.kv_num_blocks)
+    with E.Plan(wl.shape, wl.old, wl.new, host_only=True) as plan:
+        src = WD.alloc_filled(plan.arena_bytes(E.PHASE_KV, E.SIDE_OLD), wl.seed, W.KIND_KV)
+        expect = [np.full(n, WD.FILL_BYTE, np.uint8) for n in sizes_new]
+        oracle.reshard_kv(wl.shape, wl.old, wl.new, [t.cpu().numpy() for t in src], expect)
+        for r in (0, wl.new.tp - 1):
+            plan.set_local_rank(r)
+            mine = WD.alloc_const([sizes_new[r]])[0]
+            plan.reshard_kv_static(src, [mine if k == r else None for k in range(wl.new.tp)])
+            torch.cuda.synchronize()
+            assert np.array_equal(mine.cpu().numpy(), expect[r]), "rank %d" % r
 
 
 def test_static_entry_rejects_more_pairs_than_its_array_holds():

@@ -3,9 +3,9 @@
 Shapes and reconfigurations follow the benchmark definition of this project
 (tiny / mid-size / fine-grained / large-expert-count / overlap).  The
 fine-grained and large-expert-count shapes mirror the 64-routed-expert and
-128-expert models of the paper's evaluation (Sec. 7.1 "Models and
+128-expert models of the paper's evaluation (Sec. 7.2 "Models and
 Baselines"); sequence lengths mirror its request mix of about 2000 prompt
-tokens plus 500-750 decode tokens (Sec. 7.3).  Trained weights and request
+tokens plus 500-750 decode tokens (Sec. 7.6 "SLO Compliance Analysis").  Trained weights and request
 traces are not needed: the path moves bytes and never looks at them.
 
 Nothing in this module computes a re-layout: placements and block tables are
