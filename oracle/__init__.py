@@ -33,6 +33,8 @@ def lib() -> ctypes.CDLL:
         L.emoe_oracle_reshard_attn.argtypes = [i32] * 8 + [p, p]
         L.emoe_oracle_reshard_kv.restype = i32
         L.emoe_oracle_reshard_kv.argtypes = [i32] * 11 + [p, p, p, p, p, i32]
+        L.emoe_oracle_reshard_attn_fused_qkv.restype = i32
+        L.emoe_oracle_reshard_attn_fused_qkv.argtypes = [i32] * 8 + [p, p]
         L.emoe_oracle_inplace_slots.restype = i32
         L.emoe_oracle_inplace_slots.argtypes = [i32, p, p, i32, p, p, p, p]
         L.emoe_oracle_reshard_experts_inplace.restype = i32
@@ -98,11 +100,14 @@ def reshard_experts(shape, old_placement, new_placement, src: Sequence[np.ndarra
         raise ValueError("oracle: an expert of the new placement is absent from the old one")
 
 
-def reshard_attn(shape, tp_old: int, tp_new: int, src, dst) -> None:
+def reshard_attn(shape, tp_old: int, tp_new: int, src, dst, fused_qkv: bool = False) -> None:
+    """fused_qkv: per rank and layer one [qkv_t | o_t] arena whose qkv rows are grouped by
+    KV head (the group's query heads, then the k head, then the v head)."""
     if ([a.size for a in src] != attn_arena_bytes(shape, tp_old)
             or [a.size for a in dst] != attn_arena_bytes(shape, tp_new)):
         raise ValueError("attention arena sizes do not match")
-    rc = lib().emoe_oracle_reshard_attn(shape.n_layers, shape.d_model, shape.n_q_heads,
+    fn = lib().emoe_oracle_reshard_attn_fused_qkv if fused_qkv else lib().emoe_oracle_reshard_attn
+    rc = fn(shape.n_layers, shape.d_model, shape.n_q_heads,
                                        shape.n_kv_heads, shape.head_dim, shape.elem_bytes,
                                        tp_old, tp_new, _ptrs(src), _ptrs(dst))
     if rc != 0:

@@ -37,6 +37,13 @@
 //    head_major stores a KV block as [local head][token][hd] instead of
 //    [token][local head][hd].  Both are re-orderings of the same logical data.
 //
+//  * fused qkv (the paper leaves the attention tensors' form open; serving engines keep
+//    one fused projection per rank): the q, k and v rows of a rank form ONE matrix whose
+//    rows are grouped by KV head - for every KV head the rank holds, the rows of the
+//    query heads of that head's group that the rank holds, then the head's k rows, then
+//    its v rows.  With T <= Hkv a rank holds Hkv/T whole groups; with T > Hkv it holds
+//    one KV head and Hq/T of its group's query heads.  o is unchanged.
+//
 //  * in-place expert step (Sec. 4.1 "Virtual Expert Management", Sec. 5.2 "Expert
 //    Weights", App. D.5, App. E): a device that stays keeps the experts it already
 //    holds where they are and only arrivals are transferred.  Read here for a dense
@@ -313,6 +320,59 @@ int emoe_oracle_reshard_experts_inplace(int n_layers, int64_t m, int ep_old, con
     base += cap;
   }
   (void)want_off; (void)want_ids;
+  return 0;
+}
+
+// ---- attention with a fused qkv matrix per rank -------------------------------------
+//
+// Arena of rank t of a TP=T group, per layer: [qkv_t | o_t].  qkv_t has
+// (Hq/T + 2 * kvh) * hd rows of D*b bytes, kvh = KV heads per rank, grouped by KV head:
+//   group j (KV head kv_first_head(t) + j):  qpg query heads | k head | v head,
+//   qpg = (Hq/T) / kvh query heads per group on this rank.
+// o_t is stored after it exactly as in the unfused arena.
+int emoe_oracle_reshard_attn_fused_qkv(int n_layers, int d_model, int hq, int hkv, int hd, int b, int c,
+                                       int d, const uint8_t *const *src, uint8_t *const *dst) {
+  if (hq % c || hq % d || hq % hkv || !kv_tp_ok(hkv, c) || !kv_tp_ok(hkv, d)) return -1;
+  const int64_t D = d_model, row = D * b, head = (int64_t)hd * row;  // one head's rows, contiguous
+  auto kvh = [&](int T) { return kv_heads_per_rank(hkv, T); };
+  auto qpg = [&](int T) { return (int64_t)(hq / T) / kvh(T); };
+  auto qkv_bytes = [&](int T) { return ((int64_t)(hq / T) + 2 * kvh(T)) * head; };
+  auto o_bytes = [&](int T) { return (int64_t)(hq / T) * hd * row; };
+  auto layer_bytes = [&](int T) { return qkv_bytes(T) + o_bytes(T); };
+  // byte offset, inside a layer of rank (h / (hq/T)), of global query head h
+  auto q_off = [&](int T, int64_t h) {
+    const int64_t local = h % (hq / T), j = local / qpg(T), i = local % qpg(T);
+    return (j * (qpg(T) + 2) + i) * head;
+  };
+  // ... of the k (which = 0) or v (which = 1) rows of the rank's local KV head j
+  auto kv_off = [&](int T, int64_t j, int which) { return (j * (qpg(T) + 2) + qpg(T) + which) * head; };
+
+  for (int l = 0; l < n_layers; ++l) {
+    for (int64_t h = 0; h < hq; ++h) {   // query heads: each lives on exactly one rank per side
+      const int64_t ro = h / (hq / c), rn = h / (hq / d);
+      std::memcpy(dst[rn] + l * layer_bytes(d) + q_off(d, h), src[ro] + l * layer_bytes(c) + q_off(c, h),
+                  (size_t)head);
+    }
+    for (int which = 0; which < 2; ++which)   // k and v heads of every new rank
+      for (int rn = 0; rn < d; ++rn)
+        for (int64_t jn = 0; jn < kvh(d); ++jn) {
+          const int64_t g = kv_first_head(hkv, d, rn) + jn;
+          const int64_t ro = kv_source_rank(hkv, c, g, rn);
+          const int64_t jo = g - kv_first_head(hkv, c, ro);
+          std::memcpy(dst[rn] + l * layer_bytes(d) + kv_off(d, jn, which),
+                      src[ro] + l * layer_bytes(c) + kv_off(c, jo, which), (size_t)head);
+        }
+    // o: exactly as in the unfused arena (stored row i, head h owns columns [h*hd, (h+1)*hd))
+    const int64_t cols_c = (int64_t)(hq / c) * hd, cols_d = (int64_t)(hq / d) * hd;
+    for (int64_t i = 0; i < D; ++i)
+      for (int h = 0; h < hq; ++h) {
+        const int64_t col = (int64_t)h * hd;
+        const int64_t ro = col / cols_c, lo = col % cols_c;
+        const int64_t rn = col / cols_d, ln = col % cols_d;
+        std::memcpy(dst[rn] + l * layer_bytes(d) + qkv_bytes(d) + (i * cols_d + ln) * b,
+                    src[ro] + l * layer_bytes(c) + qkv_bytes(c) + (i * cols_c + lo) * b, (size_t)hd * b);
+      }
+  }
   return 0;
 }
 

@@ -90,6 +90,33 @@ def attn_arenas(logical, tp, head_dim=None):
     return out
 
 
+def attn_arenas_fused_qkv(logical, tp, n_q_heads, n_kv_heads, head_dim):
+    """Rank t: per layer [qkv_t | o_t]; qkv_t = for every KV head of the rank, the rank's
+    query heads of that head's group, then the k head, then the v head (numpy.concatenate
+    of head slices of the logical matrices)."""
+    L = logical["q"].shape[0]
+    q = logical["q"].reshape(L, n_q_heads, head_dim, -1)
+    k = logical["k"].reshape(L, n_kv_heads, head_dim, -1)
+    v = logical["v"].reshape(L, n_kv_heads, head_dim, -1)
+    os_ = np.split(logical["o"], tp, axis=2)
+    q_per_kv = n_q_heads // n_kv_heads
+    out = []
+    for t in range(tp):
+        my_q = list(range(t * n_q_heads // tp, (t + 1) * n_q_heads // tp))
+        per_layer = []
+        for l in range(L):
+            pieces = []
+            for g in kv_heads_of_rank(n_kv_heads, tp, t):
+                for h in my_q:
+                    if h // q_per_kv == g:
+                        pieces.append(q[l, h])
+                pieces += [k[l, g], v[l, g]]
+            per_layer.append(np.concatenate([np.concatenate(pieces).reshape(-1),
+                                             np.ascontiguousarray(os_[t][l]).reshape(-1)]))
+        out.append(np.concatenate(per_layer))
+    return out
+
+
 # ---- KV --------------------------------------------------------------------------------
 
 def logical_kv(shape, cfg, key=3):

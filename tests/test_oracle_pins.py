@@ -619,3 +619,66 @@ def test_inplace_paper_scenario_fixture(case):
             for l in range(2):
                 for p in range(3):
                     assert set(got[l, p, s]) == {tag(ro, so, l, p)}, (r, s)
+
+
+# ================================================================= fused qkv ===========
+
+from helpers import attn_arenas_fused_qkv  # noqa: E402
+
+
+@pytest.mark.parametrize("hq,hkv,c,d", [(8, 4, 1, 2), (8, 4, 4, 2), (8, 8, 2, 4), (8, 2, 1, 2),
+                                        (8, 2, 2, 4), (8, 2, 8, 2), (8, 2, 4, 8), (16, 4, 2, 2)])
+@pytest.mark.parametrize("elem_bytes", [1, 2])
+def test_attn_fused_qkv_equals_numpy_concatenate_of_head_slices(hq, hkv, c, d, elem_bytes):
+    sh = tiny_shape(n_q_heads=hq, n_kv_heads=hkv, head_dim=3, d_model=5, elem_bytes=elem_bytes, n_layers=2)
+    logical = logical_attn(sh)
+    src = attn_arenas_fused_qkv(logical, c, hq, hkv, sh.head_dim)
+    want = attn_arenas_fused_qkv(logical, d, hq, hkv, sh.head_dim)
+    assert [a.size for a in want] == oracle.attn_arena_bytes(sh, d)
+    dst = filled([a.size for a in want])
+    oracle.reshard_attn(sh, c, d, src, dst, fused_qkv=True)
+    for r, (g, w) in enumerate(zip(dst, want)):
+        assert np.array_equal(g, w), "rank %d" % r
+
+
+def test_attn_fused_qkv_hand_written():
+    """4 query heads, 2 KV heads, head_dim 1, d_model 1, one byte per element, one layer.
+    Logical rows tagged q: 10..13, k: 20,21, v: 30,31, o (one row of 4 columns): 40..43.
+    TP1 arena: [q0 q1 k0 v0 | q2 q3 k1 v1 | o0 o1 o2 o3];
+    TP2 arenas: rank 0 [q0 q1 k0 v0 | o0 o1], rank 1 [q2 q3 k1 v1 | o2 o3];
+    TP4 arenas: rank t [q_t k_(t//2) v_(t//2) | o_t]."""
+    sh = tiny_shape(n_layers=1, n_q_heads=4, n_kv_heads=2, head_dim=1, d_model=1, elem_bytes=1)
+    tp1 = [np.array([10, 11, 20, 30, 12, 13, 21, 31, 40, 41, 42, 43], np.uint8)]
+    tp2 = [np.array([10, 11, 20, 30, 40, 41], np.uint8), np.array([12, 13, 21, 31, 42, 43], np.uint8)]
+    tp4 = [np.array([10, 20, 30, 40], np.uint8), np.array([11, 20, 30, 41], np.uint8),
+           np.array([12, 21, 31, 42], np.uint8), np.array([13, 21, 31, 43], np.uint8)]
+    for a, b in ((tp1, tp2), (tp2, tp1), (tp1, tp4), (tp4, tp2), (tp2, tp4), (tp4, tp1)):
+        dst = filled([x.size for x in b])
+        oracle.reshard_attn(sh, len(a), len(b), a, dst, fused_qkv=True)
+        assert all(np.array_equal(g, w) for g, w in zip(dst, b)), (len(a), len(b))
+
+
+def test_attn_fused_qkv_with_one_query_head_per_kv_head_interleaves_q_k_v():
+    """Hq == Hkv: the fused matrix is [q0 k0 v0 q1 k1 v1 ...]; un-fusing it with a numpy
+    reshape gives the plain q | k | v pieces."""
+    sh = tiny_shape(n_q_heads=4, n_kv_heads=4, head_dim=2, d_model=3, elem_bytes=2, n_layers=2)
+    logical = logical_attn(sh)
+    fused = attn_arenas_fused_qkv(logical, 2, 4, 4, 2)
+    plain = attn_arenas(logical, 2)
+    row = 3 * 2
+    for f, p in zip(fused, plain):
+        f = f.reshape(2, -1)
+        p = p.reshape(2, -1)
+        n_qkv = 3 * 2 * 2 * row                                   # 2 heads per rank, q k v, hd rows
+        x = f[:, :n_qkv].reshape(2, 2, 3, 2 * row)                # [layer, head, q|k|v, head bytes]
+        unfused = np.concatenate([x[:, :, 0].reshape(2, -1), x[:, :, 1].reshape(2, -1),
+                                  x[:, :, 2].reshape(2, -1)], axis=1)
+        assert np.array_equal(unfused, p[:, :n_qkv])
+        assert np.array_equal(f[:, n_qkv:], p[:, n_qkv:])          # o is the same
+
+
+def test_attn_fused_qkv_rejects_query_heads_not_divisible_by_kv_heads():
+    sh = tiny_shape(n_q_heads=6, n_kv_heads=4, head_dim=2)
+    with pytest.raises(ValueError):
+        oracle.reshard_attn(sh, 1, 2, [np.zeros(oracle.attn_arena_bytes(sh, 1)[0], np.uint8)],
+                            filled(oracle.attn_arena_bytes(sh, 2)), fused_qkv=True)
