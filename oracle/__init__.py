@@ -35,6 +35,12 @@ def lib() -> ctypes.CDLL:
         L.emoe_oracle_reshard_kv.argtypes = [i32] * 11 + [p, p, p, p, p, i32]
         L.emoe_oracle_reshard_attn_fused_qkv.restype = i32
         L.emoe_oracle_reshard_attn_fused_qkv.argtypes = [i32] * 8 + [p, p]
+        L.emoe_oracle_scaled_expert_scale_base.restype = i64
+        L.emoe_oracle_scaled_expert_scale_base.argtypes = [i32, i32, i64]
+        L.emoe_oracle_scaled_expert_arena_bytes.restype = i64
+        L.emoe_oracle_scaled_expert_arena_bytes.argtypes = [i32, i32, i64, i64]
+        L.emoe_oracle_reshard_experts_scaled.restype = i32
+        L.emoe_oracle_reshard_experts_scaled.argtypes = [i32, i64, i64, i32, p, p, i32, p, p, p, p]
         L.emoe_oracle_inplace_slots.restype = i32
         L.emoe_oracle_inplace_slots.argtypes = [i32, p, p, i32, p, p, p, p]
         L.emoe_oracle_reshard_experts_inplace.restype = i32
@@ -65,7 +71,16 @@ def _vp(a: np.ndarray):
 
 def expert_arena_bytes(shape, placement) -> List[int]:
     m = shape.d_model * shape.d_ff * shape.elem_bytes
+    ms = getattr(shape, "expert_scale_bytes", 0)
+    if ms:
+        return [lib().emoe_oracle_scaled_expert_arena_bytes(shape.n_layers, len(p), m, ms) for p in placement]
     return [lib().emoe_oracle_expert_arena_bytes(shape.n_layers, len(p), m) for p in placement]
+
+
+def expert_scale_base(shape, n_slots: int) -> int:
+    """Offset of the scale tensor inside the arena of a rank with n_slots experts."""
+    m = shape.d_model * shape.d_ff * shape.elem_bytes
+    return lib().emoe_oracle_scaled_expert_scale_base(shape.n_layers, n_slots, m)
 
 
 def attn_arena_bytes(shape, tp: int) -> List[int]:
@@ -93,6 +108,16 @@ def reshard_experts(shape, old_placement, new_placement, src: Sequence[np.ndarra
     need_d = expert_arena_bytes(shape, new_placement)
     if [a.size for a in src] != need_s or [a.size for a in dst] != need_d:
         raise ValueError("expert arena sizes do not match the placements")
+    ms = getattr(shape, "expert_scale_bytes", 0)
+    if ms:      # every matrix travels with its scale tensor (weights first, scales after them)
+        if fused_w13:
+            raise ValueError("oracle: scale tensors go with the plain [L][3][n][m] layout")
+        rc = lib().emoe_oracle_reshard_experts_scaled(shape.n_layers, m, ms, len(old_placement), _vp(oo),
+                                                     _vp(oi), len(new_placement), _vp(no), _vp(ni),
+                                                     _ptrs(src), _ptrs(dst))
+        if rc != 0:
+            raise ValueError("oracle: an expert of the new placement is absent from the old one")
+        return
     rc = lib().emoe_oracle_reshard_experts(shape.n_layers, m, len(old_placement), _vp(oo), _vp(oi),
                                           len(new_placement), _vp(no), _vp(ni), _ptrs(src),
                                           _ptrs(dst), int(bool(fused_w13)))

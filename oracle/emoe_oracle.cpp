@@ -44,6 +44,12 @@
 //    its v rows.  With T <= Hkv a rank holds Hkv/T whole groups; with T > Hkv it holds
 //    one KV head and Hq/T of its group's query heads.  o is unchanged.
 //
+//  * quantised experts with block scales (the paper's largest model, Sec. 7.2, ships FP8
+//    weights with one scale per 128 x 128 block): every expert matrix has a second, small
+//    tensor that must travel with it.  Read here as one arena per rank holding the weight
+//    tensor [L][3][n_r][m] and, from the next multiple of 256 bytes on, the scale tensor
+//    [L][3][n_r][ms]; both are re-packed by the same placement.
+//
 //  * in-place expert step (Sec. 4.1 "Virtual Expert Management", Sec. 5.2 "Expert
 //    Weights", App. D.5, App. E): a device that stays keeps the experts it already
 //    holds where they are and only arrivals are transferred.  Read here for a dense
@@ -372,6 +378,41 @@ int emoe_oracle_reshard_attn_fused_qkv(int n_layers, int d_model, int hq, int hk
         std::memcpy(dst[rn] + l * layer_bytes(d) + qkv_bytes(d) + (i * cols_d + ln) * b,
                     src[ro] + l * layer_bytes(c) + qkv_bytes(c) + (i * cols_c + lo) * b, (size_t)hd * b);
       }
+  }
+  return 0;
+}
+
+// ---- experts with a scale tensor per matrix ------------------------------------------
+//
+// Arena of a rank with n slots: weights [L][3][n][m], then - at the next multiple of 256
+// bytes - scales [L][3][n][ms].  Bytes between the two parts belong to nobody.
+int64_t emoe_oracle_scaled_expert_scale_base(int n_layers, int n_slots, int64_t m) {
+  const int64_t w = (int64_t)n_layers * 3 * n_slots * m;
+  return (w + 255) / 256 * 256;
+}
+int64_t emoe_oracle_scaled_expert_arena_bytes(int n_layers, int n_slots, int64_t m, int64_t ms) {
+  return emoe_oracle_scaled_expert_scale_base(n_layers, n_slots, m) + (int64_t)n_layers * 3 * n_slots * ms;
+}
+
+int emoe_oracle_reshard_experts_scaled(int n_layers, int64_t m, int64_t ms, int ep_old,
+                                       const int32_t *old_off, const int32_t *old_ids, int ep_new,
+                                       const int32_t *new_off, const int32_t *new_ids,
+                                       const uint8_t *const *src, uint8_t *const *dst) {
+  Csr po{ep_old, old_off, old_ids}, pn{ep_new, new_off, new_ids};
+  for (int rn = 0; rn < ep_new; ++rn) {
+    const int64_t n_new = pn.count(rn);
+    const int64_t sb_new = emoe_oracle_scaled_expert_scale_base(n_layers, (int)n_new, m);
+    for (int l = 0; l < n_layers; ++l)
+      for (int p = 0; p < 3; ++p)
+        for (int sn = 0; sn < n_new; ++sn) {
+          int ro, so;
+          if (!find_source(po, pn.id(rn, sn), rn, &ro, &so)) return -1;
+          const int64_t n_old = po.count(ro);
+          const int64_t sb_old = emoe_oracle_scaled_expert_scale_base(n_layers, (int)n_old, m);
+          const int64_t at_new = ((int64_t)l * 3 + p) * n_new + sn, at_old = ((int64_t)l * 3 + p) * n_old + so;
+          std::memcpy(dst[rn] + at_new * m, src[ro] + at_old * m, (size_t)m);                      // the matrix
+          std::memcpy(dst[rn] + sb_new + at_new * ms, src[ro] + sb_old + at_old * ms, (size_t)ms);  // its scales
+        }
   }
   return 0;
 }

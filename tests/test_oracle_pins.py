@@ -682,3 +682,48 @@ def test_attn_fused_qkv_rejects_query_heads_not_divisible_by_kv_heads():
     with pytest.raises(ValueError):
         oracle.reshard_attn(sh, 1, 2, [np.zeros(oracle.attn_arena_bytes(sh, 1)[0], np.uint8)],
                             filled(oracle.attn_arena_bytes(sh, 2)), fused_qkv=True)
+
+
+# ==================================================== experts with scale tensors =======
+
+def scaled_arenas(weights, scales, placement):
+    """Arena of a rank = its experts' weights [L,3,n,m] flattened, zero padding up to a
+    multiple of 256 bytes, then their scales [L,3,n,ms] flattened (numpy.concatenate)."""
+    out = []
+    for p in placement:
+        w = np.ascontiguousarray(weights[:, :, list(p)]).reshape(-1)
+        pad = np.zeros(-w.size % 256, np.uint8)
+        out.append(np.concatenate([w, pad, np.ascontiguousarray(scales[:, :, list(p)]).reshape(-1)]))
+    return out
+
+
+@pytest.mark.parametrize("name", sorted(PLACEMENTS))
+@pytest.mark.parametrize("ms", [4, 24])
+def test_experts_with_scales_equal_numpy_gather_of_both_logical_tensors(name, ms):
+    sh = dataclasses.replace(tiny_shape(elem_bytes=1, d_model=9, d_ff=7), expert_scale_bytes=ms)
+    po, pn = (f() for f in PLACEMENTS[name])
+    weights = logical_experts(sh, key=41)
+    scales = rand_bytes(42, sh.n_layers * 3 * sh.n_experts * ms).reshape(sh.n_layers, 3, sh.n_experts, ms)
+    src = scaled_arenas(weights, scales, po)
+    want = scaled_arenas(weights, scales, pn)
+    assert [a.size for a in want] == oracle.expert_arena_bytes(sh, pn)
+    dst = [np.zeros(a.size, np.uint8) for a in want]       # padding is written by nobody: stays zero
+    oracle.reshard_experts(sh, po, pn, src, dst)
+    for r, (g, w) in enumerate(zip(dst, want)):
+        assert np.array_equal(g, w), "rank %d" % r
+        assert oracle.expert_scale_base(sh, len(pn[r])) % 256 == 0
+
+
+def test_experts_with_scales_hand_written():
+    """One layer, matrices of 2 bytes, scales of 1 byte.  Rank with 2 experts: weights
+    occupy 3*2*2 = 12 bytes, scales start at byte 256."""
+    sh = dataclasses.replace(tiny_shape(n_layers=1, n_routed=2, d_model=1, d_ff=1, elem_bytes=2),
+                             expert_scale_bytes=1)
+    old = np.zeros(256 + 6, np.uint8)
+    old[:12] = [1, 1, 2, 2, 3, 3, 4, 4, 5, 5, 6, 6]       # gate e0,e1 | up e0,e1 | down e0,e1
+    old[256:262] = [11, 12, 13, 14, 15, 16]
+    dst = [np.zeros(256 + 3, np.uint8), np.zeros(256 + 3, np.uint8)]
+    oracle.reshard_experts(sh, [[0, 1]], [[1], [0]], [old], dst)
+    assert list(dst[0][:6]) == [2, 2, 4, 4, 6, 6] and list(dst[0][256:]) == [12, 14, 16]
+    assert list(dst[1][:6]) == [1, 1, 3, 3, 5, 5] and list(dst[1][256:]) == [11, 13, 15]
+    assert not dst[0][6:256].any() and not dst[1][6:256].any()

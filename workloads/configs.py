@@ -41,6 +41,7 @@ class Shape:
     head_dim: int
     kv_block_tokens: int = 16
     elem_bytes: int = 2
+    expert_scale_bytes: int = 0   # bytes of the scale tensor that goes with every expert matrix (0: none)
 
     @property
     def n_experts(self) -> int:
@@ -68,6 +69,7 @@ class Workload:
     victim: Optional[dict] = field(default=None)   # C5: the concurrent GEMM's shape
     fused_w13: bool = False        # layout variant: per layer [n][gate|up] then [n][down]
     kv_head_major: bool = False    # layout variant: KV blocks [local head][token][hd]
+    fused_qkv: bool = False        # layout variant: attention arena [qkv_t | o_t], rows grouped by KV head
 
     def with_layers(self, n_layers: int) -> "Workload":
         """Same workload cut to n_layers (layers are independent in every phase)."""
