@@ -118,6 +118,12 @@ typedef struct {
 #define EMOE_LAYOUT_FUSED_W13 4u     /* expert arena per layer: [n_r][gate|up] (2m per slot),  */
                                      /* then [n_r][down], instead of [3][n_r][m]               */
 #define EMOE_LAYOUT_KV_HEAD_MAJOR 8u /* KV block [Hkv/T][B][hd] instead of [B][Hkv/T][hd]     */
+#define EMOE_LAYOUT_FUSED_QKV 16u    /* attention arena per layer: [qkv_t | o_t], the rows of  */
+                                     /* qkv_t grouped by KV head - for every KV head of the    */
+                                     /* rank: the rank's query heads of that head's group,     */
+                                     /* then the k head, then the v head (as fused-projection  */
+                                     /* checkpoints of grouped-query models store them).       */
+                                     /* Needs n_q_heads % n_kv_heads == 0; sizes are unchanged */
 
 /* phase / side selectors of the query helpers */
 #define EMOE_PHASE_EXPERTS 0
@@ -147,6 +153,28 @@ typedef struct {
 emoe_status_t emoe_plan_create(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
                                const emoe_config_t *new_cfg, uint32_t flags,
                                emoe_plan_t **out);
+
+/*
+ * emoe_plan_create_ex - emoe_plan_create with options (NULL options = emoe_plan_create).
+ *
+ * expert_scale_bytes > 0: every expert matrix travels with a scale tensor of that many
+ * bytes - block-quantised weights, as the largest model of the paper's evaluation
+ * (Sec. 7.2) ships them: FP8 matrices with one fp32 scale per 128 x 128 block.  The
+ * expert arena of a rank with n_r slots is then
+ *      weights [L][3][n_r][m]   followed, from the next multiple of 256 bytes on, by
+ *      scales  [L][3][n_r][expert_scale_bytes],
+ * and ONE plan - one call, one launch set - moves both by the same placement.  Bytes
+ * between the two parts are never written.  Not combinable with EMOE_LAYOUT_FUSED_W13
+ * (EMOE_ERR_UNSUPPORTED); such a plan's emoe_reshard_step_host runs serially.
+ * reserved: must be zero.
+ */
+typedef struct {
+  int64_t expert_scale_bytes;
+  int64_t reserved[7];
+} emoe_plan_options_t;
+emoe_status_t emoe_plan_create_ex(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
+                                  const emoe_config_t *new_cfg, uint32_t flags,
+                                  const emoe_plan_options_t *options, emoe_plan_t **out);
 
 /*
  * emoe_reshard_experts - expert re-pack EP=a -> EP=b (Sec. 4.1 "Virtual
@@ -528,6 +556,50 @@ emoe_status_t emoe_plan_set_tuning(emoe_plan_t *plan, const emoe_tuning_t *tunin
 emoe_status_t emoe_place_min_transfer(int32_t n_experts, const emoe_config_t *old_cfg,
                                       int32_t ep_new, int32_t *new_off, int32_t *new_ids,
                                       int32_t *n_kept);
+
+/* ---- plans for scaling sequences ------------------------------------------
+ *
+ * A serving system that scales up and down in steps (the paper's step patterns add or
+ * remove devices a few at a time, Sec. 7.4; scale-down mirrors scale-up, App. E) meets
+ * the same (old, new) pairs again.  A plan is a pure function of its inputs, so a cache
+ * can hand out the plan made earlier: emoe_plan_cache_get returns the cached plan when
+ * shape, flags, options and everything emoe_plan_create reads from the two configurations
+ * (placements, TP/EP degrees, pool sizes, sequence lengths, the mapped block-table
+ * entries) are byte-for-byte the same, and otherwise creates one (on the current CUDA
+ * device unless EMOE_PLAN_HOST_ONLY) and keeps it.  *hit (optional): 1 / 0.
+ * The cache OWNS its plans: never pass them to emoe_plan_destroy.  It keeps at most
+ * `capacity` plans; inserting one more destroys the least recently used one, so a plan
+ * obtained earlier may die in a later emoe_plan_cache_get - do not hold more plans than
+ * the capacity across calls, and have no launch of an evicted plan in flight.
+ * Invalid inputs return the planner's error and are not stored.  Thread-safe.
+ * Weights and KV can be cached separately: a plan whose configurations list no sequences
+ * (n_seqs = 0) covers experts and attention and does not depend on block tables. */
+typedef struct emoe_plan_cache emoe_plan_cache_t;
+emoe_status_t emoe_plan_cache_create(int32_t capacity, emoe_plan_cache_t **out);
+emoe_status_t emoe_plan_cache_get(emoe_plan_cache_t *cache, const emoe_shape_t *shape,
+                                  const emoe_config_t *old_cfg, const emoe_config_t *new_cfg,
+                                  uint32_t flags, const emoe_plan_options_t *options,
+                                  emoe_plan_t **plan, int32_t *hit);
+emoe_status_t emoe_plan_cache_stats(emoe_plan_cache_t *cache, uint64_t *hits, uint64_t *misses,
+                                    uint64_t *evictions, int32_t *size);
+void emoe_plan_cache_destroy(emoe_plan_cache_t *cache);
+
+/* emoe_kv_compact_table - a destination block table that COMPACTS the cache while it
+ * moves: the mapped blocks of the sequences, in table order (sequence by sequence, block
+ * by block), get the lowest-numbered blocks of the destination pool that are free.  The
+ * paper leaves block allocation across the two instances open (App. C names coordinating
+ * it as future work); this is the allocation a scale-down wants, where the surviving pool
+ * should end up dense.
+ * in_use [n_in_use]: blocks of the destination pool (size nb_new) that are already taken -
+ * e.g. by sequences the new instance serves already - and must not be handed out; NULL /
+ * 0 for a fresh pool, which yields the identity order 0, 1, 2, ...
+ * table_out: [n_seqs][max_blocks], -1 padded; *n_mapped (optional): blocks assigned.
+ * Errors: EMOE_ERR_BLOCK_TABLE (an in_use id out of range or listed twice, a sequence
+ * longer than max_blocks blocks), EMOE_ERR_TOO_LARGE (not enough free blocks).
+ * Host only.  Use the result as new_cfg->block_table of emoe_plan_create. */
+emoe_status_t emoe_kv_compact_table(int32_t block_tokens, int32_t n_seqs, int32_t max_blocks,
+                                    const int32_t *seq_lens, int32_t nb_new, const int32_t *in_use,
+                                    int32_t n_in_use, int32_t *table_out, int32_t *n_mapped);
 
 /* ---- one rank per GPU: pull-based exchange --------------------------------
  *

@@ -21,6 +21,7 @@ PLAN_HOST_ONLY = 1
 PLAN_HOST_STEP = 2
 LAYOUT_FUSED_W13 = 4
 LAYOUT_KV_HEAD_MAJOR = 8
+LAYOUT_FUSED_QKV = 16
 MAX_RANKS = 64
 
 _i32, _u32, _u64, _vp = ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_void_p
@@ -43,6 +44,10 @@ class _Config(ctypes.Structure):
     _fields_ = [("ep", _i32), ("tp", _i32), ("place_off", _i32p), ("place_ids", _i32p),
                 ("kv_num_blocks", _i32), ("n_seqs", _i32), ("max_blocks", _i32),
                 ("seq_lens", _i32p), ("block_table", _i32p)]
+
+
+class _PlanOptions(ctypes.Structure):
+    _fields_ = [("expert_scale_bytes", ctypes.c_int64), ("reserved", ctypes.c_int64 * 7)]
 
 
 class _Segment(ctypes.Structure):
@@ -69,7 +74,7 @@ SEGMENT_DTYPE = np.dtype([("src_off", "<u8"), ("dst_off", "<u8"), ("run_bytes", 
                           ("src_pitch", "<u8"), ("dst_pitch", "<u8"), ("n_runs", "<u4"),
                           ("src_rank", "<u4"), ("dst_rank", "<u4"), ("group", "<u4")])
 
-EXPORTS = ("emoe_plan_create", "emoe_reshard_experts", "emoe_reshard_attn", "emoe_reshard_kv",
+EXPORTS = ("emoe_plan_create", "emoe_plan_create_ex", "emoe_reshard_experts", "emoe_reshard_attn", "emoe_reshard_kv",
            "emoe_reshard_kv_static", "emoe_reshard_step", "emoe_plan_create_inplace",
            "emoe_plan_slot_table", "emoe_reshard_experts_inplace",
            "emoe_reshard_step_host", "emoe_plan_destroy", "emoe_plan_num_ranks",
@@ -77,7 +82,8 @@ EXPORTS = ("emoe_plan_create", "emoe_reshard_experts", "emoe_reshard_attn", "emo
            "emoe_plan_segments",
            "emoe_plan_device_status", "emoe_plan_clear_device_status", "emoe_plan_set_tuning",
            "emoe_strerror",
-           "emoe_place_min_transfer", "emoe_plan_set_local_rank", "emoe_ipc_export", "emoe_ipc_open", "emoe_ipc_close",
+           "emoe_plan_cache_create", "emoe_plan_cache_get", "emoe_plan_cache_stats", "emoe_plan_cache_destroy",
+           "emoe_kv_compact_table", "emoe_place_min_transfer", "emoe_plan_set_local_rank", "emoe_ipc_export", "emoe_ipc_open", "emoe_ipc_close",
            "emoe_vmm_create", "emoe_vmm_reshard", "emoe_vmm_dry_run", "emoe_vmm_num_ranks", "emoe_vmm_arena",
            "emoe_vmm_write", "emoe_vmm_read", "emoe_vmm_destroy")
 
@@ -105,6 +111,10 @@ def lib() -> ctypes.CDLL:
     L.emoe_plan_create.restype = _i32
     L.emoe_plan_create.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Config),
                                    ctypes.POINTER(_Config), _u32, ctypes.POINTER(_vp)]
+    L.emoe_plan_create_ex.restype = _i32
+    L.emoe_plan_create_ex.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Config),
+                                      ctypes.POINTER(_Config), _u32, ctypes.POINTER(_PlanOptions),
+                                      ctypes.POINTER(_vp)]
     for name in ("emoe_reshard_experts", "emoe_reshard_attn", "emoe_reshard_kv",
                  "emoe_reshard_kv_static"):
         f = getattr(L, name)
@@ -142,6 +152,18 @@ def lib() -> ctypes.CDLL:
     L.emoe_plan_clear_device_status.argtypes = [_vp]
     L.emoe_plan_set_tuning.restype = _i32
     L.emoe_plan_set_tuning.argtypes = [_vp, ctypes.POINTER(_Tuning)]
+    L.emoe_plan_cache_create.restype = _i32
+    L.emoe_plan_cache_create.argtypes = [_i32, ctypes.POINTER(_vp)]
+    L.emoe_plan_cache_get.restype = _i32
+    L.emoe_plan_cache_get.argtypes = [_vp, ctypes.POINTER(_Shape), ctypes.POINTER(_Config),
+                                      ctypes.POINTER(_Config), _u32, ctypes.POINTER(_PlanOptions),
+                                      ctypes.POINTER(_vp), _i32p]
+    L.emoe_plan_cache_stats.restype = _i32
+    L.emoe_plan_cache_stats.argtypes = [_vp] + [ctypes.POINTER(_u64)] * 3 + [_i32p]
+    L.emoe_plan_cache_destroy.restype = None
+    L.emoe_plan_cache_destroy.argtypes = [_vp]
+    L.emoe_kv_compact_table.restype = _i32
+    L.emoe_kv_compact_table.argtypes = [_i32, _i32, _i32, _i32p, _i32, _i32p, _i32, _i32p, _i32p]
     L.emoe_place_min_transfer.restype = _i32
     L.emoe_place_min_transfer.argtypes = [_i32, ctypes.POINTER(_Config), _i32, _i32p, _i32p, _i32p]
     L.emoe_plan_set_local_rank.restype = _i32
@@ -239,25 +261,33 @@ class Plan:
     """A scale-step plan: emoe_plan_create ... emoe_plan_destroy."""
 
     def __init__(self, shape, old_cfg, new_cfg, host_only: bool = False, host_step: bool = False,
-                 fused_w13: bool = False, kv_head_major: bool = False):
+                 fused_w13: bool = False, kv_head_major: bool = False, fused_qkv: bool = False):
         self._h = _vp()
         keep: list = []
         sh = _Shape(shape.n_layers, shape.n_routed, shape.n_shared, shape.d_model, shape.d_ff,
                     shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.kv_block_tokens,
                     shape.elem_bytes)
         co, cn = _make_config(old_cfg, keep), _make_config(new_cfg, keep)
-        _check(lib().emoe_plan_create(ctypes.byref(sh), ctypes.byref(co), ctypes.byref(cn),
-                                      (PLAN_HOST_ONLY if host_only else 0)
-                                      | (PLAN_HOST_STEP if host_step else 0)
-                                      | (LAYOUT_FUSED_W13 if fused_w13 else 0)
-                                      | (LAYOUT_KV_HEAD_MAJOR if kv_head_major else 0),
-                                      ctypes.byref(self._h)))
+        flags = ((PLAN_HOST_ONLY if host_only else 0) | (PLAN_HOST_STEP if host_step else 0)
+                 | (LAYOUT_FUSED_W13 if fused_w13 else 0) | (LAYOUT_KV_HEAD_MAJOR if kv_head_major else 0)
+                 | (LAYOUT_FUSED_QKV if fused_qkv else 0))
+        scale = int(getattr(shape, "expert_scale_bytes", 0) or 0)
+        if scale:     # every expert matrix travels with a scale tensor
+            opt = _PlanOptions(scale)
+            _check(lib().emoe_plan_create_ex(ctypes.byref(sh), ctypes.byref(co), ctypes.byref(cn), flags,
+                                             ctypes.byref(opt), ctypes.byref(self._h)))
+        else:
+            _check(lib().emoe_plan_create(ctypes.byref(sh), ctypes.byref(co), ctypes.byref(cn), flags,
+                                          ctypes.byref(self._h)))
         self.host_only = host_only
 
     # -- life cycle
+    _owned = True     # False: the handle belongs to a PlanCache
+
     def close(self) -> None:
         if self._h:
-            lib().emoe_plan_destroy(self._h)
+            if self._owned:
+                lib().emoe_plan_destroy(self._h)
             self._h = _vp()
 
     def __del__(self):
@@ -375,6 +405,79 @@ class Plan:
 
         _check(lib().emoe_reshard_step_host(self._h, pack(h_src), pack(h_dst), pack(d_src),
                                             pack(d_dst), _stream_handle(stream)))
+
+
+def _plan_flags(host_only=False, host_step=False, fused_w13=False, kv_head_major=False, fused_qkv=False):
+    return ((PLAN_HOST_ONLY if host_only else 0) | (PLAN_HOST_STEP if host_step else 0)
+            | (LAYOUT_FUSED_W13 if fused_w13 else 0) | (LAYOUT_KV_HEAD_MAJOR if kv_head_major else 0)
+            | (LAYOUT_FUSED_QKV if fused_qkv else 0))
+
+
+class PlanCache:
+    """emoe_plan_cache_*: plans of a scaling sequence, kept and handed out again when the
+    same (shape, old, new, flags) pair comes back.  The cache owns its plans: the Plan
+    objects returned by get() must not outlive it, and at most `capacity` of them stay
+    valid (the least recently used one is destroyed when one more is inserted)."""
+
+    def __init__(self, capacity: int = 16):
+        self._h = _vp()
+        _check(lib().emoe_plan_cache_create(capacity, ctypes.byref(self._h)))
+
+    def get(self, shape, old_cfg, new_cfg, **flags):
+        """(plan, hit)"""
+        keep: list = []
+        sh = _Shape(shape.n_layers, shape.n_routed, shape.n_shared, shape.d_model, shape.d_ff,
+                    shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.kv_block_tokens,
+                    shape.elem_bytes)
+        co, cn = _make_config(old_cfg, keep), _make_config(new_cfg, keep)
+        scale = int(getattr(shape, "expert_scale_bytes", 0) or 0)
+        opt = _PlanOptions(scale)
+        h, hit = _vp(), _i32()
+        _check(lib().emoe_plan_cache_get(self._h, ctypes.byref(sh), ctypes.byref(co), ctypes.byref(cn),
+                                         _plan_flags(**flags), ctypes.byref(opt) if scale else None,
+                                         ctypes.byref(h), ctypes.byref(hit)))
+        plan = Plan.__new__(Plan)
+        plan._h, plan._owned, plan.host_only = h, False, bool(flags.get("host_only"))
+        return plan, bool(hit.value)
+
+    def stats(self) -> dict:
+        a, b, c, n = _u64(), _u64(), _u64(), _i32()
+        _check(lib().emoe_plan_cache_stats(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
+                                           ctypes.byref(n)))
+        return dict(hits=a.value, misses=b.value, evictions=c.value, size=n.value)
+
+    def close(self) -> None:
+        if self._h:
+            lib().emoe_plan_cache_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+
+def kv_compact_table(block_tokens: int, seq_lens, nb_new: int, in_use=(), max_blocks: Optional[int] = None):
+    """Destination block table [n_seqs, max_blocks] that packs the sequences' blocks into the
+    lowest free blocks of a pool of nb_new blocks (in_use: ids already taken there)."""
+    sl = _i32arr(seq_lens)
+    need = [-(-int(n) // block_tokens) for n in sl]
+    mb = max_blocks if max_blocks is not None else max(need, default=0)
+    out = np.full((len(sl), max(mb, 1)), -1, dtype=np.int32)
+    used = _i32arr(list(in_use))
+    n = _i32()
+    _check(lib().emoe_kv_compact_table(block_tokens, len(sl), mb,
+                                       sl.ctypes.data_as(_i32p) if sl.size else None, nb_new,
+                                       used.ctypes.data_as(_i32p) if used.size else None, int(used.size),
+                                       out.ctypes.data_as(_i32p), ctypes.byref(n)))
+    return out[:, :mb] if mb else out[:, :0]
 
 
 class InplacePlan(Plan):

@@ -37,13 +37,16 @@ constexpr uint64_t kSmallPhaseBytes = 256ull << 20;
 struct DevPhase {
   std::vector<DevSeg> segs;  // routed copy of the host segments (fan-out split to kMaxFanout)
   std::vector<Dst> dsts;
-  std::vector<Unit> bulk_units, vec_units;   // bulk_units: general case only (see `regular`)
-  uint64_t n_bulk = 0;                        // bulk units of the phase
-  // Regular phase: its bulk unit table is expanded on the device from these (bulk segment
-  // indices, offset of each one's units inside a run, runs per segment, units per run).
-  bool regular = false;
+  std::vector<Unit> bulk_units, vec_units;   // bulk_units: the host-built part only (see n_gen)
+  uint64_t n_bulk = 0;                        // bulk units of the phase: n_gen + bulk_units.size()
+  // The first n_gen bulk units - those of the "regular" segments: the same number of runs
+  // each, every run at least a tile long - are expanded on the device from these (segment
+  // indices, offset of each one's units inside a run, runs per segment, units per run); the
+  // units of the other bulk segments are built on the host and follow them.
+  uint64_t n_gen = 0;
   std::vector<uint32_t> gen_seg, gen_pre;
   uint32_t gen_runs = 0, gen_upr = 0;
+  uint64_t rest_off[3] = {0, 0, 0};           // merged set: where each phase's host-built units start in bulk_units
   DevSeg *d_segs = nullptr;
   Dst *d_dsts = nullptr;
   Unit *d_bulk_units = nullptr, *d_vec_units = nullptr;
@@ -170,7 +173,7 @@ void build_tables(emoe_plan *p, int phase) {
   DevPhase &dp = p->dev[phase];
   dp.segs.clear(); dp.dsts.clear(); dp.bulk_units.clear(); dp.vec_units.clear();
   dp.gen_seg.clear(); dp.gen_pre.clear();
-  dp.regular = false; dp.n_bulk = 0; dp.gen_runs = dp.gen_upr = 0;
+  dp.n_gen = 0; dp.n_bulk = 0; dp.gen_runs = dp.gen_upr = 0;
   for (bool &b : p->reads_src[phase]) b = false;
   const uint32_t T = bulk_tile(p);
 
@@ -234,35 +237,37 @@ void build_tables(emoe_plan *p, int phase) {
       else for_each_unit(idx, s, kVecTile, [&](uint32_t, const Unit &u) { dp.vec_units.push_back(u); });
     }
   }
-  // Bulk units in run-major order.  Regular phase (every bulk segment has the same number
-  // of runs, each at least a tile long - all bench phases): only each segment's offset inside
-  // a run is computed here, the table itself is written by a kernel at upload time.
-  bool regular = p->tuning.unit_order % 2 == 0 && !bulk_segs.empty();
-  for (uint32_t idx : bulk_segs)
-    regular = regular && dp.segs[idx].run_bytes >= T && dp.segs[idx].n_runs == dp.segs[bulk_segs[0]].n_runs;
-  if (regular) {
+  // Bulk units in run-major order.  The regular segments (run >= tile, and as many runs as the
+  // first such segment - all long runs of the bench phases) only get their offset inside a run
+  // computed here: that part of the table is written by a kernel at upload time.  The units of
+  // the remaining bulk segments (short rows packed into tiles, other run counts) are few and
+  // are built here; they follow the generated part.
+  std::vector<uint32_t> rest;
+  if (p->tuning.unit_order % 2 == 0) {
+    uint32_t runs0 = 0;
+    for (uint32_t idx : bulk_segs)
+      if (dp.segs[idx].run_bytes >= T) { runs0 = dp.segs[idx].n_runs; break; }
     uint64_t upr = 0;
-    dp.gen_pre.reserve(bulk_segs.size());
     for (uint32_t idx : bulk_segs) {
+      if (runs0 == 0 || dp.segs[idx].run_bytes < T || dp.segs[idx].n_runs != runs0) { rest.push_back(idx); continue; }
+      dp.gen_seg.push_back(idx);
       dp.gen_pre.push_back((uint32_t)upr);
       const uint64_t tpr = (dp.segs[idx].run_bytes + T - 1) / T;
       upr += (tpr + kUnitTiles - 1) / kUnitTiles;
     }
-    dp.gen_runs = dp.segs[bulk_segs[0]].n_runs;
-    regular = upr * dp.gen_runs < 0xffffffffull;
-    if (regular) {
-      dp.regular = true;
-      dp.gen_seg = bulk_segs;
+    if (upr * runs0 < 0xffffffffull && upr < 0xffffffffull) {
+      dp.gen_runs = runs0;
       dp.gen_upr = (uint32_t)upr;
-      dp.n_bulk = upr * dp.gen_runs;
-    } else {
-      dp.gen_pre.clear();
+      dp.n_gen = upr * runs0;
+    } else {  // too many for 32-bit unit indices in the generator: everything on the host
+      dp.gen_seg.clear(); dp.gen_pre.clear();
+      rest = bulk_segs;
     }
+  } else {
+    rest = bulk_segs;
   }
-  if (!dp.regular) {
-    expand_units_on_host(&dp, bulk_segs, T, p->tuning.unit_order % 2 == 0);
-    dp.n_bulk = dp.bulk_units.size();
-  }
+  expand_units_on_host(&dp, rest, T, p->tuning.unit_order % 2 == 0);
+  dp.n_bulk = dp.n_gen + dp.bulk_units.size();
   if (phase == EMOE_PHASE_KV) {  // block pairs of the head re-split, in launch order
     const KvPlan &kv = p->hp.kv;
     if (kv.head_split_changes && !kv.pair_old.empty())
@@ -301,26 +306,22 @@ void build_merged(emoe_plan *p) {
   p->merged = ns <= EMOE_MAX_RANKS && nd <= EMOE_MAX_RANKS;
   if (!p->merged) return;
   all.gen_seg.clear(); all.gen_pre.clear();
-  all.regular = false; all.n_bulk = 0;
-  // the merged bulk table is written on the device too if every phase's is
-  bool regular = true;
-  for (int ph = 0; ph < 3; ++ph) regular = regular && (p->dev[ph].n_bulk == 0 || p->dev[ph].regular);
-  size_t n_seg = 0, n_dst = 0, n_vec = 0;
+  all.n_gen = 0; all.n_bulk = 0;
+  size_t n_seg = 0, n_dst = 0, n_vec = 0, n_rest = 0;
   uint64_t n_bulk = 0;
   for (int ph = 0; ph < 3; ++ph) {
-    DevPhase &dp = p->dev[ph];
+    const DevPhase &dp = p->dev[ph];
     p->merged_seg0[ph] = (uint32_t)n_seg;
-    p->merged_unit0[ph] = n_bulk;
-    if (!regular && dp.regular && dp.bulk_units.empty())   // its units are needed on the host after all
-      expand_units_on_host(&dp, dp.gen_seg, bulk_tile(p), true);
+    p->merged_unit0[ph] = n_bulk;          // the phase's generated units, then its host-built ones
+    all.rest_off[ph] = n_rest;
     n_seg += dp.segs.size(); n_dst += dp.dsts.size();
-    n_bulk += dp.n_bulk; n_vec += dp.vec_units.size();
+    n_bulk += dp.n_bulk; n_vec += dp.vec_units.size(); n_rest += dp.bulk_units.size();
+    all.n_gen += dp.n_gen;
   }
   if (n_bulk >= 0xffffffffull) { p->merged = false; return; }
-  all.regular = regular && n_bulk > 0;
   all.n_bulk = n_bulk;
   all.segs.resize(n_seg); all.dsts.resize(n_dst); all.vec_units.resize(n_vec);
-  if (!all.regular) all.bulk_units.resize(n_bulk);
+  all.bulk_units.resize(n_rest);
   size_t i_seg = 0, i_dst = 0, i_bulk = 0, i_vec = 0;
   for (int ph = 0; ph < 3; ++ph) {
     const DevPhase &dp = p->dev[ph];
@@ -337,8 +338,7 @@ void build_merged(emoe_plan *p) {
       d = d0;
       d.rank += p->dst_base[ph];
     }
-    if (!all.regular)
-      for (const Unit &u0 : dp.bulk_units) { Unit &u = all.bulk_units[i_bulk++]; u = u0; u.seg += seg0; }
+    for (const Unit &u0 : dp.bulk_units) { Unit &u = all.bulk_units[i_bulk++]; u = u0; u.seg += seg0; }
     for (const Unit &u0 : dp.vec_units) { Unit &u = all.vec_units[i_vec++]; u = u0; u.seg += seg0; }
   }
 }
@@ -403,19 +403,24 @@ emoe_status_t upload_phase(emoe_plan *p, int phase) {
   if ((e = upload(dp.segs, &dp.d_segs)) != cudaSuccess) return cuda_status(e);
   if ((e = upload(dp.dsts, &dp.d_dsts)) != cudaSuccess) return cuda_status(e);
   if ((e = upload(dp.vec_units, &dp.d_vec_units)) != cudaSuccess) return cuda_status(e);
-  if (!dp.regular) {
-    if ((e = upload(dp.bulk_units, &dp.d_bulk_units)) != cudaSuccess) return cuda_status(e);
-    return EMOE_OK;
-  }
-  // regular: the table is written by a kernel (for the merged set, phase by phase)
+  // bulk unit table: generated part(s) written by a kernel, host-built part(s) copied after them
   if (dp.d_bulk_units) { cudaFree(dp.d_bulk_units); dp.d_bulk_units = nullptr; }
+  if (dp.n_bulk == 0) return EMOE_OK;
   if ((e = cudaMalloc((void **)&dp.d_bulk_units, dp.n_bulk * sizeof(Unit))) != cudaSuccess) return cuda_status(e);
-  if (phase < 3) return cuda_status(gen_units(p, phase, dp.d_segs, 0, dp.d_bulk_units));
-  for (int q = 0; q < 3; ++q)
-    if (p->dev[q].n_bulk) {
-      e = gen_units(p, q, dp.d_segs, p->merged_seg0[q], dp.d_bulk_units + p->merged_unit0[q]);
-      if (e != cudaSuccess) return cuda_status(e);
-    }
+  auto copy_rest = [&](const Unit *host, uint64_t n, Unit *dev) {
+    return n ? cudaMemcpy(dev, host, n * sizeof(Unit), cudaMemcpyHostToDevice) : cudaSuccess;
+  };
+  if (phase < 3) {
+    if (dp.n_gen && (e = gen_units(p, phase, dp.d_segs, 0, dp.d_bulk_units)) != cudaSuccess) return cuda_status(e);
+    return cuda_status(copy_rest(dp.bulk_units.data(), dp.bulk_units.size(), dp.d_bulk_units + dp.n_gen));
+  }
+  for (int q = 0; q < 3; ++q) {
+    const DevPhase &dq = p->dev[q];
+    Unit *at = dp.d_bulk_units + p->merged_unit0[q];
+    if (dq.n_gen && (e = gen_units(p, q, dp.d_segs, p->merged_seg0[q], at)) != cudaSuccess) return cuda_status(e);
+    e = copy_rest(dp.bulk_units.data() + dp.rest_off[q], dq.bulk_units.size(), at + dq.n_gen);
+    if (e != cudaSuccess) return cuda_status(e);
+  }
   return EMOE_OK;
 }
 
@@ -485,8 +490,12 @@ BulkConfig bulk_config(const emoe_plan *p, uint32_t grid) {
                 p->tuning.bulk_hints > 0 ? (uint32_t)p->tuning.bulk_hints - 1 : kDefaultHints, 0, wait_ns(p)};
   if (p->tuning.bw_limit_gbs > 0 && grid > 0) {
     // The limit counts bytes read plus bytes written, so loads get half of it; spread over
-    // the CTAs of the launch that is one tile per CTA every tile * grid / (limit / 2) ns.
-    const double ns = 2.0 * bc.tile_bytes * grid / (double)p->tuning.bw_limit_gbs;
+    // the CTAs that run at the same time - the grid, or what fits the SMs when the grid is
+    // larger - that is one tile per CTA every tile * CTAs / (limit / 2) ns.
+    const size_t per_cta = bulk_smem_bytes(bc.tile_bytes, bc.stages) + 2048;
+    const uint64_t fit = (uint64_t)p->sm_count * std::max<size_t>(1, (227 * 1024) / per_cta);
+    const double ctas = (double)std::min<uint64_t>(grid, fit);
+    const double ns = 2.0 * bc.tile_bytes * ctas / (double)p->tuning.bw_limit_gbs;
     bc.pace_ns = ns < 1.0 ? 1u : ns > 1e6 ? 1000000u : (uint32_t)ns;
   }
   return bc;
@@ -556,7 +565,8 @@ KvTables kv_tables(const KvPlan &kv, const uint32_t *d_pair_old, const uint32_t 
 void destroy_host_step(HostStep *hs);
 
 emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
-                          const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out);
+                          const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out,
+                          uint64_t expert_scale_bytes = 0);
 
 // Chunk plans, streams and events of the pipelined host-buffer step.  Leaves p->hs null
 // (the step then runs serially) when a layer slice of some arena is not 16-byte aligned.
@@ -645,13 +655,15 @@ emoe_status_t finish_device_plan(emoe_plan *p) {
 }
 
 emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
-                          const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out) {
+                          const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out,
+                          uint64_t expert_scale_bytes) {
   if (!shape || !old_cfg || !new_cfg || !out) return EMOE_ERR_INVALID_ARG;
+  if (expert_scale_bytes && (flags & EMOE_LAYOUT_FUSED_W13)) return EMOE_ERR_UNSUPPORTED;
   emoe_plan *p = new (std::nothrow) emoe_plan();
   if (!p) return EMOE_ERR_OOM;
   emoe_status_t st;
   try {
-    st = build_host_plan(*shape, *old_cfg, *new_cfg, flags, &p->hp);
+    st = build_host_plan(*shape, *old_cfg, *new_cfg, flags, expert_scale_bytes, &p->hp);
     if (st == EMOE_OK) {
       build_all_tables(p);
     }
@@ -662,9 +674,10 @@ emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cf
   p->host_only = (flags & EMOE_PLAN_HOST_ONLY) != 0;
   if (!p->host_only) {
     st = finish_device_plan(p);
-    if (st == EMOE_OK && (flags & EMOE_PLAN_HOST_STEP)) {
+    // (an expert arena with a scale part is not layer-major: such a plan's host step stays serial)
+    if (st == EMOE_OK && (flags & EMOE_PLAN_HOST_STEP) && !expert_scale_bytes) {
       st = make_host_step(p, *shape, old_cfg, new_cfg,
-                          flags & (EMOE_LAYOUT_FUSED_W13 | EMOE_LAYOUT_KV_HEAD_MAJOR));
+                          flags & (EMOE_LAYOUT_FUSED_W13 | EMOE_LAYOUT_KV_HEAD_MAJOR | EMOE_LAYOUT_FUSED_QKV));
       if (st != EMOE_OK) free_device(p);
     }
     if (st != EMOE_OK) { delete p; return st; }
@@ -714,6 +727,19 @@ extern "C" {
 emoe_status_t emoe_plan_create(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
                                const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out) {
   return create_plan(shape, old_cfg, new_cfg, flags, out);
+}
+
+emoe_status_t emoe_plan_create_ex(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
+                                  const emoe_config_t *new_cfg, uint32_t flags,
+                                  const emoe_plan_options_t *options, emoe_plan_t **out) {
+  uint64_t scale = 0;
+  if (options) {
+    if (options->expert_scale_bytes < 0) return EMOE_ERR_INVALID_ARG;
+    for (int64_t r : options->reserved)
+      if (r != 0) return EMOE_ERR_INVALID_ARG;
+    scale = (uint64_t)options->expert_scale_bytes;
+  }
+  return create_plan(shape, old_cfg, new_cfg, flags, out, scale);
 }
 
 void emoe_plan_destroy(emoe_plan_t *p) {

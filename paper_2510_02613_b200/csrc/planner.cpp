@@ -102,12 +102,16 @@ struct ExpertMove { int rs, ss, rd, sd; };
 // Moves -> segments.  slots_old / slots_new: slots per arena (the slot stride of a layer slab).
 // Single-destination sources: runs of consecutive slots on both sides merge (dense layout
 // only); a source with several destinations becomes one segment that is read once.
+// m: bytes of the tensor that moves per (layer, projection, slot) - the expert matrix, or the
+// scale tensor that goes with it; base_old / base_new: where that tensor's [L][3][n] array
+// starts inside each arena (null: at 0).
 void emit_expert_moves(const emoe_shape_t &sh, const std::vector<uint64_t> &slots_old,
-                       const std::vector<uint64_t> &slots_new, uint64_t slab,
+                       const std::vector<uint64_t> &slots_new, uint64_t slab, uint64_t m,
+                       const std::vector<uint64_t> *base_old, const std::vector<uint64_t> *base_new,
                        const std::vector<ExpertMove> &moves, std::map<std::pair<int, int>, int> &fan,
                        bool fused_w13, PhasePlan *pp) {
-  const uint64_t m = (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes;
   const uint32_t runs = (uint32_t)sh.n_layers * 3;
+  const size_t seg0 = pp->segs.size();
   // single-destination sources: merge runs of consecutive slots on both sides (dense layout only)
   std::map<std::pair<int, int>, std::vector<Dst>> multi;
   size_t i = 0;
@@ -173,6 +177,16 @@ void emit_expert_moves(const emoe_shape_t &sh, const std::vector<uint64_t> &slot
       finish_segment(pp, s, d2);
     }
   }
+  // the tensor's array does not start at the arena's first byte: shift what was just emitted
+  if (base_old || base_new)
+    for (size_t k = seg0; k < pp->segs.size(); ++k) {
+      Segment &sg = pp->segs[k];
+      if (base_old) sg.src_off += (*base_old)[sg.src_rank];
+      for (uint32_t j = 0; j < sg.n_dst; ++j) {
+        Dst &dd = pp->dsts[sg.dst_first + j];
+        if (base_new) dd.off += (*base_new)[dd.rank];
+      }
+    }
 }
 
 
@@ -181,13 +195,23 @@ void emit_expert_moves(const emoe_shape_t &sh, const std::vector<uint64_t> &slot
 // a destination slot whose source sits on the same rank index is recorded there instead
 // of being copied (that device already holds the bytes).
 // fused_w13 (dense layout only): per layer a [n][gate|up] tensor, then the [n][down] one.
+// scale_bytes > 0: every matrix travels with a scale tensor of that many bytes; an arena is
+// then the weight array [L][3][n][m], and from the next multiple of 256 bytes on the scale
+// array [L][3][n][scale_bytes].
 void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &pn, uint64_t slab,
-                  std::vector<Remap> *remaps, bool fused_w13, PhasePlan *pp) {
+                  std::vector<Remap> *remaps, bool fused_w13, uint64_t scale_bytes, PhasePlan *pp) {
   const uint64_t m = (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes;
   const uint32_t runs = (uint32_t)sh.n_layers * 3;
   const int n_experts = sh.n_routed + sh.n_shared;
-  for (int r = 0; r < po.ep; ++r) pp->arena_old.push_back(runs * po.ids[r].size() * slab);
-  for (int r = 0; r < pn.ep; ++r) pp->arena_new.push_back(runs * pn.ids[r].size() * slab);
+  std::vector<uint64_t> scale_base_old, scale_base_new;
+  auto arena = [&](uint64_t n, std::vector<uint64_t> *bases) {
+    const uint64_t w = runs * n * slab;
+    if (!scale_bytes) return w;
+    bases->push_back((w + 255) / 256 * 256);
+    return bases->back() + runs * n * scale_bytes;
+  };
+  for (int r = 0; r < po.ep; ++r) pp->arena_old.push_back(arena(po.ids[r].size(), &scale_base_old));
+  for (int r = 0; r < pn.ep; ++r) pp->arena_new.push_back(arena(pn.ids[r].size(), &scale_base_new));
 
   // every old copy of every expert, in (rank, slot) order
   std::vector<std::vector<std::pair<int, int>>> copies(n_experts);
@@ -214,12 +238,65 @@ void plan_experts(const emoe_shape_t &sh, const Placement &po, const Placement &
       fan[src]++;
     }
 
-  emit_expert_moves(sh, slots_old, slots_new, slab, moves, fan, fused_w13, pp);
+  emit_expert_moves(sh, slots_old, slots_new, slab, m, nullptr, nullptr, moves, fan, fused_w13, pp);
+  if (scale_bytes)   // the same moves once more for the scale tensors (plain [L][3][n] array)
+    emit_expert_moves(sh, slots_old, slots_new, scale_bytes, scale_bytes, &scale_base_old, &scale_base_new,
+                      moves, fan, false, pp);
 }
 
 // ---- attention --------------------------------------------------------------------------
 
-void plan_attn(const emoe_shape_t &sh, int c, int d, PhasePlan *pp) {
+// q, k and v rows of the fused-qkv arena: one move per head (a head's hd rows are contiguous
+// on both sides), moves that are neighbours on both sides merged, one strided segment
+// (a run per layer) per merged move.  Row groups: for every KV head of a rank, the rank's
+// query heads of that group, then the k head, then the v head.
+void plan_fused_qkv(const emoe_shape_t &sh, int c, int d, uint64_t layer_c, uint64_t layer_d,
+                    PhasePlan *pp) {
+  const uint64_t head = (uint64_t)sh.head_dim * sh.d_model * sh.elem_bytes;
+  const uint32_t hq = sh.n_q_heads, hkv = sh.n_kv_heads;
+  auto kvh = [&](int T) { return (uint64_t)kv_heads_per_rank(hkv, T); };
+  auto qpg = [&](int T) { return (uint64_t)(hq / T) / kvh(T); };
+  auto q_off = [&](int T, uint64_t h) {
+    const uint64_t local = h % (hq / T), j = local / qpg(T), i = local % qpg(T);
+    return (j * (qpg(T) + 2) + i) * head;
+  };
+  auto kv_off = [&](int T, uint64_t j, int which) { return (j * (qpg(T) + 2) + qpg(T) + which) * head; };
+  struct Mv { uint32_t ro, rn; uint64_t so, dn, bytes; };
+  std::vector<Mv> mv;
+  for (uint32_t h = 0; h < hq; ++h)
+    mv.push_back({h / (hq / c), h / (hq / d), q_off(c, h), q_off(d, h), head});
+  for (int which = 0; which < 2; ++which)
+    for (int rn = 0; rn < d; ++rn)
+      for (uint32_t jn = 0; jn < kvh(d); ++jn) {
+        const uint32_t g = kv_first_head(hkv, d, rn) + jn;
+        const uint32_t ro = kv_source_rank(hkv, c, g, rn);
+        mv.push_back({ro, (uint32_t)rn, kv_off(c, g - kv_first_head(hkv, c, ro), which),
+                      kv_off(d, jn, which), head});
+      }
+  std::sort(mv.begin(), mv.end(), [](const Mv &a, const Mv &b) {
+    return a.rn != b.rn ? a.rn < b.rn : a.dn < b.dn;
+  });
+  size_t i = 0;
+  while (i < mv.size()) {
+    Mv a = mv[i];
+    size_t j = i + 1;
+    while (j < mv.size() && mv[j].rn == a.rn && mv[j].ro == a.ro && mv[j].dn == a.dn + a.bytes &&
+           mv[j].so == a.so + a.bytes) {
+      a.bytes += mv[j].bytes;
+      ++j;
+    }
+    Segment s{};
+    s.src_off = a.so;
+    s.run_bytes = a.bytes;
+    s.src_pitch = layer_c;
+    s.n_runs = (uint32_t)sh.n_layers;
+    s.src_rank = a.ro;
+    finish_segment(pp, s, {Dst{a.dn, layer_d, a.rn, 0}});
+    i = j;
+  }
+}
+
+void plan_attn(const emoe_shape_t &sh, int c, int d, bool fused_qkv, PhasePlan *pp) {
   const uint64_t D = sh.d_model, b = sh.elem_bytes, hd = sh.head_dim;
   const uint64_t row = D * b;
   const uint32_t hkv = sh.n_kv_heads;
@@ -241,8 +318,9 @@ void plan_attn(const emoe_shape_t &sh, int c, int d, PhasePlan *pp) {
     }
     return;
   }
+  if (fused_qkv) plan_fused_qkv(sh, c, d, layer_bytes(c), layer_bytes(d), pp);
   // q: intersect old and new row ranges of the logical matrix
-  {
+  if (!fused_qkv) {
     const uint64_t rows = (uint64_t)sh.n_q_heads * hd;
     const uint64_t rc = rows / c, rd = rows / d;
     for (int ro = 0; ro < c; ++ro)
@@ -260,7 +338,7 @@ void plan_attn(const emoe_shape_t &sh, int c, int d, PhasePlan *pp) {
   }
   // k, v: every new rank's heads, grouped into runs of heads that are consecutive on one
   // old rank (with more ranks than KV heads a head has several holders: see kv_source_rank)
-  for (int t = 1; t < 3; ++t) {
+  for (int t = 1; t < 3 && !fused_qkv; ++t) {
     auto piece = [&](int T) { return t == 1 ? q_bytes(T) : q_bytes(T) + kv_bytes(T); };
     const uint32_t hn = kv_heads_per_rank(hkv, d);
     for (int rn = 0; rn < d; ++rn) {
@@ -404,7 +482,8 @@ uint32_t kv_source_rank(uint32_t hkv, uint32_t c, uint32_t g, uint32_t r_new) {
 }
 
 emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
-                              const emoe_config_t &n, uint32_t flags, HostPlan *hp) {
+                              const emoe_config_t &n, uint32_t flags, uint64_t expert_scale_bytes,
+                              HostPlan *hp) {
   if (sh.n_layers <= 0 || sh.n_routed <= 0 || sh.n_shared < 0 || sh.d_model <= 0 ||
       sh.d_ff <= 0 || sh.n_q_heads <= 0 || sh.n_kv_heads <= 0 || sh.head_dim <= 0 ||
       sh.kv_block_tokens <= 0 || sh.elem_bytes <= 0)
@@ -427,8 +506,9 @@ emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
   hp->shape = sh;
   hp->ep_old = o.ep; hp->ep_new = n.ep; hp->tp_old = o.tp; hp->tp_new = n.tp;
   plan_experts(sh, po, pn, (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes, nullptr,
-               (flags & EMOE_LAYOUT_FUSED_W13) != 0, &hp->phase[EMOE_PHASE_EXPERTS]);
-  plan_attn(sh, o.tp, n.tp, &hp->phase[EMOE_PHASE_ATTN]);
+               (flags & EMOE_LAYOUT_FUSED_W13) != 0, expert_scale_bytes, &hp->phase[EMOE_PHASE_EXPERTS]);
+  if ((flags & EMOE_LAYOUT_FUSED_QKV) && sh.n_q_heads % sh.n_kv_heads) return EMOE_ERR_SHAPE;
+  plan_attn(sh, o.tp, n.tp, (flags & EMOE_LAYOUT_FUSED_QKV) != 0, &hp->phase[EMOE_PHASE_ATTN]);
   plan_kv(sh, o, n, std::move(pair_old), std::move(pair_new), (flags & EMOE_LAYOUT_KV_HEAD_MAJOR) != 0, hp);
   return EMOE_OK;
 }
@@ -445,7 +525,7 @@ emoe_status_t build_paged_expert_plan(const emoe_shape_t &sh, const emoe_config_
   if (st != EMOE_OK) return st;
   st = read_placement(n, sh.n_routed + sh.n_shared, &pn);
   if (st != EMOE_OK) return st;
-  plan_experts(sh, po, pn, slab, remaps, false, pp);
+  plan_experts(sh, po, pn, slab, remaps, false, 0, pp);
   return EMOE_OK;
 }
 
@@ -519,7 +599,7 @@ emoe_status_t build_inplace_expert_plan(const emoe_shape_t &sh, int ep_old, cons
       ++next_free;
     }
   }
-  emit_expert_moves(sh, slots_old, slots_new, m, moves, fan, false, pp);
+  emit_expert_moves(sh, slots_old, slots_new, m, m, nullptr, nullptr, moves, fan, false, pp);
   return EMOE_OK;
 }
 

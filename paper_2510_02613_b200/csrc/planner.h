@@ -74,9 +74,11 @@ struct HostPlan {
 };
 
 // Validates and plans.  Returns EMOE_OK or the first validation error.
-// flags: the EMOE_LAYOUT_* bits of emoe_plan_create.
+// flags: the EMOE_LAYOUT_* bits of emoe_plan_create.  expert_scale_bytes: size of the scale
+// tensor that goes with every expert matrix (0: none).
 emoe_status_t build_host_plan(const emoe_shape_t &shape, const emoe_config_t &old_cfg,
-                              const emoe_config_t &new_cfg, uint32_t flags, HostPlan *out);
+                              const emoe_config_t &new_cfg, uint32_t flags, uint64_t expert_scale_bytes,
+                              HostPlan *out);
 
 // A destination slot that keeps the bytes its rank already holds (paged expert store).
 struct Remap {

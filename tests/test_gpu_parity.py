@@ -398,6 +398,22 @@ def test_layout_variants_one_layer(name):
                 check_phase_full(w, plan, phase)
 
 
+@pytest.mark.parametrize("name,c,d", [("c1_tiny", 1, 2), ("c4_large", 2, 4), ("c4_large", 4, 2),
+                                      ("c4_large", 2, 8), ("c4_large", 8, 1), ("c3_fine", 2, 4)])
+def test_fused_qkv_layout(name, c, d):
+    """Attention re-slice with one fused qkv matrix per rank (rows grouped by KV head), at
+    full width, alone and as part of the whole step."""
+    from gpu_util import make_plan
+    wl = W.make_workload(name, n_layers=2)
+    wl = R(wl, fused_qkv=True, old=R(wl.old, tp=c), new=R(wl.new, tp=d),
+           shape=R(wl.shape, d_ff=64))
+    with make_plan(wl) as plan:
+        check_phase_full(wl, plan, E.PHASE_ATTN)
+        check_step_full(wl, plan)
+        plan.set_tuning(path=2, max_ctas=11)
+        check_phase_full(wl, plan, E.PHASE_ATTN)
+
+
 def test_scaling_sequence_with_chosen_placements():
     """A sequence of scale steps in the paper's step pattern (+2 devices per step, then
     back down), each new placement chosen by emoe_place_min_transfer from the previous
@@ -524,15 +540,25 @@ def test_kv_delta_plan_recopies_blocks_written_during_the_migration():
         assert moved * 8 < p_all.stats(E.PHASE_KV)["bytes_moved"]      # the delta is small
 
 
-def test_fp8_weights_with_block_scales_as_two_plans():
+def test_fp8_weights_with_block_scales_in_one_plan():
     """FP8 expert weights (elem_bytes = 1) and their per-128x128-block fp32 scale tensors
-    move with the same placement through two plans: one for the weights, one whose
-    "matrix" is the scale tensor of an expert ([d_ff/128][d_model/128] floats)."""
-    base = W.make_workload("c3_fine", n_layers=1)
-    weights = R(base, shape=R(base.shape, elem_bytes=1))
-    scales = R(base, shape=R(base.shape, d_model=base.shape.d_model // 128,
-                             d_ff=base.shape.d_ff // 128, elem_bytes=4))
-    assert scales.shape.d_model * scales.shape.d_ff * 4 == 16 * 11 * 4
-    for wl in (weights, scales):
-        with E.Plan(wl.shape, wl.old, wl.new) as plan:
-            check_phase_full(wl, plan, E.PHASE_EXPERTS)
+    ([d_ff/128][d_model/128] floats per matrix) move with the same placement through ONE plan
+    and one call: the arena of a rank holds the weights and, after them, the scales."""
+    base = W.make_workload("c3_fine", n_layers=2)
+    scale_bytes = (base.shape.d_model // 128) * (base.shape.d_ff // 128) * 4
+    assert scale_bytes == 16 * 11 * 4
+    wl = R(base, shape=R(base.shape, elem_bytes=1, expert_scale_bytes=scale_bytes))
+    for w in (wl, wl.swapped()):
+        with E.Plan(w.shape, w.old, w.new) as plan:
+            check_phase_full(w, plan, E.PHASE_EXPERTS)
+            check_step_full(w, plan)
+            assert plan.num_launches(E.PHASE_STEP) <= 2
+            plan.set_tuning(path=2, max_ctas=13)
+            check_phase_full(w, plan, E.PHASE_EXPERTS)
+            plan.set_tuning(path=1)
+            check_phase_full(w, plan, E.PHASE_EXPERTS)
+    # odd sizes: scale tensors that are not multiples of 16 bytes
+    odd = R(base, shape=R(base.shape, n_layers=3, d_model=24, d_ff=20, elem_bytes=1, expert_scale_bytes=6))
+    with E.Plan(odd.shape, odd.old, odd.new) as plan:
+        check_phase_full(odd, plan, E.PHASE_EXPERTS)
+        check_step_full(odd, plan)

@@ -727,3 +727,23 @@ def test_experts_with_scales_hand_written():
     assert list(dst[0][:6]) == [2, 2, 4, 4, 6, 6] and list(dst[0][256:]) == [12, 14, 16]
     assert list(dst[1][:6]) == [1, 1, 3, 3, 5, 5] and list(dst[1][256:]) == [11, 13, 15]
     assert not dst[0][6:256].any() and not dst[1][6:256].any()
+
+
+# ============================================================ compacting block table ===
+
+def test_compact_block_table_hand_written_and_properties():
+    """Two sequences of 5 and 3 tokens in 2-token blocks need 3 + 2 blocks; in a pool of 8
+    with blocks 1 and 4 taken they get 0, 2, 3 and 5, 6 (written by hand)."""
+    t = oracle.compact_block_table([5, 3], 2, 8, in_use=[1, 4])
+    assert t.tolist() == [[0, 2, 3], [5, 6, -1]]
+    assert oracle.compact_block_table([5, 3], 2, 5).tolist() == [[0, 1, 2], [3, 4, -1]]   # fresh pool: identity
+    rng = np.random.default_rng(3)
+    for _ in range(20):
+        nb = int(rng.integers(6, 30))
+        in_use = [int(x) for x in rng.permutation(nb)[:int(rng.integers(0, nb // 2))]]
+        free = sorted(set(range(nb)) - set(in_use))
+        lens = [int(x) for x in rng.integers(0, 8, size=3)]
+        if sum(-(-n // 3) for n in lens) > len(free):
+            continue
+        flat = [int(x) for row in oracle.compact_block_table(lens, 3, nb, in_use) for x in row if x >= 0]
+        assert flat == free[:len(flat)]

@@ -55,7 +55,7 @@ def run_oracle(wl, phase, src, dst):
         oracle.reshard_experts(wl.shape, wl.old.placement, wl.new.placement, src, dst,
                                fused_w13=wl.fused_w13)
     elif phase == E.PHASE_ATTN:
-        oracle.reshard_attn(wl.shape, wl.old.tp, wl.new.tp, src, dst)
+        oracle.reshard_attn(wl.shape, wl.old.tp, wl.new.tp, src, dst, fused_qkv=wl.fused_qkv)
     else:
         oracle.reshard_kv(wl.shape, wl.old, wl.new, src, dst, head_major=wl.kv_head_major)
 
@@ -276,3 +276,74 @@ print("ok")
     env = dict(os.environ, CUDA_VISIBLE_DEVICES="", PYTHONPATH=ROOT)
     out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, cwd=ROOT)
     assert out.returncode == 0 and out.stdout.strip() == "ok", out.stderr[-2000:]
+
+
+@pytest.mark.parametrize("name,c,d", [("c1_tiny", 1, 2), ("c1_tiny", 4, 2), ("c4_large", 2, 4),
+                                      ("c4_large", 4, 1), ("c4_large", 2, 8), ("c4_large", 16, 4),
+                                      ("c2_mid", 2, 2)])
+def test_fused_qkv_segment_replay_equals_oracle(name, c, d):
+    """The attention phase with a fused qkv matrix per rank: replayed segments == oracle,
+    destinations tile the arena exactly once."""
+    wl = small(name)
+    wl = dataclasses.replace(wl, fused_qkv=True, old=dataclasses.replace(wl.old, tp=c),
+                             new=dataclasses.replace(wl.new, tp=d))
+    with E.Plan(wl.shape, wl.old, wl.new, host_only=True, fused_qkv=True) as plan, \
+            E.Plan(wl.shape, wl.old, wl.new, host_only=True) as plain:
+        so, sn = oracle_sizes(wl, E.PHASE_ATTN)
+        assert plan.arena_bytes(E.PHASE_ATTN, E.SIDE_NEW) == sn
+        src = arenas(so, 31)
+        want = [np.full(n, FILL, np.uint8) for n in sn]
+        got = [np.full(n, FILL, np.uint8) for n in sn]
+        run_oracle(wl, E.PHASE_ATTN, src, want)
+        segs = plan.segments(E.PHASE_ATTN)
+        replay(segs, src, got)
+        for r in range(len(sn)):
+            assert np.array_equal(got[r], want[r]), r
+        cover = [np.zeros(n, np.uint8) for n in sn]
+        for s in segs:
+            for i in range(int(s["n_runs"])):
+                b = int(s["dst_off"]) + i * int(s["dst_pitch"])
+                cover[int(s["dst_rank"])][b:b + int(s["run_bytes"])] += 1
+        assert all(cv.min(initial=1) == 1 and cv.max(initial=1) == 1 for cv in cover)
+        assert plan.stats(E.PHASE_ATTN)["bytes_moved"] == plain.stats(E.PHASE_ATTN)["bytes_moved"]
+
+
+def test_fused_qkv_needs_whole_query_groups():
+    wl = small("c1_tiny")
+    sh = dataclasses.replace(wl.shape, n_q_heads=12, n_kv_heads=8)   # 12 % 8 != 0
+    cfg = lambda c: dataclasses.replace(c, tp=1)
+    with pytest.raises(E.EmoeError) as ei:
+        E.Plan(sh, cfg(wl.old), cfg(wl.new), host_only=True, fused_qkv=True)
+    assert ei.value.code == 2
+
+
+@pytest.mark.parametrize("name", ["c2_mid", "c3_fine", "c4_large"])
+@pytest.mark.parametrize("ms", [4, 48])
+def test_expert_scales_travel_with_their_matrices_in_one_plan(name, ms):
+    """emoe_plan_create_ex with expert_scale_bytes: replayed segments == oracle over the
+    whole arena (weights, the gap nobody writes, scales)."""
+    wl = small(name)
+    wl = dataclasses.replace(wl, shape=dataclasses.replace(wl.shape, elem_bytes=1, expert_scale_bytes=ms))
+    for w in (wl, wl.swapped()):
+        with E.Plan(w.shape, w.old, w.new, host_only=True) as plan:
+            so, sn = oracle_sizes(w, E.PHASE_EXPERTS)
+            assert plan.arena_bytes(E.PHASE_EXPERTS, E.SIDE_OLD) == so
+            assert plan.arena_bytes(E.PHASE_EXPERTS, E.SIDE_NEW) == sn
+            src = arenas(so, 51)
+            want = [np.full(n, FILL, np.uint8) for n in sn]
+            got = [np.full(n, FILL, np.uint8) for n in sn]
+            run_oracle(w, E.PHASE_EXPERTS, src, want)
+            replay(plan.segments(E.PHASE_EXPERTS), src, got)
+            for r in range(len(sn)):
+                assert np.array_equal(got[r], want[r]), r
+            m = w.shape.d_model * w.shape.d_ff
+            slots = sum(len(p) for p in w.new.placement)
+            assert plan.stats(E.PHASE_EXPERTS)["bytes_moved"] == w.shape.n_layers * 3 * slots * (m + ms)
+
+
+def test_plan_options_are_validated():
+    wl = small("c2_mid")
+    sh = dataclasses.replace(wl.shape, expert_scale_bytes=8)
+    with pytest.raises(E.EmoeError) as ei:
+        E.Plan(sh, wl.old, wl.new, host_only=True, fused_w13=True)     # scales + fused gate|up
+    assert ei.value.code == 9

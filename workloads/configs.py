@@ -193,6 +193,10 @@ def _kv_configs(seed: int, total_blocks: int, block_tokens: int, seq_lens: Optio
 # ---- the five workloads ----------------------------------------------------------------
 
 WORKLOAD_NAMES = ("c1_tiny", "c2_mid", "c3_fine", "c4_large", "c5_overlap")
+# beyond the five benchmark configurations: shaped like the largest model of the paper's
+# evaluation (256 routed experts, wider d_model, FP8 weights with block scales), cut to the
+# layers that fit one GPU
+EXTRA_WORKLOAD_NAMES = ("c6_wide_fp8",)
 
 
 def make_workload(name: str, n_layers: Optional[int] = None, new_order: str = "random") -> Workload:
@@ -225,6 +229,17 @@ def make_workload(name: str, n_layers: Optional[int] = None, new_order: str = "r
         old = ParallelConfig(3, 2, place_contiguous(128, 3), nbo, sl, bto)
         new = ParallelConfig(5, 4, place_hot_replicated(load, 5, 8), nbn, sl, btn)
         notes = "EP3 -> EP5 with the 8 hottest experts (Zipf 1.2) held twice; TP2 -> TP4"
+    elif name == "c6_wide_fp8":
+        # 256 routed experts + 1 shared, d_model 7168, expert d_ff 2048, one byte per weight and
+        # one fp32 scale per 128 x 128 block (56 x 16 x 4 bytes per matrix); 5 of the model's
+        # layers: old + new expert arenas are then 117 GB
+        seed = MASTER_SEED + 5
+        sh = Shape(5, 256, 1, 7168, 2048, 128, 8, 128, 16, 1, 56 * 16 * 4)
+        sl, nbo, bto, nbn, btn = _kv_configs(seed, 65536 // 16, 16, None, new_order=new_order)
+        old = ParallelConfig(8, 1, with_shared(place_contiguous(256, 8), [256]), nbo, sl, bto)
+        new = ParallelConfig(12, 1, with_shared(place_contiguous(256, 12), [256]), nbn, sl, btn)
+        notes = ("EP8 -> EP12, 256 routed experts + 1 shared on every rank, FP8 weights with "
+                 "128x128-block fp32 scales moved by the same plan, TP1")
     else:
         raise KeyError(name)
     victim = None
