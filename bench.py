@@ -682,6 +682,33 @@ def run_vmm(torch, E, wl, copy_all_ms):
     return out
 
 
+def run_vmm_slots(torch, E, wl, copy_all_ms):
+    """The paged store with slot tables (ranges kept across steps, only changed slots mapped,
+    copied or unmapped, arrivals served from pages created beforehand) on the workload's
+    expert placements, on uninitialised pages.  Host wall-clock of the synchronous call."""
+    torch.cuda.empty_cache()
+    want = [list(p) for p in wl.new.placement]
+    old, arrivals = [], 0
+    for r, p in enumerate(wl.old.placement):
+        k = len([e for e in want[r] if e not in p]) if r < len(want) else 0
+        old.append(list(p) + [-1] * k)
+    cap_new = [len(t) for t in old][:len(want)] + [len(want[r]) for r in range(len(old), len(want))]
+    arrivals = sum(len([e for e in w if r >= len(wl.old.placement) or e not in wl.old.placement[r]])
+                   for r, w in enumerate(want))
+    try:
+        with E.VmmSlots(wl.shape, old, spare_slots=arrivals) as pool:
+            torch.cuda.synchronize()
+            st = pool.reshard(want, cap_new)
+            back = pool.reshard([list(p) for p in wl.old.placement], [len(t) for t in old])  # and down again
+    except E.EmoeError as e:
+        return {"error": str(e)}
+    out = {k: (round(v, 3) if isinstance(v, float) else v) for k, v in st.items()}
+    out["step_back_total_ms"] = round(back["total_ms"], 3)
+    out["step_back_alloc_ms"] = round(back["alloc_ms"], 3)
+    out["dense_copy_all_ms"] = round(copy_all_ms, 3)
+    return out
+
+
 # ---- reference arm: the oracle on the host cores -----------------------------------------
 
 def run_reference(args):
@@ -724,6 +751,106 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ---- exchange mode: one rank per GPU, the step as a pull over the interconnect -----------
+
+def run_exchange(args):
+    """bench.py --gpus N --mode exchange (under torchrun): rank = GPU.  Every process owns the
+    old and the new arenas of its rank index, builds the same plan, restricts it to its own
+    destination rank and PULLS what it needs from its peers' old arenas through CUDA IPC
+    mappings - the library's own kernels reading peer memory (plain loads, non-multicast bulk
+    copies); torch.distributed carries handles, barriers and the max of the step times only.
+    value = 2 x bytes all ranks wrote / slowest rank's time."""
+    import torch
+    import torch.distributed as dist
+    import paper_2510_02613_b200 as E
+    from paper_2510_02613_b200 import exchange, replicas
+    import workloads as W
+    from workloads import device as WD
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world < 2:
+        raise SystemExit("--mode exchange needs at least two ranks (torchrun --nproc-per-node N)")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the re-layout has no CPU path")
+    local = local % torch.cuda.device_count()
+    torch.cuda.set_device(local)
+    backend = os.environ.get("EMOE_BENCH_BACKEND", "nccl")
+    if backend == "nccl":
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        dist.init_process_group(backend)
+    peak, peak_kind = measured_peak()
+    wl = W.make_exchange_workload(world, n_layers=args.layers)
+    kinds = (W.KIND_EXPERTS, W.KIND_ATTN, W.KIND_KV)
+    stream = torch.cuda.Stream()
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        old, new = [], []
+        for ph in range(3):
+            so, sn = plan.arena_bytes(ph, E.SIDE_OLD), plan.arena_bytes(ph, E.SIDE_NEW)
+            mine = None
+            if rank < len(so):      # this process owns rank index `rank` of either side
+                mine = torch.empty(so[rank], dtype=torch.uint8, device="cuda")
+                W.rng.torch_fill_bytes(mine, W.arena_key(wl.seed, kinds[ph], rank))
+            old.append(mine)
+            new.append(WD.alloc_const([sn[rank]])[0] if rank < len(sn) else None)
+        torch.cuda.synchronize()
+        dist.barrier()
+        ex = exchange.Exchange(dist, plan, rank, old, new)
+        try:
+            pulled = ex.bytes_pulled()
+            for _ in range(args.warmup):
+                ex.step(stream)
+            stream.synchronize()
+            dist.barrier()
+            torch.cuda.synchronize()
+            sampler = ClockSampler(local)
+            sampler.start()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.steps):
+                ex.step(stream)
+            e1.record(stream)
+            stream.synchronize()
+            torch.cuda.synchronize()
+            clocks = sampler.stop()
+            dist.barrier()
+            local_ms = e0.elapsed_time(e1)
+            dev = "cuda" if backend == "nccl" else "cpu"
+            total_ms = replicas.job_time_ms(local_ms, dist, device=dev)
+            status = plan.device_status()
+            n_launch = sum(plan.num_launches(ph) for ph in range(3)
+                           if rank < plan.num_ranks(ph, E.SIDE_NEW))
+            per_rank = [None] * world
+            dist.all_gather_object(per_rank, dict(rank=rank, ms_per_step=round(local_ms / args.steps, 4),
+                                                  bytes_written=pulled["written"],
+                                                  bytes_from_peers=pulled["from_peers"],
+                                                  pull_gbs=round(pulled["from_peers"] / (local_ms / args.steps) / 1e6, 1),
+                                                  launches_per_step=n_launch, device_status=status))
+        finally:
+            ex.close()
+    if rank == 0:
+        moved = sum(r["bytes_written"] for r in per_rank)
+        ms = total_ms / args.steps
+        line = {"metric": METRIC, "value": round(2 * moved / ms / 1e6, 1), "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 4),
+                "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "u8",
+                "data": "synthetic", "mode": "exchange",
+                "config": {"workload": wl.name if args.layers is None
+                           else "%s cut to %d layers" % (wl.name, args.layers),
+                           "reconfig": wl.notes, "parallelism": "one rank per GPU, pull over peer mappings",
+                           "l2": "inputs_larger_than_l2", "value_convention": "2 x bytes written by all ranks / slowest rank's time",
+                           "control_plane": backend},
+                "clocks": clocks, "per_rank": per_rank,
+                "bytes_from_peers_total": sum(r["bytes_from_peers"] for r in per_rank),
+                "e2e": {"value": None, "unit": UNIT, "note": "measured in the default mode at --gpus 1 only"},
+                "gpu_launches": sum(r["launches_per_step"] for r in per_rank) * args.steps}
+        print(json.dumps(line))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
 # ---- main --------------------------------------------------------------------------------
 
 def main():
@@ -733,6 +860,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c2_mid")
     ap.add_argument("--impl", default="emoe", choices=["emoe", "reference"])
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "exchange"],
+                    help="replicas (default): every GPU runs the whole workload on its own; exchange: one "
+                         "rank per GPU, the step pulled over the interconnect (needs --gpus >= 2)")
     ap.add_argument("--only-main", action="store_true",
                     help="skip the other configs, the overlap case, e2e and the CPU baseline")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -753,6 +883,9 @@ def main():
 
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.mode == "exchange":
+        run_exchange(args)
         return
 
     import torch
@@ -856,6 +989,7 @@ def main():
     if rank == 0 and not args.only_main:
         rep["inplace_expert_step"] = run_inplace(torch, E, wl, rep["phases"]["experts"]["ms"], peak)
         rep["vmm_expert_step"] = run_vmm(torch, E, wl, rep["phases"]["experts"]["ms"])
+        rep["vmm_slots_expert_step"] = run_vmm_slots(torch, E, wl, rep["phases"]["experts"]["ms"])
 
     if not args.only_main and world == 1:
         others = {}
@@ -887,6 +1021,7 @@ def main():
             if name in ("c2_mid", "c3_fine", "c4_large"):
                 r["inplace_expert_step"] = run_inplace(torch, E, wl2, r["phases"]["experts"]["ms"], peak)
                 r["vmm_expert_step"] = run_vmm(torch, E, wl2, r["phases"]["experts"]["ms"])
+                r["vmm_slots_expert_step"] = run_vmm_slots(torch, E, wl2, r["phases"]["experts"]["ms"])
         line["configs"] = others
 
     if dist:

@@ -194,7 +194,10 @@ emoe_status_t emoe_plan_create_ex(const emoe_shape_t *shape, const emoe_config_t
  * Calls may be enqueued on any streams; at most 4 launches of the SAME phase of
  * the SAME plan may be in flight on the GPU at once (they claim work through
  * per-launch counters of which the plan has 4 per phase) - more must be
- * ordered by the caller.  Calls on one stream are always fine.
+ * ordered by the caller.  Calls on one stream are always fine.  A call that is
+ * being captured into a CUDA graph uses no counter (its CTAs take their work
+ * round-robin), so a graph never holds on to one and may be replayed beside
+ * live calls.
  */
 emoe_status_t emoe_reshard_experts(const emoe_plan_t *plan, const void *const *src,
                                    void *const *dst, void *cuda_stream);
@@ -301,7 +304,12 @@ emoe_status_t emoe_reshard_step_host(const emoe_plan_t *plan, const void *const 
  * emoe_reshard_kv, whether or not the TP degree changes.
  *
  * Each call first copies the plan's pair list into the fixed array on
- * cuda_stream, then launches the kernel on the same stream.  All calls on a
+ * cuda_stream, then launches the kernel on the same stream.  The list lives
+ * in ordinary (pageable) host memory of the plan, so the driver stages that
+ * copy and the CALL may wait until cuda_stream has reached it - up to two
+ * copies of 256 KiB; the plan must stay alive until the stream has passed the
+ * call.  With emoe_plan_set_local_rank in force only that rank's blocks are
+ * written, as for emoe_reshard_kv (other dst[] entries may then be NULL).  All calls on a
  * device share that one array, and it keeps the previous call's list: two
  * calls whose GPU work can overlap (different streams without an ordering
  * between them) race on it and must be serialised by the caller.  Nothing in
@@ -447,6 +455,46 @@ emoe_status_t emoe_vmm_read(const emoe_vmm_pool_t *pool, int rank, void *host_de
 
 /* Unmaps and frees everything (synchronises the device first).  NULL-safe. */
 void emoe_vmm_destroy(emoe_vmm_pool_t *pool);
+
+/* ---- paged expert store with slot tables: a step touches only what changes ---
+ *
+ * The store above builds every range anew at every step.  This variant keeps a device's
+ * range for as long as the device exists and follows the in-place expert step
+ * (emoe_plan_create_inplace: same slot tables, same rules): the range of device r is
+ * RESERVED for cap_r slots, [L][3][cap_r][slab], and only occupied slots have pages.  A
+ * step leaves kept experts alone (no driver call, no copy), maps pages into the slots of
+ * arrivals - taken from a list of spare pages, so that no physical memory is created
+ * inside a step as long as the list lasts - fills them with the copy kernels, and after
+ * the copies unmaps the slots of experts that left, whose pages go back to the spare
+ * list.  Driver work and bytes copied are proportional to the slots that change.
+ *
+ * emoe_vmm_slots_create: slot_off [ep+1] / slot_ids: CSR slot tables (-1 = free; capacity
+ *   of device r = slot_off[r+1] - slot_off[r]); spare_slots: slots' worth of physical pages
+ *   (3 * n_layers slabs each) created up front for the arrivals of later steps.
+ * emoe_vmm_slots_reshard: cap_new / want_off / want_ids as for emoe_plan_create_inplace
+ *   (same errors, reported before anything is touched).  SYNCHRONOUS: returns after the
+ *   copies and the unmapping.  On failure the store is unchanged.  stats (optional):
+ *   slabs_remapped counts slabs kept in place, slabs_copied those of arrivals.
+ * emoe_vmm_slots_info: base address, capacity and slot table of `rank` (rank < 0: only the
+ *   pool-wide outputs: slab size, device count, spare slabs).  NULL outputs are skipped.
+ *   A free slot has NO memory behind it: only occupied slots may be read or written.
+ * emoe_vmm_slots_write / _read: one occupied slot as a dense host image [L][3][m].
+ * emoe_vmm_slots_destroy: synchronises the device, unmaps and frees everything. */
+typedef struct emoe_vmm_slots emoe_vmm_slots_t;
+emoe_status_t emoe_vmm_slots_create(const emoe_shape_t *shape, int32_t ep, const int32_t *slot_off,
+                                    const int32_t *slot_ids, int32_t spare_slots,
+                                    emoe_vmm_slots_t **out);
+emoe_status_t emoe_vmm_slots_reshard(emoe_vmm_slots_t *pool, int32_t ep_new, const int32_t *cap_new,
+                                     const int32_t *want_off, const int32_t *want_ids,
+                                     void *cuda_stream, emoe_vmm_stats_t *stats);
+emoe_status_t emoe_vmm_slots_info(const emoe_vmm_slots_t *pool, int32_t rank, void **base,
+                                  uint64_t *slab_bytes, int32_t *cap, int32_t *ids_out,
+                                  int32_t ids_cap, int32_t *n_ranks, int64_t *spare_slabs);
+emoe_status_t emoe_vmm_slots_write(emoe_vmm_slots_t *pool, int32_t rank, int32_t slot,
+                                   const void *host, void *cuda_stream);
+emoe_status_t emoe_vmm_slots_read(const emoe_vmm_slots_t *pool, int32_t rank, int32_t slot,
+                                  void *host, void *cuda_stream);
+void emoe_vmm_slots_destroy(emoe_vmm_slots_t *pool);
 
 /* emoe_plan_destroy - frees host state and device descriptor buffers.
  * NULL-safe.  No kernel using the plan may still be in flight. */

@@ -85,7 +85,9 @@ EXPORTS = ("emoe_plan_create", "emoe_plan_create_ex", "emoe_reshard_experts", "e
            "emoe_plan_cache_create", "emoe_plan_cache_get", "emoe_plan_cache_stats", "emoe_plan_cache_destroy",
            "emoe_kv_compact_table", "emoe_place_min_transfer", "emoe_plan_set_local_rank", "emoe_ipc_export", "emoe_ipc_open", "emoe_ipc_close",
            "emoe_vmm_create", "emoe_vmm_reshard", "emoe_vmm_dry_run", "emoe_vmm_num_ranks", "emoe_vmm_arena",
-           "emoe_vmm_write", "emoe_vmm_read", "emoe_vmm_destroy")
+           "emoe_vmm_write", "emoe_vmm_read", "emoe_vmm_destroy",
+           "emoe_vmm_slots_create", "emoe_vmm_slots_reshard", "emoe_vmm_slots_info", "emoe_vmm_slots_write",
+           "emoe_vmm_slots_read", "emoe_vmm_slots_destroy")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -192,6 +194,19 @@ def lib() -> ctypes.CDLL:
         f.argtypes = [_vp, _i32, _vp, _vp]
     L.emoe_vmm_destroy.restype = None
     L.emoe_vmm_destroy.argtypes = [_vp]
+    L.emoe_vmm_slots_create.restype = _i32
+    L.emoe_vmm_slots_create.argtypes = [ctypes.POINTER(_Shape), _i32, _i32p, _i32p, _i32, ctypes.POINTER(_vp)]
+    L.emoe_vmm_slots_reshard.restype = _i32
+    L.emoe_vmm_slots_reshard.argtypes = [_vp, _i32, _i32p, _i32p, _i32p, _vp, ctypes.POINTER(_VmmStats)]
+    L.emoe_vmm_slots_info.restype = _i32
+    L.emoe_vmm_slots_info.argtypes = [_vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_u64), _i32p, _i32p, _i32,
+                                      _i32p, ctypes.POINTER(ctypes.c_int64)]
+    for name in ("emoe_vmm_slots_write", "emoe_vmm_slots_read"):
+        f = getattr(L, name)
+        f.restype = _i32
+        f.argtypes = [_vp, _i32, _i32, _vp, _vp]
+    L.emoe_vmm_slots_destroy.restype = None
+    L.emoe_vmm_slots_destroy.argtypes = [_vp]
     L.emoe_strerror.restype = ctypes.c_char_p
     L.emoe_strerror.argtypes = [_i32]
     _lib = L
@@ -640,3 +655,81 @@ class VmmPool:
         _check(lib().emoe_vmm_reshard(self._h, ctypes.byref(self._config(new_cfg)),
                                       _stream_handle(stream), ctypes.byref(st)))
         return {n: getattr(st, n) for n, _ in _VmmStats._fields_}
+
+
+def _csr_i32(lists):
+    off = np.zeros(len(lists) + 1, dtype=np.int32)
+    off[1:] = np.cumsum([len(x) for x in lists])
+    ids = _i32arr([e for x in lists for e in x])
+    return off, (ids if ids.size else np.zeros(1, dtype=np.int32))
+
+
+class VmmSlots:
+    """Paged expert store with slot tables: emoe_vmm_slots_create ... _destroy.  slots: per
+    device a list of expert ids or -1 (free), as long as the device's capacity."""
+
+    def __init__(self, shape, slots, spare_slots: int = 0):
+        self._h = _vp()
+        self.shape = shape
+        sh = _Shape(shape.n_layers, shape.n_routed, shape.n_shared, shape.d_model, shape.d_ff,
+                    shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.kv_block_tokens,
+                    shape.elem_bytes)
+        off, ids = _csr_i32(slots)
+        p = lambda a: a.ctypes.data_as(_i32p)
+        _check(lib().emoe_vmm_slots_create(ctypes.byref(sh), len(slots), p(off), p(ids), spare_slots,
+                                           ctypes.byref(self._h)))
+
+    def close(self) -> None:
+        if self._h:
+            lib().emoe_vmm_slots_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    def info(self) -> dict:
+        n, spare, slab = _i32(), ctypes.c_int64(), _u64()
+        _check(lib().emoe_vmm_slots_info(self._h, -1, None, ctypes.byref(slab), None, None, 0,
+                                         ctypes.byref(n), ctypes.byref(spare)))
+        return dict(n_ranks=n.value, spare_slabs=spare.value, slab_bytes=slab.value)
+
+    def tables(self):
+        out = []
+        for r in range(self.info()["n_ranks"]):
+            cap = _i32()
+            _check(lib().emoe_vmm_slots_info(self._h, r, None, None, ctypes.byref(cap), None, 0, None, None))
+            t = np.zeros(max(cap.value, 1), dtype=np.int32)
+            _check(lib().emoe_vmm_slots_info(self._h, r, None, None, None, t.ctypes.data_as(_i32p), cap.value,
+                                             None, None))
+            out.append([int(x) for x in t[:cap.value]])
+        return out
+
+    def base(self, rank: int) -> int:
+        b = _vp()
+        _check(lib().emoe_vmm_slots_info(self._h, rank, ctypes.byref(b), None, None, None, 0, None, None))
+        return b.value or 0
+
+    def write_slot(self, rank: int, slot: int, host, stream=None) -> None:
+        _check(lib().emoe_vmm_slots_write(self._h, rank, slot, _ptr_array([host])[0], _stream_handle(stream)))
+
+    def read_slot(self, rank: int, slot: int, host, stream=None) -> None:
+        _check(lib().emoe_vmm_slots_read(self._h, rank, slot, _ptr_array([host])[0], _stream_handle(stream)))
+
+    def reshard(self, want, cap_new, stream=None) -> dict:
+        off, ids = _csr_i32(want)
+        cap = _i32arr(cap_new)
+        p = lambda a: a.ctypes.data_as(_i32p)
+        st = _VmmStats()
+        _check(lib().emoe_vmm_slots_reshard(self._h, len(want), p(cap), p(off), p(ids), _stream_handle(stream),
+                                            ctypes.byref(st)))
+        return {n: getattr(st, n) for n, _ in _VmmStats._fields_}
+

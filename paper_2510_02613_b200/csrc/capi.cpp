@@ -860,7 +860,7 @@ emoe_status_t emoe_plan_create_inplace(const emoe_shape_t *shape, int32_t ep_old
   emoe_status_t st;
   try {
     st = build_inplace_expert_plan(*shape, ep_old, slot_off_old, slot_ids_old, ep_new, cap_new, want_off,
-                                   want_ids, &p->hp.phase[EMOE_PHASE_EXPERTS], &p->slot_new);
+                                   want_ids, 0, &p->hp.phase[EMOE_PHASE_EXPERTS], &p->slot_new);
     if (st == EMOE_OK) {
       p->inplace = true;
       p->hp.shape = *shape;

@@ -531,7 +531,7 @@ emoe_status_t build_paged_expert_plan(const emoe_shape_t &sh, const emoe_config_
 
 emoe_status_t build_inplace_expert_plan(const emoe_shape_t &sh, int ep_old, const int32_t *off_old,
                                         const int32_t *ids_old, int ep_new, const int32_t *cap_new,
-                                        const int32_t *want_off, const int32_t *want_ids,
+                                        const int32_t *want_off, const int32_t *want_ids, uint64_t slab,
                                         PhasePlan *pp, std::vector<std::vector<int32_t>> *slot_new) {
   if (sh.n_layers <= 0 || sh.n_routed <= 0 || sh.n_shared < 0 || sh.d_model <= 0 || sh.d_ff <= 0 ||
       sh.elem_bytes <= 0)
@@ -555,11 +555,13 @@ emoe_status_t build_inplace_expert_plan(const emoe_shape_t &sh, int ep_old, cons
     }
   }
   const uint64_t m = (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes;
+  if (slab == 0) slab = m;
+  if (slab < m) return EMOE_ERR_INVALID_ARG;
   const uint32_t runs = (uint32_t)sh.n_layers * 3;
   std::vector<uint64_t> slots_old, slots_new;
   for (int r = 0; r < ep_old; ++r) {
     slots_old.push_back((uint64_t)(off_old[r + 1] - off_old[r]));
-    pp->arena_old.push_back(runs * slots_old.back() * m);
+    pp->arena_old.push_back(runs * slots_old.back() * slab);
   }
   slot_new->assign(ep_new, {});
   std::vector<ExpertMove> moves;
@@ -569,7 +571,7 @@ emoe_status_t build_inplace_expert_plan(const emoe_shape_t &sh, int ep_old, cons
     const bool stays = r < ep_old;
     if (stays && (uint64_t)cap_new[r] != slots_old[r]) return EMOE_ERR_INVALID_ARG;  // same arena
     slots_new.push_back((uint64_t)cap_new[r]);
-    pp->arena_new.push_back(runs * slots_new.back() * m);
+    pp->arena_new.push_back(runs * slots_new.back() * slab);
     std::vector<int32_t> &mine = (*slot_new)[r];
     mine.assign(cap_new[r], -1);
     std::vector<char> free_before(cap_new[r], 1), wanted(n_experts, 0);
@@ -599,7 +601,7 @@ emoe_status_t build_inplace_expert_plan(const emoe_shape_t &sh, int ep_old, cons
       ++next_free;
     }
   }
-  emit_expert_moves(sh, slots_old, slots_new, m, m, nullptr, nullptr, moves, fan, false, pp);
+  emit_expert_moves(sh, slots_old, slots_new, slab, m, nullptr, nullptr, moves, fan, false, pp);
   return EMOE_OK;
 }
 

@@ -94,10 +94,11 @@ emoe_status_t build_paged_expert_plan(const emoe_shape_t &shape, const emoe_conf
 // In-place expert step on capacity-strided arenas [L][3][cap_r][m] (see
 // emoe_plan_create_inplace): segments for arrivals only, and the slot tables after the step.
 // arena_old / arena_new of *pp are sized by the capacities; rank r of both sides is the same
-// arena when r exists on both.
+// arena when r exists on both.  slab: distance between consecutive slots (0: one matrix; the
+// paged store pads every matrix to its allocation granularity).
 emoe_status_t build_inplace_expert_plan(const emoe_shape_t &shape, int ep_old, const int32_t *off_old,
                                         const int32_t *ids_old, int ep_new, const int32_t *cap_new,
-                                        const int32_t *want_off, const int32_t *want_ids,
+                                        const int32_t *want_off, const int32_t *want_ids, uint64_t slab,
                                         PhasePlan *pp, std::vector<std::vector<int32_t>> *slot_new);
 
 // Expands a phase into flat emoe_segment_t records (one per destination).  For a

@@ -12,6 +12,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <chrono>
 #include <cstring>
 #include <map>
@@ -410,3 +411,331 @@ emoe_status_t emoe_vmm_reshard(emoe_vmm_pool_t *pool, const emoe_config_t *new_c
 }
 
 }  // extern "C"
+
+// ---- paged store with slot tables: a step touches only the slots that change ------------
+//
+// The store above rebuilds every range at every step.  This one keeps a device's range for
+// as long as the device exists: the range is RESERVED for `cap` slots per (layer,
+// projection), [L][3][cap][slab], and only occupied slots have pages behind them.  A step
+// follows the in-place expert step (emoe_plan_create_inplace): kept experts are not
+// touched at all, an arrival gets pages mapped into a slot that was free before the step
+// and is filled by the copy kernels, a leaving expert's pages are unmapped AFTER the copies
+// and go back to a list of spare pages, from which later arrivals are served - so that, in
+// the steady state, a step neither creates nor releases physical memory and its driver work
+// is proportional to the slots that change.
+
+namespace {
+
+struct SlotRange {
+  CUdeviceptr base = 0;
+  uint64_t bytes = 0;
+  uint32_t cap = 0;
+  std::vector<int32_t> ids;                          // expert per slot, -1 free
+  std::vector<CUmemGenericAllocationHandle> slabs;   // index run * cap + slot; 0 = nothing mapped
+};
+
+}  // namespace
+
+struct emoe_vmm_slots {
+  emoe_shape_t shape{};
+  int device = 0;
+  uint64_t m = 0, slab = 0;
+  uint32_t runs = 0;
+  std::vector<SlotRange> ranges;
+  std::vector<CUmemGenericAllocationHandle> spare;   // physical slabs that no slot maps
+  CUmemAllocationProp prop{};
+  CUmemAccessDesc access{};
+};
+
+namespace {
+
+CUdeviceptr slot_addr(const emoe_vmm_slots *pool, const SlotRange &rg, uint32_t run, uint32_t slot) {
+  return rg.base + ((uint64_t)run * rg.cap + slot) * pool->slab;
+}
+
+emoe_status_t take_slab(emoe_vmm_slots *pool, CUmemGenericAllocationHandle *h, double *alloc_ms) {
+  if (!pool->spare.empty()) {
+    *h = pool->spare.back();
+    pool->spare.pop_back();
+    return EMOE_OK;
+  }
+  const double t = now_ms();
+  const CUresult r = driver().MemCreate(h, pool->slab, &pool->prop, 0);
+  if (alloc_ms) *alloc_ms += now_ms() - t;
+  if (r == CUDA_ERROR_OUT_OF_MEMORY) return EMOE_ERR_OOM;
+  return r == CUDA_SUCCESS ? EMOE_OK : EMOE_ERR_CUDA;
+}
+
+// Pages behind every (layer, projection) of one slot.  On failure what was mapped stays
+// recorded in rg.slabs, so that unmap_slot / the destructor undo it.
+emoe_status_t map_slot(emoe_vmm_slots *pool, SlotRange *rg, uint32_t slot, double *alloc_ms, double *access_ms) {
+  for (uint32_t run = 0; run < pool->runs; ++run) {
+    CUmemGenericAllocationHandle h = 0;
+    emoe_status_t st = take_slab(pool, &h, alloc_ms);
+    if (st != EMOE_OK) return st;
+    const CUdeviceptr at = slot_addr(pool, *rg, run, slot);
+    if (driver().MemMap(at, pool->slab, 0, h, 0) != CUDA_SUCCESS) {
+      pool->spare.push_back(h);
+      return EMOE_ERR_CUDA;
+    }
+    rg->slabs[(size_t)run * rg->cap + slot] = h;
+    const double t = now_ms();
+    const CUresult r = driver().MemSetAccess(at, pool->slab, &pool->access, 1);
+    if (access_ms) *access_ms += now_ms() - t;
+    if (r != CUDA_SUCCESS) return EMOE_ERR_CUDA;
+  }
+  return EMOE_OK;
+}
+
+void unmap_slot(emoe_vmm_slots *pool, SlotRange *rg, uint32_t slot) {
+  for (uint32_t run = 0; run < pool->runs; ++run) {
+    CUmemGenericAllocationHandle &h = rg->slabs[(size_t)run * rg->cap + slot];
+    if (!h) continue;
+    driver().MemUnmap(slot_addr(pool, *rg, run, slot), pool->slab);
+    pool->spare.push_back(h);
+    h = 0;
+  }
+}
+
+emoe_status_t reserve_slots(emoe_vmm_slots *pool, uint32_t cap, SlotRange *rg) {
+  rg->cap = cap;
+  rg->bytes = (uint64_t)pool->runs * cap * pool->slab;
+  rg->ids.assign(cap, -1);
+  rg->slabs.assign((size_t)pool->runs * cap, 0);
+  rg->base = 0;
+  if (!rg->bytes) return EMOE_OK;
+  const CUresult r = driver().MemAddressReserve(&rg->base, rg->bytes, 0, 0, 0);
+  if (r != CUDA_SUCCESS) {
+    rg->base = 0;
+    return r == CUDA_ERROR_OUT_OF_MEMORY ? EMOE_ERR_OOM : EMOE_ERR_CUDA;
+  }
+  return EMOE_OK;
+}
+
+void drop_range(emoe_vmm_slots *pool, SlotRange *rg) {
+  if (!rg->base) return;
+  for (uint32_t s = 0; s < rg->cap; ++s) unmap_slot(pool, rg, s);
+  driver().MemAddressFree(rg->base, rg->bytes);
+  rg->base = 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+emoe_status_t emoe_vmm_slots_create(const emoe_shape_t *shape, int32_t ep, const int32_t *slot_off,
+                                    const int32_t *slot_ids, int32_t spare_slots,
+                                    emoe_vmm_slots_t **out) {
+  if (!shape || !slot_off || !slot_ids || !out || ep < 1 || spare_slots < 0) return EMOE_ERR_INVALID_ARG;
+  if (ep > EMOE_MAX_RANKS) return EMOE_ERR_UNSUPPORTED;
+  try {  // validation of shape and tables: plan the step that changes nothing
+    PhasePlan pp;
+    std::vector<std::vector<int32_t>> tables;
+    std::vector<int32_t> cap(ep), want_off(ep + 1, 0), want;
+    for (int r = 0; r < ep; ++r) {
+      if (slot_off[r + 1] < slot_off[r]) return EMOE_ERR_PLACEMENT;
+      cap[r] = slot_off[r + 1] - slot_off[r];
+      for (int i = slot_off[r]; i < slot_off[r + 1]; ++i)
+        if (slot_ids[i] >= 0) want.push_back(slot_ids[i]);
+      want_off[r + 1] = (int32_t)want.size();
+    }
+    if (want.empty()) want.push_back(0);
+    const emoe_status_t st = build_inplace_expert_plan(*shape, ep, slot_off, slot_ids, ep, cap.data(),
+                                                       want_off.data(), want.data(), 0, &pp, &tables);
+    if (st != EMOE_OK) return st;
+  } catch (const std::bad_alloc &) {
+    return EMOE_ERR_OOM;
+  }
+  if (cudaFree(nullptr) != cudaSuccess) { (void)cudaGetLastError(); return EMOE_ERR_CUDA; }
+  if (!driver().ok) return EMOE_ERR_UNSUPPORTED;
+  emoe_vmm_slots *pool = new (std::nothrow) emoe_vmm_slots();
+  if (!pool) return EMOE_ERR_OOM;
+  emoe_status_t st = EMOE_OK;
+  try {
+    pool->shape = *shape;
+    if (cudaGetDevice(&pool->device) != cudaSuccess) { delete pool; return EMOE_ERR_CUDA; }
+    pool->prop.type = CU_MEM_ALLOCATION_TYPE_PINNED;
+    pool->prop.location.type = CU_MEM_LOCATION_TYPE_DEVICE;
+    pool->prop.location.id = pool->device;
+    pool->access.location = pool->prop.location;
+    pool->access.flags = CU_MEM_ACCESS_FLAGS_PROT_READWRITE;
+    size_t gran = 0;
+    if (driver().MemGetAllocationGranularity(&gran, &pool->prop, CU_MEM_ALLOC_GRANULARITY_MINIMUM) !=
+            CUDA_SUCCESS || gran == 0) {
+      delete pool;
+      return EMOE_ERR_UNSUPPORTED;
+    }
+    pool->m = (uint64_t)shape->d_model * shape->d_ff * shape->elem_bytes;
+    pool->slab = (pool->m + gran - 1) / gran * gran;
+    pool->runs = 3u * (uint32_t)shape->n_layers;
+    pool->ranges.resize(ep);
+    for (int r = 0; st == EMOE_OK && r < ep; ++r) {
+      SlotRange &rg = pool->ranges[r];
+      st = reserve_slots(pool, (uint32_t)(slot_off[r + 1] - slot_off[r]), &rg);
+      for (uint32_t s = 0; st == EMOE_OK && s < rg.cap; ++s) {
+        rg.ids[s] = slot_ids[slot_off[r] + s];
+        if (rg.ids[s] >= 0) st = map_slot(pool, &rg, s, nullptr, nullptr);
+      }
+    }
+    // spare pages for the arrivals of later steps: created now, outside any step
+    for (int64_t i = 0; st == EMOE_OK && i < (int64_t)spare_slots * pool->runs; ++i) {
+      CUmemGenericAllocationHandle h = 0;
+      const CUresult r = driver().MemCreate(&h, pool->slab, &pool->prop, 0);
+      if (r != CUDA_SUCCESS) { st = r == CUDA_ERROR_OUT_OF_MEMORY ? EMOE_ERR_OOM : EMOE_ERR_CUDA; break; }
+      pool->spare.push_back(h);
+    }
+  } catch (const std::bad_alloc &) {
+    st = EMOE_ERR_OOM;
+  }
+  if (st != EMOE_OK) {
+    emoe_vmm_slots_destroy(pool);
+    return st;
+  }
+  *out = pool;
+  return EMOE_OK;
+}
+
+void emoe_vmm_slots_destroy(emoe_vmm_slots_t *pool) {
+  if (!pool) return;
+  (void)cudaDeviceSynchronize();
+  for (SlotRange &rg : pool->ranges) drop_range(pool, &rg);
+  for (CUmemGenericAllocationHandle h : pool->spare) driver().MemRelease(h);
+  delete pool;
+}
+
+emoe_status_t emoe_vmm_slots_info(const emoe_vmm_slots_t *pool, int32_t rank, void **base,
+                                  uint64_t *slab_bytes, int32_t *cap, int32_t *ids_out, int32_t ids_cap,
+                                  int32_t *n_ranks, int64_t *spare_slabs) {
+  if (!pool) return EMOE_ERR_INVALID_ARG;
+  if (n_ranks) *n_ranks = (int32_t)pool->ranges.size();
+  if (spare_slabs) *spare_slabs = (int64_t)pool->spare.size();
+  if (slab_bytes) *slab_bytes = pool->slab;
+  if (rank < 0) return EMOE_OK;                       // pool-wide figures only
+  if (rank >= (int)pool->ranges.size() || (ids_cap > 0 && !ids_out)) return EMOE_ERR_INVALID_ARG;
+  const SlotRange &rg = pool->ranges[rank];
+  if (base) *base = reinterpret_cast<void *>(rg.base);
+  if (cap) *cap = (int32_t)rg.cap;
+  for (int32_t i = 0; i < ids_cap && i < (int32_t)rg.cap; ++i) ids_out[i] = rg.ids[i];
+  return EMOE_OK;
+}
+
+// One slot as a dense host image [L][3][m] <-> its pages.
+emoe_status_t emoe_vmm_slots_write(emoe_vmm_slots_t *pool, int32_t rank, int32_t slot, const void *host,
+                                   void *stream) {
+  if (!pool || rank < 0 || rank >= (int)pool->ranges.size() || !host) return EMOE_ERR_INVALID_ARG;
+  const SlotRange &rg = pool->ranges[rank];
+  if (slot < 0 || slot >= (int)rg.cap || rg.ids[slot] < 0) return EMOE_ERR_INVALID_ARG;
+  const cudaError_t e = cudaMemcpy2DAsync(reinterpret_cast<void *>(slot_addr(pool, rg, 0, (uint32_t)slot)),
+                                          (size_t)rg.cap * pool->slab, host, pool->m, pool->m, pool->runs,
+                                          cudaMemcpyHostToDevice, (cudaStream_t)stream);
+  if (e != cudaSuccess) { (void)cudaGetLastError(); return EMOE_ERR_CUDA; }
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_vmm_slots_read(const emoe_vmm_slots_t *pool, int32_t rank, int32_t slot, void *host,
+                                  void *stream) {
+  if (!pool || rank < 0 || rank >= (int)pool->ranges.size() || !host) return EMOE_ERR_INVALID_ARG;
+  const SlotRange &rg = pool->ranges[rank];
+  if (slot < 0 || slot >= (int)rg.cap || rg.ids[slot] < 0) return EMOE_ERR_INVALID_ARG;
+  const cudaError_t e = cudaMemcpy2DAsync(host, pool->m,
+                                          reinterpret_cast<const void *>(slot_addr(pool, rg, 0, (uint32_t)slot)),
+                                          (size_t)rg.cap * pool->slab, pool->m, pool->runs,
+                                          cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  if (e != cudaSuccess) { (void)cudaGetLastError(); return EMOE_ERR_CUDA; }
+  return EMOE_OK;
+}
+
+emoe_status_t emoe_vmm_slots_reshard(emoe_vmm_slots_t *pool, int32_t ep_new, const int32_t *cap_new,
+                                     const int32_t *want_off, const int32_t *want_ids, void *stream,
+                                     emoe_vmm_stats_t *stats) {
+  if (!pool || !cap_new || !want_off || !want_ids) return EMOE_ERR_INVALID_ARG;
+  if (ep_new < 1 || ep_new > EMOE_MAX_RANKS) return EMOE_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  emoe_vmm_stats_t s{};
+  const double t0 = now_ms();
+  emoe_status_t rc = EMOE_OK;
+  const int ep_old = (int)pool->ranges.size();
+  try {
+    std::vector<int32_t> off(ep_old + 1, 0), ids;
+    for (int r = 0; r < ep_old; ++r) {
+      off[r + 1] = off[r] + (int32_t)pool->ranges[r].cap;
+      ids.insert(ids.end(), pool->ranges[r].ids.begin(), pool->ranges[r].ids.end());
+    }
+    if (ids.empty()) ids.push_back(-1);
+    PhasePlan pp;
+    std::vector<std::vector<int32_t>> slot_new;
+    rc = build_inplace_expert_plan(pool->shape, ep_old, off.data(), ids.data(), ep_new, cap_new, want_off,
+                                   want_ids, pool->slab, &pp, &slot_new);
+    if (rc != EMOE_OK) return rc;            // nothing has been touched yet
+
+    // 1. ranges of added devices, pages behind every arrival's slot
+    const size_t n_dev = (size_t)std::max(ep_old, (int)ep_new);
+    if (pool->ranges.size() < n_dev) pool->ranges.resize(n_dev);
+    std::vector<std::pair<int, uint32_t>> arrived;    // (rank, slot) mapped by this step
+    for (int r = 0; rc == EMOE_OK && r < ep_new; ++r) {
+      SlotRange &rg = pool->ranges[r];
+      if (r >= ep_old) rc = reserve_slots(pool, (uint32_t)cap_new[r], &rg);
+      for (uint32_t sl = 0; rc == EMOE_OK && sl < rg.cap; ++sl) {
+        const int32_t e = slot_new[r][sl];
+        if (e < 0 || (r < ep_old && rg.ids[sl] == e)) continue;   // free, or kept: not touched
+        arrived.push_back({r, sl});
+        rc = map_slot(pool, &rg, sl, &s.alloc_ms, &s.access_ms);
+        s.slabs_copied += pool->runs;
+      }
+    }
+    const double t1 = now_ms();
+    s.map_ms = t1 - t0;
+
+    // 2. the copy kernels fill the arrivals from their sources (ranges as they are now)
+    if (rc == EMOE_OK && !pp.segs.empty()) {
+      RankPtrs ptrs;
+      std::memset(&ptrs, 0, sizeof(ptrs));
+      for (int r = 0; r < ep_old; ++r) ptrs.src[r] = reinterpret_cast<const uint8_t *>(pool->ranges[r].base);
+      for (int r = 0; r < ep_new; ++r) ptrs.dst[r] = reinterpret_cast<uint8_t *>(pool->ranges[r].base);
+      rc = run_phase_once(pp, ptrs, st);
+      s.bytes_copied = pp.bytes_moved;
+      s.bytes_read = pp.bytes_read;
+    } else if (rc == EMOE_OK) {
+      if (cudaStreamSynchronize(st) != cudaSuccess) { (void)cudaGetLastError(); rc = EMOE_ERR_CUDA; }
+    }
+    const double t2 = now_ms();
+    s.copy_ms = t2 - t1;
+    if (rc != EMOE_OK) {   // undo: the pool is as it was before the call
+      for (auto &a : arrived) unmap_slot(pool, &pool->ranges[a.first], a.second);
+      for (size_t r = ep_old; r < pool->ranges.size(); ++r) drop_range(pool, &pool->ranges[r]);
+      pool->ranges.resize(ep_old);
+      return rc;
+    }
+
+    // 3. experts that left: their pages go back to the spare list; removed devices go whole
+    for (int r = 0; r < ep_old; ++r) {
+      SlotRange &rg = pool->ranges[r];
+      if (r >= ep_new) { drop_range(pool, &rg); continue; }
+      for (uint32_t sl = 0; sl < rg.cap; ++sl)
+        if (rg.ids[sl] >= 0 && slot_new[r][sl] != rg.ids[sl]) unmap_slot(pool, &rg, sl);
+    }
+    pool->ranges.resize(ep_new);
+    uint64_t kept = 0;
+    for (int r = 0; r < ep_new; ++r) {
+      for (uint32_t sl = 0; sl < pool->ranges[r].cap; ++sl)
+        if (slot_new[r][sl] >= 0 && r < ep_old && pool->ranges[r].ids[sl] == slot_new[r][sl]) ++kept;
+      pool->ranges[r].ids = slot_new[r];
+    }
+    s.slabs_remapped = kept * pool->runs;      // kept in place: no driver call at all
+    s.unmap_ms = now_ms() - t2;
+  } catch (const std::bad_alloc &) {
+    return EMOE_ERR_OOM;
+  }
+  s.total_ms = now_ms() - t0;
+  s.slab_bytes = pool->slab;
+  s.matrix_bytes = pool->m;
+  uint64_t mapped = 0;
+  for (const SlotRange &rg : pool->ranges)
+    for (CUmemGenericAllocationHandle h : rg.slabs) mapped += h != 0;
+  s.physical_bytes = (mapped + pool->spare.size()) * pool->slab;
+  if (stats) *stats = s;
+  return EMOE_OK;
+}
+
+}  // extern "C"
+

@@ -41,6 +41,56 @@ class PeerArenas:
                 self.ptrs.append(opened[handle] + offset)
 
 
+class Exchange:
+    """A prepared exchange: the plan restricted to this rank, the peers' old arenas mapped.
+    Set-up and tear-down talk to the other processes (all of them must create and close
+    their Exchange together); step() only enqueues this rank's kernels."""
+
+    def __init__(self, dist, plan: "B.Plan", rank: int, old_arenas, new_arenas):
+        self.dist, self.plan, self.rank = dist, plan, rank
+        self.opened: dict = {}
+        self.calls = []
+        plan.set_local_rank(rank)
+        run = (plan.reshard_experts, plan.reshard_attn, plan.reshard_kv)
+        try:
+            for phase in range(3):
+                n_old = plan.num_ranks(phase, B.SIDE_OLD)
+                n_new = plan.num_ranks(phase, B.SIDE_NEW)
+                pa = PeerArenas(dist, rank, n_old, old_arenas[phase], self.opened)
+                if rank >= n_new or new_arenas[phase] is None:
+                    continue                         # nothing of this phase lands here
+                dst = [new_arenas[phase] if r == rank else None for r in range(n_new)]
+                self.calls.append((run[phase], pa.ptrs, dst))
+        except Exception:
+            self.close(barrier=False)
+            raise
+
+    def step(self, stream=None) -> None:
+        """Enqueues this rank's share of the three phases on `stream`; no synchronisation."""
+        for fn, src, dst in self.calls:
+            fn(src, dst, stream)
+
+    def bytes_pulled(self) -> dict:
+        """Bytes this rank writes, and how many of them it reads from OTHER ranks' arenas."""
+        total = remote = 0
+        for phase in range(3):
+            segs = self.plan.segments(phase)
+            mine = segs[segs["dst_rank"] == self.rank]
+            b = mine["run_bytes"].astype("int64") * mine["n_runs"].astype("int64")
+            total += int(b.sum())
+            remote += int(b[mine["src_rank"] != self.rank].sum())
+        return dict(written=total, from_peers=remote)
+
+    def close(self, barrier: bool = True) -> None:
+        if barrier:
+            self.dist.barrier()                      # nobody still reads a peer's old arena
+        for base in self.opened.values():
+            B.ipc_close(base)
+        self.opened = {}
+        self.calls = []
+        self.plan.set_local_rank(-1)
+
+
 def exchange_step(dist, plan: "B.Plan", rank: int, old_arenas, new_arenas, stream=None) -> None:
     """Runs this rank's share of the three phases.
 
@@ -51,22 +101,10 @@ def exchange_step(dist, plan: "B.Plan", rank: int, old_arenas, new_arenas, strea
     """
     import torch
 
-    plan.set_local_rank(rank)
-    run = (plan.reshard_experts, plan.reshard_attn, plan.reshard_kv)
     dist.barrier()                                   # every old arena is complete
-    opened: dict = {}
+    ex = Exchange(dist, plan, rank, old_arenas, new_arenas)
     try:
-        for phase in range(3):
-            n_old = plan.num_ranks(phase, B.SIDE_OLD)
-            n_new = plan.num_ranks(phase, B.SIDE_NEW)
-            pa = PeerArenas(dist, rank, n_old, old_arenas[phase], opened)
-            if rank >= n_new or new_arenas[phase] is None:
-                continue                             # nothing of this phase lands here
-            dst = [new_arenas[phase] if r == rank else None for r in range(n_new)]
-            run[phase](pa.ptrs, dst, stream)
+        ex.step(stream)
         (stream.synchronize() if stream is not None else torch.cuda.synchronize())
-        dist.barrier()                               # nobody still reads a peer's old arena
     finally:
-        for base in opened.values():
-            B.ipc_close(base)
-        plan.set_local_rank(-1)
+        ex.close()

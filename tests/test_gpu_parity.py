@@ -540,6 +540,59 @@ def test_kv_delta_plan_recopies_blocks_written_during_the_migration():
         assert moved * 8 < p_all.stats(E.PHASE_KV)["bytes_moved"]      # the delta is small
 
 
+def test_kv_migration_while_a_second_stream_appends_tokens():
+    """Scale while serving, for real this time: the whole-cache migration runs on one stream
+    WHILE a second stream keeps appending tokens to the last block of every sequence (the
+    writes race with the copy of those blocks, so their destination bytes are undefined for
+    the moment); afterwards a delta plan that lists just the blocks written re-copies them.
+    The final cache must equal the oracle run on the final source in one go, and the two
+    streams must really have overlapped in time."""
+    from gpu_util import oracle_phase
+    wl = W.make_workload("c4_large", n_layers=8)
+    B, L = wl.shape.kv_block_tokens, wl.shape.n_layers
+    hl = wl.shape.n_kv_heads // wl.old.tp
+    blk = B * hl * wl.shape.head_dim * wl.shape.elem_bytes
+    nblk = [-(-n // B) for n in wl.old.seq_lens]
+    last_old = np.array([[wl.old.block_table[s_, k - 1]] for s_, k in enumerate(nblk)], np.int32)
+    last_new = np.array([[wl.new.block_table[s_, k - 1]] for s_, k in enumerate(nblk)], np.int32)
+    delta = R(wl, old=R(wl.old, seq_lens=[B] * len(nblk), block_table=last_old),
+              new=R(wl.new, seq_lens=[B] * len(nblk), block_table=last_new))
+    idx = torch.from_numpy(last_old[:, 0].astype(np.int64)).cuda()
+    s_copy, s_serve = torch.cuda.Stream(), torch.cuda.Stream()
+    with E.Plan(wl.shape, wl.old, wl.new) as p_all, E.Plan(delta.shape, delta.old, delta.new) as p_delta:
+        src = WD.alloc_filled(p_all.arena_bytes(E.PHASE_KV, E.SIDE_OLD), wl.seed, W.KIND_KV)
+        dst = WD.alloc_const(p_all.arena_bytes(E.PHASE_KV, E.SIDE_NEW))
+        pools = [t.view(L * 2, wl.old.kv_num_blocks, blk) for t in src]
+        torch.cuda.synchronize()
+        overlapped = False
+        for attempt in range(4):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            ev[0].record(s_copy)
+            for _ in range(4):                    # the migration, a few times over to make it last
+                p_all.reshard_kv(src, dst, s_copy)
+            ev[1].record(s_copy)
+            with torch.cuda.stream(s_serve):
+                ev[2].record(s_serve)
+                for step in range(40):            # "decode steps": one more token per sequence each
+                    for pool in pools:
+                        pool[:, idx, (step % B) * hl * 8:(step % B) * hl * 8 + 8] += 1
+                ev[3].record(s_serve)
+            torch.cuda.synchronize()
+            # serving started before the migration ended and the migration started before serving ended
+            overlapped = ev[2].elapsed_time(ev[1]) > 0 and ev[0].elapsed_time(ev[3]) > 0
+            if overlapped:
+                break
+        assert overlapped, "the appending stream never ran beside the migration"
+        p_delta.reshard_kv(src, dst, s_copy)      # close the gap: only the blocks written since
+        s_copy.synchronize()
+        want = [np.full(t.numel(), WD.FILL_BYTE, np.uint8) for t in dst]
+        oracle_phase(wl, E.PHASE_KV, [t.cpu().numpy() for t in src], want)
+        for r, (g, w) in enumerate(zip(dst, want)):
+            assert np.array_equal(g.cpu().numpy(), w), "rank %d" % r
+        assert p_delta.stats(E.PHASE_KV)["bytes_moved"] * 20 < p_all.stats(E.PHASE_KV)["bytes_moved"]
+        assert p_all.device_status() == 0 and p_delta.device_status() == 0
+
+
 def test_fp8_weights_with_block_scales_in_one_plan():
     """FP8 expert weights (elem_bytes = 1) and their per-128x128-block fp32 scale tensors
     ([d_ff/128][d_model/128] floats per matrix) move with the same placement through ONE plan

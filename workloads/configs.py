@@ -252,6 +252,26 @@ def make_workload(name: str, n_layers: Optional[int] = None, new_order: str = "r
     return wl
 
 
+def make_exchange_workload(n_devices: int, n_layers: Optional[int] = None) -> Workload:
+    """A scale step whose ranks map onto n_devices GPUs, one rank index per GPU: the
+    fine-grained shape (64 routed + 2 shared experts), expert parallelism grown by two devices
+    as in the paper's step pattern (n_devices - 2 -> n_devices; 1 -> 2 for two devices),
+    tensor parallelism doubled (n_devices / 2 -> n_devices, capped by the 16 heads), so
+    experts, attention slices and KV heads all cross devices."""
+    if n_devices < 2 or n_devices > 16 or n_devices & (n_devices - 1):
+        raise ValueError("exchange workloads are defined for 2, 4, 8 or 16 devices")
+    seed = MASTER_SEED + 6
+    sh = Shape(27, 64, 2, 2048, 1408, 16, 16, 128)
+    sl, nbo, bto, nbn, btn = _kv_configs(seed, 65536 // 16, 16, None)
+    ep_old = n_devices - 2 if n_devices >= 4 else 1
+    old = ParallelConfig(ep_old, n_devices // 2, with_shared(place_contiguous(64, ep_old), [64, 65]), nbo, sl, bto)
+    new = ParallelConfig(n_devices, n_devices, with_shared(place_contiguous(64, n_devices), [64, 65]), nbn, sl, btn)
+    wl = Workload("exchange_%d" % n_devices, sh, old, new, seed,
+                  "EP%d,TP%d -> EP%d,TP%d, one rank per GPU, pulled over the GPU interconnect"
+                  % (ep_old, n_devices // 2, n_devices, n_devices))
+    return wl.with_layers(n_layers) if n_layers is not None else wl
+
+
 def small_variant(name: str) -> Workload:
     """A few-layer cut of a workload with the same per-layer structure, sized so
     that a CPU implementation finishes in seconds."""
