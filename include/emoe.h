@@ -556,7 +556,11 @@ emoe_status_t emoe_plan_clear_device_status(emoe_plan_t *plan);
 /* Launch tuning.  Fields set to 0 keep the library default. */
 typedef struct {
   int32_t max_ctas;        /* upper bound on CTAs per launch (SM budget when the    */
-                           /* reshard shares the GPU with a live kernel)            */
+                           /* reshard shares the GPU with a live kernel).  The ring */
+                           /* kernel keeps one CTA per SM for the whole launch and  */
+                           /* a live kernel loses those SMs: 16 keeps a concurrent  */
+                           /* GEMM within 1.5x on B200; more than the default (74)  */
+                           /* and fewer than all SMs only hurts both sides          */
   int32_t bulk_tile_bytes; /* bytes per shared-memory stage of the bulk kernel      */
   int32_t bulk_stages;     /* stages of the bulk kernel's ring                      */
   int32_t path;            /* 0 default routing, 1 force the vector kernel for all  */

@@ -479,12 +479,30 @@ emoe_status_t map_slot(emoe_vmm_slots *pool, SlotRange *rg, uint32_t slot, doubl
       return EMOE_ERR_CUDA;
     }
     rg->slabs[(size_t)run * rg->cap + slot] = h;
-    const double t = now_ms();
-    const CUresult r = driver().MemSetAccess(at, pool->slab, &pool->access, 1);
-    if (access_ms) *access_ms += now_ms() - t;
-    if (r != CUDA_SUCCESS) return EMOE_ERR_CUDA;
   }
+  (void)access_ms;
   return EMOE_OK;
+}
+
+// Enables access to freshly mapped slots: one driver call per (layer, projection) and per run
+// of neighbouring slots, since neighbouring slots are neighbours in the address range.
+emoe_status_t enable_slots(emoe_vmm_slots *pool, const SlotRange &rg, const std::vector<uint32_t> &slots,
+                           double *access_ms) {
+  const double t = now_ms();
+  emoe_status_t st = EMOE_OK;
+  for (uint32_t run = 0; st == EMOE_OK && run < pool->runs; ++run) {
+    size_t i = 0;
+    while (st == EMOE_OK && i < slots.size()) {
+      size_t j = i + 1;
+      while (j < slots.size() && slots[j] == slots[j - 1] + 1) ++j;
+      if (driver().MemSetAccess(slot_addr(pool, rg, run, slots[i]), (j - i) * pool->slab, &pool->access, 1) !=
+          CUDA_SUCCESS)
+        st = EMOE_ERR_CUDA;
+      i = j;
+    }
+  }
+  if (access_ms) *access_ms += now_ms() - t;
+  return st;
 }
 
 void unmap_slot(emoe_vmm_slots *pool, SlotRange *rg, uint32_t slot) {
@@ -572,10 +590,15 @@ emoe_status_t emoe_vmm_slots_create(const emoe_shape_t *shape, int32_t ep, const
     for (int r = 0; st == EMOE_OK && r < ep; ++r) {
       SlotRange &rg = pool->ranges[r];
       st = reserve_slots(pool, (uint32_t)(slot_off[r + 1] - slot_off[r]), &rg);
+      std::vector<uint32_t> mapped;
       for (uint32_t s = 0; st == EMOE_OK && s < rg.cap; ++s) {
         rg.ids[s] = slot_ids[slot_off[r] + s];
-        if (rg.ids[s] >= 0) st = map_slot(pool, &rg, s, nullptr, nullptr);
+        if (rg.ids[s] >= 0) {
+          st = map_slot(pool, &rg, s, nullptr, nullptr);
+          mapped.push_back(s);
+        }
       }
+      if (st == EMOE_OK) st = enable_slots(pool, rg, mapped, nullptr);
     }
     // spare pages for the arrivals of later steps: created now, outside any step
     for (int64_t i = 0; st == EMOE_OK && i < (int64_t)spare_slots * pool->runs; ++i) {
@@ -619,16 +642,21 @@ emoe_status_t emoe_vmm_slots_info(const emoe_vmm_slots_t *pool, int32_t rank, vo
   return EMOE_OK;
 }
 
-// One slot as a dense host image [L][3][m] <-> its pages.
+// One slot as a dense host image [L][3][m] <-> its pages.  One copy per (layer, projection):
+// the rows of a slot are a whole layer slab apart and what lies between them may be unmapped,
+// which a strided 2-D copy does not accept.
 emoe_status_t emoe_vmm_slots_write(emoe_vmm_slots_t *pool, int32_t rank, int32_t slot, const void *host,
                                    void *stream) {
   if (!pool || rank < 0 || rank >= (int)pool->ranges.size() || !host) return EMOE_ERR_INVALID_ARG;
   const SlotRange &rg = pool->ranges[rank];
   if (slot < 0 || slot >= (int)rg.cap || rg.ids[slot] < 0) return EMOE_ERR_INVALID_ARG;
-  const cudaError_t e = cudaMemcpy2DAsync(reinterpret_cast<void *>(slot_addr(pool, rg, 0, (uint32_t)slot)),
-                                          (size_t)rg.cap * pool->slab, host, pool->m, pool->m, pool->runs,
-                                          cudaMemcpyHostToDevice, (cudaStream_t)stream);
-  if (e != cudaSuccess) { (void)cudaGetLastError(); return EMOE_ERR_CUDA; }
+  for (uint32_t run = 0; run < pool->runs; ++run)
+    if (cudaMemcpyAsync(reinterpret_cast<void *>(slot_addr(pool, rg, run, (uint32_t)slot)),
+                        static_cast<const uint8_t *>(host) + (uint64_t)run * pool->m, pool->m,
+                        cudaMemcpyHostToDevice, (cudaStream_t)stream) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return EMOE_ERR_CUDA;
+    }
   return EMOE_OK;
 }
 
@@ -637,11 +665,13 @@ emoe_status_t emoe_vmm_slots_read(const emoe_vmm_slots_t *pool, int32_t rank, in
   if (!pool || rank < 0 || rank >= (int)pool->ranges.size() || !host) return EMOE_ERR_INVALID_ARG;
   const SlotRange &rg = pool->ranges[rank];
   if (slot < 0 || slot >= (int)rg.cap || rg.ids[slot] < 0) return EMOE_ERR_INVALID_ARG;
-  const cudaError_t e = cudaMemcpy2DAsync(host, pool->m,
-                                          reinterpret_cast<const void *>(slot_addr(pool, rg, 0, (uint32_t)slot)),
-                                          (size_t)rg.cap * pool->slab, pool->m, pool->runs,
-                                          cudaMemcpyDeviceToHost, (cudaStream_t)stream);
-  if (e != cudaSuccess) { (void)cudaGetLastError(); return EMOE_ERR_CUDA; }
+  for (uint32_t run = 0; run < pool->runs; ++run)
+    if (cudaMemcpyAsync(static_cast<uint8_t *>(host) + (uint64_t)run * pool->m,
+                        reinterpret_cast<const void *>(slot_addr(pool, rg, run, (uint32_t)slot)), pool->m,
+                        cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return EMOE_ERR_CUDA;
+    }
   return EMOE_OK;
 }
 
@@ -675,13 +705,16 @@ emoe_status_t emoe_vmm_slots_reshard(emoe_vmm_slots_t *pool, int32_t ep_new, con
     for (int r = 0; rc == EMOE_OK && r < ep_new; ++r) {
       SlotRange &rg = pool->ranges[r];
       if (r >= ep_old) rc = reserve_slots(pool, (uint32_t)cap_new[r], &rg);
+      std::vector<uint32_t> mine;
       for (uint32_t sl = 0; rc == EMOE_OK && sl < rg.cap; ++sl) {
         const int32_t e = slot_new[r][sl];
         if (e < 0 || (r < ep_old && rg.ids[sl] == e)) continue;   // free, or kept: not touched
         arrived.push_back({r, sl});
+        mine.push_back(sl);
         rc = map_slot(pool, &rg, sl, &s.alloc_ms, &s.access_ms);
         s.slabs_copied += pool->runs;
       }
+      if (rc == EMOE_OK) rc = enable_slots(pool, rg, mine, &s.access_ms);
     }
     const double t1 = now_ms();
     s.map_ms = t1 - t0;
