@@ -32,6 +32,42 @@ int main(void) {
   nc.tp = 3;                                                    /* 3 does not divide 4 heads */
   if (emoe_plan_create(&sh, &oc, &nc, EMOE_PLAN_HOST_ONLY, &plan) != EMOE_ERR_SHAPE) return 8;
   if (strcmp(emoe_strerror(EMOE_OK), "ok") != 0) return 9;
+  nc.tp = 2;
+  {
+    /* scale tensors in the same plan: weights, then (256-byte aligned) 8 bytes per matrix */
+    emoe_plan_options_t opt;
+    memset(&opt, 0, sizeof(opt));
+    opt.expert_scale_bytes = 8;
+    if (emoe_plan_create_ex(&sh, &oc, &nc, EMOE_PLAN_HOST_ONLY, &opt, &plan) != EMOE_OK) return 10;
+    if (emoe_plan_arena_bytes(plan, EMOE_PHASE_EXPERTS, EMOE_SIDE_NEW, 0, &bytes) != EMOE_OK) return 11;
+    if (bytes != 2ull * 3 * 1 * 64 * 32 * 2 + 2ull * 3 * 1 * 8) return 12;   /* 24576 is a multiple of 256 */
+    emoe_plan_destroy(plan);
+  }
+  {
+    /* in-place expert step: device 0 [0, 1, free], device 1 [2, 3, free] -> 0 wants {0, 2}, 1 wants {3, 1} */
+    int32_t slot_off[3] = {0, 3, 6}, slot_ids[6] = {0, 1, -1, 2, 3, -1};
+    int32_t cap[2] = {3, 3}, want_off[3] = {0, 2, 4}, want[4] = {0, 2, 3, 1}, table[3], n_slots = 0;
+    if (emoe_plan_create_inplace(&sh, 2, slot_off, slot_ids, 2, cap, want_off, want, EMOE_PLAN_HOST_ONLY,
+                                 &plan) != EMOE_OK) return 13;
+    if (emoe_plan_slot_table(plan, 0, table, 3, &n_slots) != EMOE_OK || n_slots != 3) return 14;
+    if (table[0] != 0 || table[1] != -1 || table[2] != 2) return 15;
+    if (emoe_plan_stats(plan, EMOE_PHASE_EXPERTS, &moved, &read, &nseg) != EMOE_OK) return 16;
+    if (moved != 2ull * 2 * 3 * 64 * 32 * 2) return 17;         /* two arrivals only */
+    emoe_plan_destroy(plan);
+  }
+  {
+    /* plan cache and the compacting block table */
+    emoe_plan_cache_t *cache = NULL;
+    int32_t hit = -1, bt[2] = {9, 9}, mapped = 0, in_use[1] = {0};
+    uint64_t hits = 0, misses = 0;
+    if (emoe_plan_cache_create(2, &cache) != EMOE_OK) return 18;
+    if (emoe_plan_cache_get(cache, &sh, &oc, &nc, EMOE_PLAN_HOST_ONLY, NULL, &plan, &hit) != EMOE_OK || hit) return 19;
+    if (emoe_plan_cache_get(cache, &sh, &oc, &nc, EMOE_PLAN_HOST_ONLY, NULL, &plan, &hit) != EMOE_OK || !hit) return 20;
+    if (emoe_plan_cache_stats(cache, &hits, &misses, NULL, NULL) != EMOE_OK || hits != 1 || misses != 1) return 21;
+    emoe_plan_cache_destroy(cache);
+    if (emoe_kv_compact_table(4, 1, 2, seq_lens, 3, in_use, 1, bt, &mapped) != EMOE_OK) return 22;
+    if (bt[0] != 1 || bt[1] != 2 || mapped != 2) return 23;
+  }
   printf("c abi ok\n");
   return 0;
 }
