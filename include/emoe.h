@@ -570,8 +570,9 @@ typedef struct {
                            /* row-mapped fast path                                  */
   int32_t bulk_hints;      /* 0 default, 1 none, 2 loads evict-first in L2, 3 stores */
                            /* evict-first, 4 both                                   */
-  int32_t kv_order;        /* order in which mapped KV blocks are visited: 0 default,   */
-                           /* 1 block-table order, 2 by old physical id, 3 by new id    */
+  int32_t kv_order;        /* order in which mapped KV blocks are visited: 0 default    */
+                           /* (= 2), 1 block-table order, 2 by old physical id (reads   */
+                           /* walk the old pool in address order), 3 by new id          */
   int32_t unit_order;      /* bulk work order: 0 default (run-major: one layer slab or  */
                            /* KV pool at a time), 1 segment-major; +2: CTAs take units  */
                            /* round-robin instead of claiming them from a counter       */

@@ -26,7 +26,7 @@ constexpr int kCtrSlots = 4;        // launches of one phase of one plan that ma
 constexpr int kTableSets = 4;        // experts, attn, kv, and the three merged for one whole step
 constexpr int kStatusWords = 1 + kTableSets * kCtrSlots * 2;
 constexpr int kDefaultKvMode = 1;   // 1 direct, 2 staged through shared memory
-constexpr int kDefaultKvOrder = 1;  // 1 table order, 2 by old block id, 3 by new block id
+constexpr int kDefaultKvOrder = 2;  // 1 table order, 2 by old block id (sequential reads: measured best), 3 by new block id
 constexpr uint32_t kDefaultBulkCtas = 74;  // measured optimum on B200: half the SMs, deep rings
 constexpr uint32_t kVecTile = 16384;
 constexpr uint64_t kBulkMinRun = 16384;  // shorter runs go to the vector kernel
@@ -45,7 +45,7 @@ struct DevPhase {
   // units of the other bulk segments are built on the host and follow them.
   uint64_t n_gen = 0;
   std::vector<uint32_t> gen_seg, gen_pre;
-  uint32_t gen_runs = 0, gen_upr = 0;
+  uint32_t gen_runs = 0, gen_upr = 0, gen_group = 1;   // gen_upr: units per group of gen_group runs
   uint64_t rest_off[3] = {0, 0, 0};           // merged set: where each phase's host-built units start in bulk_units
   DevSeg *d_segs = nullptr;
   Dst *d_dsts = nullptr;
@@ -121,12 +121,27 @@ int kv_order(const emoe_plan *p) {
 }
 
 // Cuts one segment into units of at most kUnitTiles tiles and hands each to f(first run
-// the unit touches, unit).  A unit of a long-run segment (run >= tile) stays inside one run,
-// so that units can be ordered by run.
+// the unit touches, unit).  A unit of a long-run segment (run >= tile) whose runs fill a unit
+// stays inside one run, so that units can be ordered by run; runs of fewer tiles than a unit
+// (a 64 KiB KV block is two) are taken several to a unit - runs_per_unit() consecutive runs -
+// because a unit is the grain at which CTAs claim work and fetch descriptors, and a grain of
+// two tiles costs 4-5 % of the bandwidth.
+uint32_t runs_per_unit(uint32_t tiles_per_run) {
+  return tiles_per_run >= kUnitTiles ? 1u : kUnitTiles / tiles_per_run;
+}
+
 template <typename F>
 void for_each_unit(uint32_t seg, const DevSeg &s, uint32_t T, F &&f) {
   if (s.run_bytes >= T) {
     const uint32_t tpr = (uint32_t)((s.run_bytes + T - 1) / T);
+    const uint32_t g = runs_per_unit(tpr);
+    if (g > 1) {
+      for (uint32_t run = 0; run < s.n_runs; run += g) {
+        const uint32_t n = s.n_runs - run < g ? s.n_runs - run : g;
+        f(run, Unit{seg, run * tpr, n * tpr, 0});
+      }
+      return;
+    }
     for (uint32_t run = 0; run < s.n_runs; ++run)
       for (uint32_t t = 0; t < tpr; t += kUnitTiles) {
         const uint32_t n = tpr - t < kUnitTiles ? tpr - t : kUnitTiles;
@@ -173,7 +188,7 @@ void build_tables(emoe_plan *p, int phase) {
   DevPhase &dp = p->dev[phase];
   dp.segs.clear(); dp.dsts.clear(); dp.bulk_units.clear(); dp.vec_units.clear();
   dp.gen_seg.clear(); dp.gen_pre.clear();
-  dp.n_gen = 0; dp.n_bulk = 0; dp.gen_runs = dp.gen_upr = 0;
+  dp.n_gen = 0; dp.n_bulk = 0; dp.gen_runs = dp.gen_upr = 0; dp.gen_group = 1;
   for (bool &b : p->reads_src[phase]) b = false;
   const uint32_t T = bulk_tile(p);
 
@@ -244,21 +259,31 @@ void build_tables(emoe_plan *p, int phase) {
   // are built here; they follow the generated part.
   std::vector<uint32_t> rest;
   if (p->tuning.unit_order % 2 == 0) {
-    uint32_t runs0 = 0;
+    uint32_t runs0 = 0, g0 = 1;     // run count and runs per unit of the regular segments
     for (uint32_t idx : bulk_segs)
-      if (dp.segs[idx].run_bytes >= T) { runs0 = dp.segs[idx].n_runs; break; }
-    uint64_t upr = 0;
+      if (dp.segs[idx].run_bytes >= T) {
+        runs0 = dp.segs[idx].n_runs;
+        g0 = runs_per_unit((uint32_t)((dp.segs[idx].run_bytes + T - 1) / T));
+        break;
+      }
+    uint64_t upg = 0;               // units per group of g0 runs, over all regular segments
     for (uint32_t idx : bulk_segs) {
-      if (runs0 == 0 || dp.segs[idx].run_bytes < T || dp.segs[idx].n_runs != runs0) { rest.push_back(idx); continue; }
-      dp.gen_seg.push_back(idx);
-      dp.gen_pre.push_back((uint32_t)upr);
       const uint64_t tpr = (dp.segs[idx].run_bytes + T - 1) / T;
-      upr += (tpr + kUnitTiles - 1) / kUnitTiles;
+      if (runs0 == 0 || dp.segs[idx].run_bytes < T || dp.segs[idx].n_runs != runs0 ||
+          runs_per_unit((uint32_t)tpr) != g0) {
+        rest.push_back(idx);
+        continue;
+      }
+      dp.gen_seg.push_back(idx);
+      dp.gen_pre.push_back((uint32_t)upg);
+      upg += g0 > 1 ? 1 : (tpr + kUnitTiles - 1) / kUnitTiles;
     }
-    if (upr * runs0 < 0xffffffffull && upr < 0xffffffffull) {
+    const uint64_t groups = (runs0 + g0 - 1) / g0;
+    if (upg * groups < 0xffffffffull && upg < 0xffffffffull) {
       dp.gen_runs = runs0;
-      dp.gen_upr = (uint32_t)upr;
-      dp.n_gen = upr * runs0;
+      dp.gen_group = g0;
+      dp.gen_upr = (uint32_t)upg;
+      dp.n_gen = upg * groups;
     } else {  // too many for 32-bit unit indices in the generator: everything on the host
       dp.gen_seg.clear(); dp.gen_pre.clear();
       rest = bulk_segs;
@@ -389,8 +414,8 @@ cudaError_t gen_units(const emoe_plan *p, int src_ph, const DevSeg *d_segs, uint
   if (e == cudaSuccess) e = cudaMemcpy(d_idx, dp.gen_seg.data(), bytes, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemcpy(d_pre, dp.gen_pre.data(), bytes, cudaMemcpyHostToDevice);
   if (e == cudaSuccess)
-    e = launch_gen_units(d_segs, d_idx, d_pre, (uint32_t)dp.gen_seg.size(), dp.gen_runs, dp.gen_upr,
-                         bulk_tile(p), kUnitTiles, seg_offset, out, nullptr);
+    e = launch_gen_units(d_segs, d_idx, d_pre, (uint32_t)dp.gen_seg.size(), dp.gen_runs, dp.gen_group,
+                         dp.gen_upr, bulk_tile(p), kUnitTiles, seg_offset, out, nullptr);
   if (e == cudaSuccess) e = cudaStreamSynchronize(nullptr);
   cudaFree(d_idx);
   cudaFree(d_pre);

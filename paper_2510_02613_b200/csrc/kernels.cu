@@ -1205,29 +1205,36 @@ cudaError_t launch_kv_copy(const KvTables &t, const RankPtrs &ptrs, int mode, ui
 
 namespace {
 __global__ void gen_units_kernel(const DevSeg *segs, const uint32_t *seg_idx, const uint32_t *seg_pre,
-                                 uint32_t n_segs, uint32_t n_runs, uint32_t units_per_run,
+                                 uint32_t n_segs, uint32_t n_runs, uint32_t group, uint32_t units_per_group,
                                  uint32_t tile_bytes, uint32_t unit_tiles, uint32_t seg_offset,
                                  Unit *out) {
+  const uint32_t n_groups = (n_runs + group - 1) / group;
   const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (uint64_t)n_segs * n_runs) return;
-  const uint32_t k = (uint32_t)(i % n_segs), run = (uint32_t)(i / n_segs);
+  if (i >= (uint64_t)n_segs * n_groups) return;
+  const uint32_t k = (uint32_t)(i % n_segs), grp = (uint32_t)(i / n_segs);
   const uint32_t seg = seg_idx[k] + seg_offset;
   const uint64_t run_bytes = segs[seg].run_bytes;
   const uint32_t tpr = (uint32_t)((run_bytes + tile_bytes - 1) / tile_bytes);
-  Unit *o = out + (uint64_t)run * units_per_run + seg_pre[k];
+  Unit *o = out + (uint64_t)grp * units_per_group + seg_pre[k];
+  if (group > 1) {  // runs shorter than a unit: `group` consecutive runs are one unit
+    const uint32_t run0 = grp * group, n = n_runs - run0 < group ? n_runs - run0 : group;
+    *o = Unit{seg, run0 * tpr, n * tpr, 0};
+    return;
+  }
   for (uint32_t t = 0; t < tpr; t += unit_tiles, ++o)
-    *o = Unit{seg, run * tpr + t, tpr - t < unit_tiles ? tpr - t : unit_tiles, 0};
+    *o = Unit{seg, grp * tpr + t, tpr - t < unit_tiles ? tpr - t : unit_tiles, 0};
 }
 }  // namespace
 
 cudaError_t launch_gen_units(const DevSeg *segs, const uint32_t *seg_idx, const uint32_t *seg_pre,
-                             uint32_t n_segs, uint32_t n_runs, uint32_t units_per_run,
+                             uint32_t n_segs, uint32_t n_runs, uint32_t group, uint32_t units_per_group,
                              uint32_t tile_bytes, uint32_t unit_tiles, uint32_t seg_offset, Unit *out,
                              cudaStream_t stream) {
-  const uint64_t n = (uint64_t)n_segs * n_runs;
+  if (group == 0) return cudaErrorInvalidValue;
+  const uint64_t n = (uint64_t)n_segs * ((n_runs + group - 1) / group);
   if (n == 0) return cudaSuccess;
   gen_units_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(
-      segs, seg_idx, seg_pre, n_segs, n_runs, units_per_run, tile_bytes, unit_tiles, seg_offset, out);
+      segs, seg_idx, seg_pre, n_segs, n_runs, group, units_per_group, tile_bytes, unit_tiles, seg_offset, out);
   return cudaGetLastError();
 }
 

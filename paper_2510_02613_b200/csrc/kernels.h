@@ -103,11 +103,13 @@ emoe_status_t launch_kv_copy_static(const KvTables &shape_only, const uint32_t *
                                     const uint32_t *pair_new, const RankPtrs &ptrs,
                                     cudaStream_t stream);
 
-// Writes the regular unit table of a phase on the device: for every run r < n_runs and every
-// listed segment k (index seg_idx[k] + seg_offset into segs), the units of that run at
-// out[r * units_per_run + seg_pre[k] ...], each of at most unit_tiles tiles of tile_bytes.
+// Writes the regular unit table of a phase on the device.  Runs are taken `group` at a time
+// (group > 1 only for runs of fewer tiles than a unit: those runs then form ONE unit); for
+// every group g and every listed segment k (index seg_idx[k] + seg_offset into segs) the
+// units of that group go to out[g * units_per_group + seg_pre[k] ...], each of at most
+// unit_tiles tiles of tile_bytes.
 cudaError_t launch_gen_units(const DevSeg *segs, const uint32_t *seg_idx, const uint32_t *seg_pre,
-                             uint32_t n_segs, uint32_t n_runs, uint32_t units_per_run,
+                             uint32_t n_segs, uint32_t n_runs, uint32_t group, uint32_t units_per_group,
                              uint32_t tile_bytes, uint32_t unit_tiles, uint32_t seg_offset, Unit *out,
                              cudaStream_t stream);
 
