@@ -757,8 +757,8 @@ def run_exchange(args):
     """bench.py --gpus N --mode exchange (under torchrun): rank = GPU.  Every process owns the
     old and the new arenas of its rank index, builds the same plan, restricts it to its own
     destination rank and PULLS what it needs from its peers' old arenas through CUDA IPC
-    mappings - the library's own kernels reading peer memory (plain loads, non-multicast bulk
-    copies); torch.distributed carries handles, barriers and the max of the step times only.
+    mappings - the library's own kernels reading peer memory (plain loads and bulk copies that
+    every CTA issues for itself); torch.distributed carries handles, barriers and the max of the step times only.
     value = 2 x bytes all ranks wrote / slowest rank's time."""
     import torch
     import torch.distributed as dist

@@ -237,10 +237,19 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *plan, const void *const *src,
 /*
  * emoe_reshard_step - the whole scale step (Sec. 5.2: experts, attention
  * weights and KV cache are reconfigured together): the three phases of
- * emoe_reshard_experts / _attn / _kv with the same results, enqueued as ONE
- * set of launches.  The phases touch disjoint arenas, so their copy segments
- * share a launch (no ramp-up and tail per phase); only a KV head re-split keeps
- * its own kernel.
+ * emoe_reshard_experts / _attn / _kv with the same results, enqueued as at
+ * most TWO launches.  The phases touch disjoint arenas, so all their long
+ * runs share one launch of the ring kernel (no ramp-up and tail per phase),
+ * and what cannot go through the ring - short or strided runs and a KV head
+ * re-split - shares one launch of a second kernel.  When both are present the
+ * second one is enqueued on a stream that belongs to the plan, forked from
+ * cuda_stream and joined back to it with events: it starts after everything
+ * cuda_stream held before the call, the two launches run side by side, and
+ * cuda_stream continues only after both.  The plan keeps such a stream at
+ * the least and at the greatest priority and uses the one nearer to
+ * cuda_stream's priority.  The call itself still neither allocates nor
+ * synchronises, and it can be captured into a CUDA graph.  tuning.serial = 1
+ * keeps everything on cuda_stream.
  *
  * src / dst: indexed by EMOE_PHASE_EXPERTS / _ATTN / _KV, each a HOST array of
  * DEVICE pointers as for the per-phase call.  All arguments of all phases are

@@ -4,7 +4,7 @@
 //    issues cp.async.bulk (TMA, untiled) global->shared loads into a ring of
 //    stages guarded by mbarriers; one consumer thread issues the
 //    shared->global bulk stores, once per destination of the tile, so a
-//    replicated source is read from HBM once.  No cluster, no multicast.
+//    replicated source is read from HBM once.  No thread-block cluster is used.
 //  * vec_copy_kernel  : short, strided or narrowly aligned runs.  A warp per
 //    tile, lanes walk the tile in 16-byte (or narrower) pieces, four loads in
 //    flight per lane before the stores.

@@ -4,7 +4,7 @@ Process g owns the old arenas of rank index g (where the old configuration has s
 rank) and the new arenas of rank index g.  Every process builds the same plan, restricts
 it to its own destination rank (emoe_plan_set_local_rank) and pulls what it needs from its
 peers' old arenas through CUDA IPC mappings: the library's kernels read a peer-mapped
-pointer exactly as they read a local one (plain loads and non-multicast bulk copies).
+pointer exactly as they read a local one (plain loads and per-CTA bulk copies).
 torch.distributed carries the control plane only (handles, barriers); no collective
 touches the data.
 """
