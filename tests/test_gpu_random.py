@@ -29,3 +29,33 @@ def test_drawn_cases_match_the_oracle(wl):
         check_step_full(wl, plan)
         plan.set_tuning()
         check_step_full(wl, plan)
+
+
+@settings(max_examples=40, deadline=None, derandomize=True, database=None,
+          suppress_health_check=list(HealthCheck))
+@given(__import__("test_planner_random").inplace_cases())
+def test_drawn_inplace_steps_match_the_oracle(case):
+    """The in-place expert step on drawn slot tables (holes, replicas, devices added and
+    removed), default routing and forced onto the ring kernel; whole arenas against the oracle."""
+    import numpy as np
+    import torch
+    import oracle
+    import workloads as W
+    from workloads import device as WD
+    sh, old, want, cap_new = case
+    try:
+        plan = E.InplacePlan(sh, old, want, cap_new)
+    except E.EmoeError as e:
+        assert e.code == 11
+        return
+    with plan:
+        for tuning in (dict(), dict(path=2, max_ctas=3)):
+            plan.set_tuning(**tuning)
+            dev = WD.alloc_filled(oracle.inplace_arena_bytes(sh, plan.caps), 31, W.KIND_EXPERTS)
+            expect = [t.cpu().numpy() for t in dev]
+            assert oracle.reshard_experts_inplace(sh, old, want, cap_new, expect) == plan.slot_tables()
+            plan.reshard(dev)
+            torch.cuda.synchronize()
+            assert plan.device_status() == 0
+            for r, (g, w) in enumerate(zip(dev, expect)):
+                assert np.array_equal(g.cpu().numpy(), w), (tuning, r)
