@@ -8,7 +8,7 @@ from hypothesis import HealthCheck, given, settings
 
 import paper_2510_02613_b200 as E
 from gpu_util import check_phase_full, check_step_full, make_plan
-from test_planner_random import cases
+from test_planner_random import cases, inplace_cases
 
 pytestmark = pytest.mark.gpu
 
@@ -33,7 +33,7 @@ def test_drawn_cases_match_the_oracle(wl):
 
 @settings(max_examples=40, deadline=None, derandomize=True, database=None,
           suppress_health_check=list(HealthCheck))
-@given(__import__("test_planner_random").inplace_cases())
+@given(inplace_cases())
 def test_drawn_inplace_steps_match_the_oracle(case):
     """The in-place expert step on drawn slot tables (holes, replicas, devices added and
     removed), default routing and forced onto the ring kernel; whole arenas against the oracle."""
