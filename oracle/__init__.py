@@ -125,9 +125,20 @@ def reshard_experts(shape, old_placement, new_placement, src: Sequence[np.ndarra
         raise ValueError("oracle: an expert of the new placement is absent from the old one")
 
 
-def reshard_attn(shape, tp_old: int, tp_new: int, src, dst, fused_qkv: bool = False) -> None:
+def reshard_attn(shape, tp_old: int, tp_new: int, src, dst, fused_qkv: bool = False,
+                 replicas: int = 1) -> None:
     """fused_qkv: per rank and layer one [qkv_t | o_t] arena whose qkv rows are grouped by
-    KV head (the group's query heads, then the k head, then the v head)."""
+    KV head (the group's query heads, then the k head, then the v head).
+    replicas > 1: the new side consists of that many data-parallel replicas of the TP group
+    (Sec. 5.2 "Attention Weights": added devices receive whole copies of the attention
+    tensors); dst lists them replica after replica, tp_new arenas each, and every replica is
+    by definition the same re-slice of the old shards."""
+    if replicas > 1:
+        if len(dst) != tp_new * replicas:
+            raise ValueError("attention arena sizes do not match")
+        for k in range(replicas):
+            reshard_attn(shape, tp_old, tp_new, src, dst[k * tp_new:(k + 1) * tp_new], fused_qkv)
+        return
     if ([a.size for a in src] != attn_arena_bytes(shape, tp_old)
             or [a.size for a in dst] != attn_arena_bytes(shape, tp_new)):
         raise ValueError("attention arena sizes do not match")

@@ -747,3 +747,22 @@ def test_compact_block_table_hand_written_and_properties():
             continue
         flat = [int(x) for row in oracle.compact_block_table(lens, 3, nb, in_use) for x in row if x >= 0]
         assert flat == free[:len(flat)]
+
+
+# ======================================================= attention for added replicas ===
+
+@pytest.mark.parametrize("c,d,replicas", [(2, 2, 3), (1, 2, 2), (4, 2, 2)])
+def test_attn_replicas_each_equal_the_numpy_split(c, d, replicas):
+    """Provisioning added data-parallel replicas: every replica's shard t is the numpy split of
+    the logical matrices, whatever the old TP degree; a dropped or misplaced replica shows."""
+    sh = tiny_shape(n_layers=2)
+    logical = logical_attn(sh)
+    src = attn_arenas(logical, c)
+    want = attn_arenas(logical, d)
+    dst = filled([a.size for a in want] * replicas)
+    oracle.reshard_attn(sh, c, d, src, dst, replicas=replicas)
+    for k in range(replicas):
+        for t in range(d):
+            assert np.array_equal(dst[k * d + t], want[t]), (k, t)
+    with pytest.raises(ValueError):
+        oracle.reshard_attn(sh, c, d, src, dst[:-1], replicas=replicas)
