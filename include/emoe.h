@@ -166,11 +166,24 @@ emoe_status_t emoe_plan_create(const emoe_shape_t *shape, const emoe_config_t *o
  * and ONE plan - one call, one launch set - moves both by the same placement.  Bytes
  * between the two parts are never written.  Not combinable with EMOE_LAYOUT_FUSED_W13
  * (EMOE_ERR_UNSUPPORTED); such a plan's emoe_reshard_step_host runs serially.
+ *
+ * attn_new_replicas > 1: the new side consists of that many data-parallel replicas of
+ * the TP=d group - the paper's attention step (Sec. 5.2 "Attention Weights": devices that
+ * are added receive whole copies of the attention tensors from devices that hold them).
+ * The attention phase then has tp_new * attn_new_replicas destination arenas, replica
+ * after replica (replica k's rank t is index k * tp_new + t), every replica the same
+ * re-slice of the old shards; a source run is read ONCE and stored to all replicas.
+ * emoe_plan_num_ranks / _arena_bytes report the larger rank count for EMOE_PHASE_ATTN,
+ * EMOE_SIDE_NEW, and dst of emoe_reshard_attn / emoe_reshard_step has that many entries.
+ * Experts and KV are not affected (a new replica starts with an empty KV cache).
+ * tp_new * attn_new_replicas may not exceed EMOE_MAX_RANKS (EMOE_ERR_UNSUPPORTED).
+ * 0 and 1 both mean one replica.
  * reserved: must be zero.
  */
 typedef struct {
   int64_t expert_scale_bytes;
-  int64_t reserved[7];
+  int64_t attn_new_replicas;
+  int64_t reserved[6];
 } emoe_plan_options_t;
 emoe_status_t emoe_plan_create_ex(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
                                   const emoe_config_t *new_cfg, uint32_t flags,

@@ -47,7 +47,8 @@ class _Config(ctypes.Structure):
 
 
 class _PlanOptions(ctypes.Structure):
-    _fields_ = [("expert_scale_bytes", ctypes.c_int64), ("reserved", ctypes.c_int64 * 7)]
+    _fields_ = [("expert_scale_bytes", ctypes.c_int64), ("attn_new_replicas", ctypes.c_int64),
+                ("reserved", ctypes.c_int64 * 6)]
 
 
 class _Segment(ctypes.Structure):
@@ -276,7 +277,8 @@ class Plan:
     """A scale-step plan: emoe_plan_create ... emoe_plan_destroy."""
 
     def __init__(self, shape, old_cfg, new_cfg, host_only: bool = False, host_step: bool = False,
-                 fused_w13: bool = False, kv_head_major: bool = False, fused_qkv: bool = False):
+                 fused_w13: bool = False, kv_head_major: bool = False, fused_qkv: bool = False,
+                 attn_replicas: int = 1):
         self._h = _vp()
         keep: list = []
         sh = _Shape(shape.n_layers, shape.n_routed, shape.n_shared, shape.d_model, shape.d_ff,
@@ -287,8 +289,8 @@ class Plan:
                  | (LAYOUT_FUSED_W13 if fused_w13 else 0) | (LAYOUT_KV_HEAD_MAJOR if kv_head_major else 0)
                  | (LAYOUT_FUSED_QKV if fused_qkv else 0))
         scale = int(getattr(shape, "expert_scale_bytes", 0) or 0)
-        if scale:     # every expert matrix travels with a scale tensor
-            opt = _PlanOptions(scale)
+        if scale or attn_replicas > 1:     # scale tensors with the matrices / several new DP replicas
+            opt = _PlanOptions(scale, attn_replicas)
             _check(lib().emoe_plan_create_ex(ctypes.byref(sh), ctypes.byref(co), ctypes.byref(cn), flags,
                                              ctypes.byref(opt), ctypes.byref(self._h)))
         else:
@@ -446,10 +448,11 @@ class PlanCache:
                     shape.elem_bytes)
         co, cn = _make_config(old_cfg, keep), _make_config(new_cfg, keep)
         scale = int(getattr(shape, "expert_scale_bytes", 0) or 0)
-        opt = _PlanOptions(scale)
+        replicas = int(flags.pop("attn_replicas", 1))
+        opt = _PlanOptions(scale, replicas)
         h, hit = _vp(), _i32()
         _check(lib().emoe_plan_cache_get(self._h, ctypes.byref(sh), ctypes.byref(co), ctypes.byref(cn),
-                                         _plan_flags(**flags), ctypes.byref(opt) if scale else None,
+                                         _plan_flags(**flags), ctypes.byref(opt) if scale or replicas > 1 else None,
                                          ctypes.byref(h), ctypes.byref(hit)))
         plan = Plan.__new__(Plan)
         plan._h, plan._owned, plan.host_only = h, False, bool(flags.get("host_only"))

@@ -80,7 +80,9 @@ emoe_status_t emoe_plan_cache_get(emoe_plan_cache_t *c, const emoe_shape_t *shap
     put(&key, shape, sizeof(*shape));
     put(&key, &flags, sizeof(flags));
     const int64_t scale = options ? options->expert_scale_bytes : 0;
+    const int64_t replicas = options ? options->attn_new_replicas : 0;
     put(&key, &scale, sizeof(scale));
+    put(&key, &replicas, sizeof(replicas));
     cacheable = config_key(*shape, *old_cfg, &key) && config_key(*shape, *new_cfg, &key);
   } catch (const std::bad_alloc &) {
     return EMOE_ERR_OOM;

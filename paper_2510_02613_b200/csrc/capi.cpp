@@ -464,7 +464,8 @@ void free_device(emoe_plan *p) {
 
 int ranks_of(const emoe_plan *p, int phase, int side) {
   if (phase == EMOE_PHASE_EXPERTS) return side == EMOE_SIDE_OLD ? p->hp.ep_old : p->hp.ep_new;
-  return side == EMOE_SIDE_OLD ? p->hp.tp_old : p->hp.tp_new;
+  if (side == EMOE_SIDE_OLD) return p->hp.tp_old;
+  return phase == EMOE_PHASE_ATTN ? p->hp.tp_new * (int)p->hp.attn_replicas : p->hp.tp_new;
 }
 
 // Host-side argument checks of a reshard call; fills the by-value pointer table.
@@ -591,7 +592,7 @@ void destroy_host_step(HostStep *hs);
 
 emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
                           const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out,
-                          uint64_t expert_scale_bytes = 0);
+                          uint64_t expert_scale_bytes = 0, uint32_t attn_replicas = 1);
 
 // Chunk plans, streams and events of the pipelined host-buffer step.  Leaves p->hs null
 // (the step then runs serially) when a layer slice of some arena is not 16-byte aligned.
@@ -611,10 +612,10 @@ emoe_status_t make_host_step(emoe_plan *p, const emoe_shape_t &shape, const emoe
   hs->n_chunks = n_full + (tail ? 1 : 0);
   emoe_shape_t sh = shape;
   sh.n_layers = hs->lc;
-  emoe_status_t st = create_plan(&sh, old_cfg, new_cfg, layout_flags, &hs->chunk);
+  emoe_status_t st = create_plan(&sh, old_cfg, new_cfg, layout_flags, &hs->chunk, 0, p->hp.attn_replicas);
   if (st == EMOE_OK && tail) {
     sh.n_layers = tail;
-    st = create_plan(&sh, old_cfg, new_cfg, layout_flags, &hs->tail);
+    st = create_plan(&sh, old_cfg, new_cfg, layout_flags, &hs->tail, 0, p->hp.attn_replicas);
   }
   cudaError_t e = cudaSuccess;
   if (st == EMOE_OK) e = cudaStreamCreateWithFlags(&hs->s_in, cudaStreamNonBlocking);
@@ -681,14 +682,14 @@ emoe_status_t finish_device_plan(emoe_plan *p) {
 
 emoe_status_t create_plan(const emoe_shape_t *shape, const emoe_config_t *old_cfg,
                           const emoe_config_t *new_cfg, uint32_t flags, emoe_plan_t **out,
-                          uint64_t expert_scale_bytes) {
+                          uint64_t expert_scale_bytes, uint32_t attn_replicas) {
   if (!shape || !old_cfg || !new_cfg || !out) return EMOE_ERR_INVALID_ARG;
   if (expert_scale_bytes && (flags & EMOE_LAYOUT_FUSED_W13)) return EMOE_ERR_UNSUPPORTED;
   emoe_plan *p = new (std::nothrow) emoe_plan();
   if (!p) return EMOE_ERR_OOM;
   emoe_status_t st;
   try {
-    st = build_host_plan(*shape, *old_cfg, *new_cfg, flags, expert_scale_bytes, &p->hp);
+    st = build_host_plan(*shape, *old_cfg, *new_cfg, flags, expert_scale_bytes, attn_replicas, &p->hp);
     if (st == EMOE_OK) {
       build_all_tables(p);
     }
@@ -758,13 +759,17 @@ emoe_status_t emoe_plan_create_ex(const emoe_shape_t *shape, const emoe_config_t
                                   const emoe_config_t *new_cfg, uint32_t flags,
                                   const emoe_plan_options_t *options, emoe_plan_t **out) {
   uint64_t scale = 0;
+  uint32_t replicas = 1;
   if (options) {
-    if (options->expert_scale_bytes < 0) return EMOE_ERR_INVALID_ARG;
+    if (options->expert_scale_bytes < 0 || options->attn_new_replicas < 0 ||
+        options->attn_new_replicas > EMOE_MAX_RANKS)
+      return EMOE_ERR_INVALID_ARG;
     for (int64_t r : options->reserved)
       if (r != 0) return EMOE_ERR_INVALID_ARG;
     scale = (uint64_t)options->expert_scale_bytes;
+    if (options->attn_new_replicas > 1) replicas = (uint32_t)options->attn_new_replicas;
   }
-  return create_plan(shape, old_cfg, new_cfg, flags, out, scale);
+  return create_plan(shape, old_cfg, new_cfg, flags, out, scale, replicas);
 }
 
 void emoe_plan_destroy(emoe_plan_t *p) {

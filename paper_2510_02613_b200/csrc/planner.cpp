@@ -481,9 +481,32 @@ uint32_t kv_source_rank(uint32_t hkv, uint32_t c, uint32_t g, uint32_t r_new) {
   return 0;  // not reached for valid degrees
 }
 
+// The attention phase again for `replicas` data-parallel copies of the new TP group: every
+// segment keeps its source and gets one destination per replica (replica k's rank t is
+// new-rank index k * d + t), so a shard is read once however many devices receive it.
+void replicate_attn(PhasePlan *pp, int d, uint32_t replicas) {
+  if (replicas <= 1) return;
+  PhasePlan one = std::move(*pp);
+  *pp = PhasePlan();
+  pp->arena_old = one.arena_old;
+  for (uint32_t k = 0; k < replicas; ++k)
+    pp->arena_new.insert(pp->arena_new.end(), one.arena_new.begin(), one.arena_new.end());
+  for (const Segment &s0 : one.segs) {
+    std::vector<Dst> dsts;
+    for (uint32_t k = 0; k < replicas; ++k)
+      for (uint32_t j = 0; j < s0.n_dst; ++j) {
+        Dst dd = one.dsts[s0.dst_first + j];
+        dd.rank += k * (uint32_t)d;
+        dsts.push_back(dd);
+      }
+    Segment s = s0;
+    finish_segment(pp, s, dsts);
+  }
+}
+
 emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
                               const emoe_config_t &n, uint32_t flags, uint64_t expert_scale_bytes,
-                              HostPlan *hp) {
+                              uint32_t attn_replicas, HostPlan *hp) {
   if (sh.n_layers <= 0 || sh.n_routed <= 0 || sh.n_shared < 0 || sh.d_model <= 0 ||
       sh.d_ff <= 0 || sh.n_q_heads <= 0 || sh.n_kv_heads <= 0 || sh.head_dim <= 0 ||
       sh.kv_block_tokens <= 0 || sh.elem_bytes <= 0)
@@ -508,7 +531,11 @@ emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
   plan_experts(sh, po, pn, (uint64_t)sh.d_model * sh.d_ff * sh.elem_bytes, nullptr,
                (flags & EMOE_LAYOUT_FUSED_W13) != 0, expert_scale_bytes, &hp->phase[EMOE_PHASE_EXPERTS]);
   if ((flags & EMOE_LAYOUT_FUSED_QKV) && sh.n_q_heads % sh.n_kv_heads) return EMOE_ERR_SHAPE;
+  if (attn_replicas < 1) attn_replicas = 1;
+  if ((uint64_t)n.tp * attn_replicas > EMOE_MAX_RANKS) return EMOE_ERR_UNSUPPORTED;
+  hp->attn_replicas = attn_replicas;
   plan_attn(sh, o.tp, n.tp, (flags & EMOE_LAYOUT_FUSED_QKV) != 0, &hp->phase[EMOE_PHASE_ATTN]);
+  replicate_attn(&hp->phase[EMOE_PHASE_ATTN], n.tp, attn_replicas);
   plan_kv(sh, o, n, std::move(pair_old), std::move(pair_new), (flags & EMOE_LAYOUT_KV_HEAD_MAJOR) != 0, hp);
   return EMOE_OK;
 }

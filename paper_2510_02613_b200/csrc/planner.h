@@ -69,6 +69,7 @@ uint32_t kv_source_rank(uint32_t hkv, uint32_t c, uint32_t g, uint32_t r_new);
 struct HostPlan {
   emoe_shape_t shape;
   int ep_old, ep_new, tp_old, tp_new;
+  uint32_t attn_replicas = 1;  // new attention arenas: tp_new per replica, replica after replica
   PhasePlan phase[3];  // experts, attn, kv (kv.segs filled only when the head split is kept)
   KvPlan kv;
 };
@@ -76,9 +77,10 @@ struct HostPlan {
 // Validates and plans.  Returns EMOE_OK or the first validation error.
 // flags: the EMOE_LAYOUT_* bits of emoe_plan_create.  expert_scale_bytes: size of the scale
 // tensor that goes with every expert matrix (0: none).
+// attn_replicas: data-parallel copies of the new TP group that receive the attention shards.
 emoe_status_t build_host_plan(const emoe_shape_t &shape, const emoe_config_t &old_cfg,
                               const emoe_config_t &new_cfg, uint32_t flags, uint64_t expert_scale_bytes,
-                              HostPlan *out);
+                              uint32_t attn_replicas, HostPlan *out);
 
 // A destination slot that keeps the bytes its rank already holds (paged expert store).
 struct Remap {

@@ -19,7 +19,8 @@ def oracle_phase(wl, phase, src, dst):
         oracle.reshard_experts(wl.shape, wl.old.placement, wl.new.placement, src, dst,
                                fused_w13=wl.fused_w13)
     elif phase == E.PHASE_ATTN:
-        oracle.reshard_attn(wl.shape, wl.old.tp, wl.new.tp, src, dst, fused_qkv=wl.fused_qkv)
+        oracle.reshard_attn(wl.shape, wl.old.tp, wl.new.tp, src, dst, fused_qkv=wl.fused_qkv,
+                            replicas=wl.attn_replicas)
     else:
         oracle.reshard_kv(wl.shape, wl.old, wl.new, src, dst, head_major=wl.kv_head_major)
 
@@ -27,7 +28,8 @@ def oracle_phase(wl, phase, src, dst):
 def make_plan(wl, **kw):
     """A plan with the workload's layout variants."""
     return E.Plan(wl.shape, wl.old, wl.new, fused_w13=wl.fused_w13,
-                  kv_head_major=wl.kv_head_major, fused_qkv=wl.fused_qkv, **kw)
+                  kv_head_major=wl.kv_head_major, fused_qkv=wl.fused_qkv,
+                  attn_replicas=wl.attn_replicas, **kw)
 
 
 def run_phase(plan, phase, src, dst, stream=None):

@@ -414,6 +414,24 @@ def test_fused_qkv_layout(name, c, d):
         check_phase_full(wl, plan, E.PHASE_ATTN)
 
 
+@pytest.mark.parametrize("name,c,d,replicas", [("c3_fine", 2, 2, 3), ("c4_large", 2, 4, 2), ("c4_large", 4, 2, 5)])
+def test_attention_for_added_replicas(name, c, d, replicas):
+    """The paper's attention step: added data-parallel replicas receive whole copies of the
+    attention shards (here together with a TP change); every replica against the oracle, alone
+    and inside the whole step, the shards read once and stored to all replicas."""
+    from gpu_util import make_plan
+    wl = W.make_workload(name, n_layers=2)
+    wl = R(wl, attn_replicas=replicas, old=R(wl.old, tp=c), new=R(wl.new, tp=d), shape=R(wl.shape, d_ff=64))
+    with make_plan(wl) as plan:
+        assert plan.num_ranks(E.PHASE_ATTN, E.SIDE_NEW) == d * replicas
+        check_phase_full(wl, plan, E.PHASE_ATTN)
+        check_step_full(wl, plan)
+        plan.set_tuning(path=2, max_ctas=7)
+        check_phase_full(wl, plan, E.PHASE_ATTN)
+        st = plan.stats(E.PHASE_ATTN)
+        assert st["bytes_moved"] == replicas * st["bytes_read"]
+
+
 def test_scaling_sequence_with_chosen_placements():
     """A sequence of scale steps in the paper's step pattern (+2 devices per step, then
     back down), each new placement chosen by emoe_place_min_transfer from the previous

@@ -55,7 +55,8 @@ def run_oracle(wl, phase, src, dst):
         oracle.reshard_experts(wl.shape, wl.old.placement, wl.new.placement, src, dst,
                                fused_w13=wl.fused_w13)
     elif phase == E.PHASE_ATTN:
-        oracle.reshard_attn(wl.shape, wl.old.tp, wl.new.tp, src, dst, fused_qkv=wl.fused_qkv)
+        oracle.reshard_attn(wl.shape, wl.old.tp, wl.new.tp, src, dst, fused_qkv=wl.fused_qkv,
+                            replicas=wl.attn_replicas)
     else:
         oracle.reshard_kv(wl.shape, wl.old, wl.new, src, dst, head_major=wl.kv_head_major)
 
@@ -347,3 +348,35 @@ def test_plan_options_are_validated():
     with pytest.raises(E.EmoeError) as ei:
         E.Plan(sh, wl.old, wl.new, host_only=True, fused_w13=True)     # scales + fused gate|up
     assert ei.value.code == 9
+
+
+@pytest.mark.parametrize("name,c,d,replicas,fused", [("c2_mid", 2, 2, 3, False), ("c4_large", 2, 4, 2, False),
+                                                    ("c4_large", 4, 2, 2, True), ("c1_tiny", 1, 1, 9, False)])
+def test_attention_onto_several_new_replicas_reads_every_source_once(name, c, d, replicas, fused):
+    """emoe_plan_create_ex with attn_new_replicas: replayed segments == oracle on all
+    d * replicas arenas; bytes written grow with the replicas, bytes read do not."""
+    wl = small(name)
+    wl = dataclasses.replace(wl, fused_qkv=fused, attn_replicas=replicas, old=dataclasses.replace(wl.old, tp=c),
+                             new=dataclasses.replace(wl.new, tp=d))
+    with E.Plan(wl.shape, wl.old, wl.new, host_only=True, fused_qkv=fused, attn_replicas=replicas) as plan, \
+            E.Plan(wl.shape, wl.old, wl.new, host_only=True, fused_qkv=fused) as one:
+        so = oracle.attn_arena_bytes(wl.shape, c)
+        sn = oracle.attn_arena_bytes(wl.shape, d) * replicas
+        assert plan.num_ranks(E.PHASE_ATTN, E.SIDE_NEW) == d * replicas
+        assert plan.num_ranks(E.PHASE_KV, E.SIDE_NEW) == d          # experts and KV are not affected
+        assert plan.arena_bytes(E.PHASE_ATTN, E.SIDE_NEW) == sn
+        src = arenas(so, 71)
+        want = [np.full(n, FILL, np.uint8) for n in sn]
+        got = [np.full(n, FILL, np.uint8) for n in sn]
+        run_oracle(wl, E.PHASE_ATTN, src, want)
+        segs = plan.segments(E.PHASE_ATTN)
+        replay(segs, src, got)
+        for r in range(len(sn)):
+            assert np.array_equal(got[r], want[r]), r
+        a, b = plan.stats(E.PHASE_ATTN), one.stats(E.PHASE_ATTN)
+        assert a["bytes_moved"] == replicas * b["bytes_moved"] and a["bytes_read"] == b["bytes_read"]
+        assert len(set(int(g) for g in segs["group"])) == b["n_segments"]      # one read per source run
+    if d > 1:       # d * 64 attention arenas are more than the library takes
+        with pytest.raises(E.EmoeError) as ei:
+            E.Plan(wl.shape, wl.old, wl.new, host_only=True, attn_replicas=E.MAX_RANKS)
+        assert ei.value.code == 9

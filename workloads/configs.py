@@ -70,6 +70,7 @@ class Workload:
     fused_w13: bool = False        # layout variant: per layer [n][gate|up] then [n][down]
     kv_head_major: bool = False    # layout variant: KV blocks [local head][token][hd]
     fused_qkv: bool = False        # layout variant: attention arena [qkv_t | o_t], rows grouped by KV head
+    attn_replicas: int = 1         # data-parallel replicas of the new TP group that receive the attention shards
 
     def with_layers(self, n_layers: int) -> "Workload":
         """Same workload cut to n_layers (layers are independent in every phase)."""
