@@ -987,23 +987,26 @@ def main():
     plan.close()
     torch.cuda.empty_cache()
     if rank == 0 and not args.only_main:
-        rep["inplace_expert_step"] = run_inplace(torch, E, wl, rep["phases"]["experts"]["ms"], peak)
-        rep["vmm_expert_step"] = run_vmm(torch, E, wl, rep["phases"]["experts"]["ms"])
-        rep["vmm_slots_expert_step"] = run_vmm_slots(torch, E, wl, rep["phases"]["experts"]["ms"])
+        for key, fn in (("inplace_expert_step", lambda: run_inplace(torch, E, wl, rep["phases"]["experts"]["ms"], peak)),
+                        ("vmm_expert_step", lambda: run_vmm(torch, E, wl, rep["phases"]["experts"]["ms"])),
+                        ("vmm_slots_expert_step", lambda: run_vmm_slots(torch, E, wl, rep["phases"]["experts"]["ms"]))):
+            try:
+                rep[key] = fn()
+            except Exception as e:      # report, never hide
+                rep[key] = {"error": repr(e)[:300]}
+                torch.cuda.empty_cache()
 
-    if not args.only_main and world == 1:
-        others = {}
-        for name in W.WORKLOAD_NAMES + W.EXTRA_WORKLOAD_NAMES:
-            if name == args.workload:
-                others[name] = rep
-                continue
-            wl2, plan2, src2, dst2, pms = setup(name, torch, E, W, WD)
+    def measure_config(name):
+        wl2, plan2, src2, dst2, pms = setup(name, torch, E, W, WD)
+        try:
             # at least 100 steps and about a second of timed region each; the tiny config is
             # timed without per-step events (an event costs a tenth of its step)
             k = {"c1_tiny": 2000}.get(name, max(100, args.steps // 2))
             tot, each2 = time_steps(torch, plan2, src2, dst2, k, 3, stream, per_step=name != "c1_tiny")
             ph = time_phases(torch, plan2, src2, dst2, 20, stream)
             r = config_report(E, plan2, wl2, tot, each2, ph, k, peak, peak_kind, pms, traffic)
+            if plan2.device_status() != 0:
+                r["error"] = "device status word set: a bounded wait expired"
             if name == "c1_tiny":    # launch-bound: also as a CUDA-graph replay
                 g_ms = time_graph_steps(torch, plan2, src2, dst2, k, 3, stream)
                 r["cuda_graph"] = {"scale_step_ms": round(g_ms, 4),
@@ -1014,14 +1017,34 @@ def main():
                 r["overlap"] = run_overlap(torch, E, plan2, wl2, src2, dst2, peak,
                                            W.make_workload("c5_overlap").victim,
                                            points=(dict(), dict(bw_limit_gbs=4500), dict(bw_limit_gbs=2500)))
-            others[name] = r
+        finally:
             del src2, dst2
             plan2.close()
             torch.cuda.empty_cache()
-            if name in ("c2_mid", "c3_fine", "c4_large"):
-                r["inplace_expert_step"] = run_inplace(torch, E, wl2, r["phases"]["experts"]["ms"], peak)
-                r["vmm_expert_step"] = run_vmm(torch, E, wl2, r["phases"]["experts"]["ms"])
-                r["vmm_slots_expert_step"] = run_vmm_slots(torch, E, wl2, r["phases"]["experts"]["ms"])
+        if name in ("c2_mid", "c3_fine", "c4_large"):
+            for key, fn in (("inplace_expert_step", lambda: run_inplace(torch, E, wl2, r["phases"]["experts"]["ms"], peak)),
+                            ("vmm_expert_step", lambda: run_vmm(torch, E, wl2, r["phases"]["experts"]["ms"])),
+                            ("vmm_slots_expert_step", lambda: run_vmm_slots(torch, E, wl2, r["phases"]["experts"]["ms"]))):
+                try:
+                    r[key] = fn()
+                except Exception as e:
+                    r[key] = {"error": repr(e)[:300]}
+                    torch.cuda.empty_cache()
+        return r
+
+    if not args.only_main and world == 1:
+        others = {}
+        for name in W.WORKLOAD_NAMES + W.EXTRA_WORKLOAD_NAMES:
+            if name == args.workload:
+                others[name] = rep
+                continue
+            # a config that cannot be measured (out of memory on a smaller device, ...) is
+            # reported as such in its place; it does not take the line down with it
+            try:
+                others[name] = measure_config(name)
+            except Exception as e:
+                others[name] = {"workload": name, "error": repr(e)[:300]}
+                torch.cuda.empty_cache()
         line["configs"] = others
 
     if dist:
