@@ -261,8 +261,9 @@ emoe_status_t emoe_reshard_kv(const emoe_plan_t *plan, const void *const *src,
  * cuda_stream continues only after both.  The plan keeps such a stream at
  * the least and at the greatest priority and uses the one nearer to
  * cuda_stream's priority.  The call itself still neither allocates nor
- * synchronises, and it can be captured into a CUDA graph.  tuning.serial = 1
- * keeps everything on cuda_stream.
+ * synchronises, and it can be captured into a CUDA graph (the plan's stream
+ * then belongs to the capture until it ends: make no other whole-step call on
+ * that plan meanwhile).  tuning.serial = 1 keeps everything on cuda_stream.
  *
  * src / dst: indexed by EMOE_PHASE_EXPERTS / _ATTN / _KV, each a HOST array of
  * DEVICE pointers as for the per-phase call.  All arguments of all phases are

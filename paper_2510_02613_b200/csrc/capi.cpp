@@ -90,6 +90,7 @@ struct emoe_plan {
   // side[0] has the least priority, side[1] the greatest; the one nearer the caller's
   // stream is used.  The mutex orders the record / wait pairs of concurrent callers.
   cudaStream_t side[2] = {nullptr, nullptr};
+  int prio_least = 0, prio_greatest = 0;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   mutable std::mutex fork_mu;
   emoe_plan() { for (auto &a : launch_seq) a.store(0); }
@@ -668,10 +669,9 @@ emoe_status_t finish_device_plan(emoe_plan *p) {
   if (st == EMOE_OK) {
     cudaError_t e3 = cudaMalloc((void **)&p->d_status, kStatusWords * sizeof(int));
     if (e3 == cudaSuccess) e3 = cudaMemset(p->d_status, 0, kStatusWords * sizeof(int));
-    int least = 0, greatest = 0;
-    if (e3 == cudaSuccess) e3 = cudaDeviceGetStreamPriorityRange(&least, &greatest);
-    if (e3 == cudaSuccess) e3 = cudaStreamCreateWithPriority(&p->side[0], cudaStreamNonBlocking, least);
-    if (e3 == cudaSuccess) e3 = cudaStreamCreateWithPriority(&p->side[1], cudaStreamNonBlocking, greatest);
+    if (e3 == cudaSuccess) e3 = cudaDeviceGetStreamPriorityRange(&p->prio_least, &p->prio_greatest);
+    if (e3 == cudaSuccess) e3 = cudaStreamCreateWithPriority(&p->side[0], cudaStreamNonBlocking, p->prio_least);
+    if (e3 == cudaSuccess) e3 = cudaStreamCreateWithPriority(&p->side[1], cudaStreamNonBlocking, p->prio_greatest);
     if (e3 == cudaSuccess) e3 = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
     if (e3 == cudaSuccess) e3 = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
     st = cuda_status(e3);
@@ -847,11 +847,10 @@ emoe_status_t emoe_reshard_step(const emoe_plan_t *p, const void *const *const s
   cudaStream_t st2 = st;
   std::unique_lock<std::mutex> lock(p->fork_mu, std::defer_lock);
   if (fork) {
-    int prio = 0, least = 0, greatest = 0;
+    int prio = 0;
     cudaError_t e = cudaStreamGetPriority(st, &prio);
-    if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&least, &greatest);
     if (e != cudaSuccess) return cuda_status(e);
-    st2 = (prio - greatest) < (least - prio) ? p->side[1] : p->side[0];
+    st2 = (prio - p->prio_greatest) < (p->prio_least - prio) ? p->side[1] : p->side[0];
     lock.lock();
     e = cudaEventRecord(p->ev_fork, st);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(st2, p->ev_fork, 0);
