@@ -73,7 +73,8 @@ typedef enum {
   EMOE_ERR_CUDA = 8,         /* a CUDA runtime call failed (no device, bad stream...) */
   EMOE_ERR_UNSUPPORTED = 9,  /* more ranks than EMOE_MAX_RANKS, no virtual memory API   */
   EMOE_ERR_DEVICE_TIMEOUT = 10, /* a bounded device-side wait expired                 */
-  EMOE_ERR_TOO_LARGE = 11    /* the problem exceeds a fixed capacity of the entry point */
+  EMOE_ERR_TOO_LARGE = 11,   /* the problem exceeds a fixed capacity of the entry point */
+  EMOE_ERR_PLAN_CHECK = 12   /* a segment list failed emoe_segments_validate            */
 } emoe_status_t;
 
 /* Model shape.  All fields must be > 0 except n_shared (>= 0). */
@@ -565,6 +566,26 @@ typedef struct {
  * old rank, new rank) overlap, its runs being the block's token rows. */
 emoe_status_t emoe_plan_segments(const emoe_plan_t *plan, int phase, emoe_segment_t *out,
                                  uint64_t cap, uint64_t *n);
+
+/* emoe_segments_validate / emoe_plan_validate - the host-side bounds and race check.
+ * Copy kernels can only fault by leaving an arena and only race by writing one byte twice;
+ * both are properties of the segment list.  Checks, for segments as emoe_plan_segments
+ * exports them and arena sizes in bytes: every source run and every destination run lies
+ * inside its arena (ranks in range, no arithmetic overflow), a segment's own runs do not
+ * overlap, destination runs of one arena are pairwise disjoint, and - with must_tile - they
+ * cover the arena exactly (weights: every byte of a new arena is written once).
+ * Returns EMOE_OK or EMOE_ERR_PLAN_CHECK with the index of an offending segment in
+ * *bad_segment (optional; n_segs if an arena's tail is not covered).  Host only.
+ * emoe_plan_validate runs it on a plan's own three phases (experts and attention must tile;
+ * the KV phase need not: unmapped blocks are not written; an in-place plan must not tile
+ * either: kept slots are not written) and stores the failing phase in *bad_phase.  A plan made
+ * by this library passes; the call exists for callers that want the guarantee re-checked
+ * (after an upgrade, under test) and costs time proportional to the number of runs. */
+emoe_status_t emoe_segments_validate(const emoe_segment_t *segs, uint64_t n_segs,
+                                     const uint64_t *arena_old, int32_t n_old,
+                                     const uint64_t *arena_new, int32_t n_new, int32_t must_tile,
+                                     uint64_t *bad_segment);
+emoe_status_t emoe_plan_validate(const emoe_plan_t *plan, int32_t *bad_phase, uint64_t *bad_segment);
 
 /* Reads the plan's device status word (EMOE_OK or EMOE_ERR_DEVICE_TIMEOUT).
  * Synchronises the device copy on the legacy default stream; call it after

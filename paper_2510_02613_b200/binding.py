@@ -82,6 +82,7 @@ EXPORTS = ("emoe_plan_create", "emoe_plan_create_ex", "emoe_reshard_experts", "e
            "emoe_plan_arena_bytes", "emoe_plan_stats", "emoe_plan_num_launches", "emoe_plan_launch_work",
            "emoe_plan_segments",
            "emoe_plan_device_status", "emoe_plan_clear_device_status", "emoe_plan_set_tuning",
+           "emoe_segments_validate", "emoe_plan_validate",
            "emoe_strerror",
            "emoe_plan_cache_create", "emoe_plan_cache_get", "emoe_plan_cache_stats", "emoe_plan_cache_destroy",
            "emoe_kv_compact_table", "emoe_place_min_transfer", "emoe_plan_set_local_rank", "emoe_ipc_export", "emoe_ipc_open", "emoe_ipc_close",
@@ -151,6 +152,11 @@ def lib() -> ctypes.CDLL:
     L.emoe_plan_segments.argtypes = [_vp, _i32, _vp, _u64, ctypes.POINTER(_u64)]
     L.emoe_plan_device_status.restype = _i32
     L.emoe_plan_device_status.argtypes = [_vp, ctypes.POINTER(_i32)]
+    L.emoe_segments_validate.restype = _i32
+    L.emoe_segments_validate.argtypes = [_vp, _u64, ctypes.POINTER(_u64), _i32, ctypes.POINTER(_u64), _i32,
+                                         _i32, ctypes.POINTER(_u64)]
+    L.emoe_plan_validate.restype = _i32
+    L.emoe_plan_validate.argtypes = [_vp, _i32p, ctypes.POINTER(_u64)]
     L.emoe_plan_clear_device_status.restype = _i32
     L.emoe_plan_clear_device_status.argtypes = [_vp]
     L.emoe_plan_set_tuning.restype = _i32
@@ -360,6 +366,14 @@ class Plan:
                                             ctypes.byref(n)))
         return out
 
+    def validate(self) -> None:
+        """Host-side bounds and race check of the plan's segments; raises EmoeError (status 12)
+        naming the phase and segment if a run leaves its arena or two runs write one byte."""
+        ph, seg = _i32(-1), _u64(0)
+        code = lib().emoe_plan_validate(self._h, ctypes.byref(ph), ctypes.byref(seg))
+        if code != 0:
+            raise EmoeError(code, "%s (phase %d, segment %d)" % (strerror(code), ph.value, seg.value))
+
     def device_status(self) -> int:
         s = _i32()
         _check(lib().emoe_plan_device_status(self._h, ctypes.byref(s)))
@@ -542,6 +556,23 @@ class InplacePlan(Plan):
 
 
 IPC_HANDLE_BYTES = 64
+
+
+def segments_validate(segs: np.ndarray, arena_old, arena_new, must_tile: bool = False) -> int:
+    """emoe_segments_validate on a SEGMENT_DTYPE array; returns -1 if the list passes, else the
+    index of an offending segment."""
+    segs = np.ascontiguousarray(segs, dtype=SEGMENT_DTYPE)
+    ao = np.ascontiguousarray(arena_old, dtype=np.uint64)
+    an = np.ascontiguousarray(arena_new, dtype=np.uint64)
+    bad = _u64(0)
+    u64p = ctypes.POINTER(_u64)
+    code = lib().emoe_segments_validate(segs.ctypes.data_as(_vp), len(segs), ao.ctypes.data_as(u64p), len(ao),
+                                        an.ctypes.data_as(u64p), len(an), int(must_tile), ctypes.byref(bad))
+    if code == 0:
+        return -1
+    if code != 12:
+        _check(code)
+    return int(bad.value)
 
 
 def ipc_export(device_ptr: int):

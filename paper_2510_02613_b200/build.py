@@ -7,7 +7,7 @@ import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = ["planner.cpp", "capi.cpp", "vmm.cpp", "placement.cpp", "cache.cpp", "kernels.cu"]
+SOURCES = ["planner.cpp", "capi.cpp", "vmm.cpp", "placement.cpp", "cache.cpp", "validate.cpp", "kernels.cu"]
 HEADERS = ["planner.h", "kernels.h", "internal.h", os.path.join("..", "..", "include", "emoe.h")]
 OUT = os.path.join(HERE, "libemoe.so")
 

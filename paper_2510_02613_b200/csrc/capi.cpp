@@ -1179,6 +1179,32 @@ emoe_status_t emoe_plan_segments(const emoe_plan_t *p, int phase, emoe_segment_t
   return EMOE_OK;
 }
 
+emoe_status_t emoe_plan_validate(const emoe_plan_t *p, int32_t *bad_phase, uint64_t *bad_segment) {
+  if (!p) return EMOE_ERR_INVALID_ARG;
+  try {
+    for (int ph = 0; ph < 3; ++ph) {
+      if (p->inplace && ph != EMOE_PHASE_EXPERTS) continue;
+      std::vector<emoe_segment_t> v;
+      export_segments(p->hp, ph, &v);
+      const PhasePlan &pp = p->hp.phase[ph];
+      // weights must fill their new arenas exactly; not so the KV phase (unmapped blocks), the
+      // in-place step (kept slots) and expert arenas with the gap before their scale part
+      const bool tile = ph != EMOE_PHASE_KV && !p->inplace &&
+                        !(ph == EMOE_PHASE_EXPERTS && p->hp.expert_scale_bytes);
+      const emoe_status_t st = emoe_segments_validate(v.data(), v.size(), pp.arena_old.data(),
+                                                      (int32_t)pp.arena_old.size(), pp.arena_new.data(),
+                                                      (int32_t)pp.arena_new.size(), tile ? 1 : 0, bad_segment);
+      if (st != EMOE_OK) {
+        if (bad_phase) *bad_phase = ph;
+        return st;
+      }
+    }
+  } catch (const std::bad_alloc &) {
+    return EMOE_ERR_OOM;
+  }
+  return EMOE_OK;
+}
+
 emoe_status_t emoe_plan_device_status(const emoe_plan_t *p, int32_t *status) {
   if (!p || !status) return EMOE_ERR_INVALID_ARG;
   if (p->host_only) return EMOE_ERR_CUDA;
@@ -1329,6 +1355,7 @@ const char *emoe_strerror(emoe_status_t s) {
     case EMOE_ERR_UNSUPPORTED: return "unsupported configuration";
     case EMOE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
     case EMOE_ERR_TOO_LARGE: return "problem exceeds the fixed capacity of this entry point";
+    case EMOE_ERR_PLAN_CHECK: return "a copy run leaves its arena or two runs write the same byte";
   }
   return "unknown status";
 }

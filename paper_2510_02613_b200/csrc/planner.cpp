@@ -534,6 +534,7 @@ emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
   if (attn_replicas < 1) attn_replicas = 1;
   if ((uint64_t)n.tp * attn_replicas > EMOE_MAX_RANKS) return EMOE_ERR_UNSUPPORTED;
   hp->attn_replicas = attn_replicas;
+  hp->expert_scale_bytes = expert_scale_bytes;
   plan_attn(sh, o.tp, n.tp, (flags & EMOE_LAYOUT_FUSED_QKV) != 0, &hp->phase[EMOE_PHASE_ATTN]);
   replicate_attn(&hp->phase[EMOE_PHASE_ATTN], n.tp, attn_replicas);
   plan_kv(sh, o, n, std::move(pair_old), std::move(pair_new), (flags & EMOE_LAYOUT_KV_HEAD_MAJOR) != 0, hp);

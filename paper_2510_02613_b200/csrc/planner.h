@@ -70,6 +70,7 @@ struct HostPlan {
   emoe_shape_t shape;
   int ep_old, ep_new, tp_old, tp_new;
   uint32_t attn_replicas = 1;  // new attention arenas: tp_new per replica, replica after replica
+  uint64_t expert_scale_bytes = 0;  // > 0: expert arenas hold a scale array after a 256-byte-aligned gap
   PhasePlan phase[3];  // experts, attn, kv (kv.segs filled only when the head split is kept)
   KvPlan kv;
 };
