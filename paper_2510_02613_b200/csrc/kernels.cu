@@ -1011,7 +1011,6 @@ cudaError_t launch_vec_kv_copy(const SegTables &t, const RankPtrs &ptrs, uint32_
                                bool unbounded, cudaStream_t stream) {
   const uint64_t n_tiles = (uint64_t)kv.n_pairs * kv.n_lk;
   if (n_tiles == 0) return launch_vec_copy(t, ptrs, tile_bytes, unbounded ? 0xffffffffu : grid, stream);
-  if (t.n_units == 0 && n_tiles == 0) return cudaSuccess;
   VecKvParams p{};
   p.t = t;
   p.tile_bytes = tile_bytes;
