@@ -206,9 +206,10 @@ emoe_status_t emoe_plan_create_ex(const emoe_shape_t *shape, const emoe_config_t
  * The call only enqueues work on the stream: it neither synchronises nor
  * allocates.  The pointer arrays are read before the call returns.
  * Calls may be enqueued on any streams; at most 4 launches of the SAME phase of
- * the SAME plan may be in flight on the GPU at once (they claim work through
- * per-launch counters of which the plan has 4 per phase) - more must be
- * ordered by the caller.  Calls on one stream are always fine.  A call that is
+ * the SAME plan (a whole-step call counts as a phase of its own) may be
+ * enqueued and unfinished at once when they are on different streams (they
+ * claim work through per-launch counters of which the plan has 4 per phase,
+ * used in turn) - more must be ordered by the caller.  Calls on one stream are always fine.  A call that is
  * being captured into a CUDA graph uses no counter (its CTAs take their work
  * round-robin), so a graph never holds on to one and may be replayed beside
  * live calls.

@@ -558,6 +558,45 @@ def test_kv_delta_plan_recopies_blocks_written_during_the_migration():
         assert moved * 8 < p_all.stats(E.PHASE_KV)["bytes_moved"]      # the delta is small
 
 
+@pytest.mark.parametrize("name", ["c2_mid", "c4_large"])
+def test_one_plan_on_several_streams_at_once(name):
+    """The header allows up to four launches of one phase of one plan in flight at once (they
+    claim work through per-launch counters) and whole-step calls from several streams (they
+    share the plan's side stream).  Three streams run the same step into three sets of
+    destination arenas without any ordering between them, twice over; every set must equal
+    the oracle."""
+    from gpu_util import oracle_phase
+    wl = W.make_workload(name, n_layers=1)
+    with E.Plan(wl.shape, wl.old, wl.new) as plan:
+        src = [WD.alloc_filled(plan.arena_bytes(ph, E.SIDE_OLD), wl.seed, KINDS[ph]) for ph in range(3)]
+        want = []
+        for ph in range(3):
+            w = [np.full(n, WD.FILL_BYTE, np.uint8) for n in plan.arena_bytes(ph, E.SIDE_NEW)]
+            oracle_phase(wl, ph, [t.cpu().numpy() for t in src[ph]], w)
+            want.append(w)
+        sets = [[WD.alloc_const(plan.arena_bytes(ph, E.SIDE_NEW)) for ph in range(3)] for _ in range(3)]
+        streams = [torch.cuda.Stream() for _ in range(3)]
+        torch.cuda.synchronize()
+        for tuning in (dict(), dict(path=2, max_ctas=20)):
+            plan.set_tuning(**tuning)
+            for dst in sets:
+                for g in dst:
+                    for t in g:
+                        t.fill_(WD.FILL_BYTE)
+            torch.cuda.synchronize()
+            for rounds in range(2):
+                for st, dst in zip(streams, sets):
+                    plan.reshard_step(src, dst, st)
+                for st, dst in zip(streams, sets):          # and the per-phase calls on top
+                    plan.reshard_experts(src[0], dst[0], st)
+                torch.cuda.synchronize()                    # at most four unfinished launches per phase
+            assert plan.device_status() == 0
+            for k, dst in enumerate(sets):
+                for ph in range(3):
+                    for r, (t, w) in enumerate(zip(dst[ph], want[ph])):
+                        assert np.array_equal(t.cpu().numpy(), w), (tuning, k, ph, r)
+
+
 def test_kv_migration_while_a_second_stream_appends_tokens():
     """Scale while serving, for real this time: the whole-cache migration runs on one stream
     WHILE a second stream keeps appending tokens to the last block of every sequence (the
