@@ -613,7 +613,12 @@ def run_inplace(torch, E, wl, copy_all_ms, peak, reps=30):
     placements: the workload's own, and (when every expert is held once) the balanced
     placement that keeps the most experts in place.  Arena contents are left uninitialised:
     byte movement does not depend on values."""
-    out = {"dense_copy_all_ms": round(copy_all_ms, 4), "variants": []}
+    m_bytes = wl.shape.d_model * wl.shape.d_ff * wl.shape.elem_bytes * wl.shape.n_layers * 3
+    out = {"dense_copy_all_ms": round(copy_all_ms, 4),
+           # device memory an expert step needs while it runs: copy-all holds the old AND the new arenas
+           "dense_copy_all_peak_bytes": m_bytes * (sum(len(p) for p in wl.old.placement)
+                                                   + sum(len(p) for p in wl.new.placement)),
+           "variants": []}
     held_once = all(sum(e in p for p in wl.old.placement) == 1 for e in range(wl.shape.n_experts))
     wants = [("workload placement", [list(p) for p in wl.new.placement])]
     if held_once:
@@ -654,7 +659,8 @@ def run_inplace(torch, E, wl, copy_all_ms, peak, reps=30):
             "wanted": label, "experts_kept_in_place": sum(len(set(want[r]) & set(wl.old.placement[r]))
                                                           for r in range(min(len(want), wl.old.ep))),
             "expert_slots_wanted": sum(len(w) for w in want),
-            "bytes_moved": st["bytes_moved"], "ms": round(ms, 4), "min_ms": round(min(each), 4),
+            "bytes_moved": st["bytes_moved"], "peak_bytes": m_bytes * sum(plan.caps),
+            "ms": round(ms, 4), "min_ms": round(min(each), 4),
             "reshard_gbs": round(2 * st["bytes_moved"] / ms / 1e6, 1),
             "hbm_gbs": round(alg / ms / 1e6, 1), "frac_of_measured_peak": round(alg / ms / 1e6 / peak, 4),
             "speedup_over_copy_all": round(copy_all_ms / ms, 2), "device_status_ok": ok})
@@ -797,7 +803,7 @@ def run_exchange(args):
             new.append(WD.alloc_const([sn[rank]])[0] if rank < len(sn) else None)
         torch.cuda.synchronize()
         dist.barrier()
-        ex = exchange.Exchange(dist, plan, rank, old, new)
+        ex = exchange.Exchange(dist, plan, rank, old, new, whole_step=True)
         try:
             pulled = ex.bytes_pulled()
             for _ in range(args.warmup):
@@ -820,8 +826,7 @@ def run_exchange(args):
             dev = "cuda" if backend == "nccl" else "cpu"
             total_ms = replicas.job_time_ms(local_ms, dist, device=dev)
             status = plan.device_status()
-            n_launch = sum(plan.num_launches(ph) for ph in range(3)
-                           if rank < plan.num_ranks(ph, E.SIDE_NEW))
+            n_launch = plan.num_launches(E.PHASE_STEP)
             per_rank = [None] * world
             dist.all_gather_object(per_rank, dict(rank=rank, ms_per_step=round(local_ms / args.steps, 4),
                                                   bytes_written=pulled["written"],

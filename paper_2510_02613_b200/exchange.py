@@ -46,10 +46,14 @@ class Exchange:
     Set-up and tear-down talk to the other processes (all of them must create and close
     their Exchange together); step() only enqueues this rank's kernels."""
 
-    def __init__(self, dist, plan: "B.Plan", rank: int, old_arenas, new_arenas):
+    def __init__(self, dist, plan: "B.Plan", rank: int, old_arenas, new_arenas, whole_step: bool = False):
+        """whole_step: run the three phases through ONE emoe_reshard_step call (its launch sets
+        merged and side by side) instead of one call per phase."""
         self.dist, self.plan, self.rank = dist, plan, rank
+        self.whole_step = whole_step
         self.opened: dict = {}
         self.calls = []
+        self.step_src, self.step_dst = [], []
         plan.set_local_rank(rank)
         run = (plan.reshard_experts, plan.reshard_attn, plan.reshard_kv)
         try:
@@ -57,16 +61,22 @@ class Exchange:
                 n_old = plan.num_ranks(phase, B.SIDE_OLD)
                 n_new = plan.num_ranks(phase, B.SIDE_NEW)
                 pa = PeerArenas(dist, rank, n_old, old_arenas[phase], self.opened)
-                if rank >= n_new or new_arenas[phase] is None:
-                    continue                         # nothing of this phase lands here
-                dst = [new_arenas[phase] if r == rank else None for r in range(n_new)]
-                self.calls.append((run[phase], pa.ptrs, dst))
+                lands = rank < n_new and new_arenas[phase] is not None
+                dst = [new_arenas[phase] if (lands and r == rank) else None for r in range(n_new)]
+                self.step_src.append(pa.ptrs)
+                self.step_dst.append(dst)
+                if lands:                            # else nothing of this phase lands here
+                    self.calls.append((run[phase], pa.ptrs, dst))
         except Exception:
             self.close(barrier=False)
             raise
 
     def step(self, stream=None) -> None:
         """Enqueues this rank's share of the three phases on `stream`; no synchronisation."""
+        if self.whole_step:
+            if self.calls:
+                self.plan.reshard_step(self.step_src, self.step_dst, stream)
+            return
         for fn, src, dst in self.calls:
             fn(src, dst, stream)
 
@@ -91,7 +101,8 @@ class Exchange:
         self.plan.set_local_rank(-1)
 
 
-def exchange_step(dist, plan: "B.Plan", rank: int, old_arenas, new_arenas, stream=None) -> None:
+def exchange_step(dist, plan: "B.Plan", rank: int, old_arenas, new_arenas, stream=None,
+                  whole_step: bool = False) -> None:
     """Runs this rank's share of the three phases.
 
     old_arenas / new_arenas: per phase (experts, attn, kv) this process's own device tensor
@@ -102,7 +113,7 @@ def exchange_step(dist, plan: "B.Plan", rank: int, old_arenas, new_arenas, strea
     import torch
 
     dist.barrier()                                   # every old arena is complete
-    ex = Exchange(dist, plan, rank, old_arenas, new_arenas)
+    ex = Exchange(dist, plan, rank, old_arenas, new_arenas, whole_step=whole_step)
     try:
         ex.step(stream)
         (stream.synchronize() if stream is not None else torch.cuda.synchronize())

@@ -34,7 +34,7 @@ def _workload(world: int):
     return wl        # world 4: EP 2 -> 4, TP 1 -> 2 as defined
 
 
-def _worker(rank: int, world: int, port: int, out, force_bulk: bool = False):
+def _worker(rank: int, world: int, port: int, out, force_bulk: bool = False, whole_step: bool = False):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
     torch.cuda.set_device(0)
     dist.init_process_group("gloo", rank=rank, world_size=world)
@@ -58,7 +58,7 @@ def _worker(rank: int, world: int, port: int, out, force_bulk: bool = False):
                 old.append(mine)
                 new.append(WD.alloc_const([sn[rank]])[0] if rank < len(sn) else None)
             torch.cuda.synchronize()
-            exchange.exchange_step(dist, plan, rank, old, new)
+            exchange.exchange_step(dist, plan, rank, old, new, whole_step=whole_step)
             assert plan.device_status() == 0
             out.put((rank, [None if t is None else t.cpu().numpy() for t in new]))
         dist.barrier()
@@ -66,15 +66,16 @@ def _worker(rank: int, world: int, port: int, out, force_bulk: bool = False):
         dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("world,force_bulk", [(2, False), (4, False), (2, True)])
-def test_ranks_as_processes_pull_their_share(world, force_bulk):
+@pytest.mark.parametrize("world,force_bulk,whole_step", [(2, False, False), (4, False, False), (2, True, False),
+                                                         (4, False, True), (2, True, True)])
+def test_ranks_as_processes_pull_their_share(world, force_bulk, whole_step):
     import oracle
     from gpu_util import oracle_phase
     from workloads import device as WD
     ctx = mp.get_context("spawn")
     out = ctx.Queue()
     port = _free_port()
-    procs = [ctx.Process(target=_worker, args=(r, world, port, out, force_bulk)) for r in range(world)]
+    procs = [ctx.Process(target=_worker, args=(r, world, port, out, force_bulk, whole_step)) for r in range(world)]
     for p in procs:
         p.start()
     got = dict(out.get(timeout=300) for _ in range(world))
