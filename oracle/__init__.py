@@ -230,19 +230,23 @@ def reshard_experts_inplace(shape, old_slots, want, cap_new, arenas: Sequence[np
 
 # ---- compacting block table ---------------------------------------------------------------
 
-def compact_block_table(seq_lens, block_tokens: int, nb_new: int, in_use=()) -> np.ndarray:
+def compact_block_table(seq_lens, block_tokens: int, nb_new: int, in_use=(), old_table=None) -> np.ndarray:
     """The definition of "compacted": going through the sequences in order and through each
     sequence's blocks in order, every block gets the smallest block id of the destination
     pool that is neither in use there already nor handed out before (the paper leaves block
-    allocation across instances open, App. C).  Returns int32 [n_seqs, max blocks], -1 padded."""
+    allocation across instances open, App. C).  Returns int32 [n_seqs, max blocks], -1 padded.
+    old_table (same shape of mapped entries): the blocks are served in the order of their OLD
+    physical id instead, so that old and new addresses rise together."""
     need = [-(-int(n) // block_tokens) for n in seq_lens]
     out = np.full((len(need), max(need, default=0)), -1, dtype=np.int32)
     taken = set(int(x) for x in in_use)
-    for s, n in enumerate(need):
-        for j in range(n):
-            b = min(x for x in range(nb_new) if x not in taken)    # ValueError if the pool is full
-            out[s, j] = b
-            taken.add(b)
+    todo = [(s, j) for s, n in enumerate(need) for j in range(n)]
+    if old_table is not None:
+        todo.sort(key=lambda sj: int(old_table[sj[0]][sj[1]]))
+    for s, j in todo:
+        b = min(x for x in range(nb_new) if x not in taken)    # ValueError if the pool is full
+        out[s, j] = b
+        taken.add(b)
     return out
 
 

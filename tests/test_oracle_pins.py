@@ -766,3 +766,13 @@ def test_attn_replicas_each_equal_the_numpy_split(c, d, replicas):
             assert np.array_equal(dst[k * d + t], want[t]), (k, t)
     with pytest.raises(ValueError):
         oracle.reshard_attn(sh, c, d, src, dst[:-1], replicas=replicas)
+
+
+def test_compact_block_table_in_old_address_order_hand_written():
+    """Same two sequences; their old blocks are 7, 2, 5 and 3, 6.  Served in old-id order
+    (2, 3, 5, 6, 7) from the free ids 0, 2, 3, 5, 6: old 2 -> 0, 3 -> 2, 5 -> 3, 6 -> 5, 7 -> 6."""
+    old = np.array([[7, 2, 5], [3, 6, -1]], np.int32)
+    t = oracle.compact_block_table([5, 3], 2, 8, in_use=[1, 4], old_table=old)
+    assert t.tolist() == [[6, 0, 3], [2, 5, -1]]
+    pairs = sorted((int(old[s, j]), int(t[s, j])) for s in range(2) for j in range(3) if old[s, j] >= 0)
+    assert [b for _, b in pairs] == sorted(b for _, b in pairs)          # new ids rise with old ids
