@@ -607,31 +607,38 @@ def verify_layer(torch, E, plan, wl, src, dst, layer):
 # ---- KV phase into a compacting (identity-order) new table --------------------------------
 
 def run_kv_compacting(torch, E, W, WD, name, random_ms, reps=30):
-    """The KV phase of the workload once more, with the new block table in compacting order
-    (mapped blocks get the destination ids 0, 1, 2, ... in table order, as a scale-down that
-    packs the surviving pool would choose) instead of a random permutation: writes then walk
-    the new pool in address order too."""
-    wl = W.make_workload(name, new_order="identity")
+    """The KV phase of the workload once more, with the new block table COMPACTING the pool
+    (emoe_kv_compact_table: mapped blocks get the destination ids 0, 1, 2, ...) instead of a
+    random permutation - as a scale-down that packs the surviving pool would choose: once with
+    the ids handed out in table order, once in the order of the blocks' old physical ids, so
+    that the migration writes the new pool in address order as it reads the old one."""
+    import dataclasses
+    wl = W.make_workload(name)
+    B = wl.shape.kv_block_tokens
+    out = {"random_new_table_ms": round(random_ms, 4)}
     stream = torch.cuda.Stream()
-    with E.Plan(wl.shape, wl.old, wl.new) as plan:
-        src = WD.alloc_filled(plan.arena_bytes(E.PHASE_KV, E.SIDE_OLD), wl.seed, W.KIND_KV)
-        dst = WD.alloc_const(plan.arena_bytes(E.PHASE_KV, E.SIDE_NEW))
-        torch.cuda.synchronize()
-        for _ in range(3):
-            plan.reshard_kv(src, dst, stream)
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
-        ev[0].record(stream)
-        for i in range(reps):
-            plan.reshard_kv(src, dst, stream)
-            ev[i + 1].record(stream)
-        stream.synchronize()
-        ms = statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(reps))
-        st = plan.stats(E.PHASE_KV)
-        ok = plan.device_status() == 0
-    del src, dst
-    torch.cuda.empty_cache()
-    return {"ms": round(ms, 4), "gbs": round(2 * st["bytes_moved"] / ms / 1e6, 1),
-            "random_new_table_ms": round(random_ms, 4), "device_status_ok": ok}
+    for label, old_table in (("table_order", None), ("old_address_order", wl.old.block_table)):
+        table = E.kv_compact_table(B, wl.old.seq_lens, wl.new.kv_num_blocks, old_table=old_table)
+        w2 = dataclasses.replace(wl, new=dataclasses.replace(wl.new, block_table=table))
+        with E.Plan(w2.shape, w2.old, w2.new) as plan:
+            src = WD.alloc_filled(plan.arena_bytes(E.PHASE_KV, E.SIDE_OLD), w2.seed, W.KIND_KV)
+            dst = WD.alloc_const(plan.arena_bytes(E.PHASE_KV, E.SIDE_NEW))
+            torch.cuda.synchronize()
+            for _ in range(3):
+                plan.reshard_kv(src, dst, stream)
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+            ev[0].record(stream)
+            for i in range(reps):
+                plan.reshard_kv(src, dst, stream)
+                ev[i + 1].record(stream)
+            stream.synchronize()
+            ms = statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(reps))
+            st = plan.stats(E.PHASE_KV)
+            out[label] = {"ms": round(ms, 4), "gbs": round(2 * st["bytes_moved"] / ms / 1e6, 1),
+                          "device_status_ok": plan.device_status() == 0}
+        del src, dst
+        torch.cuda.empty_cache()
+    return out
 
 
 # ---- in-place expert step: only arrivals move ---------------------------------------------

@@ -691,13 +691,19 @@ void emoe_plan_cache_destroy(emoe_plan_cache_t *cache);
  * in_use [n_in_use]: blocks of the destination pool (size nb_new) that are already taken -
  * e.g. by sequences the new instance serves already - and must not be handed out; NULL /
  * 0 for a fresh pool, which yields the identity order 0, 1, 2, ...
+ * old_table (optional, [n_seqs][max_blocks]): the table the blocks are read through.  If
+ * given, the blocks are served in the order of their OLD physical id instead of table order:
+ * the free ids are the same, but old and new addresses then rise together, and a migration
+ * - which visits the blocks in old-pool order - reads AND writes in address order (measured
+ * on B200: the KV phase 0.8 to 1.3 % faster than with the ids handed out in table order).
  * table_out: [n_seqs][max_blocks], -1 padded; *n_mapped (optional): blocks assigned.
  * Errors: EMOE_ERR_BLOCK_TABLE (an in_use id out of range or listed twice, a sequence
- * longer than max_blocks blocks), EMOE_ERR_TOO_LARGE (not enough free blocks).
- * Host only.  Use the result as new_cfg->block_table of emoe_plan_create. */
+ * longer than max_blocks blocks, an unmapped old entry), EMOE_ERR_TOO_LARGE (not enough free
+ * blocks).  Host only.  Use the result as new_cfg->block_table of emoe_plan_create. */
 emoe_status_t emoe_kv_compact_table(int32_t block_tokens, int32_t n_seqs, int32_t max_blocks,
                                     const int32_t *seq_lens, int32_t nb_new, const int32_t *in_use,
-                                    int32_t n_in_use, int32_t *table_out, int32_t *n_mapped);
+                                    int32_t n_in_use, const int32_t *old_table, int32_t *table_out,
+                                    int32_t *n_mapped);
 
 /* ---- one rank per GPU: pull-based exchange --------------------------------
  *

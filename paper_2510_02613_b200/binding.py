@@ -172,7 +172,7 @@ def lib() -> ctypes.CDLL:
     L.emoe_plan_cache_destroy.restype = None
     L.emoe_plan_cache_destroy.argtypes = [_vp]
     L.emoe_kv_compact_table.restype = _i32
-    L.emoe_kv_compact_table.argtypes = [_i32, _i32, _i32, _i32p, _i32, _i32p, _i32, _i32p, _i32p]
+    L.emoe_kv_compact_table.argtypes = [_i32, _i32, _i32, _i32p, _i32, _i32p, _i32, _i32p, _i32p, _i32p]
     L.emoe_place_min_transfer.restype = _i32
     L.emoe_place_min_transfer.argtypes = [_i32, ctypes.POINTER(_Config), _i32, _i32p, _i32p, _i32p]
     L.emoe_plan_set_local_rank.restype = _i32
@@ -496,18 +496,28 @@ class PlanCache:
         self.close()
 
 
-def kv_compact_table(block_tokens: int, seq_lens, nb_new: int, in_use=(), max_blocks: Optional[int] = None):
+def kv_compact_table(block_tokens: int, seq_lens, nb_new: int, in_use=(), max_blocks: Optional[int] = None,
+                     old_table=None):
     """Destination block table [n_seqs, max_blocks] that packs the sequences' blocks into the
-    lowest free blocks of a pool of nb_new blocks (in_use: ids already taken there)."""
+    lowest free blocks of a pool of nb_new blocks (in_use: ids already taken there), in table
+    order or - with old_table - in the order of the blocks' old physical ids."""
     sl = _i32arr(seq_lens)
     need = [-(-int(n) // block_tokens) for n in sl]
     mb = max_blocks if max_blocks is not None else max(need, default=0)
+    old = None
+    if old_table is not None:
+        old = np.full((len(sl), max(mb, 1)), -1, dtype=np.int32)
+        src = np.asarray(old_table, dtype=np.int32).reshape(len(sl), -1)[:, :mb]
+        old[:, :src.shape[1]] = src
     out = np.full((len(sl), max(mb, 1)), -1, dtype=np.int32)
+    if mb == 0:
+        return out[:, :0]
     used = _i32arr(list(in_use))
     n = _i32()
-    _check(lib().emoe_kv_compact_table(block_tokens, len(sl), mb,
+    _check(lib().emoe_kv_compact_table(block_tokens, len(sl), max(mb, 1),
                                        sl.ctypes.data_as(_i32p) if sl.size else None, nb_new,
                                        used.ctypes.data_as(_i32p) if used.size else None, int(used.size),
+                                       old.ctypes.data_as(_i32p) if old is not None else None,
                                        out.ctypes.data_as(_i32p), ctypes.byref(n)))
     return out[:, :mb] if mb else out[:, :0]
 

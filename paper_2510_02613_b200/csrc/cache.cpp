@@ -5,6 +5,7 @@
 // and scale-down mirrors scale-up, App. E).  A plan is a pure function of the model shape,
 // the two configurations and the flags, so it can be kept and reused; only plans whose
 // inputs are byte-for-byte the same are shared.
+#include <algorithm>
 #include <cstdint>
 #include <cstring>
 #include <list>
@@ -135,10 +136,13 @@ void emoe_plan_cache_destroy(emoe_plan_cache_t *c) {
 }
 
 // New block table that packs the mapped blocks into the lowest free blocks of the
-// destination pool, in table order.
+// destination pool: in table order, or - given the old table - in the order of the blocks'
+// old physical ids, so that a migration that walks the old pool in address order also writes
+// the new pool in address order.
 emoe_status_t emoe_kv_compact_table(int32_t block_tokens, int32_t n_seqs, int32_t max_blocks,
                                     const int32_t *seq_lens, int32_t nb_new, const int32_t *in_use,
-                                    int32_t n_in_use, int32_t *table_out, int32_t *n_mapped) {
+                                    int32_t n_in_use, const int32_t *old_table, int32_t *table_out,
+                                    int32_t *n_mapped) {
   if (block_tokens < 1 || n_seqs < 0 || max_blocks < 0 || nb_new < 0 || n_in_use < 0) return EMOE_ERR_INVALID_ARG;
   if ((n_seqs && (!seq_lens || !table_out)) || (n_in_use && !in_use)) return EMOE_ERR_INVALID_ARG;
   try {
@@ -147,7 +151,8 @@ emoe_status_t emoe_kv_compact_table(int32_t block_tokens, int32_t n_seqs, int32_
       if (in_use[i] < 0 || in_use[i] >= nb_new || taken[in_use[i]]) return EMOE_ERR_BLOCK_TABLE;
       taken[in_use[i]] = 1;
     }
-    int32_t next = 0, mapped = 0;
+    // the mapped entries, as positions in the table, in the order in which they are served
+    std::vector<int64_t> todo;
     for (int32_t s = 0; s < n_seqs; ++s) {
       if (seq_lens[s] < 0) return EMOE_ERR_BLOCK_TABLE;
       const int64_t n = ((int64_t)seq_lens[s] + block_tokens - 1) / block_tokens;
@@ -155,13 +160,23 @@ emoe_status_t emoe_kv_compact_table(int32_t block_tokens, int32_t n_seqs, int32_
       int32_t *row = table_out + (int64_t)s * max_blocks;
       for (int64_t j = 0; j < max_blocks; ++j) row[j] = -1;
       for (int64_t j = 0; j < n; ++j) {
-        while (next < nb_new && taken[next]) ++next;
-        if (next >= nb_new) return EMOE_ERR_TOO_LARGE;   // the pool has fewer free blocks than needed
-        row[j] = next++;
-        ++mapped;
+        if (old_table && old_table[(int64_t)s * max_blocks + j] < 0) return EMOE_ERR_BLOCK_TABLE;
+        todo.push_back((int64_t)s * max_blocks + j);
       }
     }
-    if (n_mapped) *n_mapped = mapped;
+    if (old_table)
+      std::stable_sort(todo.begin(), todo.end(),
+                       [&](int64_t a, int64_t b) { return old_table[a] < old_table[b]; });
+    int32_t next = 0;
+    for (int64_t at : todo) {
+      while (next < nb_new && taken[next]) ++next;
+      if (next >= nb_new) {   // the pool has fewer free blocks than needed: hand out nothing
+        for (int64_t k = 0; k < (int64_t)n_seqs * max_blocks; ++k) table_out[k] = -1;
+        return EMOE_ERR_TOO_LARGE;
+      }
+      table_out[at] = next++;
+    }
+    if (n_mapped) *n_mapped = (int32_t)todo.size();
   } catch (const std::bad_alloc &) {
     return EMOE_ERR_OOM;
   }

@@ -65,7 +65,7 @@ int main(void) {
     if (emoe_plan_cache_get(cache, &sh, &oc, &nc, EMOE_PLAN_HOST_ONLY, NULL, &plan, &hit) != EMOE_OK || !hit) return 20;
     if (emoe_plan_cache_stats(cache, &hits, &misses, NULL, NULL) != EMOE_OK || hits != 1 || misses != 1) return 21;
     emoe_plan_cache_destroy(cache);
-    if (emoe_kv_compact_table(4, 1, 2, seq_lens, 3, in_use, 1, bt, &mapped) != EMOE_OK) return 22;
+    if (emoe_kv_compact_table(4, 1, 2, seq_lens, 3, in_use, 1, NULL, bt, &mapped) != EMOE_OK) return 22;
     if (bt[0] != 1 || bt[1] != 2 || mapped != 2) return 23;
   }
   printf("c abi ok\n");

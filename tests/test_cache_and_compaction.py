@@ -90,6 +90,25 @@ def test_compact_table_equals_the_definition(seed):
     assert np.array_equal(got, want)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_compact_table_in_old_address_order_equals_the_definition(seed):
+    rng = np.random.default_rng(100 + seed)
+    B = int(rng.integers(1, 9))
+    seq_lens = [int(x) for x in rng.integers(0, 40, size=int(rng.integers(1, 7)))]
+    need = sum(-(-n // B) for n in seq_lens)
+    nb_old, nb = need + int(rng.integers(0, 5)), need + int(rng.integers(0, 12))
+    old = W.make_block_table(W.rng.stream_key(seed, 3), seq_lens, B, nb_old) if need else np.zeros((len(seq_lens), 0), np.int32)
+    in_use = [int(x) for x in rng.permutation(nb)[:nb - need]][:int(rng.integers(0, nb - need + 1))]
+    got = E.kv_compact_table(B, seq_lens, nb, in_use, old_table=old)
+    want = oracle.compact_block_table(seq_lens, B, nb, in_use, old_table=old)
+    assert np.array_equal(got, want)
+    pairs = sorted((int(o), int(n)) for o, n in zip(old.reshape(-1), got.reshape(-1)) if o >= 0)
+    assert [n for _, n in pairs] == sorted(n for _, n in pairs)        # old and new ids rise together
+    # the set of ids handed out does not depend on the order they are served in
+    plain = E.kv_compact_table(B, seq_lens, nb, in_use)
+    assert sorted(int(x) for x in got.reshape(-1) if x >= 0) == sorted(int(x) for x in plain.reshape(-1) if x >= 0)
+
+
 def test_compact_table_properties():
     """What "compacted" means, checked without the oracle: the blocks handed out are exactly
     the n smallest free ids, they increase along (sequence, block), a fresh pool gives the
