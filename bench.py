@@ -61,10 +61,10 @@ def load_traffic():
     return t.get("captures", {})
 
 
-def traffic_per_launch(traffic, wl_name, kernel, full_layers):
-    """Read + written DRAM bytes of one launch of `kernel` at full size (kernel None: of all
-    kernels of one step): the capture's bytes scaled by layers (every layer has identical
-    units, so traffic grows in proportion)."""
+def traffic_split(traffic, wl_name, kernel, full_layers):
+    """(read, written) DRAM bytes of one launch of `kernel` at full size (kernel None: of all
+    kernels of one step), or None: the capture's bytes scaled by layers (every layer has
+    identical units, so traffic grows in proportion)."""
     cap = traffic.get({"c5_overlap": "c3_fine"}.get(wl_name, wl_name))   # the overlap case runs the c3 reshard
     if not cap:
         return None
@@ -72,8 +72,16 @@ def traffic_per_launch(traffic, wl_name, kernel, full_layers):
     pick = list(ks.values()) if kernel is None else [ks[kernel]] if kernel in ks else []
     if not pick:
         return None
-    per = sum((k["dram_bytes_read"] + k["dram_bytes_write"]) / max(k["launches"], 1) for k in pick)
-    return int(per * full_layers / cap["layers"])
+    scale = full_layers / cap["layers"]
+    rd = sum(k["dram_bytes_read"] / max(k["launches"], 1) for k in pick)
+    wr = sum(k["dram_bytes_write"] / max(k["launches"], 1) for k in pick)
+    return int(rd * scale), int(wr * scale)
+
+
+def traffic_per_launch(traffic, wl_name, kernel, full_layers):
+    """Read + written DRAM bytes of one launch (see traffic_split), or None."""
+    t = traffic_split(traffic, wl_name, kernel, full_layers)
+    return None if t is None else t[0] + t[1]
 
 
 def record_traffic(args):
@@ -297,6 +305,11 @@ def config_rooflines(E, plan, wl, step_ms, phase_ms, peak, peak_kind, traffic, f
     out = {"step": roofline_block(" + ".join(names) + (" (vector and KV work in one kernel)" if fused else ""),
                                   sum(alg), step_ms, peak, peak_kind, tr(None)),
            "kernels": []}
+    # read and written bytes apart: a source that feeds several destinations must show up once
+    out["step"]["algorithmic_bytes_read"] = sum(x["bytes_read"] for x in st)
+    out["step"]["algorithmic_bytes_written"] = sum(x["bytes_moved"] for x in st)
+    split = None if cut else traffic_split(traffic, wl.name, None, full_layers)
+    out["step"]["traffic_read"], out["step"]["traffic_written"] = split if split else (None, None)
     if len(names) == 1:
         out["kernels"].append(dict(out["step"], kernel=names[0], timed_as="the whole step (one launch)"))
         return out
