@@ -165,7 +165,8 @@ def test_argument_errors_launch_nothing():
 
 def _step_on_host_buffers(wl, host_step):
     from gpu_util import oracle_phase
-    with E.Plan(wl.shape, wl.old, wl.new, host_step=host_step) as plan:
+    with E.Plan(wl.shape, wl.old, wl.new, host_step=host_step, fused_w13=wl.fused_w13,
+                kv_head_major=wl.kv_head_major, fused_qkv=wl.fused_qkv, attn_replicas=wl.attn_replicas) as plan:
         h_src, h_dst, d_src, d_dst, want = [], [], [], [], []
         for phase in range(3):
             so, sn = plan.arena_bytes(phase, E.SIDE_OLD), plan.arena_bytes(phase, E.SIDE_NEW)
@@ -195,6 +196,16 @@ def _step_on_host_buffers(wl, host_step):
 @pytest.mark.parametrize("host_step", [False, True], ids=["serial", "pipelined"])
 def test_step_on_host_buffers_matches_oracle(host_step):
     _step_on_host_buffers(W.make_workload("c1_tiny"), host_step)
+
+
+def test_host_step_with_layout_options():
+    """The host-buffer step with attention replicas and a fused qkv matrix (pipelined), and
+    with scale tensors (whose arenas are not layer-major: the step then runs serially)."""
+    wl = W.make_workload("c1_tiny", n_layers=6)
+    _step_on_host_buffers(R(wl, attn_replicas=3, fused_qkv=True), True)
+    scaled = R(wl, shape=R(wl.shape, elem_bytes=1, expert_scale_bytes=40))
+    _step_on_host_buffers(scaled, True)
+    _step_on_host_buffers(scaled, False)
 
 
 def test_pipelined_host_step_with_a_ragged_last_chunk():
