@@ -481,6 +481,7 @@ OVERLAP_POINTS = (
     dict(bw_limit_gbs=2500), dict(bw_limit_gbs=1500), dict(bw_limit_gbs=3500, bulk_hints=2),
     dict(max_ctas=37, bw_limit_gbs=3000), dict(max_ctas=24, bulk_stages=2), dict(max_ctas=16, bw_limit_gbs=1000),
     dict(max_ctas=1000000, bulk_tile_bytes=16384, bulk_stages=12),   # one short-lived CTA per unit
+    dict(path=3),                                                    # driver copies on the copy engines: no SM taken
 )
 
 

@@ -605,11 +605,16 @@ typedef struct {
                            /* kernel keeps one CTA per SM for the whole launch and  */
                            /* a live kernel loses those SMs: 16 keeps a concurrent  */
                            /* GEMM within 1.5x on B200; more than the default (74)  */
-                           /* and fewer than all SMs only hurts both sides          */
+                           /* and fewer than all SMs only hurts both sides.  (path  */
+                           /* = 3 takes no SM at all, at the copy engines' rate.)   */
   int32_t bulk_tile_bytes; /* bytes per shared-memory stage of the bulk kernel      */
   int32_t bulk_stages;     /* stages of the bulk kernel's ring                      */
   int32_t path;            /* 0 default routing, 1 force the vector kernel for all  */
-                           /* segments, 2 force the bulk kernel where aligned       */
+                           /* segments, 2 force the bulk kernel where aligned, 3    */
+                           /* one driver copy (cudaMemcpy2DAsync, copy engines) per */
+                           /* segment and destination instead of the kernels - no   */
+                           /* SM is taken from a kernel that runs beside it; a KV   */
+                           /* head re-split still uses its kernel                   */
   int32_t kv_mode;         /* 0 default, 1 direct, 2 staged through shared memory,  */
                            /* 3 tiled TMA loads and stores, 4 direct without the    */
                            /* row-mapped fast path                                  */

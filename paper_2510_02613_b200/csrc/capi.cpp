@@ -569,7 +569,31 @@ emoe_status_t run_vec(const emoe_plan *p, int set, const RankPtrs &ptrs, cudaStr
                                      ptrs, kVecTile, vec_grid(p), st));
 }
 
+// path = 3: the segments of a phase as driver copies - one (strided) device-to-device copy
+// per segment and destination, which the driver hands to the GPU's copy engines: no SM, no
+// shared memory is taken from a kernel that runs beside the reshard.  Only for comparison and
+// for sharing the GPU: a replicated source is read once per destination, every segment is an
+// API call, and the rate is the copy engines'.
+emoe_status_t run_segments_by_copy_engine(const emoe_plan *p, int phase, const RankPtrs &ptrs, cudaStream_t st) {
+  const PhasePlan &pp = p->hp.phase[phase];
+  for (const Segment &s : pp.segs)
+    for (uint32_t j = 0; j < s.n_dst; ++j) {
+      const Dst &d = pp.dsts[s.dst_first + j];
+      if (p->local_rank >= 0 && (int)d.rank != p->local_rank) continue;
+      const uint8_t *src = ptrs.src[s.src_rank] + s.src_off;
+      uint8_t *dst = ptrs.dst[d.rank] + d.off;
+      cudaError_t e;
+      if (s.n_runs == 1)
+        e = cudaMemcpyAsync(dst, src, s.run_bytes, cudaMemcpyDeviceToDevice, st);
+      else
+        e = cudaMemcpy2DAsync(dst, d.pitch, src, s.src_pitch, s.run_bytes, s.n_runs, cudaMemcpyDeviceToDevice, st);
+      if (e != cudaSuccess) return cuda_status(e);
+    }
+  return EMOE_OK;
+}
+
 emoe_status_t run_segments(const emoe_plan *p, int phase, const RankPtrs &ptrs, cudaStream_t st) {
+  if (p->tuning.path == 3 && phase < 3) return run_segments_by_copy_engine(p, phase, ptrs, st);
   const emoe_status_t rc = run_bulk(p, phase, ptrs, st);
   return rc != EMOE_OK ? rc : run_vec(p, phase, ptrs, st);
 }
@@ -835,7 +859,7 @@ emoe_status_t emoe_reshard_step(const emoe_plan_t *p, const void *const *const s
   cudaStream_t st = (cudaStream_t)stream;
   const KvPlan &kv = p->hp.kv;
   emoe_status_t rc = EMOE_OK;
-  if (!p->merged) {  // too many ranks for one pointer table: phase by phase
+  if (!p->merged || p->tuning.path == 3) {  // too many ranks for one pointer table, or driver copies: phase by phase
     for (int ph = 0; rc == EMOE_OK && ph < 3; ++ph) rc = run_segments(p, ph, ph_ptrs[ph], st);
     if (rc == EMOE_OK && kv.head_split_changes) {
       KvTables t = kv_tables(kv, p->d_pair_old, p->d_pair_new, p->local_rank);
@@ -1140,6 +1164,11 @@ emoe_status_t emoe_plan_stats(const emoe_plan_t *p, int phase, uint64_t *bytes_m
 
 emoe_status_t emoe_plan_num_launches(const emoe_plan_t *p, int phase, int32_t *n) {
   if (!p || !n || phase < 0 || phase > EMOE_PHASE_STEP) return EMOE_ERR_INVALID_ARG;
+  if (p->tuning.path == 3) {  // driver copies: the only kernel left is a KV head re-split
+    const bool kv_here = phase == EMOE_PHASE_KV || phase == EMOE_PHASE_STEP;
+    *n = kv_here && p->hp.kv.head_split_changes && !p->hp.kv.pair_old.empty() ? 1 : 0;
+    return EMOE_OK;
+  }
   if (phase == EMOE_PHASE_STEP) {  // launches of one emoe_reshard_step call
     const int kv_pairs = p->hp.kv.head_split_changes && !p->hp.kv.pair_old.empty() ? 1 : 0;
     int k = 0;
@@ -1254,7 +1283,7 @@ emoe_status_t emoe_plan_clear_device_status(emoe_plan_t *p) {
 emoe_status_t emoe_plan_set_tuning(emoe_plan_t *p, const emoe_tuning_t *t) {
   if (!p || !t) return EMOE_ERR_INVALID_ARG;
   if (t->max_ctas < 0 || t->bulk_tile_bytes < 0 || t->bulk_stages < 0 || t->path < 0 ||
-      t->path > 2 || t->kv_mode < 0 || t->kv_mode > 4 || t->bulk_hints < 0 ||
+      t->path > 3 || t->kv_mode < 0 || t->kv_mode > 4 || t->bulk_hints < 0 ||
       t->bulk_hints > 4 || t->kv_order < 0 || t->kv_order > 3 || t->unit_order < 0 ||
       t->unit_order > 3 || t->wait_limit_us < -1 || t->bw_limit_gbs < 0 || t->bulk_min_run < 0 ||
       t->serial < 0 || t->serial > 2)

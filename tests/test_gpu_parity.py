@@ -60,7 +60,7 @@ TUNINGS = [dict(path=1), dict(path=2), dict(bulk_tile_bytes=8192, bulk_stages=3)
            dict(unit_order=3, path=2, max_ctas=5), dict(path=2, max_ctas=1),
            dict(serial=1, path=2), dict(serial=2), dict(bw_limit_gbs=300, path=2),
            dict(bw_limit_gbs=4000, path=2, max_ctas=16), dict(bulk_min_run=256, path=2),
-           dict(bulk_min_run=1024), dict(wait_limit_us=2000000, path=2)]
+           dict(bulk_min_run=1024), dict(wait_limit_us=2000000, path=2), dict(path=3), dict(path=3, max_ctas=8)]
 
 
 @pytest.mark.parametrize("tuning", TUNINGS, ids=lambda t: "-".join("%s%s" % kv for kv in t.items()))
