@@ -69,6 +69,8 @@ def traffic_split(traffic, wl_name, kernel, full_layers):
     if not cap:
         return None
     ks = cap.get("kernels", {})
+    if kernel is not None and kernel not in ks:
+        ks = cap.get("phase_kernels", {})       # a kernel that only the per-phase entry points launch
     pick = list(ks.values()) if kernel is None else [ks[kernel]] if kernel in ks else []
     if not pick:
         return None
@@ -117,9 +119,16 @@ def record_traffic(args):
     t["note"] = ("DRAM counters (dram__bytes_read.sum / dram__bytes_write.sum, summed over the captured "
                  "launches) of small cuts of the workloads; bench.py scales them by layers and drops them "
                  "when the kernel sources no longer hash to kernel_sources_sha256")
-    t["captures"][args.workload] = {"layers": args.layers, "command": args.traffic_command or "",
-                                    "kernels": {n: {k: (int(v) if k != "duration_us" else round(v, 1))
-                                                    for k, v in d.items()} for n, d in kernels.items()}}
+    new = {n: {k: (int(v) if k != "duration_us" else round(v, 1)) for k, v in d.items()}
+           for n, d in kernels.items()}
+    old = t["captures"].get(args.workload)
+    if args.traffic_merge and old and old.get("layers") == args.layers:
+        # kernels of the per-phase entry points, captured apart from the whole-step kernels
+        old.setdefault("phase_kernels", {}).update(new)
+        old["phase_command"] = args.traffic_command or ""
+    else:
+        t["captures"][args.workload] = {"layers": args.layers, "command": args.traffic_command or "",
+                                        "kernels": new}
     with open(TRAFFIC_FILE, "w") as f:
         json.dump(t, f, indent=1, sort_keys=True)
         f.write("\n")
@@ -318,8 +327,10 @@ def config_rooflines(E, plan, wl, step_ms, phase_ms, peak, peak_kind, traffic, f
         k = kernels_of(w)
         if len(k) != 1 or phase_ms[ph] <= 0:
             continue
-        b = roofline_block(k[0], alg[ph], phase_ms[ph], peak, peak_kind,
-                           tr(k[0]) if k[0] == "bulk_copy_kernel" and work["ring_units"] == w["ring_units"] else None)
+        # the ring kernel's capture is the whole step's launch: it stands for a phase only if
+        # that phase is all the ring work of the step
+        same = k[0] != "bulk_copy_kernel" or work["ring_units"] == w["ring_units"]
+        b = roofline_block(k[0], alg[ph], phase_ms[ph], peak, peak_kind, tr(k[0]) if same else None)
         b["timed_as"] = "the %s phase through its own entry point" % pname
         out["kernels"].append(b)
     return out
@@ -931,6 +942,9 @@ def main():
                     help="do not run: parse `ncu -i X.ncu-rep --page raw --csv` of a capture of "
                          "`bench.py --only-main --steps-only --workload W --layers N` into profiles/traffic.json")
     ap.add_argument("--traffic-command", default=None, help="the capture's command line, stored with --record-traffic")
+    ap.add_argument("--traffic-merge", action="store_true",
+                    help="with --record-traffic: add the capture's kernels to the workload's entry as the kernels "
+                         "of the per-phase entry points instead of replacing the entry")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "emoe" else args.warmup
     if args.record_traffic:
