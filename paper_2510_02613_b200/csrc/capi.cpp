@@ -582,11 +582,16 @@ emoe_status_t run_segments_by_copy_engine(const emoe_plan *p, int phase, const R
       if (p->local_rank >= 0 && (int)d.rank != p->local_rank) continue;
       const uint8_t *src = ptrs.src[s.src_rank] + s.src_off;
       uint8_t *dst = ptrs.dst[d.rank] + d.off;
-      cudaError_t e;
-      if (s.n_runs == 1)
-        e = cudaMemcpyAsync(dst, src, s.run_bytes, cudaMemcpyDeviceToDevice, st);
-      else
+      // a strided copy takes pitches below 2 GiB; runs that are further apart go one by one
+      const bool strided = s.n_runs > 1 && d.pitch < (1ull << 31) && s.src_pitch < (1ull << 31);
+      cudaError_t e = cudaSuccess;
+      if (strided) {
         e = cudaMemcpy2DAsync(dst, d.pitch, src, s.src_pitch, s.run_bytes, s.n_runs, cudaMemcpyDeviceToDevice, st);
+      } else {
+        for (uint32_t r = 0; e == cudaSuccess && r < s.n_runs; ++r)
+          e = cudaMemcpyAsync(dst + (uint64_t)r * d.pitch, src + (uint64_t)r * s.src_pitch, s.run_bytes,
+                              cudaMemcpyDeviceToDevice, st);
+      }
       if (e != cudaSuccess) return cuda_status(e);
     }
   return EMOE_OK;
