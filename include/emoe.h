@@ -203,6 +203,15 @@ emoe_status_t emoe_plan_create_ex(const emoe_shape_t *shape, const emoe_config_t
  * cuda_stream: a cudaStream_t (NULL = legacy default stream).
  * Arenas are caller-owned, sized by emoe_plan_arena_bytes, 16-byte aligned,
  * and no source arena may intersect a destination arena (out of place).
+ * One exception, the paper's zero-copy case (Sec. 5.2: with TP kept, attention
+ * weights and KV cache stay where they are and the new configuration goes on
+ * using them): when a phase changes nothing - same rank count, same arena
+ * sizes, every byte written comes from the same offset of the same rank index
+ * (TP kept and, for the KV cache, block table and pool size kept; for experts,
+ * placement kept) - the caller may pass dst[r] == src[r] for EVERY rank; the
+ * call then returns EMOE_OK and enqueues nothing for that phase.  Any other
+ * intersection is still EMOE_ERR_OVERLAP.  emoe_plan_phase_is_identity tells
+ * whether a phase qualifies.
  * The call only enqueues work on the stream: it neither synchronises nor
  * allocates.  The pointer arrays are read before the call returns.
  * Calls may be enqueued on any streams; at most 4 launches of the SAME phase of
@@ -227,6 +236,13 @@ emoe_status_t emoe_reshard_experts(const emoe_plan_t *plan, const void *const *s
  */
 emoe_status_t emoe_reshard_attn(const emoe_plan_t *plan, const void *const *src,
                                 void *const *dst, void *cuda_stream);
+
+/*
+ * emoe_plan_phase_is_identity - 1 when the phase moves every byte onto its own
+ * place (see the zero-copy exception under emoe_reshard_experts; Sec. 5.2),
+ * 0 when not, -1 on a bad argument.  Pure host query.
+ */
+int32_t emoe_plan_phase_is_identity(const emoe_plan_t *plan, int32_t phase);
 
 /*
  * emoe_reshard_kv - paged KV cache head re-split and re-paging (Sec. 5.2

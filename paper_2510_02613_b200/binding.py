@@ -80,6 +80,7 @@ EXPORTS = ("emoe_plan_create", "emoe_plan_create_ex", "emoe_reshard_experts", "e
            "emoe_plan_slot_table", "emoe_reshard_experts_inplace",
            "emoe_reshard_step_host", "emoe_plan_destroy", "emoe_plan_num_ranks",
            "emoe_plan_arena_bytes", "emoe_plan_stats", "emoe_plan_num_launches", "emoe_plan_launch_work",
+           "emoe_plan_phase_is_identity",
            "emoe_plan_segments",
            "emoe_plan_device_status", "emoe_plan_clear_device_status", "emoe_plan_set_tuning",
            "emoe_segments_validate", "emoe_plan_validate",
@@ -146,6 +147,8 @@ def lib() -> ctypes.CDLL:
     L.emoe_plan_stats.argtypes = [_vp, _i32] + [ctypes.POINTER(_u64)] * 3
     L.emoe_plan_num_launches.restype = _i32
     L.emoe_plan_num_launches.argtypes = [_vp, _i32, ctypes.POINTER(_i32)]
+    L.emoe_plan_phase_is_identity.restype = _i32
+    L.emoe_plan_phase_is_identity.argtypes = [_vp, _i32]
     L.emoe_plan_launch_work.restype = _i32
     L.emoe_plan_launch_work.argtypes = [_vp, _i32] + [ctypes.POINTER(_u64)] * 3
     L.emoe_plan_segments.restype = _i32
@@ -349,6 +352,14 @@ class Plan:
         n = _i32()
         _check(lib().emoe_plan_num_launches(self._h, phase, ctypes.byref(n)))
         return n.value
+
+    def phase_is_identity(self, phase: int) -> bool:
+        """True when the phase moves every byte onto its own place: src arenas may then be
+        passed as dst arenas and nothing is launched (the zero-copy case, Sec. 5.2)."""
+        r = lib().emoe_plan_phase_is_identity(self._h, phase)
+        if r < 0:
+            raise EmoeError(1, strerror(1))
+        return bool(r)
 
     def launch_work(self, phase: int) -> dict:
         """Work items per kind of kernel for one call of this phase (PHASE_STEP: a whole step)."""

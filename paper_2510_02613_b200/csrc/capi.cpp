@@ -480,13 +480,22 @@ int ranks_of(const emoe_plan *p, int phase, int side) {
 }
 
 // Host-side argument checks of a reshard call; fills the by-value pointer table.
+// *zero_copy (optional) is set when the phase changes nothing AND the caller passed, for every
+// rank, the very arena it already has (dst[r] == src[r]): the paper's zero-copy case - the new
+// configuration goes on using the memory in place and nothing is launched.
 emoe_status_t check_arenas(const emoe_plan *p, int phase, const void *const *src, void *const *dst,
-                           RankPtrs *out) {
+                           RankPtrs *out, bool *zero_copy = nullptr) {
+  if (zero_copy) *zero_copy = false;
   if (!p || !src || !dst || p->inplace) return EMOE_ERR_INVALID_ARG;
   if (p->host_only) return EMOE_ERR_CUDA;
   const PhasePlan &pp = p->hp.phase[phase];
   const int ns = ranks_of(p, phase, EMOE_SIDE_OLD), nd = ranks_of(p, phase, EMOE_SIDE_NEW);
   std::memset(out, 0, sizeof(*out));
+  if (zero_copy && pp.identity && ns == nd) {
+    bool same = true;
+    for (int r = 0; r < ns; ++r) same = same && src[r] == dst[r] && (src[r] || !pp.arena_old[r]);
+    if (same) { *zero_copy = true; return EMOE_OK; }
+  }
   // With a local rank set, only that rank's destination arena and the source arenas its
   // work reads are needed; the other entries may be NULL and are never dereferenced.
   const bool local = p->local_rank >= 0;
@@ -823,8 +832,9 @@ emoe_status_t emoe_reshard_experts(const emoe_plan_t *p, const void *const *src,
                                    void *stream) {
   TraceRange trace("emoe_reshard_experts");
   RankPtrs ptrs;
-  emoe_status_t st = check_arenas(p, EMOE_PHASE_EXPERTS, src, dst, &ptrs);
-  if (st != EMOE_OK) return st;
+  bool zero_copy = false;
+  emoe_status_t st = check_arenas(p, EMOE_PHASE_EXPERTS, src, dst, &ptrs, &zero_copy);
+  if (st != EMOE_OK || zero_copy) return st;
   return run_segments(p, EMOE_PHASE_EXPERTS, ptrs, (cudaStream_t)stream);
 }
 
@@ -832,17 +842,24 @@ emoe_status_t emoe_reshard_attn(const emoe_plan_t *p, const void *const *src, vo
                                 void *stream) {
   TraceRange trace("emoe_reshard_attn");
   RankPtrs ptrs;
-  emoe_status_t st = check_arenas(p, EMOE_PHASE_ATTN, src, dst, &ptrs);
-  if (st != EMOE_OK) return st;
+  bool zero_copy = false;
+  emoe_status_t st = check_arenas(p, EMOE_PHASE_ATTN, src, dst, &ptrs, &zero_copy);
+  if (st != EMOE_OK || zero_copy) return st;
   return run_segments(p, EMOE_PHASE_ATTN, ptrs, (cudaStream_t)stream);
+}
+
+int32_t emoe_plan_phase_is_identity(const emoe_plan_t *p, int32_t phase) {
+  if (!p || phase < 0 || phase > 2 || p->inplace) return -1;
+  return p->hp.phase[phase].identity ? 1 : 0;
 }
 
 emoe_status_t emoe_reshard_kv(const emoe_plan_t *p, const void *const *src, void *const *dst,
                               void *stream) {
   TraceRange trace("emoe_reshard_kv");
   RankPtrs ptrs;
-  emoe_status_t st = check_arenas(p, EMOE_PHASE_KV, src, dst, &ptrs);
-  if (st != EMOE_OK) return st;
+  bool zero_copy = false;
+  emoe_status_t st = check_arenas(p, EMOE_PHASE_KV, src, dst, &ptrs, &zero_copy);
+  if (st != EMOE_OK || zero_copy) return st;
   if (!p->hp.kv.head_split_changes) return run_segments(p, EMOE_PHASE_KV, ptrs, (cudaStream_t)stream);
   const KvPlan &kv = p->hp.kv;
   KvTables t = kv_tables(kv, p->d_pair_old, p->d_pair_new, p->local_rank);
@@ -856,16 +873,21 @@ emoe_status_t emoe_reshard_step(const emoe_plan_t *p, const void *const *const s
   TraceRange trace("emoe_reshard_step");
   if (!p || !src || !dst || p->inplace) return EMOE_ERR_INVALID_ARG;
   RankPtrs ph_ptrs[3];
+  bool zero_copy[3], any_zero_copy = false;
   for (int ph = 0; ph < 3; ++ph) {  // every argument is checked before anything is enqueued
     if (!src[ph] || !dst[ph]) return EMOE_ERR_INVALID_ARG;
-    const emoe_status_t st = check_arenas(p, ph, src[ph], dst[ph], &ph_ptrs[ph]);
+    const emoe_status_t st = check_arenas(p, ph, src[ph], dst[ph], &ph_ptrs[ph], &zero_copy[ph]);
     if (st != EMOE_OK) return st;
+    any_zero_copy = any_zero_copy || zero_copy[ph];
   }
   cudaStream_t st = (cudaStream_t)stream;
   const KvPlan &kv = p->hp.kv;
   emoe_status_t rc = EMOE_OK;
-  if (!p->merged || p->tuning.path == 3) {  // too many ranks for one pointer table, or driver copies: phase by phase
-    for (int ph = 0; rc == EMOE_OK && ph < 3; ++ph) rc = run_segments(p, ph, ph_ptrs[ph], st);
+  // Phase by phase: too many ranks for one pointer table, driver copies, or a phase that stays
+  // where it is (zero-copy: that phase launches nothing).
+  if (!p->merged || p->tuning.path == 3 || any_zero_copy) {
+    for (int ph = 0; rc == EMOE_OK && ph < 3; ++ph)
+      if (!zero_copy[ph]) rc = run_segments(p, ph, ph_ptrs[ph], st);
     if (rc == EMOE_OK && kv.head_split_changes) {
       KvTables t = kv_tables(kv, p->d_pair_old, p->d_pair_new, p->local_rank);
       rc = cuda_status(launch_kv_copy(t, ph_ptrs[2], kv_mode(p), cta_budget(p), p->tuning.max_ctas <= 0,

@@ -504,6 +504,16 @@ void replicate_attn(PhasePlan *pp, int d, uint32_t replicas) {
   }
 }
 
+bool phase_is_identity(const PhasePlan &pp) {
+  if (pp.arena_old != pp.arena_new) return false;
+  for (const Segment &s : pp.segs) {
+    if (s.n_dst != 1) return false;
+    const Dst &d = pp.dsts[s.dst_first];
+    if (d.rank != s.src_rank || d.off != s.src_off || (s.n_runs > 1 && d.pitch != s.src_pitch)) return false;
+  }
+  return true;
+}
+
 emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
                               const emoe_config_t &n, uint32_t flags, uint64_t expert_scale_bytes,
                               uint32_t attn_replicas, HostPlan *hp) {
@@ -538,6 +548,8 @@ emoe_status_t build_host_plan(const emoe_shape_t &sh, const emoe_config_t &o,
   plan_attn(sh, o.tp, n.tp, (flags & EMOE_LAYOUT_FUSED_QKV) != 0, &hp->phase[EMOE_PHASE_ATTN]);
   replicate_attn(&hp->phase[EMOE_PHASE_ATTN], n.tp, attn_replicas);
   plan_kv(sh, o, n, std::move(pair_old), std::move(pair_new), (flags & EMOE_LAYOUT_KV_HEAD_MAJOR) != 0, hp);
+  for (int ph = 0; ph < 3; ++ph) hp->phase[ph].identity = phase_is_identity(hp->phase[ph]);
+  if (hp->kv.head_split_changes) hp->phase[EMOE_PHASE_KV].identity = false;
   return EMOE_OK;
 }
 

@@ -40,6 +40,10 @@ struct PhasePlan {
   std::vector<Dst> dsts;
   std::vector<uint64_t> arena_old, arena_new;  // bytes per rank
   uint64_t bytes_moved = 0, bytes_read = 0;
+  // Every byte the phase writes comes from the same offset of the same rank index, and the
+  // arenas have the same sizes: the phase changes nothing (TP kept and, for the KV cache, the
+  // block table kept - the paper's zero-copy case).  Set by build_host_plan.
+  bool identity = false;
 };
 
 // KV phase when the head split changes: block pairs + shape constants.

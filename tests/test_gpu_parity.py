@@ -12,7 +12,7 @@ import oracle
 import paper_2510_02613_b200 as E
 import workloads as W
 from workloads import device as WD
-from gpu_util import KINDS, check_phase_full, check_phase_layers, check_step_full, run_phase
+from gpu_util import KINDS, check_phase_full, check_phase_layers, check_step_full, make_plan, run_phase
 
 pytestmark = pytest.mark.gpu
 R = dataclasses.replace
@@ -161,6 +161,50 @@ def test_argument_errors_launch_nothing():
         assert ei.value.code == 1
         torch.cuda.synchronize()
         assert bool((big == 0xCD).all())
+
+
+def test_zero_copy_phases_accept_their_own_arenas_and_launch_nothing():
+    """Sec. 5.2: with TP and the block table kept, attention weights and KV cache are used in
+    place.  Such a phase accepts dst == src and leaves the arenas alone, alone or inside the
+    whole step; a partly aliased call is still refused."""
+    import dataclasses
+    from gpu_util import oracle_phase
+    base = W.make_workload("c4_large").with_layers(2)
+    kept = dataclasses.replace(base.new, tp=base.old.tp, kv_num_blocks=base.old.kv_num_blocks,
+                               block_table=base.old.block_table)
+    wl = dataclasses.replace(base, new=kept)
+    with make_plan(wl) as plan:
+        assert [plan.phase_is_identity(ph) for ph in range(3)] == [False, True, True]
+        src = [WD.alloc_filled(plan.arena_bytes(ph, E.SIDE_OLD), wl.seed, KINDS[ph]) for ph in range(3)]
+        before = [[t.clone() for t in g] for g in src]
+        plan.reshard_attn(src[1], src[1])
+        plan.reshard_kv(src[2], src[2])
+        dst0 = WD.alloc_const(plan.arena_bytes(E.PHASE_EXPERTS, E.SIDE_NEW))
+        plan.reshard_step(src, [dst0, src[1], src[2]])
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        for ph in (1, 2):
+            h = [t.cpu().numpy() for t in before[ph]]
+            want = [a.copy() for a in h]
+            oracle_phase(wl, ph, h, want)          # the oracle on a copy of the input changes nothing either
+            for g, w, x in zip(src[ph], want, h):
+                assert np.array_equal(w, x) and np.array_equal(g.cpu().numpy(), x)
+        want = [np.full(t.numel(), WD.FILL_BYTE, np.uint8) for t in dst0]
+        oracle_phase(wl, 0, [t.cpu().numpy() for t in src[0]], want)
+        for g, w in zip(dst0, want):
+            assert np.array_equal(g.cpu().numpy(), w)
+        # one rank aliased, the other not: not the zero-copy case
+        other = torch.empty_like(src[2][1])
+        with pytest.raises(E.EmoeError) as ei:
+            plan.reshard_kv(src[2], [src[2][0], other])
+        assert ei.value.code == 6
+        # a phase that does move bytes never accepts its own arenas
+        with pytest.raises(E.EmoeError) as ei:
+            plan.reshard_experts(src[0], src[0][:1] + dst0[1:])
+        assert ei.value.code == 6
+        # and the same phases still copy when given separate arenas
+        for ph in (1, 2):
+            check_phase_full(wl, plan, ph)
 
 
 def _step_on_host_buffers(wl, host_step):

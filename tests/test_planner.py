@@ -137,6 +137,31 @@ def test_identity_plan_is_one_run_per_arena():
             assert list(segs["run_bytes"]) == plan.arena_bytes(phase, E.SIDE_OLD)
 
 
+def test_phases_that_stay_in_place_are_flagged_for_zero_copy():
+    """Sec. 5.2: with TP kept, attention weights and KV cache are used where they are.  The plan
+    flags a phase as identity exactly when old and new agree on everything that phase sees."""
+    wl = small("c2_mid")
+    with E.Plan(wl.shape, wl.old, wl.old, host_only=True) as plan:
+        assert [plan.phase_is_identity(ph) for ph in range(3)] == [True, True, True]
+    with E.Plan(wl.shape, wl.old, wl.new, host_only=True) as plan:       # EP and the KV tables change, TP kept
+        assert [plan.phase_is_identity(ph) for ph in range(3)] == [False, True, False]
+    w4 = small("c4_large")                                               # TP 2 -> 4 as well
+    with E.Plan(w4.shape, w4.old, w4.new, host_only=True) as plan:
+        assert [plan.phase_is_identity(ph) for ph in range(3)] == [False, False, False]
+    # the paper's own step: experts re-placed, TP and the KV table kept
+    import dataclasses
+    kept = dataclasses.replace(wl.new, kv_num_blocks=wl.old.kv_num_blocks, block_table=wl.old.block_table)
+    with E.Plan(wl.shape, wl.old, kept, host_only=True) as plan:
+        assert [plan.phase_is_identity(ph) for ph in range(3)] == [False, True, True]
+    # same TP and table but a larger pool: the arenas differ in size, so the KV cache has to be copied
+    grown = dataclasses.replace(kept, kv_num_blocks=wl.old.kv_num_blocks + 1)
+    with E.Plan(wl.shape, wl.old, grown, host_only=True) as plan:
+        assert [plan.phase_is_identity(ph) for ph in range(3)] == [False, True, False]
+    # attention onto extra replicas is a copy even with TP kept
+    with E.Plan(wl.shape, wl.old, kept, host_only=True, attn_replicas=2) as plan:
+        assert not plan.phase_is_identity(E.PHASE_ATTN)
+
+
 # ---- validation ------------------------------------------------------------------------
 
 def _plan_code(shape, old, new):
