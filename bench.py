@@ -481,7 +481,34 @@ def run_e2e(torch, plan, src, dst, steps, stream):
     e1.record(stream)
     stream.synchronize()
     ms = e0.elapsed_time(e1) / steps
-    return ms, h2d, d2h
+    return ms, h2d, d2h, host_link_rates(torch, h_src, h_dst, src, dst)
+
+
+def host_link_rates(torch, h_src, h_dst, src, dst):
+    """The yardstick for the end-to-end number: plain pinned copies of the largest old arena
+    host->device and the largest new arena device->host, on two streams at once (no kernel in
+    between), GB/s per direction while both run."""
+    hs, ds = max(((h, d) for hg, dg in zip(h_src, src) for h, d in zip(hg, dg)), key=lambda x: x[0].numel())
+    hd, dd = max(((h, d) for hg, dg in zip(h_dst, dst) for h, d in zip(hg, dg)), key=lambda x: x[0].numel())
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    reps = 3
+    torch.cuda.synchronize()
+    for timed in (False, True):
+        with torch.cuda.stream(s_in):
+            ev[0].record()
+            for _ in range(reps if timed else 1):
+                ds.copy_(hs, non_blocking=True)
+            ev[1].record()
+        with torch.cuda.stream(s_out):
+            ev[2].record()
+            for _ in range(reps if timed else 1):
+                hd.copy_(dd, non_blocking=True)
+            ev[3].record()
+        torch.cuda.synchronize()
+    return {"h2d_gbs": round(reps * hs.numel() / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9, 2),
+            "d2h_gbs": round(reps * hd.numel() / (ev[2].elapsed_time(ev[3]) * 1e-3) / 1e9, 2),
+            "bytes_each_way": [hs.numel(), hd.numel()], "how": "pinned copies both ways at once, no kernel"}
 
 
 # ---- C5: reshard on a low-priority stream beside a grouped expert GEMM -------------------
@@ -1037,10 +1064,14 @@ def main():
                 raise MemoryError("host has %.0f GB available, the step needs %.0f GB pinned"
                                   % (psutil.virtual_memory().available / 1e9, need / 1e9))
             with E.Plan(wl.shape, wl.old, wl.new, host_step=True) as e2e_plan:   # pipelined form
-                e_ms, h2d, d2h = run_e2e(torch, e2e_plan, src, dst, args.e2e_steps, stream)
+                e_ms, h2d, d2h, link = run_e2e(torch, e2e_plan, src, dst, args.e2e_steps, stream)
+            # the step cannot beat the slower direction of the host link carrying its bytes
+            link_ms = max(h2d / link["h2d_gbs"], d2h / link["d2h_gbs"]) / 1e6
             line["e2e"] = {"value": round(2 * rep["bytes_moved"] / (e_ms * 1e-3) / 1e9, 2),
                            "unit": UNIT, "ms_per_step": round(e_ms, 2), "steps": args.e2e_steps,
-                           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+                           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                           "host_link": link, "host_link_bound_ms": round(link_ms, 2),
+                           "frac_of_host_link": round(link_ms / e_ms, 3)}
         except Exception as e:  # report, never hide
             line["e2e"] = {"value": None, "unit": UNIT, "error": repr(e)[:200]}
         # CPU baseline: the oracle on sampled layers of the same arenas
