@@ -685,7 +685,8 @@ emoe_status_t emoe_place_min_transfer(int32_t n_experts, const emoe_config_t *ol
  * shape, flags, options and everything emoe_plan_create reads from the two configurations
  * (placements, TP/EP degrees, pool sizes, sequence lengths, the mapped block-table
  * entries) are byte-for-byte the same, and otherwise creates one (on the current CUDA
- * device unless EMOE_PLAN_HOST_ONLY) and keeps it.  *hit (optional): 1 / 0.
+ * device unless EMOE_PLAN_HOST_ONLY; the device is part of the key) and keeps it.
+ * *hit (optional): 1 / 0.
  * The cache OWNS its plans: never pass them to emoe_plan_destroy.  It keeps at most
  * `capacity` plans; inserting one more destroys the least recently used one, so a plan
  * obtained earlier may die in a later emoe_plan_cache_get - do not hold more plans than

@@ -5,6 +5,8 @@
 // and scale-down mirrors scale-up, App. E).  A plan is a pure function of the model shape,
 // the two configurations and the flags, so it can be kept and reused; only plans whose
 // inputs are byte-for-byte the same are shared.
+#include <cuda_runtime_api.h>
+
 #include <algorithm>
 #include <cstdint>
 #include <cstring>
@@ -84,6 +86,10 @@ emoe_status_t emoe_plan_cache_get(emoe_plan_cache_t *c, const emoe_shape_t *shap
     const int64_t replicas = options ? options->attn_new_replicas : 0;
     put(&key, &scale, sizeof(scale));
     put(&key, &replicas, sizeof(replicas));
+    // a plan's tables live on the device that was current when it was made
+    int device = -1;
+    if (!(flags & EMOE_PLAN_HOST_ONLY) && cudaGetDevice(&device) != cudaSuccess) device = -1;
+    put_i32(&key, device);
     cacheable = config_key(*shape, *old_cfg, &key) && config_key(*shape, *new_cfg, &key);
   } catch (const std::bad_alloc &) {
     return EMOE_ERR_OOM;
@@ -91,7 +97,7 @@ emoe_status_t emoe_plan_cache_get(emoe_plan_cache_t *c, const emoe_shape_t *shap
   std::lock_guard<std::mutex> lock(c->mu);
   if (cacheable)
     for (auto it = c->lru.begin(); it != c->lru.end(); ++it)
-      if (it->key == key) {
+      if (!it->key.empty() && it->key == key) {
         c->lru.splice(c->lru.begin(), c->lru, it);
         ++c->hits;
         *plan = c->lru.front().plan;
@@ -102,6 +108,9 @@ emoe_status_t emoe_plan_cache_get(emoe_plan_cache_t *c, const emoe_shape_t *shap
   const emoe_status_t st = emoe_plan_create_ex(shape, old_cfg, new_cfg, flags, options, &p);
   if (st != EMOE_OK) return st;   // invalid inputs are reported, never stored
   ++c->misses;
+  // An input the planner accepts although its key could not be formed completely is owned
+  // and evicted like any other plan but never found again: a lookup compares complete keys only.
+  if (!cacheable) key.clear();
   try {
     c->lru.push_front(Entry{std::move(key), p});
   } catch (const std::bad_alloc &) {
