@@ -214,6 +214,8 @@ emoe_status_t emoe_plan_create_ex(const emoe_shape_t *shape, const emoe_config_t
  * whether a phase qualifies.
  * The call only enqueues work on the stream: it neither synchronises nor
  * allocates.  The pointer arrays are read before the call returns.
+ * The device the plan was created on must be the current device of the calling
+ * thread (EMOE_ERR_CUDA otherwise, nothing enqueued).
  * Calls may be enqueued on any streams; at most 4 launches of the SAME phase of
  * the SAME plan (a whole-step call counts as a phase of its own) may be
  * enqueued and unfinished at once when they are on different streams (they

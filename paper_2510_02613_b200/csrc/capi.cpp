@@ -488,6 +488,9 @@ emoe_status_t check_arenas(const emoe_plan *p, int phase, const void *const *src
   if (zero_copy) *zero_copy = false;
   if (!p || !src || !dst || p->inplace) return EMOE_ERR_INVALID_ARG;
   if (p->host_only) return EMOE_ERR_CUDA;
+  // the plan's tables, counters and streams belong to the device it was made on
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev != p->device) return EMOE_ERR_CUDA;
   const PhasePlan &pp = p->hp.phase[phase];
   const int ns = ranks_of(p, phase, EMOE_SIDE_OLD), nd = ranks_of(p, phase, EMOE_SIDE_NEW);
   std::memset(out, 0, sizeof(*out));
@@ -987,6 +990,8 @@ emoe_status_t emoe_reshard_experts_inplace(const emoe_plan_t *p, void *const *ar
   TraceRange trace("emoe_reshard_experts_inplace");
   if (!p || !arenas || !p->inplace) return EMOE_ERR_INVALID_ARG;
   if (p->host_only) return EMOE_ERR_CUDA;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev != p->device) return EMOE_ERR_CUDA;
   const PhasePlan &pp = p->hp.phase[EMOE_PHASE_EXPERTS];
   const int ns = p->hp.ep_old, nd = p->hp.ep_new, n = ns > nd ? ns : nd;
   RankPtrs ptrs;
