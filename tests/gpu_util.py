@@ -62,10 +62,13 @@ def check_phase_full(wl, plan, phase, src=None):
 
 def check_phase_layers(wl, plan, phase, src, dst, layers):
     """Full-size run already done into dst: compare the given layers with the oracle
-    run on those layers alone (layers are independent in every phase)."""
+    run on those layers alone (layers are independent in every phase).  A few layers are
+    in flight at once: the oracle call and the comparisons release the interpreter lock."""
+    from concurrent.futures import ThreadPoolExecutor
     L = wl.shape.n_layers
     wl1 = wl.with_layers(1)
-    for l in layers:
+
+    def one(l):
         h_src = []
         for t in src:
             per = t.numel() // L
@@ -79,6 +82,10 @@ def check_phase_layers(wl, plan, phase, src, dst, layers):
                 bad = np.flatnonzero(g != w)
                 raise AssertionError("%s phase %d layer %d rank %d: %d bytes differ, first at %d"
                                      % (wl.name, phase, l, r, bad.size, bad[0]))
+
+    with ThreadPoolExecutor(max_workers=4) as pool:
+        for _ in pool.map(one, layers):
+            pass
 
 
 def check_step_full(wl, plan):
