@@ -208,8 +208,9 @@ emoe_status_t emoe_plan_create_ex(const emoe_shape_t *shape, const emoe_config_t
  * using them): when a phase changes nothing - same rank count, same arena
  * sizes, every byte written comes from the same offset of the same rank index
  * (TP kept and, for the KV cache, block table and pool size kept; for experts,
- * placement kept) - the caller may pass dst[r] == src[r] for EVERY rank; the
- * call then returns EMOE_OK and enqueues nothing for that phase.  Any other
+ * placement kept) - the caller may pass dst[r] == src[r] for EVERY rank (after
+ * emoe_plan_set_local_rank: for that rank); the call then returns EMOE_OK and
+ * enqueues nothing for that phase.  Any other
  * intersection is still EMOE_ERR_OVERLAP.  emoe_plan_phase_is_identity tells
  * whether a phase qualifies.
  * The call only enqueues work on the stream: it neither synchronises nor

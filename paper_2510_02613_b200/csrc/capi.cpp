@@ -495,8 +495,10 @@ emoe_status_t check_arenas(const emoe_plan *p, int phase, const void *const *src
   const int ns = ranks_of(p, phase, EMOE_SIDE_OLD), nd = ranks_of(p, phase, EMOE_SIDE_NEW);
   std::memset(out, 0, sizeof(*out));
   if (zero_copy && pp.identity && ns == nd) {
-    bool same = true;
-    for (int r = 0; r < ns; ++r) same = same && src[r] == dst[r] && (src[r] || !pp.arena_old[r]);
+    bool same = true;   // with a local rank set only that rank's arena is looked at
+    for (int r = 0; r < ns; ++r)
+      if (p->local_rank < 0 || r == p->local_rank)
+        same = same && src[r] == dst[r] && (src[r] || !pp.arena_old[r]);
     if (same) { *zero_copy = true; return EMOE_OK; }
   }
   // With a local rank set, only that rank's destination arena and the source arenas its

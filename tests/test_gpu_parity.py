@@ -202,6 +202,14 @@ def test_zero_copy_phases_accept_their_own_arenas_and_launch_nothing():
         with pytest.raises(E.EmoeError) as ei:
             plan.reshard_experts(src[0], src[0][:1] + dst0[1:])
         assert ei.value.code == 6
+        # one rank per process: only the local rank's arena is looked at
+        plan.set_local_rank(1)
+        plan.reshard_kv([None, src[2][1]], [None, src[2][1]])
+        plan.reshard_attn([None, src[1][1]], [None, src[1][1]])
+        plan.set_local_rank(-1)
+        torch.cuda.synchronize()
+        for ph in (1, 2):
+            assert all(torch.equal(a, b) for a, b in zip(src[ph], before[ph]))
         # and the same phases still copy when given separate arenas
         for ph in (1, 2):
             check_phase_full(wl, plan, ph)
